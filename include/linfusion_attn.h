@@ -1,0 +1,150 @@
+/*
+ * linfusion_attn.h — C ABI of the B200 (sm_100a) normalized non-causal linear attention.
+ *
+ * The operation is the token mixer of the LinFusion module (Sec. 2.3, Prop. 2 / Prop. 3,
+ * with the normalization of Sec. 2.2 / Eq. 5 in its non-causal form).  For every
+ * (batch, head) slab, with Q = f'(X), K = g'(X), V = X W_V already computed by the caller:
+ *
+ *     S   = sum_j phi(K_j)^T V_j          d x d state      (g'(X)^T X of Prop. 2)
+ *     z   = sum_j phi(K_j)                1 x d normalizer (Z of Eq. 5, scan replaced by the sum)
+ *     Y_i = phi(Q_i) S / (phi(Q_i) . z + eps)
+ *
+ * phi is the non-negative activation of Sec. 2.2 (the paper gives no closed form; this
+ * library implements phi(x) = elu(x) + 1, and the identity for callers whose features are
+ * already non-negative).  eps is this library's guard on the denominator; the paper has none.
+ *
+ * Unless a function says otherwise, tensor arguments are DEVICE pointers to dense row-major
+ * bf16 [B, H, N, d] (token rows of d contiguous channels, one slab of N rows per (b, h)),
+ * 16-byte aligned.  Y must not overlap Q, K or V.  The caller owns Q, K, V, Y and the stream.
+ * The handle owns an fp32 workspace on its device unless the caller lends one (set_workspace).
+ *
+ * Every function returns a status code; nothing throws or aborts across this boundary.
+ * forward() only enqueues work on the given stream and returns without synchronizing; it
+ * allocates nothing.  Results are bit-identical from call to call for identical inputs
+ * (fixed split of N, fixed summation order, no floating-point atomics).
+ * One forward may be in flight per handle at a time (the workspace is shared).
+ */
+#ifndef LINFUSION_ATTN_H
+#define LINFUSION_ATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct linfusion_attn linfusion_attn_t; /* opaque handle */
+
+typedef enum {
+    LINFUSION_OK = 0,
+    LINFUSION_ERR_INVALID_ARG = 1, /* null / misaligned pointer, non-positive size, bad eps   */
+    LINFUSION_ERR_UNSUPPORTED = 2, /* head dim, phi, flags or device this build cannot serve  */
+    LINFUSION_ERR_ALLOC = 3,       /* device workspace could not be allocated / is too small   */
+    LINFUSION_ERR_CUDA = 4,        /* a CUDA runtime or driver call failed                     */
+    LINFUSION_ERR_TIMEOUT = 5      /* a bounded device-side wait expired (see status())        */
+} linfusion_status_t;
+
+typedef enum {
+    LINFUSION_PHI_ELU_PLUS_ONE = 0, /* phi(x) = x + 1 (x > 0), exp(x) (x <= 0)  */
+    LINFUSION_PHI_IDENTITY = 1      /* phi(x) = x: inputs are non-negative features already */
+} linfusion_phi_t;
+
+/* flags: kernel-variant selection.  0 lets the library choose from (N, d, B*H). */
+#define LINFUSION_VARIANT_AUTO 0u
+#define LINFUSION_VARIANT_SPLIT 1u   /* three launches: split-N state, reduction, apply (any supported d) */
+#define LINFUSION_VARIANT_STREAM 2u  /* three launches, TMA-pipelined persistent kernels (d = 64 only)    */
+#define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N)               */
+#define LINFUSION_VARIANT_MASK 0xFu
+
+typedef struct {
+    int32_t B;      /* batch                                   > 0 */
+    int32_t H;      /* heads                                   > 0 */
+    int32_t N;      /* tokens per slab                         > 0 */
+    int32_t d;      /* head dim: one of 32, 40, 64, 80, 128, 160   */
+    int32_t phi;    /* linfusion_phi_t                             */
+    float eps;      /* finite, >= 0; added once to phi(Q_i) . z    */
+    int32_t device; /* CUDA device ordinal the handle lives on     */
+    uint32_t flags; /* LINFUSION_VARIANT_*                         */
+} linfusion_attn_desc_t;
+
+/*
+ * Create a handle for one problem shape (Prop. 2's token mixer at fixed B, H, N, d).
+ * Validates the descriptor, checks that `device` is compute capability 10.x, fixes the
+ * split of N and allocates the workspace (cudaMalloc) on that device.
+ * Errors: INVALID_ARG (null pointers, sizes <= 0, eps negative or not finite),
+ * UNSUPPORTED (d, phi, variant, device architecture), ALLOC, CUDA.  *out is NULL on error.
+ */
+linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linfusion_attn_t** out);
+
+/*
+ * Enqueue Y = norm-linear-attention(Q, K, V) on `cuda_stream` (a cudaStream_t / CUstream;
+ * NULL is the legacy default stream).  q, k, v: const bf16 [B,H,N,d] device memory;
+ * y: bf16 [B,H,N,d] device memory, written in full, rounded to nearest even from fp32.
+ * Steps: split-N state reduction (S_p, z_p per chunk p of the tokens; Prop. 2 and Eq. 5),
+ * fixed-order reduction to (S, z), apply — or all three in one clustered launch for small N.
+ * Errors: INVALID_ARG (null handle or pointer, pointer not 16-byte aligned, y overlapping an
+ * input), CUDA (launch or tensor-map encoding failed).  A bounded device-side wait that
+ * expired is reported by status(), not here.
+ */
+linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, const void* k,
+                                          const void* v, void* y, void* cuda_stream);
+
+/*
+ * The same operation for callers whose tensors live in HOST memory (pinned memory makes the
+ * copies asynchronous): copies K, V, Q to device staging buffers owned by the handle, runs
+ * forward() on them and copies Y back, all enqueued on `cuda_stream`.  The staging buffers
+ * (4 x B*H*N*d*2 bytes) are allocated with cudaMalloc by the first call on a handle and freed
+ * by destroy().  y_host is valid after the stream has been synchronized.
+ * Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* q_host,
+                                               const void* k_host, const void* v_host, void* y_host,
+                                               void* cuda_stream);
+
+/* Free the handle, the workspace it owns and its staging buffers.  destroy(NULL) is OK. */
+linfusion_status_t linfusion_attn_destroy(linfusion_attn_t* h);
+
+/* Static, NUL-terminated description of a status code. */
+const char* linfusion_status_string(linfusion_status_t s);
+
+/*
+ * Bytes of device workspace a handle for `desc` needs, for callers that want to own it:
+ * fp32 partial states S_p | z_p of the split of N, the reduced state S | z per slab, and one
+ * status word.  Pure host computation (no CUDA call) for a given SM count; `sm_count` <= 0
+ * means 148 (B200).  Errors: INVALID_ARG, UNSUPPORTED.
+ */
+linfusion_status_t linfusion_attn_workspace_bytes(const linfusion_attn_desc_t* desc, int sm_count,
+                                                  size_t* bytes);
+
+/*
+ * Lend a device workspace (256-byte aligned, at least workspace_bytes) to the handle, which
+ * stops using — and frees — its own.  The caller keeps ownership and must keep it alive
+ * until the handle is destroyed.  Errors: INVALID_ARG, ALLOC (too small).
+ */
+linfusion_status_t linfusion_attn_set_workspace(linfusion_attn_t* h, void* dev_ptr, size_t bytes);
+
+/*
+ * Synchronize the handle's last stream and read the device status word: OK, or TIMEOUT if
+ * a kernel gave up on a bounded wait (its outputs are then undefined), or CUDA.
+ */
+linfusion_status_t linfusion_attn_status(linfusion_attn_t* h);
+
+/*
+ * Copy the reduced state of the last forward to HOST buffers (fp32): S [B*H][d][d] (row =
+ * feature c of K, column = channel e of V) and z [B*H][d].  Synchronizes the handle's last
+ * stream.  Either pointer may be NULL.  This is the c' x c quantity that the paper's
+ * distributed inference exchanges between devices (Sec. 4.3).  Errors: INVALID_ARG, CUDA.
+ */
+linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host, float* z_host);
+
+/* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
+const char* linfusion_attn_variant_name(const linfusion_attn_t* h);
+
+/* Number of kernel launches one forward() enqueues for this handle. */
+int32_t linfusion_attn_launches_per_forward(const linfusion_attn_t* h);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LINFUSION_ATTN_H */

@@ -1,0 +1,214 @@
+"""ctypes binding over the C ABI in ``include/linfusion_attn.h``.
+
+Argument marshalling only: every step of the attention runs in the CUDA library.  There is no
+CPU fallback; loading fails loudly when ``liblinfusion_attn.so`` has not been built
+(``python -m paper_2409_02097_b200.build``).  PyTorch is used for device memory and streams.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "liblinfusion_attn.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(6)
+PHI_ELU_PLUS_ONE, PHI_IDENTITY = 0, 1
+VARIANT_AUTO, VARIANT_SPLIT, VARIANT_STREAM, VARIANT_CLUSTER = 0, 1, 2, 3
+VARIANTS = {"auto": VARIANT_AUTO, "split": VARIANT_SPLIT, "stream": VARIANT_STREAM,
+            "cluster": VARIANT_CLUSTER}
+
+EXPORTED = [
+    "linfusion_attn_create", "linfusion_attn_forward", "linfusion_attn_forward_host",
+    "linfusion_attn_destroy", "linfusion_status_string", "linfusion_attn_workspace_bytes",
+    "linfusion_attn_set_workspace", "linfusion_attn_status", "linfusion_attn_read_state",
+    "linfusion_attn_variant_name", "linfusion_attn_launches_per_forward",
+]
+
+
+class Desc(ctypes.Structure):
+    """Mirror of ``linfusion_attn_desc_t``."""
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32),
+                ("d", ctypes.c_int32), ("phi", ctypes.c_int32), ("eps", ctypes.c_float),
+                ("device", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class LinFusionError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        super().__init__(f"{what}: {status_string(code)} (status {code})")
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Load the CUDA library; raises if it is missing (there is no other implementation)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} not found: build it with `python -m paper_2409_02097_b200.build` "
+            "(nvcc, sm_100a).  This package has no CPU or PyTorch fallback.")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, st = ctypes.c_void_p, ctypes.c_int
+    lib.linfusion_attn_create.restype = st
+    lib.linfusion_attn_create.argtypes = [ctypes.POINTER(Desc), ctypes.POINTER(vp)]
+    lib.linfusion_attn_forward.restype = st
+    lib.linfusion_attn_forward.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.linfusion_attn_forward_host.restype = st
+    lib.linfusion_attn_forward_host.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.linfusion_attn_destroy.restype = st
+    lib.linfusion_attn_destroy.argtypes = [vp]
+    lib.linfusion_status_string.restype = ctypes.c_char_p
+    lib.linfusion_status_string.argtypes = [st]
+    lib.linfusion_attn_workspace_bytes.restype = st
+    lib.linfusion_attn_workspace_bytes.argtypes = [ctypes.POINTER(Desc), ctypes.c_int,
+                                                   ctypes.POINTER(ctypes.c_size_t)]
+    lib.linfusion_attn_set_workspace.restype = st
+    lib.linfusion_attn_set_workspace.argtypes = [vp, vp, ctypes.c_size_t]
+    lib.linfusion_attn_status.restype = st
+    lib.linfusion_attn_status.argtypes = [vp]
+    lib.linfusion_attn_read_state.restype = st
+    lib.linfusion_attn_read_state.argtypes = [vp, vp, vp]
+    lib.linfusion_attn_variant_name.restype = ctypes.c_char_p
+    lib.linfusion_attn_variant_name.argtypes = [vp]
+    lib.linfusion_attn_launches_per_forward.restype = ctypes.c_int32
+    lib.linfusion_attn_launches_per_forward.argtypes = [vp]
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().linfusion_status_string(int(code)).decode()
+
+
+def make_desc(B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto") -> Desc:
+    flags = VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    return Desc(int(B), int(H), int(N), int(d), int(phi), float(eps), int(device), flags)
+
+
+def linfusion_attn_workspace_bytes(desc: Desc, sm_count: int = 0) -> int:
+    out = ctypes.c_size_t(0)
+    rc = load_library().linfusion_attn_workspace_bytes(ctypes.byref(desc), int(sm_count),
+                                                       ctypes.byref(out))
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_workspace_bytes")
+    return int(out.value)
+
+
+def linfusion_attn_create(desc: Desc) -> ctypes.c_void_p:
+    handle = ctypes.c_void_p()
+    rc = load_library().linfusion_attn_create(ctypes.byref(desc), ctypes.byref(handle))
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_create")
+    return handle
+
+
+def linfusion_attn_forward(handle, q_ptr: int, k_ptr: int, v_ptr: int, y_ptr: int,
+                           stream_ptr: int = 0) -> None:
+    rc = load_library().linfusion_attn_forward(handle, q_ptr, k_ptr, v_ptr, y_ptr, stream_ptr)
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_forward")
+
+
+def linfusion_attn_forward_host(handle, q_ptr: int, k_ptr: int, v_ptr: int, y_ptr: int,
+                                stream_ptr: int = 0) -> None:
+    rc = load_library().linfusion_attn_forward_host(handle, q_ptr, k_ptr, v_ptr, y_ptr, stream_ptr)
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_forward_host")
+
+
+def linfusion_attn_destroy(handle) -> None:
+    rc = load_library().linfusion_attn_destroy(handle)
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_destroy")
+
+
+class LinFusionAttention:
+    """One handle per shape.  ``forward`` takes bf16 CUDA tensors [B, H, N, d]."""
+
+    def __init__(self, B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto"):
+        self.desc = make_desc(B, H, N, d, phi, eps, device, variant)
+        self.shape = (int(B), int(H), int(N), int(d))
+        self._lib = load_library()
+        self._h = linfusion_attn_create(self.desc)
+        self._lent_ws = None
+
+    # -- properties -------------------------------------------------------------------------
+    @property
+    def variant(self) -> str:
+        return self._lib.linfusion_attn_variant_name(self._h).decode()
+
+    @property
+    def launches_per_forward(self) -> int:
+        return int(self._lib.linfusion_attn_launches_per_forward(self._h))
+
+    # -- calls ------------------------------------------------------------------------------
+    def _check(self, t, name):
+        import torch
+        if tuple(t.shape) != self.shape or t.dtype != torch.bfloat16 or not t.is_contiguous():
+            raise ValueError(f"{name}: expected contiguous bf16 tensor of shape {self.shape}")
+
+    def forward(self, q, k, v, y=None, stream: Optional[int] = None):
+        import torch
+        for t, n in ((q, "q"), (k, "k"), (v, "v")):
+            self._check(t, n)
+            if not t.is_cuda:
+                raise ValueError(f"{n}: expected a CUDA tensor")
+        if y is None:
+            y = torch.empty_like(q)
+        else:
+            self._check(y, "y")
+        if stream is None:
+            stream = torch.cuda.current_stream(q.device).cuda_stream
+        linfusion_attn_forward(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(), y.data_ptr(),
+                               stream)
+        return y
+
+    def forward_host(self, q, k, v, y, stream: Optional[int] = None):
+        """q, k, v, y: CPU (ideally pinned) bf16 tensors; y is valid after a stream sync."""
+        import torch
+        for t, n in ((q, "q"), (k, "k"), (v, "v"), (y, "y")):
+            self._check(t, n)
+            if t.is_cuda:
+                raise ValueError(f"{n}: expected a host tensor")
+        if stream is None:
+            stream = torch.cuda.current_stream(self.desc.device).cuda_stream
+        linfusion_attn_forward_host(self._h, q.data_ptr(), k.data_ptr(), v.data_ptr(),
+                                    y.data_ptr(), stream)
+        return y
+
+    def status(self) -> int:
+        return int(self._lib.linfusion_attn_status(self._h))
+
+    def read_state(self):
+        """(S [B,H,d,d], z [B,H,d]) of the last forward as fp32 numpy arrays."""
+        import numpy as np
+        B, H, _, d = self.shape
+        S = np.empty((B, H, d, d), dtype=np.float32)
+        z = np.empty((B, H, d), dtype=np.float32)
+        rc = self._lib.linfusion_attn_read_state(self._h, S.ctypes.data, z.ctypes.data)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_read_state")
+        return S, z
+
+    def set_workspace(self, tensor) -> None:
+        rc = self._lib.linfusion_attn_set_workspace(self._h, tensor.data_ptr(),
+                                                    tensor.numel() * tensor.element_size())
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_set_workspace")
+        self._lent_ws = tensor
+
+    def close(self) -> None:
+        if self._h is not None and self._h.value:
+            linfusion_attn_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

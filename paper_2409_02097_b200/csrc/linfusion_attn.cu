@@ -1,0 +1,629 @@
+// Host side of the C ABI declared in include/linfusion_attn.h: descriptor validation, the
+// fixed split of N, workspace layout, tensor-map encoding and kernel launches.
+#include "../../include/linfusion_attn.h"
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "split_kernels.cuh"
+#include "stream_kernels.cuh"
+
+using namespace lf;
+
+namespace {
+
+constexpr int kDefaultSmCount = 148;
+constexpr int kStreamApplyWarps = 12;
+using ApplyCfg = StreamApplyCfg<kStreamApplyWarps>;
+
+enum Variant { kSplit = 1, kStream = 2, kCluster = 3 };
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+bool supported_d(int d)
+{
+    return d == 32 || d == 40 || d == 64 || d == 80 || d == 128 || d == 160;
+}
+
+// Everything that follows from (descriptor, SM count) alone.
+struct Plan {
+    int variant = 0;
+    int slabs = 0;
+    int state_floats = 0;
+    // split
+    int chunks_state = 0, chunks_apply = 0;
+    // stream
+    int tiles_state = 0, tiles_apply = 0;  // per slab
+    long long W_state = 0, W_apply = 0;
+    int G_state = 0, G_apply = 0, spans = 0;
+    // cluster
+    int cluster_size = 0;
+    // workspace (bytes, offsets)
+    size_t partial_bytes = 0, state_off = 0, status_off = 0, total_bytes = 0;
+    int launches = 0;
+};
+
+int tile_q_of(int d) { return 16 * ((d + 15) / 16); }
+
+linfusion_status_t validate(const linfusion_attn_desc_t* d)
+{
+    if (d == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    if (d->B <= 0 || d->H <= 0 || d->N <= 0 || d->d <= 0) return LINFUSION_ERR_INVALID_ARG;
+    if (!std::isfinite(d->eps) || d->eps < 0.0f) return LINFUSION_ERR_INVALID_ARG;
+    if (d->device < 0) return LINFUSION_ERR_INVALID_ARG;
+    if (static_cast<long long>(d->B) * d->H > 65535) return LINFUSION_ERR_UNSUPPORTED;
+    if (!supported_d(d->d)) return LINFUSION_ERR_UNSUPPORTED;
+    if (d->phi != LINFUSION_PHI_ELU_PLUS_ONE && d->phi != LINFUSION_PHI_IDENTITY)
+        return LINFUSION_ERR_UNSUPPORTED;
+    if ((d->flags & ~LINFUSION_VARIANT_MASK) != 0u) return LINFUSION_ERR_UNSUPPORTED;
+    uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
+    if (v > LINFUSION_VARIANT_CLUSTER) return LINFUSION_ERR_UNSUPPORTED;
+    if (v == LINFUSION_VARIANT_STREAM && d->d != kStreamD) return LINFUSION_ERR_UNSUPPORTED;
+    return LINFUSION_OK;
+}
+
+int largest_cluster(int tiles_kv)
+{
+    int c = 8;
+    while (c > 1 && c > tiles_kv) c >>= 1;
+    return c;
+}
+
+linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan* p)
+{
+    linfusion_status_t st = validate(d);
+    if (st != LINFUSION_OK) return st;
+    if (sm_count <= 0) sm_count = kDefaultSmCount;
+    *p = Plan();
+    const int slabs = d->B * d->H;
+    p->slabs = slabs;
+    p->state_floats = d->d * (d->d + 1);
+    const int tiles_kv = (d->N + 63) / 64;
+    const int tiles_q = (d->N + tile_q_of(d->d) - 1) / tile_q_of(d->d);
+
+    uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
+    if (v == LINFUSION_VARIANT_AUTO) {
+        const long long tokens = static_cast<long long>(slabs) * d->N;
+        const int cl = largest_cluster(tiles_kv);
+        if (d->d == kStreamD && slabs <= sm_count && tokens >= 4ll * sm_count * StreamStateCfg::TILE)
+            v = LINFUSION_VARIANT_STREAM;
+        else if (static_cast<long long>(slabs) * cl <= 2ll * sm_count && d->N <= 1024 * cl)
+            v = LINFUSION_VARIANT_CLUSTER;
+        else
+            v = LINFUSION_VARIANT_SPLIT;
+    }
+    if (v == LINFUSION_VARIANT_STREAM && slabs > sm_count) return LINFUSION_ERR_UNSUPPORTED;
+    p->variant = static_cast<int>(v);
+
+    size_t partial_floats = 0;
+    if (v == LINFUSION_VARIANT_SPLIT) {
+        int cs = (2 * sm_count + slabs - 1) / slabs;
+        p->chunks_state = cs < 1 ? 1 : (cs > tiles_kv ? tiles_kv : cs);
+        int ca = (4 * sm_count + slabs - 1) / slabs;
+        p->chunks_apply = ca < 1 ? 1 : (ca > tiles_q ? tiles_q : ca);
+        partial_floats = static_cast<size_t>(slabs) * p->chunks_state * p->state_floats;
+        p->launches = 3;
+    } else if (v == LINFUSION_VARIANT_STREAM) {
+        p->tiles_state = (d->N + StreamStateCfg::TILE - 1) / StreamStateCfg::TILE;
+        p->tiles_apply = (d->N + ApplyCfg::TILE - 1) / ApplyCfg::TILE;
+        p->W_state = static_cast<long long>(slabs) * p->tiles_state;
+        p->W_apply = static_cast<long long>(slabs) * p->tiles_apply;
+        long long gs = static_cast<long long>(sm_count) * StreamStateCfg::CTAS_PER_SM;
+        p->G_state = static_cast<int>(gs < p->W_state ? gs : p->W_state);
+        long long ga = sm_count;
+        p->G_apply = static_cast<int>(ga < p->W_apply ? ga : p->W_apply);
+        int spans = 1;
+        for (int g = 0; g < p->G_state; ++g) {
+            long long b = unit_begin(g, p->W_state, p->G_state);
+            long long e = unit_begin(g + 1, p->W_state, p->G_state);
+            if (e > b) {
+                int s = static_cast<int>((e - 1) / p->tiles_state - b / p->tiles_state) + 1;
+                if (s > spans) spans = s;
+            }
+        }
+        p->spans = spans;
+        partial_floats = static_cast<size_t>(p->G_state) * spans * 2 * kStreamStateFloats;
+        p->launches = 3;
+    } else {
+        p->cluster_size = largest_cluster(tiles_kv);
+        partial_floats = 0;
+        p->launches = 1;
+    }
+    p->partial_bytes = align_up(partial_floats * sizeof(float), 256);
+    p->state_off = p->partial_bytes;
+    p->status_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
+    p->total_bytes = p->status_off + 256;
+    return LINFUSION_OK;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (fn == nullptr) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 [slabs][N][64] -> boxes of [1][tile_rows][64], 128-byte swizzle, zero fill past N.
+bool encode_slab_map(CUtensorMap* map, const void* base, int slabs, int N, int tile_rows)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(kStreamD), static_cast<cuuint64_t>(N),
+                          static_cast<cuuint64_t>(slabs)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(kStreamRowBytes),
+                             static_cast<cuuint64_t>(N) * kStreamRowBytes};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(kStreamD), static_cast<cuuint32_t>(tile_rows), 1u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+                    estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+struct linfusion_attn {
+    linfusion_attn_desc_t desc;
+    Plan plan;
+    int sm_count;
+    void* ws;  // device workspace in use
+    bool owns_ws;
+    float* partials;
+    float* state;
+    uint32_t* status;
+    cudaStream_t last_stream;
+    void* stage[4];  // staging for the host-buffer entry point (allocated on first use)
+};
+
+namespace {
+
+void bind_workspace(linfusion_attn* h, void* ws)
+{
+    h->ws = ws;
+    unsigned char* base = static_cast<unsigned char*>(ws);
+    h->partials = reinterpret_cast<float*>(base);
+    h->state = reinterpret_cast<float*>(base + h->plan.state_off);
+    h->status = reinterpret_cast<uint32_t*>(base + h->plan.status_off);
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || (cudaSetDevice(dev) == cudaSuccess);
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+template <int D, int PHI>
+cudaError_t set_split_attrs()
+{
+    using C = SplitCfg<D>;
+    cudaError_t e;
+    e = cudaFuncSetAttribute(state_partial_kernel<D, PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(apply_kernel<D, PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(cluster_fused_kernel<D, PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             C::SMEM_CLUSTER);
+    return e;
+}
+
+template <int PHI>
+cudaError_t set_stream_attrs()
+{
+    cudaError_t e;
+    e = cudaFuncSetAttribute(stream_state_kernel<PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             StreamStateCfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(stream_apply_kernel<PHI, kStreamApplyWarps>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg::SMEM_BYTES);
+    return e;
+}
+
+template <int D, int PHI>
+cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                         const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
+{
+    using C = SplitCfg<D>;
+    const Plan& p = h->plan;
+    const int N = h->desc.N;
+    state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
+        k, v, h->partials, N, p.chunks_state);
+    state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
+        h->partials, h->state, C::STATE_FLOATS, p.chunks_state);
+    apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
+        q, h->state, y, N, p.chunks_apply, h->desc.eps);
+    return cudaGetLastError();
+}
+
+template <int D>
+void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cluster_size, int slabs,
+                    cudaStream_t s)
+{
+    using C = SplitCfg<D>;
+    memset(cfg, 0, sizeof(*cfg));
+    cfg->gridDim = dim3(cluster_size, slabs, 1);
+    cfg->blockDim = dim3(C::NT, 1, 1);
+    cfg->dynamicSmemBytes = C::SMEM_CLUSTER;
+    cfg->stream = s;
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cluster_size;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg->attrs = attr;
+    cfg->numAttrs = 1;
+}
+
+template <int D, int PHI>
+cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                           const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
+{
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
+    return cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state, h->desc.N,
+                              h->desc.eps);
+}
+
+template <int PHI>
+cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                          const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
+{
+    const Plan& p = h->plan;
+    const int N = h->desc.N;
+    CUtensorMap mq, mk, mv;
+    if (!encode_slab_map(&mk, k, p.slabs, N, StreamStateCfg::TILE) ||
+        !encode_slab_map(&mv, v, p.slabs, N, StreamStateCfg::TILE) ||
+        !encode_slab_map(&mq, q, p.slabs, N, ApplyCfg::TILE))
+        return cudaErrorInvalidValue;
+    stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
+        mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans);
+    stream_reduce_kernel<<<dim3((kStreamStateFloats + 255) / 256, p.slabs), 256, 0, s>>>(
+        h->partials, h->state, p.tiles_state, p.W_state, p.G_state, p.spans);
+    stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
+        mq, h->state, y, h->status, N, p.tiles_apply, p.W_apply, h->desc.eps);
+    return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t set_attrs_d(int phi)
+{
+    return phi == LINFUSION_PHI_IDENTITY ? set_split_attrs<D, kPhiIdentity>()
+                                         : set_split_attrs<D, kPhiEluPlusOne>();
+}
+
+template <int D>
+cudaError_t launch_d(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                     const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
+{
+    const bool ident = h->desc.phi == LINFUSION_PHI_IDENTITY;
+    if (h->plan.variant == kCluster)
+        return ident ? launch_cluster<D, kPhiIdentity>(h, q, k, v, y, s)
+                     : launch_cluster<D, kPhiEluPlusOne>(h, q, k, v, y, s);
+    return ident ? launch_split<D, kPhiIdentity>(h, q, k, v, y, s)
+                 : launch_split<D, kPhiEluPlusOne>(h, q, k, v, y, s);
+}
+
+#define LF_DISPATCH_D(dval, CALL)   \
+    switch (dval) {                 \
+        case 32: CALL(32); break;   \
+        case 40: CALL(40); break;   \
+        case 64: CALL(64); break;   \
+        case 80: CALL(80); break;   \
+        case 128: CALL(128); break; \
+        case 160: CALL(160); break; \
+        default: break;             \
+    }
+
+template <int D>
+bool cluster_fits(int phi, int cluster_size, int slabs)
+{
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    cluster_config<D>(&cfg, attr, cluster_size, slabs, nullptr);
+    int n = 0;
+    cudaError_t e = phi == LINFUSION_PHI_IDENTITY
+                        ? cudaOccupancyMaxActiveClusters(&n, cluster_fused_kernel<D, kPhiIdentity>, &cfg)
+                        : cudaOccupancyMaxActiveClusters(&n, cluster_fused_kernel<D, kPhiEluPlusOne>, &cfg);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return n > 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* linfusion_status_string(linfusion_status_t s)
+{
+    switch (s) {
+        case LINFUSION_OK: return "ok";
+        case LINFUSION_ERR_INVALID_ARG: return "invalid argument";
+        case LINFUSION_ERR_UNSUPPORTED: return "unsupported head dim, activation, variant or device";
+        case LINFUSION_ERR_ALLOC: return "workspace allocation failed or workspace too small";
+        case LINFUSION_ERR_CUDA: return "CUDA call failed";
+        case LINFUSION_ERR_TIMEOUT: return "a bounded device-side wait expired";
+        default: return "unknown status";
+    }
+}
+
+linfusion_status_t linfusion_attn_workspace_bytes(const linfusion_attn_desc_t* desc, int sm_count,
+                                                  size_t* bytes)
+{
+    if (bytes == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    Plan p;
+    linfusion_status_t st = make_plan(desc, sm_count, &p);
+    if (st != LINFUSION_OK) return st;
+    *bytes = p.total_bytes;
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linfusion_attn_t** out)
+{
+    if (out == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    *out = nullptr;
+    linfusion_status_t st = validate(desc);
+    if (st != LINFUSION_OK) return st;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    if (desc->device >= ndev) return LINFUSION_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, desc->device) != cudaSuccess) return LINFUSION_ERR_CUDA;
+    if (prop.major != 10) return LINFUSION_ERR_UNSUPPORTED;
+
+    DeviceGuard guard(desc->device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+
+    linfusion_attn* h = new (std::nothrow) linfusion_attn();
+    if (h == nullptr) return LINFUSION_ERR_ALLOC;
+    h->desc = *desc;
+    h->sm_count = prop.multiProcessorCount;
+    h->ws = nullptr;
+    h->owns_ws = false;
+    h->last_stream = nullptr;
+    for (int i = 0; i < 4; ++i) h->stage[i] = nullptr;
+    st = make_plan(desc, h->sm_count, &h->plan);
+    if (st != LINFUSION_OK) {
+        delete h;
+        return st;
+    }
+
+    cudaError_t e = cudaSuccess;
+#define LF_SET(DV) e = set_attrs_d<DV>(desc->phi)
+    LF_DISPATCH_D(desc->d, LF_SET)
+#undef LF_SET
+    if (e == cudaSuccess && desc->d == kStreamD)
+        e = desc->phi == LINFUSION_PHI_IDENTITY ? set_stream_attrs<kPhiIdentity>()
+                                                : set_stream_attrs<kPhiEluPlusOne>();
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        delete h;
+        return LINFUSION_ERR_CUDA;
+    }
+
+    if (h->plan.variant == kCluster) {
+        // Shrink the cluster until the device can co-schedule it; else fall back to three launches.
+        bool fits = false;
+        const bool forced = (desc->flags & LINFUSION_VARIANT_MASK) == LINFUSION_VARIANT_CLUSTER;
+        while (true) {
+#define LF_FIT(DV) fits = cluster_fits<DV>(desc->phi, h->plan.cluster_size, h->plan.slabs)
+            LF_DISPATCH_D(desc->d, LF_FIT)
+#undef LF_FIT
+            if (fits || h->plan.cluster_size == 1) break;
+            h->plan.cluster_size >>= 1;
+        }
+        if (!fits) {
+            if (forced) {
+                delete h;
+                return LINFUSION_ERR_UNSUPPORTED;
+            }
+            linfusion_attn_desc_t d2 = *desc;
+            d2.flags = (d2.flags & ~LINFUSION_VARIANT_MASK) | LINFUSION_VARIANT_SPLIT;
+            make_plan(&d2, h->sm_count, &h->plan);
+        }
+    }
+
+    void* ws = nullptr;
+    if (cudaMalloc(&ws, h->plan.total_bytes) != cudaSuccess) {
+        cudaGetLastError();
+        delete h;
+        return LINFUSION_ERR_ALLOC;
+    }
+    h->owns_ws = true;
+    bind_workspace(h, ws);
+    if (cudaMemset(h->status, 0, 256) != cudaSuccess) {
+        cudaFree(ws);
+        delete h;
+        return LINFUSION_ERR_CUDA;
+    }
+    *out = h;
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_set_workspace(linfusion_attn_t* h, void* dev_ptr, size_t bytes)
+{
+    if (h == nullptr || dev_ptr == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(dev_ptr) & 255u) != 0) return LINFUSION_ERR_INVALID_ARG;
+    if (bytes < h->plan.total_bytes) return LINFUSION_ERR_ALLOC;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    cudaStreamSynchronize(h->last_stream);
+    if (h->owns_ws && h->ws != nullptr) cudaFree(h->ws);
+    h->owns_ws = false;
+    bind_workspace(h, dev_ptr);
+    if (cudaMemset(h->status, 0, 256) != cudaSuccess) return LINFUSION_ERR_CUDA;
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, const void* k,
+                                          const void* v, void* y, void* cuda_stream)
+{
+    if (h == nullptr || q == nullptr || k == nullptr || v == nullptr || y == nullptr)
+        return LINFUSION_ERR_INVALID_ARG;
+    const uintptr_t pq = reinterpret_cast<uintptr_t>(q), pk = reinterpret_cast<uintptr_t>(k),
+                    pv = reinterpret_cast<uintptr_t>(v), py = reinterpret_cast<uintptr_t>(y);
+    if (((pq | pk | pv | py) & 15u) != 0) return LINFUSION_ERR_INVALID_ARG;
+    const size_t bytes = static_cast<size_t>(h->plan.slabs) * h->desc.N * h->desc.d * 2;
+    auto overlaps = [&](uintptr_t a) { return a < py + bytes && py < a + bytes; };
+    if (overlaps(pq) || overlaps(pk) || overlaps(pv)) return LINFUSION_ERR_INVALID_ARG;
+
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const __nv_bfloat16* Q = static_cast<const __nv_bfloat16*>(q);
+    const __nv_bfloat16* K = static_cast<const __nv_bfloat16*>(k);
+    const __nv_bfloat16* V = static_cast<const __nv_bfloat16*>(v);
+    __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
+
+    cudaError_t e = cudaErrorInvalidValue;
+    if (h->plan.variant == kStream) {
+        e = h->desc.phi == LINFUSION_PHI_IDENTITY ? launch_stream<kPhiIdentity>(h, Q, K, V, Y, s)
+                                                  : launch_stream<kPhiEluPlusOne>(h, Q, K, V, Y, s);
+    } else {
+#define LF_LAUNCH(DV) e = launch_d<DV>(h, Q, K, V, Y, s)
+        LF_DISPATCH_D(h->desc.d, LF_LAUNCH)
+#undef LF_LAUNCH
+    }
+    h->last_stream = s;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* q_host,
+                                               const void* k_host, const void* v_host, void* y_host,
+                                               void* cuda_stream)
+{
+    if (h == nullptr || q_host == nullptr || k_host == nullptr || v_host == nullptr || y_host == nullptr)
+        return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    const size_t bytes = static_cast<size_t>(h->plan.slabs) * h->desc.N * h->desc.d * 2;
+    if (h->stage[0] == nullptr) {
+        for (int i = 0; i < 4; ++i) {
+            if (cudaMalloc(&h->stage[i], bytes) != cudaSuccess) {
+                cudaGetLastError();
+                for (int j = 0; j < i; ++j) cudaFree(h->stage[j]);
+                for (int j = 0; j < 4; ++j) h->stage[j] = nullptr;
+                return LINFUSION_ERR_ALLOC;
+            }
+        }
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    // K and V first: they feed the first kernel.
+    if (cudaMemcpyAsync(h->stage[1], k_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(h->stage[2], v_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(h->stage[0], q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    linfusion_status_t st = linfusion_attn_forward(h, h->stage[0], h->stage[1], h->stage[2], h->stage[3], s);
+    if (st != LINFUSION_OK) return st;
+    if (cudaMemcpyAsync(y_host, h->stage[3], bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_status(linfusion_attn_t* h)
+{
+    if (h == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    uint32_t word = 0;
+    if (cudaMemcpy(&word, h->status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return word == kStatusOk ? LINFUSION_OK : LINFUSION_ERR_TIMEOUT;
+}
+
+linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host, float* z_host)
+{
+    if (h == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    const int d = h->desc.d, sf = h->plan.state_floats;
+    for (int s = 0; s < h->plan.slabs; ++s) {
+        const float* src = h->state + static_cast<size_t>(s) * sf;
+        if (S_host != nullptr &&
+            cudaMemcpy(S_host + static_cast<size_t>(s) * d * d, src, sizeof(float) * d * d,
+                       cudaMemcpyDeviceToHost) != cudaSuccess)
+            return LINFUSION_ERR_CUDA;
+        if (z_host != nullptr &&
+            cudaMemcpy(z_host + static_cast<size_t>(s) * d, src + d * d, sizeof(float) * d,
+                       cudaMemcpyDeviceToHost) != cudaSuccess)
+            return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
+
+const char* linfusion_attn_variant_name(const linfusion_attn_t* h)
+{
+    if (h == nullptr) return "";
+    switch (h->plan.variant) {
+        case kSplit: return "split";
+        case kStream: return "stream";
+        case kCluster: return "cluster";
+        default: return "";
+    }
+}
+
+int32_t linfusion_attn_launches_per_forward(const linfusion_attn_t* h)
+{
+    return h == nullptr ? 0 : h->plan.launches;
+}
+
+linfusion_status_t linfusion_attn_destroy(linfusion_attn_t* h)
+{
+    if (h == nullptr) return LINFUSION_OK;
+    DeviceGuard guard(h->desc.device);
+    linfusion_status_t st = LINFUSION_OK;
+    if (guard.ok) {
+        if (h->owns_ws && h->ws != nullptr && cudaFree(h->ws) != cudaSuccess) st = LINFUSION_ERR_CUDA;
+        for (int i = 0; i < 4; ++i)
+            if (h->stage[i] != nullptr && cudaFree(h->stage[i]) != cudaSuccess) st = LINFUSION_ERR_CUDA;
+    } else {
+        st = LINFUSION_ERR_CUDA;
+    }
+    delete h;
+    return st;
+}
+
+}  // extern "C"

@@ -1,0 +1,375 @@
+// Kernels for any supported head dim D (multiple of 8, up to 160), built on warp-level
+// tensor-core MMAs with operands staged in shared memory by plain 16-byte loads:
+//
+//   state_partial_kernel  — split-N partial state  S_p = sum_{j in chunk} phi(K_j)^T V_j,
+//                           z_p = sum phi(K_j)                        (Prop. 2, Eq. 5)
+//   state_reduce_kernel   — fixed-order sum of the partials into S | z
+//   apply_kernel          — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps)
+//   cluster_fused_kernel  — all three in one launch: one thread-block cluster per slab, the
+//                           partial states summed in rank order through distributed shared memory
+//
+// MMA roles.  State: D[c][e] += A[c][j] B[j][e] with A = phi(K)^T and B = V, the contraction
+// running over tokens j; one warp owns one 16-row block of c and every column block of e,
+// plus one extra column block fed with ones, which yields z.  Apply: D[i][e] += A[i][c] B[c][e]
+// with A = phi(Q) and B = S (held transposed, as bf16), one warp per 16 tokens, plus one
+// extra column block holding z in every column, which yields the denominator.
+#pragma once
+
+#include <cooperative_groups.h>
+
+#include "common.cuh"
+
+namespace lf {
+
+namespace cg = cooperative_groups;
+
+template <int D>
+struct SplitCfg {
+    static_assert(D % 8 == 0 && D >= 8 && D <= 160, "head dim must be a multiple of 8 in [8, 160]");
+    static constexpr int DP = (D + 15) / 16 * 16;  // channels padded to the MMA's 16
+    static constexpr int MB = DP / 16;             // 16-row blocks of the state = warps per CTA
+    static constexpr int NBV = D / 8;              // 8-column blocks over V channels
+    static constexpr int NBT = NBV + 1;            // + the ones / z block
+    static constexpr int CH = DP / 8;              // 16-byte chunks per padded row
+    static constexpr int PITCH = ((DP / 8) | 1) * 16;  // smem row pitch, odd in 16-byte units
+    static constexpr int NT = 32 * MB;             // threads per CTA
+    static constexpr int TILE_KV = 64;             // tokens per K/V tile
+    static constexpr int TILE_Q = 16 * MB;         // tokens per Q tile (one m16 block per warp)
+    static constexpr int LD_KV = TILE_KV * CH / NT;  // 16-byte chunks per thread per tile
+    static constexpr int LD_Q = TILE_Q * CH / NT;
+    static_assert(TILE_KV * CH % NT == 0 && TILE_Q * CH % NT == 0, "tile must split evenly");
+    static constexpr int ST_ROWS = (D + 8 + 15) / 16 * 16;  // S^T rows: D channels, 8 z rows, pad
+    static constexpr int STATE_FLOATS = D * (D + 1);        // S [D][D] then z [D]
+
+    static constexpr int SMEM_KV = 2 * TILE_KV * PITCH;  // phi(K) tile + V tile
+    static constexpr int SMEM_Q = TILE_Q * PITCH;
+    static constexpr int SMEM_ST = ST_ROWS * PITCH;
+    static constexpr int SMEM_APPLY = SMEM_ST + SMEM_Q;
+    static constexpr int SMEM_STAGE = (SMEM_KV > SMEM_Q ? SMEM_KV : SMEM_Q);
+    static constexpr int SMEM_CLUSTER = STATE_FLOATS * 4 + SMEM_ST + SMEM_STAGE;
+};
+
+// First tile of chunk `p` when `tiles` tiles are cut into `chunks` nearly equal runs.
+__host__ __device__ __forceinline__ int chunk_begin(int p, int tiles, int chunks)
+{
+    return static_cast<int>((static_cast<long long>(p) * tiles) / chunks);
+}
+
+// ---------------------------------------------------------------------------------------------
+// State accumulation over K/V tiles [tile0, tile1) of one slab.  acc[nb][.] holds this warp's
+// 16 x 8 block (rows c = 16*warp + ..., columns 8*nb + ...), acc[NBV] the z block.
+// ---------------------------------------------------------------------------------------------
+template <int D, int PHI>
+__device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict__ Ks,
+                                                 const __nv_bfloat16* __restrict__ Vs, int N,
+                                                 int tile0, int tile1, unsigned char* smem_kv,
+                                                 float (&acc)[SplitCfg<D>::NBT][4])
+{
+    using C = SplitCfg<D>;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    unsigned char* Ksm = smem_kv;
+    unsigned char* Vsm = smem_kv + C::TILE_KV * C::PITCH;
+
+#pragma unroll
+    for (int nb = 0; nb < C::NBT; ++nb)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) acc[nb][i] = 0.0f;
+
+    uint4 kreg[C::LD_KV], vreg[C::LD_KV];
+    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+
+    auto load_tile = [&](int tile) {
+#pragma unroll
+        for (int i = 0; i < C::LD_KV; ++i) {
+            int idx = tid + i * C::NT;
+            int row = idx / C::CH, ch = idx % C::CH;
+            long long j = static_cast<long long>(tile) * C::TILE_KV + row;
+            bool ok = (j < N) && (ch * 8 < D);
+            kreg[i] = ok ? ld_stream_16B(Ks + j * D + ch * 8) : zero4;
+            vreg[i] = ok ? ld_stream_16B(Vs + j * D + ch * 8) : zero4;
+        }
+    };
+    auto store_tile = [&](int tile) {
+#pragma unroll
+        for (int i = 0; i < C::LD_KV; ++i) {
+            int idx = tid + i * C::NT;
+            int row = idx / C::CH, ch = idx % C::CH;
+            long long j = static_cast<long long>(tile) * C::TILE_KV + row;
+            bool ok = (j < N) && (ch * 8 < D);
+            uint4 pk = zero4;  // rows past N and pad channels contribute nothing (not phi(0) = 1)
+            if (ok) {
+                pk.x = phi_bf16x2<PHI>(kreg[i].x);
+                pk.y = phi_bf16x2<PHI>(kreg[i].y);
+                pk.z = phi_bf16x2<PHI>(kreg[i].z);
+                pk.w = phi_bf16x2<PHI>(kreg[i].w);
+            }
+            *reinterpret_cast<uint4*>(Ksm + row * C::PITCH + ch * 16) = pk;
+            *reinterpret_cast<uint4*>(Vsm + row * C::PITCH + ch * 16) = vreg[i];
+        }
+    };
+
+    const uint32_t ksm_base = smem_u32(Ksm), vsm_base = smem_u32(Vsm);
+    // ldmatrix.trans lane addressing.  A (16 c x 16 j) from the phi(K) tile stored [j][c]:
+    // matrices (j0, c0), (j0, c0+8), (j0+8, c0), (j0+8, c0+8).  B (16 j x 16 e) from the V tile
+    // stored [j][e]: matrices (j0, e0), (j0+8, e0), (j0, e0+8), (j0+8, e0+8).
+    const uint32_t a_off = ((lane & 7) + ((lane >> 4) << 3)) * C::PITCH +
+                           (warp * 16 + ((lane >> 3) & 1) * 8) * 2;
+    const uint32_t b_off = ((lane & 7) + (((lane >> 3) & 1) << 3)) * C::PITCH + ((lane >> 4) * 8) * 2;
+    const uint32_t ones = 0x3F803F80u;  // bf16 (1, 1)
+
+    if (tile0 < tile1) load_tile(tile0);
+    for (int tile = tile0; tile < tile1; ++tile) {
+        store_tile(tile);
+        __syncthreads();
+        if (tile + 1 < tile1) load_tile(tile + 1);
+#pragma unroll
+        for (int ks = 0; ks < C::TILE_KV / 16; ++ks) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4_trans(ksm_base + ks * 16 * C::PITCH + a_off, a0, a1, a2, a3);
+#pragma unroll
+            for (int nbp = 0; nbp < (C::NBV + 1) / 2; ++nbp) {
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4_trans(vsm_base + ks * 16 * C::PITCH + b_off + nbp * 32, b0, b1, b2, b3);
+                mma_bf16_16816(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
+                if (2 * nbp + 1 < C::NBV) mma_bf16_16816(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
+            }
+            mma_bf16_16816(acc[C::NBV], a0, a1, a2, a3, ones, ones);
+        }
+        __syncthreads();
+    }
+}
+
+// Write this warp's rows of the state as fp32: S [D][D] then z [D] at `dst` (global or shared).
+template <int D>
+__device__ __forceinline__ void store_state(float* dst, const float (&acc)[SplitCfg<D>::NBT][4])
+{
+    using C = SplitCfg<D>;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int c0 = warp * 16 + g, c1 = c0 + 8;
+#pragma unroll
+    for (int nb = 0; nb < C::NBV; ++nb) {
+        int e = nb * 8 + 2 * t;
+        if (c0 < D) *reinterpret_cast<float2*>(dst + c0 * D + e) = make_float2(acc[nb][0], acc[nb][1]);
+        if (c1 < D) *reinterpret_cast<float2*>(dst + c1 * D + e) = make_float2(acc[nb][2], acc[nb][3]);
+    }
+    if (t == 0) {
+        if (c0 < D) dst[D * D + c0] = acc[C::NBV][0];
+        if (c1 < D) dst[D * D + c1] = acc[C::NBV][2];
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Apply over Q tiles [tile0, tile1) of one slab, with S^T | z resident in shared memory as bf16.
+// ---------------------------------------------------------------------------------------------
+template <int D, int PHI>
+__device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs,
+                                            __nv_bfloat16* __restrict__ Ys, int N, int tile0,
+                                            int tile1, const unsigned char* St, unsigned char* Qsm,
+                                            float eps)
+{
+    using C = SplitCfg<D>;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
+    uint4 qreg[C::LD_Q];
+
+    auto load_tile = [&](int tile) {
+#pragma unroll
+        for (int i = 0; i < C::LD_Q; ++i) {
+            int idx = tid + i * C::NT;
+            int row = idx / C::CH, ch = idx % C::CH;
+            long long r = static_cast<long long>(tile) * C::TILE_Q + row;
+            bool ok = (r < N) && (ch * 8 < D);
+            qreg[i] = ok ? ld_stream_16B(Qs + r * D + ch * 8) : zero4;
+        }
+    };
+    auto store_tile = [&](int tile) {
+#pragma unroll
+        for (int i = 0; i < C::LD_Q; ++i) {
+            int idx = tid + i * C::NT;
+            int row = idx / C::CH, ch = idx % C::CH;
+            long long r = static_cast<long long>(tile) * C::TILE_Q + row;
+            bool ok = (r < N) && (ch * 8 < D);
+            uint4 pq = zero4;
+            if (ok) {
+                pq.x = phi_bf16x2<PHI>(qreg[i].x);
+                pq.y = phi_bf16x2<PHI>(qreg[i].y);
+                pq.z = phi_bf16x2<PHI>(qreg[i].z);
+                pq.w = phi_bf16x2<PHI>(qreg[i].w);
+            }
+            *reinterpret_cast<uint4*>(Qsm + row * C::PITCH + ch * 16) = pq;
+        }
+    };
+
+    // Non-transposed ldmatrix.  A (16 i x 16 c) from the phi(Q) tile stored [i][c]: matrices
+    // (i0, c0), (i0+8, c0), (i0, c0+8), (i0+8, c0+8).  B (16 c x 16 e) from S^T stored [e][c]:
+    // matrices (e0, c0), (e0, c0+8), (e0+8, c0), (e0+8, c0+8).
+    const uint32_t q_base = smem_u32(Qsm) + (warp * 16 + (lane & 7) + (((lane >> 3) & 1) << 3)) * C::PITCH +
+                            ((lane >> 4) * 8) * 2;
+    const uint32_t s_base = smem_u32(St) + ((lane & 7) + ((lane >> 4) << 3)) * C::PITCH +
+                            (((lane >> 3) & 1) * 8) * 2;
+
+    if (tile0 < tile1) load_tile(tile0);
+    for (int tile = tile0; tile < tile1; ++tile) {
+        store_tile(tile);
+        __syncthreads();
+        if (tile + 1 < tile1) load_tile(tile + 1);
+
+        float acc[C::NBT][4];
+#pragma unroll
+        for (int nb = 0; nb < C::NBT; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[nb][i] = 0.0f;
+#pragma unroll
+        for (int kb = 0; kb < C::MB; ++kb) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(q_base + kb * 32, a0, a1, a2, a3);
+#pragma unroll
+            for (int nbp = 0; nbp < (C::NBT + 1) / 2; ++nbp) {
+                uint32_t b0, b1, b2, b3;
+                ldmatrix_x4(s_base + nbp * 16 * C::PITCH + kb * 32, b0, b1, b2, b3);
+                mma_bf16_16816(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
+                if (2 * nbp + 1 < C::NBT) mma_bf16_16816(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
+            }
+        }
+        // Every column of the z block holds phi(Q_i) . z for its row.
+        const float inv0 = 1.0f / (acc[C::NBV][0] + eps);
+        const float inv1 = 1.0f / (acc[C::NBV][2] + eps);
+        const long long r0 = static_cast<long long>(tile) * C::TILE_Q + warp * 16 + g, r1 = r0 + 8;
+#pragma unroll
+        for (int nb = 0; nb < C::NBV; ++nb) {
+            int e = nb * 8 + 2 * t;
+            if (r0 < N) st_stream_4B(Ys + r0 * D + e, pack_bf16x2(acc[nb][0] * inv0, acc[nb][1] * inv0));
+            if (r1 < N) st_stream_4B(Ys + r1 * D + e, pack_bf16x2(acc[nb][2] * inv1, acc[nb][3] * inv1));
+        }
+        __syncthreads();
+    }
+}
+
+// Fill the shared S^T | z operand (bf16, rows = output channel e, then 8 rows of z, then zero
+// rows; columns = feature c padded with zeros) from fp32 S [D][D], z [D].  `read(idx)` returns
+// element idx of that fp32 state.
+template <int D, typename ReadFn>
+__device__ __forceinline__ void fill_state_operand(unsigned char* St, ReadFn read)
+{
+    using C = SplitCfg<D>;
+    for (int idx = threadIdx.x; idx < C::DP * C::ST_ROWS; idx += blockDim.x) {
+        int c = idx / C::ST_ROWS, e = idx % C::ST_ROWS;
+        float val = 0.0f;
+        if (c < D) {
+            if (e < D) val = read(c * D + e);
+            else if (e < D + 8) val = read(D * D + c);
+        }
+        *reinterpret_cast<__nv_bfloat16*>(St + e * C::PITCH + c * 2) = __float2bfloat16_rn(val);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Kernels
+// ---------------------------------------------------------------------------------------------
+
+// grid (chunks, slabs).  partials: [slab][chunk][D*(D+1)] fp32.
+template <int D, int PHI>
+__global__ void __launch_bounds__(SplitCfg<D>::NT)
+state_partial_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
+                     float* __restrict__ partials, int N, int chunks)
+{
+    using C = SplitCfg<D>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    const int slab = blockIdx.y, p = blockIdx.x;
+    const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;
+    const size_t slab_off = static_cast<size_t>(slab) * N * D;
+    float acc[C::NBT][4];
+    accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, chunk_begin(p, tiles, chunks),
+                             chunk_begin(p + 1, tiles, chunks), smem, acc);
+    store_state<D>(partials + (static_cast<size_t>(slab) * chunks + p) * C::STATE_FLOATS, acc);
+}
+
+// grid (ceil(state_floats / 256), slabs).  Sums `chunks` partials per slab in index order.
+__global__ void __launch_bounds__(256)
+state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state, int state_floats,
+                    int chunks)
+{
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= state_floats) return;
+    const int slab = blockIdx.y;
+    const float* src = partials + static_cast<size_t>(slab) * chunks * state_floats + idx;
+    float sum = 0.0f;
+    for (int p = 0; p < chunks; ++p) sum += src[static_cast<size_t>(p) * state_floats];
+    state[static_cast<size_t>(slab) * state_floats + idx] = sum;
+}
+
+// grid (chunks, slabs).
+template <int D, int PHI>
+__global__ void __launch_bounds__(SplitCfg<D>::NT)
+apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ state,
+             __nv_bfloat16* __restrict__ Y, int N, int chunks, float eps)
+{
+    using C = SplitCfg<D>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* St = smem;
+    unsigned char* Qsm = smem + C::SMEM_ST;
+    const int slab = blockIdx.y, p = blockIdx.x;
+    const int tiles = (N + C::TILE_Q - 1) / C::TILE_Q;
+    const float* st = state + static_cast<size_t>(slab) * C::STATE_FLOATS;
+    fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); });
+    __syncthreads();
+    const size_t slab_off = static_cast<size_t>(slab) * N * D;
+    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, chunk_begin(p, tiles, chunks),
+                        chunk_begin(p + 1, tiles, chunks), St, Qsm, eps);
+}
+
+// One cluster of `cluster_size` CTAs per slab (grid.x = cluster_size, grid.y = slabs).  CTA r
+// accumulates the partial state of its run of K/V tiles into its own shared memory; after a
+// cluster barrier every CTA sums the partials of ranks 0, 1, ... in that order through
+// distributed shared memory (so all CTAs hold the same bits), then applies to its run of Q.
+// state_out (may be null) receives S | z from rank 0.
+template <int D, int PHI>
+__global__ void __launch_bounds__(SplitCfg<D>::NT)
+cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
+                     const __nv_bfloat16* __restrict__ V, __nv_bfloat16* __restrict__ Y,
+                     float* __restrict__ state_out, int N, float eps)
+{
+    using C = SplitCfg<D>;
+    extern __shared__ __align__(128) unsigned char smem[];
+    float* part = reinterpret_cast<float*>(smem);
+    unsigned char* St = smem + C::STATE_FLOATS * 4;
+    unsigned char* stage = St + C::SMEM_ST;
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int rank = static_cast<int>(cluster.block_rank());
+    const int csize = static_cast<int>(cluster.num_blocks());
+    const int slab = blockIdx.y;
+    const size_t slab_off = static_cast<size_t>(slab) * N * D;
+
+    {
+        const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;
+        float acc[C::NBT][4];
+        accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, chunk_begin(rank, tiles, csize),
+                                 chunk_begin(rank + 1, tiles, csize), stage, acc);
+        store_state<D>(part, acc);
+    }
+    cluster.sync();
+
+    fill_state_operand<D>(St, [&](int i) {
+        float sum = 0.0f;
+        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(part, r)[i];
+        return sum;
+    });
+    if (rank == 0 && state_out != nullptr) {
+        float* dst = state_out + static_cast<size_t>(slab) * C::STATE_FLOATS;
+        for (int i = threadIdx.x; i < C::STATE_FLOATS; i += blockDim.x) {
+            float sum = 0.0f;
+            for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(part, r)[i];
+            dst[i] = sum;
+        }
+    }
+    cluster.sync();  // no CTA leaves (or reuses `part`) while a peer still reads it
+
+    const int qtiles = (N + C::TILE_Q - 1) / C::TILE_Q;
+    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, chunk_begin(rank, qtiles, csize),
+                        chunk_begin(rank + 1, qtiles, csize), St, stage, eps);
+}
+
+}  // namespace lf
