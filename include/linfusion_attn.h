@@ -138,6 +138,18 @@ linfusion_status_t linfusion_attn_status(linfusion_attn_t* h);
  */
 linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host, float* z_host);
 
+/*
+ * Per-kernel timing for benchmarks.  enable(h, slots > 0) creates `slots` sets of CUDA events;
+ * from then on every forward() brackets each of its kernels with event records on its stream
+ * (set = call index modulo slots).  enable(h, 0) turns it off.  kernel_times() synchronizes the
+ * handle's last stream and returns, for the calls recorded since the last kernel_times()
+ * (at most `slots`), the summed milliseconds of each kernel in launch order — ms_sum[0] the
+ * state kernel (or the single clustered kernel), ms_sum[1] the reduction, ms_sum[2] the apply —
+ * and the number of calls summed.  Errors: INVALID_ARG, ALLOC, CUDA.
+ */
+linfusion_status_t linfusion_attn_enable_kernel_timing(linfusion_attn_t* h, int32_t slots);
+linfusion_status_t linfusion_attn_kernel_times(linfusion_attn_t* h, float* ms_sum, int32_t* calls);
+
 /* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);
 

@@ -24,6 +24,7 @@ EXPORTED = [
     "linfusion_attn_destroy", "linfusion_status_string", "linfusion_attn_workspace_bytes",
     "linfusion_attn_set_workspace", "linfusion_attn_status", "linfusion_attn_read_state",
     "linfusion_attn_variant_name", "linfusion_attn_launches_per_forward",
+    "linfusion_attn_enable_kernel_timing", "linfusion_attn_kernel_times",
 ]
 
 
@@ -77,6 +78,11 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_variant_name.argtypes = [vp]
     lib.linfusion_attn_launches_per_forward.restype = ctypes.c_int32
     lib.linfusion_attn_launches_per_forward.argtypes = [vp]
+    lib.linfusion_attn_enable_kernel_timing.restype = st
+    lib.linfusion_attn_enable_kernel_timing.argtypes = [vp, ctypes.c_int32]
+    lib.linfusion_attn_kernel_times.restype = st
+    lib.linfusion_attn_kernel_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
+                                                ctypes.POINTER(ctypes.c_int32)]
     _lib = lib
     return lib
 
@@ -194,6 +200,20 @@ class LinFusionAttention:
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_read_state")
         return S, z
+
+    def enable_kernel_timing(self, slots: int) -> None:
+        rc = self._lib.linfusion_attn_enable_kernel_timing(self._h, int(slots))
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_enable_kernel_timing")
+
+    def kernel_times(self):
+        """([ms_state, ms_reduce, ms_apply] summed, calls) since the last call of this method."""
+        ms = (ctypes.c_float * 3)()
+        calls = ctypes.c_int32(0)
+        rc = self._lib.linfusion_attn_kernel_times(self._h, ms, ctypes.byref(calls))
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_kernel_times")
+        return [float(x) for x in ms], int(calls.value)
 
     def set_workspace(self, tensor) -> None:
         rc = self._lib.linfusion_attn_set_workspace(self._h, tensor.data_ptr(),

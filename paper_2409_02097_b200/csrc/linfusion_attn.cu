@@ -186,6 +186,10 @@ struct linfusion_attn {
     uint32_t* status;
     cudaStream_t last_stream;
     void* stage[4];  // staging for the host-buffer entry point (allocated on first use)
+    // Optional per-kernel timing: `timing_slots` sets of 4 events, used round-robin by forward().
+    cudaEvent_t* events;
+    int timing_slots;
+    long long timed_calls;
 };
 
 namespace {
@@ -212,6 +216,13 @@ struct DeviceGuard {
         if (ok && prev >= 0) cudaSetDevice(prev);
     }
 };
+
+// Record timing event `i` (0..3) of the current forward, when kernel timing is enabled.
+inline void mark(const linfusion_attn* h, int i, cudaStream_t s)
+{
+    if (h->events != nullptr)
+        cudaEventRecord(h->events[(h->timed_calls % h->timing_slots) * 4 + i], s);
+}
 
 template <int D, int PHI>
 cudaError_t set_split_attrs()
@@ -246,12 +257,16 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
     using C = SplitCfg<D>;
     const Plan& p = h->plan;
     const int N = h->desc.N;
+    mark(h, 0, s);
     state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
         k, v, h->partials, N, p.chunks_state);
+    mark(h, 1, s);
     state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
         h->partials, h->state, C::STATE_FLOATS, p.chunks_state);
+    mark(h, 2, s);
     apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
         q, h->state, y, N, p.chunks_apply, h->desc.eps);
+    mark(h, 3, s);
     return cudaGetLastError();
 }
 
@@ -280,8 +295,11 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
-    return cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state, h->desc.N,
-                              h->desc.eps);
+    mark(h, 0, s);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state,
+                                       h->desc.N, h->desc.eps);
+    mark(h, 1, s);
+    return e;
 }
 
 template <int PHI>
@@ -295,12 +313,16 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
         !encode_slab_map(&mv, v, p.slabs, N, StreamStateCfg::TILE) ||
         !encode_slab_map(&mq, q, p.slabs, N, ApplyCfg::TILE))
         return cudaErrorInvalidValue;
+    mark(h, 0, s);
     stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
         mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans);
+    mark(h, 1, s);
     stream_reduce_kernel<<<dim3((kStreamStateFloats + 255) / 256, p.slabs), 256, 0, s>>>(
         h->partials, h->state, p.tiles_state, p.W_state, p.G_state, p.spans);
+    mark(h, 2, s);
     stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
         mq, h->state, y, h->status, N, p.tiles_apply, p.W_apply, h->desc.eps);
+    mark(h, 3, s);
     return cudaGetLastError();
 }
 
@@ -407,6 +429,9 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     h->owns_ws = false;
     h->last_stream = nullptr;
     for (int i = 0; i < 4; ++i) h->stage[i] = nullptr;
+    h->events = nullptr;
+    h->timing_slots = 0;
+    h->timed_calls = 0;
     st = make_plan(desc, h->sm_count, &h->plan);
     if (st != LINFUSION_OK) {
         delete h;
@@ -510,10 +535,69 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
 #undef LF_LAUNCH
     }
     h->last_stream = s;
+    if (h->events != nullptr) ++h->timed_calls;
     if (e != cudaSuccess) {
         cudaGetLastError();
         return LINFUSION_ERR_CUDA;
     }
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_enable_kernel_timing(linfusion_attn_t* h, int32_t slots)
+{
+    if (h == nullptr || slots < 0 || slots > 4096) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    if (h->events != nullptr) {
+        cudaStreamSynchronize(h->last_stream);
+        for (int i = 0; i < h->timing_slots * 4; ++i) cudaEventDestroy(h->events[i]);
+        delete[] h->events;
+        h->events = nullptr;
+    }
+    h->timing_slots = 0;
+    h->timed_calls = 0;
+    if (slots == 0) return LINFUSION_OK;
+    cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[slots * 4];
+    if (ev == nullptr) return LINFUSION_ERR_ALLOC;
+    for (int i = 0; i < slots * 4; ++i) {
+        if (cudaEventCreate(&ev[i]) != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(ev[j]);
+            delete[] ev;
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+    }
+    h->events = ev;
+    h->timing_slots = slots;
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_kernel_times(linfusion_attn_t* h, float* ms_sum, int32_t* calls)
+{
+    if (h == nullptr || ms_sum == nullptr || calls == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    ms_sum[0] = ms_sum[1] = ms_sum[2] = 0.0f;
+    *calls = 0;
+    if (h->events == nullptr) return LINFUSION_OK;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    const int n = static_cast<int>(h->timed_calls < h->timing_slots ? h->timed_calls : h->timing_slots);
+    const int kernels = h->plan.launches;
+    for (int c = 0; c < n; ++c) {
+        for (int k = 0; k < kernels; ++k) {
+            float ms = 0.0f;
+            if (cudaEventElapsedTime(&ms, h->events[c * 4 + k], h->events[c * 4 + k + 1]) != cudaSuccess) {
+                cudaGetLastError();
+                return LINFUSION_ERR_CUDA;
+            }
+            ms_sum[k] += ms;
+        }
+    }
+    *calls = n;
+    h->timed_calls = 0;
     return LINFUSION_OK;
 }
 
@@ -619,6 +703,10 @@ linfusion_status_t linfusion_attn_destroy(linfusion_attn_t* h)
         if (h->owns_ws && h->ws != nullptr && cudaFree(h->ws) != cudaSuccess) st = LINFUSION_ERR_CUDA;
         for (int i = 0; i < 4; ++i)
             if (h->stage[i] != nullptr && cudaFree(h->stage[i]) != cudaSuccess) st = LINFUSION_ERR_CUDA;
+        if (h->events != nullptr) {
+            for (int i = 0; i < h->timing_slots * 4; ++i) cudaEventDestroy(h->events[i]);
+            delete[] h->events;
+        }
     } else {
         st = LINFUSION_ERR_CUDA;
     }

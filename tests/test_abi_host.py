@@ -1,0 +1,127 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every declared
+symbol, and rejects bad descriptors before touching CUDA."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2409_02097_b200 import attn, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build_library()
+    return attn.load_library()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "linfusion_attn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(linfusion_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = _declared_symbols()
+    assert "linfusion_attn_create" in names and "linfusion_attn_forward" in names
+    assert "linfusion_attn_destroy" in names
+    for name in names:
+        assert hasattr(lib, name), f"{name} declared in the header but not exported"
+    assert set(attn.EXPORTED) <= set(names)
+
+
+def test_status_strings(lib):
+    seen = set()
+    for code in range(6):
+        s = attn.status_string(code)
+        assert s and s not in seen
+        seen.add(s)
+    assert attn.status_string(0) == "ok"
+    assert "unknown" in attn.status_string(99)
+
+
+def _ws(desc, sm=148):
+    return attn.linfusion_attn_workspace_bytes(desc, sm)
+
+
+def test_workspace_bytes_is_pure_host_and_monotone():
+    small = _ws(attn.make_desc(2, 8, 4096, 40, variant="split"))
+    assert small > 2 * 8 * 40 * 41 * 4
+    # split: partials scale with the chunk count, never with N beyond the tile count
+    a = _ws(attn.make_desc(2, 10, 524288, 64, variant="split"))
+    b = _ws(attn.make_desc(2, 10, 2 * 524288, 64, variant="split"))
+    assert a == b
+    # stream: G * spans * 2 partials + state + status word
+    s = _ws(attn.make_desc(2, 10, 524288, 64, variant="stream"))
+    assert s == 296 * 2 * 2 * 4160 * 4 + 20 * 4160 * 4 + 256
+    # cluster: no partials in global memory
+    c = _ws(attn.make_desc(2, 8, 256, 160, variant="cluster"))
+    assert c == (16 * 160 * 161 * 4 + 255) // 256 * 256 + 256
+    # the plan depends on the SM count it is given
+    assert _ws(attn.make_desc(2, 10, 524288, 64, variant="stream"), 74) < s
+
+
+@pytest.mark.parametrize("kw", [
+    dict(B=0), dict(H=0), dict(N=0), dict(N=-5), dict(eps=-1.0), dict(eps=float("nan")),
+    dict(eps=float("inf")), dict(device=-1),
+])
+def test_invalid_descriptors(kw):
+    args = dict(B=2, H=8, N=4096, d=40, eps=1e-6, device=0)
+    args.update(kw)
+    desc = attn.make_desc(**args)
+    with pytest.raises(attn.LinFusionError) as e:
+        _ws(desc)
+    assert e.value.code == attn.ERR_INVALID_ARG
+    with pytest.raises(attn.LinFusionError) as e:
+        attn.linfusion_attn_create(desc)
+    assert e.value.code == attn.ERR_INVALID_ARG
+
+
+@pytest.mark.parametrize("kw", [
+    dict(d=48), dict(d=7), dict(d=256), dict(phi=7), dict(variant=9), dict(variant=0x10),
+    dict(d=40, variant="stream"),
+])
+def test_unsupported_descriptors(kw):
+    args = dict(B=2, H=8, N=4096, d=64, eps=1e-6, device=0)
+    args.update(kw)
+    desc = attn.make_desc(**args)
+    with pytest.raises(attn.LinFusionError) as e:
+        _ws(desc)
+    assert e.value.code == attn.ERR_UNSUPPORTED
+    with pytest.raises(attn.LinFusionError) as e:
+        attn.linfusion_attn_create(desc)
+    assert e.value.code == attn.ERR_UNSUPPORTED
+
+
+def test_null_arguments(lib):
+    assert lib.linfusion_attn_create(None, None) == attn.ERR_INVALID_ARG
+    out = ctypes.c_void_p()
+    assert lib.linfusion_attn_create(None, ctypes.byref(out)) == attn.ERR_INVALID_ARG
+    assert not out.value
+    assert lib.linfusion_attn_forward(None, 16, 16, 16, 16, None) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_forward_host(None, 16, 16, 16, 16, None) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_destroy(None) == attn.OK
+    assert lib.linfusion_attn_status(None) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_read_state(None, None, None) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_set_workspace(None, None, 0) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_workspace_bytes(None, 0, None) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_launches_per_forward(None) == 0
+    assert lib.linfusion_attn_variant_name(None) == b""
+
+
+def test_create_without_a_device_fails_cleanly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a CUDA device is present")
+    with pytest.raises(attn.LinFusionError) as e:
+        attn.linfusion_attn_create(attn.make_desc(2, 8, 4096, 40))
+    assert e.value.code in (attn.ERR_CUDA, attn.ERR_INVALID_ARG)
+
+
+def test_binding_has_no_fallback(monkeypatch):
+    monkeypatch.setattr(attn, "_lib", None)
+    monkeypatch.setattr(attn, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
+    with pytest.raises(ImportError):
+        attn.load_library()

@@ -1,0 +1,219 @@
+"""GPU parity: the CUDA library (through its C ABI) against the fp64 CPU oracle on the same
+seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2409_02097_b200 import attn, workloads as wl
+
+from _util import EPS, assert_parity, error_metrics, oracle_y, to_f64
+
+pytestmark = pytest.mark.gpu
+
+SMALL_SHAPES = [s for cfg in wl.CONFIGS[:4] for s in cfg]
+SMALL_SHAPES = list({s.name: s for s in SMALL_SHAPES}.values())
+BIG_SHAPES = wl.CONFIGS[4]
+
+
+def run_gpu(q, k, v, variant="auto", eps=EPS, phi=attn.PHI_ELU_PLUS_ONE):
+    B, H, N, d = q.shape
+    op = attn.LinFusionAttention(B, H, N, d, phi=phi, eps=eps, device=q.device.index or 0,
+                                 variant=variant)
+    y = op.forward(q, k, v)
+    torch.cuda.synchronize()
+    assert op.status() == attn.OK
+    return y, op
+
+
+def variants_for(shape):
+    out = ["auto", "split"]
+    if shape.d == 64:
+        out.append("stream")
+    if shape.N <= 16384:
+        out.append("cluster")
+    return out
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES, ids=lambda s: s.name)
+def test_workload_shapes_all_variants(shape):
+    q, k, v = wl.make_qkv(shape, seed=wl.BASE_SEED, device="cuda")
+    ref = oracle_y(q, k, v)
+    for variant in variants_for(shape):
+        y, op = run_gpu(q, k, v, variant)
+        assert_parity(y, ref, f"{shape.name}/{variant}->{op.variant}")
+        op.close()
+
+
+@pytest.mark.parametrize("shape", SMALL_SHAPES, ids=lambda s: s.name)
+def test_workload_shapes_shifted_v(shape):
+    """V ~ N(1, 1): |Y| ~ 1, where the absolute gate bites (at |Y| in [1, 2) bf16 output rounding
+    alone has a mean error of about 1.95e-3, in [0.5, 1) half of that)."""
+    q, k, v = wl.make_qkv(shape, seed=wl.BASE_SEED + 1, device="cuda", v_mean=1.0)
+    ref = oracle_y(q, k, v)
+    y, op = run_gpu(q, k, v)
+    assert_parity(y, ref, f"{shape.name}/v_mean=1")
+    op.close()
+
+
+@pytest.mark.parametrize("shape", BIG_SHAPES, ids=lambda s: s.name)
+def test_full_size_16k_shapes_sampled_slabs(shape):
+    """Full size, in the configuration the benchmark times; the oracle checks whole slabs
+    (first, a middle one, last) and the reduced state of those slabs."""
+    q, k, v = wl.make_qkv(shape, seed=wl.BASE_SEED, device="cuda")
+    y, op = run_gpu(q, k, v)
+    assert op.variant == "stream"
+    assert torch.isfinite(y.view(-1)[:: 4097].float()).all()
+    S_gpu, z_gpu = op.read_state()
+    for b, h in [(0, 0), (1, shape.H // 2), (shape.B - 1, shape.H - 1)]:
+        kq, kk, kv = q[b, h], k[b, h], v[b, h]
+        S, z = oracle.state(to_f64(kk), to_f64(kv))
+        ref = oracle.apply(to_f64(kq), S, z, EPS)
+        assert_parity(y[b, h], ref, f"{shape.name}[{b},{h}]")
+        # state: relative to its own scale (entries are sums of N terms)
+        assert np.abs(z_gpu[b, h] - z).max() <= 2e-3 * np.abs(z).max()
+        assert np.linalg.norm(S_gpu[b, h] - S) <= 5e-3 * np.linalg.norm(S)
+    op.close()
+
+
+EDGE_CASES = [
+    # (B, H, N, d): ragged tails, tiny N, N around tile sizes, odd slab counts
+    (1, 1, 1, 64), (1, 1, 1, 40), (1, 3, 7, 160), (2, 1, 63, 64), (1, 2, 65, 64),
+    (1, 1, 127, 64), (1, 1, 129, 64), (1, 5, 191, 64), (1, 1, 193, 64), (3, 1, 1000, 80),
+    (1, 7, 333, 40), (1, 1, 4097, 128), (2, 3, 257, 32), (1, 2, 12289, 64), (1, 148, 64, 64),
+]
+
+
+@pytest.mark.parametrize("dims", EDGE_CASES, ids=lambda d: "x".join(map(str, d)))
+def test_edge_shapes_all_variants(dims):
+    B, H, N, d = dims
+    q, k, v = wl.make_small(B, H, N, d, seed=11, device="cuda")
+    ref = oracle_y(q, k, v)
+    for variant in variants_for(wl.AttnShape("e", B, H, N, d)):
+        y, op = run_gpu(q, k, v, variant)
+        assert_parity(y, ref, f"{dims}/{variant}->{op.variant}")
+        op.close()
+
+
+def test_stream_variant_tail_and_slab_crossing():
+    """Many slabs, ragged N: every CTA's run crosses slab boundaries and tail tiles are masked."""
+    for (B, H, N) in [(2, 37, 1000), (1, 100, 130), (2, 20, 2500)]:
+        q, k, v = wl.make_small(B, H, N, 64, seed=5, device="cuda")
+        ref = oracle_y(q, k, v)
+        y, op = run_gpu(q, k, v, "stream")
+        assert op.variant == "stream"
+        assert_parity(y, ref, f"stream {(B, H, N)}")
+        op.close()
+
+
+def test_bit_reproducible_run_to_run():
+    for shape, variant in [(wl.find_shape("sdxl_2048_L2"), "stream"),
+                           (wl.find_shape("sd15_512_L1"), "split"),
+                           (wl.find_shape("sd15_512_L2"), "cluster")]:
+        q, k, v = wl.make_qkv(shape, seed=3, device="cuda")
+        y1, op = run_gpu(q, k, v, variant)
+        y2 = op.forward(q, k, v)
+        torch.cuda.synchronize()
+        op.close()
+        y3, op3 = run_gpu(q, k, v, variant)
+        op3.close()
+        assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
+        assert torch.equal(y1.view(torch.int16), y3.view(torch.int16))
+
+
+def test_state_matches_oracle_state():
+    shape = wl.find_shape("sd21_768_L2")
+    q, k, v = wl.make_qkv(shape, seed=9, device="cuda")
+    S, z = oracle.state(to_f64(k), to_f64(v))
+    for variant in ("split", "stream", "cluster"):
+        _, op = run_gpu(q, k, v, variant)
+        S_gpu, z_gpu = op.read_state()
+        op.close()
+        assert np.abs(z_gpu - z).max() <= 2e-3 * np.abs(z).max(), variant
+        assert np.linalg.norm(S_gpu - S) <= 5e-3 * np.linalg.norm(S), variant
+
+
+def test_constant_v_and_zero_qk_properties():
+    B, H, N, d = 1, 2, 3000, 64
+    q, k, _ = wl.make_small(B, H, N, d, seed=21, device="cuda")
+    row = torch.linspace(-2, 2, d, device="cuda").bfloat16()
+    v = row.expand(B, H, N, d).contiguous()
+    for variant in ("split", "stream", "cluster"):
+        y, op = run_gpu(q, k, v, variant)
+        op.close()
+        # row sums of the attention weights are one: constant V comes back (to bf16 rounding)
+        assert (y.float() - row.float()).abs().max().item() <= 2.0 * 2 ** -8
+    z = torch.zeros_like(q)
+    _, _, v2 = wl.make_small(B, H, N, d, seed=22, device="cuda")
+    y, op = run_gpu(z, z, v2, "stream")
+    op.close()
+    mean = v2.float().mean(dim=2, keepdim=True)
+    assert (y.float() - mean).abs().max().item() <= 2e-3
+
+
+def test_outlier_scale_inputs_and_identity_phi():
+    q, k, v = wl.make_small(1, 4, 2048, 64, seed=31, device="cuda", scale=8.0)
+    ref = oracle_y(q, k, v)
+    for variant in ("split", "stream", "cluster"):
+        y, op = run_gpu(q, k, v, variant)
+        op.close()
+        assert_parity(y, ref, f"x8/{variant}")
+    qa, ka = q.abs(), k.abs()
+    ref = oracle_y(qa, ka, v, phi_kind=oracle.PHI_IDENTITY)
+    for variant in ("split", "stream", "cluster"):
+        y, op = run_gpu(qa, ka, v, variant, phi=attn.PHI_IDENTITY)
+        op.close()
+        assert_parity(y, ref, f"identity/{variant}")
+
+
+def test_forward_host_matches_device_forward():
+    shape = wl.find_shape("sd21_768_L3")
+    q, k, v = wl.make_qkv(shape, seed=13, device="cpu")
+    qp, kp, vp = (t.pin_memory() for t in (q, k, v))
+    yp = torch.empty_like(qp).pin_memory()
+    op = attn.LinFusionAttention(shape.B, shape.H, shape.N, shape.d)
+    op.forward_host(qp, kp, vp, yp)
+    torch.cuda.synchronize()
+    y_dev = op.forward(q.cuda(), k.cuda(), v.cuda())
+    torch.cuda.synchronize()
+    assert torch.equal(yp.view(torch.int16), y_dev.cpu().view(torch.int16))
+    assert_parity(yp, oracle_y(q, k, v), "forward_host")
+    op.close()
+
+
+def test_lent_workspace_gives_same_bits():
+    shape = wl.find_shape("sdxl_2048_L2")
+    q, k, v = wl.make_qkv(shape, seed=17, device="cuda")
+    y1, op = run_gpu(q, k, v, "stream")
+    nbytes = attn.linfusion_attn_workspace_bytes(op.desc, torch.cuda.get_device_properties(0).multi_processor_count)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    off = (-ws.data_ptr()) % 256
+    op.set_workspace(ws[off:off + nbytes])
+    y2 = op.forward(q, k, v)
+    torch.cuda.synchronize()
+    assert op.status() == attn.OK
+    assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
+    with pytest.raises(attn.LinFusionError) as e:
+        op.set_workspace(ws[off:off + 256])
+    assert e.value.code == attn.ERR_ALLOC
+    op.close()
+
+
+def test_forward_argument_errors_touch_no_memory():
+    op = attn.LinFusionAttention(1, 1, 256, 64)
+    q, k, v = wl.make_small(1, 1, 256, 64, seed=1, device="cuda")
+    y = torch.empty_like(q)
+    lib = attn.load_library()
+    args = [q.data_ptr(), k.data_ptr(), v.data_ptr(), y.data_ptr()]
+    for i in range(4):
+        bad = list(args)
+        bad[i] = 0
+        assert lib.linfusion_attn_forward(op._h, *bad, None) == attn.ERR_INVALID_ARG
+        bad[i] = args[i] + 2
+        assert lib.linfusion_attn_forward(op._h, *bad, None) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_forward(op._h, args[0], args[1], args[2], args[0], None) == attn.ERR_INVALID_ARG
+    assert lib.linfusion_attn_forward(op._h, args[0], args[1], args[2], args[2] + 64, None) == attn.ERR_INVALID_ARG
+    with pytest.raises(attn.LinFusionError) as e:
+        attn.LinFusionAttention(1, 1, 256, 64, device=torch.cuda.device_count())
+    assert e.value.code == attn.ERR_INVALID_ARG
+    op.close()
