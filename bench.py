@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the normalized non-causal linear attention at the SD-XL 16K-image shapes.
+
+    python bench.py --gpus N --steps K --warmup W            # the CUDA library
+    python bench.py --impl reference --steps K --warmup W    # the fp64 CPU oracle, on host cores
+
+One step = one forward of each attention level of the 16384x8192 SD-XL workload
+(N = 524288, C = 640, H = 10 and N = 131072, C = 1280, H = 20; B = 2, d = 64, bf16), i.e. every
+stage of the path (split-N state, fixed-order reduction, apply) over one batch.  Prints ONE JSON
+line: tokens/s over all GPUs with inputs resident in HBM, the same through the host-buffer entry
+point (copies inside the timed region), the roofline of the slowest kernel, and the oracle timed
+on a bounded sample as a CPU baseline.  With N > 1 (torchrun) every rank runs the same per-GPU
+workload on its own seeded batch: independent units, no data-path collective (weak scaling).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "linear_attn_tokens_per_s"
+UNIT = "tokens/s"
+WORKLOAD = "sdxl_16k"          # both attention levels of the 16384x8192 SD-XL workload
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peak_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples taken while the benchmark runs (read-only)."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int, period_ms: int = 50):
+        self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", str(period_ms), "-i", str(gpu_index)],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is not None:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+        rows = []
+        try:
+            self.file.flush()
+            with open(self.file.name) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) < 9:
+                        continue
+                    try:
+                        ts = time.mktime(time.strptime(parts[0].split(".")[0], "%Y/%m/%d %H:%M:%S"))
+                        ts += float("0." + parts[0].split(".")[1]) if "." in parts[0] else 0.0
+                        rows.append((ts, float(parts[1]), float(parts[2]), float(parts[3]), parts[4:9]))
+                    except Exception:
+                        continue
+            os.unlink(self.file.name)
+        except Exception:
+            pass
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        inside = [r for r in rows if t0 - 0.05 <= r[0] <= t1 + 0.05]
+        window = "timed_region"
+        if len(inside) < 3:
+            # Too short a region for the sampler: use the samples taken under load in this run.
+            pmax = max(r[3] for r in rows)
+            inside = [r for r in rows if r[3] >= 0.5 * pmax]
+            window = "whole_run_under_load"
+        sm = sorted(r[1] for r in inside)
+        reasons = set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in inside:
+            for name, val in zip(names, r[4][1:]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": inside[0][2], "reasons": sorted(reasons),
+                "samples": len(inside), "window": window,
+                "power_w_max": max(r[3] for r in inside)}
+
+
+def time_oracle_sample(max_seconds: float = 20.0):
+    """Time the oracle, as it stands, on one (batch, head) slab of the larger 16K level — or on a
+    leading run of its tokens if a whole slab would take too long.  Returns a dict."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2409_02097_b200 import workloads as wl
+
+    shape = wl.find_shape("sdxl_16k_L1")
+    g = torch.Generator().manual_seed(wl.BASE_SEED)
+    probe_n = 16384
+    def draw(n):
+        return [torch.randn((n, shape.d), generator=g).bfloat16().double().numpy() for _ in range(3)]
+    q, k, v = draw(probe_n)
+    oracle.linear(q, k, v, 1e-6)                      # load the library, warm the threads
+    t = time.perf_counter()
+    oracle.linear(q, k, v, 1e-6)
+    per_token = (time.perf_counter() - t) / probe_n
+    n = int(min(shape.N, max(probe_n, max_seconds / max(per_token, 1e-12))))
+    q, k, v = draw(n)
+    t = time.perf_counter()
+    y = oracle.linear(q, k, v, 1e-6)
+    dt = time.perf_counter() - t
+    assert np.isfinite(y).all()
+    # A slab carries one of H heads of every token: n slab-rows are n / H tokens of the layer.
+    tokens = n / shape.H
+    return {"value": tokens / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{n} of {shape.N} tokens of one (b,h) slab of sdxl_16k_L1 "
+                      f"(1/{shape.B * shape.H} of the level's slabs), fp64, {dt:.2f} s",
+            "seconds": dt, "n": n}
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on a bounded sample per step."""
+    import numpy as np
+    import torch
+    import oracle
+    from paper_2409_02097_b200 import workloads as wl
+
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    shape = wl.find_shape("sdxl_16k_L1")
+    probe = time_oracle_sample(max_seconds=2.0)
+    per_token_row = probe["seconds"] / probe["n"]
+    budget = 150.0 / max(1, args.steps + args.warmup)
+    n = int(min(shape.N, max(4096, budget / per_token_row)))
+    g = torch.Generator().manual_seed(wl.BASE_SEED)
+    q, k, v = [torch.randn((n, shape.d), generator=g).bfloat16().double().numpy() for _ in range(3)]
+    for _ in range(args.warmup):
+        oracle.linear(q, k, v, 1e-6)
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        y = oracle.linear(q, k, v, 1e-6)
+    dt = time.perf_counter() - t
+    assert np.isfinite(y).all()
+    value = (n / shape.H) * args.steps / dt
+    sample = (f"per step: {n} of {shape.N} tokens of one (b,h) slab of sdxl_16k_L1, fp64 oracle "
+              f"on host cores")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * dt / args.steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_cuda(args):
+    import torch
+    from paper_2409_02097_b200 import attn, build, workloads as wl
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build_library()
+    if dist is not None:
+        dist.barrier()
+    attn.load_library()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    shapes = wl.CONFIGS[4]
+    eps = 1e-6
+    layers = []
+    for i, s in enumerate(shapes):
+        q, k, v = wl.make_qkv(s, seed=wl.BASE_SEED + 100 * rank + i, device=f"cuda:{local_rank}")
+        y = torch.empty_like(q)
+        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank)
+        layers.append((s, op, q, k, v, y))
+    tokens_per_step = sum(s.tokens for s in shapes)
+    launches_per_step = sum(op.launches_per_forward for _, op, *_ in layers)
+
+    def step():
+        for _, op, q, k, v, y in layers:
+            op.forward(q, k, v, y)
+
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    for _ in range(max(args.warmup, 3)):
+        step()
+    for _, op, *_ in layers:
+        op.enable_kernel_timing(min(args.steps, 4096))
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    ev0.record()
+    for _ in range(args.steps):
+        step()
+    ev1.record()
+    barrier()
+    t1 = time.time()
+    ms = ev0.elapsed_time(ev1)
+    for _, op, *_ in layers:
+        assert op.status() == attn.OK, "a device-side wait expired"
+    if dist is not None:
+        t = torch.tensor([ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = world * tokens_per_step * args.steps / (ms * 1e-3)
+
+    # Per-kernel durations recorded inside the timed region.
+    peak, peak_kind = measured_peak_gbs()
+    kernels = []
+    names = ["stream_state_kernel", "stream_reduce_kernel", "stream_apply_kernel"]
+    for s, op, *_ in layers:
+        sums, calls = op.kernel_times()
+        op.enable_kernel_timing(0)
+        for name, total in zip(names, sums):
+            if calls == 0:
+                continue
+            avg_ms = total / calls
+            algo = 2 * s.B * s.N * s.C * 2 if name != "stream_reduce_kernel" else 0
+            kernels.append({"kernel": name, "shape": s.name, "avg_ms": avg_ms,
+                            "algorithmic_bytes": algo,
+                            "gbs": (algo / (avg_ms * 1e-3) / 1e9) if avg_ms > 0 else None})
+    dominant = max(kernels, key=lambda r: r["avg_ms"]) if kernels else None
+    roofline = None
+    if dominant is not None:
+        roofline = {"bound": "hbm", "kernel": dominant["kernel"], "shape": dominant["shape"],
+                    "achieved": dominant["gbs"], "peak": peak, "peak_kind": f"of {peak_kind}",
+                    "unit": "GB/s", "frac": dominant["gbs"] / peak, "traffic": None,
+                    "frac_of_nominal_8TBps": dominant["gbs"] / NOMINAL_HBM_GBS}
+    step_bytes = sum(s.min_bytes for s in shapes)
+    path_gbs = step_bytes * args.steps / (ms * 1e-3) / 1e9
+
+    # End to end through the host-buffer entry point: H2D of Q, K, V and D2H of Y every step.
+    e2e = None
+    if not args.no_e2e:
+        host = []
+        for s, op, q, k, v, y in layers:
+            hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+            hy = torch.empty_like(hq).pin_memory()
+            host.append((op, hq, hk, hv, hy))
+        def e2e_step():
+            for op, hq, hk, hv, hy in host:
+                op.forward_host(hq, hk, hv, hy)
+        e2e_step()                      # allocates the staging buffers
+        e2e_step()
+        barrier()
+        k_e2e = max(1, min(args.steps, args.e2e_steps))
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(k_e2e):
+            e2e_step()
+        e1.record()
+        barrier()
+        ms_e2e = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ms_e2e], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_e2e = float(t.item())
+        h2d = sum(3 * s.B * s.N * s.C * 2 for s in shapes)
+        d2h = sum(s.B * s.N * s.C * 2 for s in shapes)
+        e2e = {"value": world * tokens_per_step * k_e2e / (ms_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": k_e2e,
+               "ms_per_step": ms_e2e / k_e2e}
+        del host
+
+    clocks = sampler.stop(t0, t1) if sampler is not None else None
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cb = time_oracle_sample(20.0)
+        cpu_baseline = {k: cb[k] for k in ("value", "unit", "cores", "kind", "sample")}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": WORKLOAD,
+                       "shapes": [{"name": s.name, "B": s.B, "H": s.H, "N": s.N, "d": s.d}
+                                  for s in shapes],
+                       "variant": [op.variant for _, op, *_ in layers],
+                       "l2": "inputs larger than L2 (8.05 GB touched per step)",
+                       "parallelism": f"independent batches x{world}"},
+            "tokens_per_s_per_gpu": value / world,
+            "hbm_gbs_whole_path": path_gbs,
+            "hbm_frac_of_nominal_8TBps": path_gbs / NOMINAL_HBM_GBS,
+            "hbm_frac_of_measured_copy": path_gbs / peak,
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=300)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_cuda(args)
+
+
+if __name__ == "__main__":
+    main()
