@@ -16,10 +16,11 @@ constexpr int kPhiIdentity = 1;
 constexpr uint32_t kStatusOk = 0u;
 constexpr uint32_t kStatusWaitExpired = 1u;
 
-// Upper bound on polls of one mbarrier wait; far beyond any legitimate wait (each failed
-// try_wait already blocks for a hardware-defined interval), so that a lost transaction ends
-// the kernel with an error word instead of a hang.
-constexpr uint32_t kMaxBarrierPolls = 1u << 20;
+// Upper bound on polls of one mbarrier wait.  Each failed try_wait already blocks for a
+// hardware-defined interval (about 4 us measured), so this is roughly a quarter of a second: far
+// beyond any legitimate wait here (microseconds), so that a lost transaction ends the kernel with
+// an error word instead of a hang.
+constexpr uint32_t kMaxBarrierPolls = 1u << 16;
 
 // ---------------------------------------------------------------------------------------------
 // phi (Sec. 2.2: non-negative activation on the K and Q features).  elu(x) + 1:
@@ -57,6 +58,29 @@ __device__ __forceinline__ uint32_t phi_bf16x2(uint32_t p)
     return pack_bf16x2(phi<PHI>(bf16_lo(p)), phi<PHI>(bf16_hi(p)));
 }
 
+// The same activation on a packed bf16 pair, entirely in bf16x2 arithmetic (6 instructions per
+// pair instead of 13 through fp32).  log2(e) is split into a bf16 head and tail so that
+// t = min(x,0) * log2(e) is the correctly rounded bf16 product (one fused rounding); rounding t
+// to bf16 adds a relative error of about |x| * 2^-9 to exp(x), and the bf16 exponential
+// instruction rounds its result toward zero (measured mean -0.27 % on the negative side, where
+// the fp32 route has none) — both of the order of the bf16 rounding the MMA operand gets anyway.
+template <int PHI>
+__device__ __forceinline__ uint32_t phi_packed_bf16x2(uint32_t p)
+{
+    if (PHI == kPhiIdentity) return p;
+    const uint32_t zero = 0u;
+    const uint32_t log2e_hi = 0x3FB93FB9u;  // bf16 pair 1.4453125
+    const uint32_t log2e_lo = 0xBB2CBB2Cu;  // bf16 pair log2(e) - 1.4453125 = -0.0026245
+    uint32_t m, u, t, e, r;
+    asm("min.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(p), "r"(zero));
+    asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(u) : "r"(m), "r"(log2e_lo));
+    asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(t) : "r"(m), "r"(log2e_hi), "r"(u));
+    asm("ex2.approx.ftz.bf16x2 %0, %1;" : "=r"(e) : "r"(t));
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(p), "r"(zero));
+    asm("add.rn.bf16x2 %0, %1, %2;" : "=r"(r) : "r"(r), "r"(e));
+    return r;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Shared-memory addressing and fragment loads
 // ---------------------------------------------------------------------------------------------
@@ -90,6 +114,17 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint3
         "{%0,%1,%2,%3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// D(16x8, fp32) = A * B (accumulator starts at zero; saves clearing the registers first)
+__device__ __forceinline__ void mma_bf16_16816_init(float (&c)[4], uint32_t a0, uint32_t a1,
+                                                    uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "{%10,%10,%10,%10};"
+        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
 }
 
 // ---------------------------------------------------------------------------------------------

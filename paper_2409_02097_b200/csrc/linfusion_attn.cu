@@ -15,7 +15,7 @@ using namespace lf;
 namespace {
 
 constexpr int kDefaultSmCount = 148;
-constexpr int kStreamApplyWarps = 12;
+constexpr int kStreamApplyWarps = 10;
 using ApplyCfg = StreamApplyCfg<kStreamApplyWarps>;
 
 enum Variant { kSplit = 1, kStream = 2, kCluster = 3 };
@@ -41,7 +41,7 @@ struct Plan {
     // cluster
     int cluster_size = 0;
     // workspace (bytes, offsets)
-    size_t partial_bytes = 0, state_off = 0, status_off = 0, total_bytes = 0;
+    size_t partial_bytes = 0, state_off = 0, frags_off = 0, counters_off = 0, status_off = 0, total_bytes = 0;
     int launches = 0;
 };
 
@@ -114,6 +114,7 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         p->G_state = static_cast<int>(gs < p->W_state ? gs : p->W_state);
         long long ga = sm_count;
         p->G_apply = static_cast<int>(ga < p->W_apply ? ga : p->W_apply);
+        if (p->G_apply < slabs) p->G_apply = slabs;  // every slab is some CTA's home
         int spans = 1;
         for (int g = 0; g < p->G_state; ++g) {
             long long b = unit_begin(g, p->W_state, p->G_state);
@@ -133,7 +134,12 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     }
     p->partial_bytes = align_up(partial_floats * sizeof(float), 256);
     p->state_off = p->partial_bytes;
-    p->status_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
+    p->frags_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
+    // Stream variant only: bf16 fragment image of S | z and one tile counter per slab.
+    const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM ? static_cast<size_t>(slabs) * kStreamFragWords * 4 : 0;
+    const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM ? align_up(static_cast<size_t>(slabs) * 4, 256) : 0;
+    p->counters_off = p->frags_off + align_up(frag_bytes, 256);
+    p->status_off = p->counters_off + counter_bytes;
     p->total_bytes = p->status_off + 256;
     return LINFUSION_OK;
 }
@@ -183,6 +189,8 @@ struct linfusion_attn {
     bool owns_ws;
     float* partials;
     float* state;
+    uint32_t* frags;
+    int* tile_counters;
     uint32_t* status;
     cudaStream_t last_stream;
     void* stage[4];  // staging for the host-buffer entry point (allocated on first use)
@@ -200,6 +208,8 @@ void bind_workspace(linfusion_attn* h, void* ws)
     unsigned char* base = static_cast<unsigned char*>(ws);
     h->partials = reinterpret_cast<float*>(base);
     h->state = reinterpret_cast<float*>(base + h->plan.state_off);
+    h->frags = reinterpret_cast<uint32_t*>(base + h->plan.frags_off);
+    h->tile_counters = reinterpret_cast<int*>(base + h->plan.counters_off);
     h->status = reinterpret_cast<uint32_t*>(base + h->plan.status_off);
 }
 
@@ -318,10 +328,10 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
         mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans);
     mark(h, 1, s);
     stream_reduce_kernel<<<dim3((kStreamStateFloats + 255) / 256, p.slabs), 256, 0, s>>>(
-        h->partials, h->state, p.tiles_state, p.W_state, p.G_state, p.spans);
+        h->partials, h->state, h->frags, h->tile_counters, p.tiles_state, p.W_state, p.G_state, p.spans);
     mark(h, 2, s);
     stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-        mq, h->state, y, h->status, N, p.tiles_apply, p.W_apply, h->desc.eps);
+        mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps);
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -481,7 +491,7 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     }
     h->owns_ws = true;
     bind_workspace(h, ws);
-    if (cudaMemset(h->status, 0, 256) != cudaSuccess) {
+    if (cudaMemset(h->frags, 0, h->plan.total_bytes - h->plan.frags_off) != cudaSuccess) {
         cudaFree(ws);
         delete h;
         return LINFUSION_ERR_CUDA;
@@ -501,7 +511,7 @@ linfusion_status_t linfusion_attn_set_workspace(linfusion_attn_t* h, void* dev_p
     if (h->owns_ws && h->ws != nullptr) cudaFree(h->ws);
     h->owns_ws = false;
     bind_workspace(h, dev_ptr);
-    if (cudaMemset(h->status, 0, 256) != cudaSuccess) return LINFUSION_ERR_CUDA;
+    if (cudaMemset(h->frags, 0, h->plan.total_bytes - h->plan.frags_off) != cudaSuccess) return LINFUSION_ERR_CUDA;
     return LINFUSION_OK;
 }
 

@@ -14,10 +14,13 @@
 //                           ldmatrix.trans, phi is applied to the A fragments in registers, and a
 //                           ninth column block of ones produces z.  Each (CTA, slab, half) writes
 //                           its own fp32 partial; nothing is combined with atomics.
-//   stream_reduce_kernel  — sums the partials of a slab in (CTA, half) order.
+//   stream_reduce_kernel  — sums the partials of a slab in (CTA, half) order; also lays S | z out
+//                           as the bf16 MMA B-fragments the apply kernel loads.
 //   stream_apply_kernel   — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps).  S | z sit in registers as
-//                           bf16 MMA B-fragments (reloaded when the CTA's run crosses into the
-//                           next slab); A = phi(Q) comes from the stage with ldmatrix; the
+//                           bf16 MMA B-fragments (reloaded when the CTA moves to another slab);
+//                           Q tiles are handed out per slab through an atomic counter (the
+//                           result of a tile does not depend on which CTA computes it);
+//                           A = phi(Q) comes from the stage with ldmatrix; the
 //                           columns of S are permuted so that every lane ends up with 8
 //                           contiguous output channels and stores them as one 16-byte vector.
 //
@@ -50,8 +53,8 @@ struct StreamApplyCfg {
     static constexpr int TILE = 16 * CW;  // tokens per stage: one m16 block per consumer warp
     static constexpr int THREADS = 32 * (CW + 1);
     static constexpr int STAGE_BYTES = TILE * kStreamRowBytes;
-    static constexpr int STAGES = (192 * 1024) / STAGE_BYTES;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 512;  // + align, barriers, meta
 };
 
 // First unit of CTA g when W units are dealt to G CTAs.
@@ -67,11 +70,18 @@ __device__ __forceinline__ void report_wait_expired(uint32_t* status)
 
 // Before the producer leaves: a bounded wait for every bulk copy it still has in flight, so
 // that no copy lands in shared memory after the CTA has gone.
+// Loads [first, issued) are waited for; a load whose stage has been armed again since (its phase
+// is then two behind and can no longer be waited on) must not be in that range.
 template <int STAGES>
-__device__ __forceinline__ void drain_loads(uint64_t* full, int issued)
+__device__ __forceinline__ void drain_loads(uint64_t* full, int first, int issued, uint32_t* status)
 {
-    const int first = issued > STAGES ? issued - STAGES : 0;
-    for (int it = first; it < issued; ++it) (void)mbar_wait(&full[it % STAGES], (it / STAGES) & 1);
+    if (first < issued - STAGES) first = issued - STAGES;
+    if (first < 0) first = 0;
+    for (int it = first; it < issued; ++it)
+        if (!mbar_wait(&full[it % STAGES], (it / STAGES) & 1)) {
+            report_wait_expired(status);
+            return;
+        }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -127,7 +137,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                 tma_load_3d(dst + C::TILE_BYTES, &tmap_v, 0, tile * C::TILE, slab, &full[s], policy);
                 ++issued;
             }
-            drain_loads<C::STAGES>(full, issued);
+            drain_loads<C::STAGES>(full, 0, issued, status);
         }
         return;
     }
@@ -196,10 +206,10 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
             for (int ks = 0; ks < 4; ++ks) {
                 uint32_t a0, a1, a2, a3;
                 ldmatrix_x4_trans(kbase + a_lane + ks * 2048, a0, a1, a2, a3);
-                a0 = phi_bf16x2<PHI>(a0);
-                a1 = phi_bf16x2<PHI>(a1);
-                a2 = phi_bf16x2<PHI>(a2);
-                a3 = phi_bf16x2<PHI>(a3);
+                a0 = phi_packed_bf16x2<PHI>(a0);
+                a1 = phi_packed_bf16x2<PHI>(a1);
+                a2 = phi_packed_bf16x2<PHI>(a2);
+                a3 = phi_packed_bf16x2<PHI>(a3);
                 if (valid < 64) {
                     // Rows past N were zero-filled by TMA, but phi(0) = 1: clear them explicitly.
                     // a0/a1 hold tokens j, j+1; a2/a3 hold j+8, j+9 with j = 16*ks + 2*t4.
@@ -227,40 +237,90 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     if (n_units > 0) flush(slab_first, cur_slab);
 }
 
-// grid (ceil(kStreamStateFloats / 256), slabs): state[slab] = sum over the CTAs whose run meets the
-// slab, in increasing CTA index, half 0 then half 1.
+// Operand image of S | z for the apply kernel: bf16 MMA B-fragments in the order the lanes load
+// them, [k block 4][column-block pair 5][lane 32][4 words] per slab.  Word w of pair p holds
+// register (w & 1) of column block 2p + (w >> 1); block 8 is z, block 9 does not exist.
+constexpr int kStreamFragWords = 4 * 5 * 32 * 4;
+
+// Output channel carried by column slot g8 of column block nb (nb < 8): with this permutation a
+// lane ends up owning channels 8*t4 .. 8*t4+7 (blocks 0-3) and 32+8*t4 .. (blocks 4-7) of its rows.
+__host__ __device__ __forceinline__ int apply_channel_of(int nb, int g8)
+{
+    return 32 * (nb >> 2) + 8 * (g8 >> 1) + 2 * (nb & 3) + (g8 & 1);
+}
+
+// grid (17, slabs), 256 threads: state[slab] = sum over the CTAs whose run meets the slab, in
+// increasing CTA index, half 0 then half 1 (fp32, fixed order).  Also writes the bf16 fragment
+// image of S | z for the apply kernel and clears the slab's tile counter for it.
 __global__ void __launch_bounds__(256)
 stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
+                     uint32_t* __restrict__ frags, int* __restrict__ tile_counters,
                      int tiles_per_slab, long long W, int G, int spans)
 {
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    if (idx >= kStreamStateFloats) return;
+    __shared__ float sums[256];
+    const int tid = threadIdx.x;
+    const int idx = blockIdx.x * 256 + tid;
     const int slab = blockIdx.y;
-    const long long lo = static_cast<long long>(slab) * tiles_per_slab, hi = lo + tiles_per_slab;
-    // First CTA whose run contains unit `lo`.
-    long long g = (lo * G) / W;
-    while (g + 1 < G && unit_begin(g + 1, W, G) <= lo) ++g;
-    while (g > 0 && unit_begin(g, W, G) > lo) --g;
+    if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
     float sum = 0.0f;
-    for (; g < G; ++g) {
-        const long long b = unit_begin(g, W, G);
-        if (b >= hi) break;
-        const int slot = slab - static_cast<int>(b / tiles_per_slab);
-        const float* src = partials + ((static_cast<size_t>(g) * spans + slot) * 2) * kStreamStateFloats + idx;
-        sum += src[0];
-        sum += src[kStreamStateFloats];
+    if (idx < kStreamStateFloats) {
+        const long long lo = static_cast<long long>(slab) * tiles_per_slab, hi = lo + tiles_per_slab;
+        // g0: the CTA whose run contains unit `lo`; g1: the first CTA whose run starts at or after `hi`.
+        long long g0 = (lo * G) / W;
+        while (g0 + 1 < G && unit_begin(g0 + 1, W, G) <= lo) ++g0;
+        while (g0 > 0 && unit_begin(g0, W, G) > lo) --g0;
+        long long g1 = (hi * G) / W;
+        while (g1 < G && unit_begin(g1, W, G) < hi) ++g1;
+        while (g1 > 0 && unit_begin(g1 - 1, W, G) >= hi) --g1;
+        const int slot0 = slab - static_cast<int>(unit_begin(g0, W, G) / tiles_per_slab);
+        const size_t F = kStreamStateFloats;
+        const float* src = partials + idx;
+        sum += src[((static_cast<size_t>(g0) * spans + slot0) * 2) * F];
+        sum += src[((static_cast<size_t>(g0) * spans + slot0) * 2 + 1) * F];
+        // Every later CTA starts inside this slab: its partial for it is in slot 0.
+#pragma unroll 4
+        for (long long g = g0 + 1; g < g1; ++g) {
+            sum += src[(static_cast<size_t>(g) * spans * 2) * F];
+            sum += src[(static_cast<size_t>(g) * spans * 2 + 1) * F];
+        }
+        state[static_cast<size_t>(slab) * F + idx] = sum;
     }
-    state[static_cast<size_t>(slab) * kStreamStateFloats + idx] = sum;
+    sums[tid] = sum;
+    __syncthreads();
+
+    uint32_t* fr = frags + static_cast<size_t>(slab) * kStreamFragWords;
+    if (blockIdx.x < 16) {
+        // rows c = 4*blockIdx.x + tid/64 of S; even rows pack (S[c][e], S[c+1][e])
+        const int r = tid >> 6, e = tid & 63;
+        if ((r & 1) == 0) {
+            const int c = 4 * blockIdx.x + r;
+            const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 64]);
+            const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
+            const int r32 = e & 31;
+            const int nb = 4 * (e >> 5) + ((r32 & 7) >> 1);
+            const int g8 = 2 * (r32 >> 3) + (r32 & 1);
+            fr[((kb * 5 + (nb >> 1)) * 32 + g8 * 4 + t4) * 4 + (nb & 1) * 2 + reg] = pair;
+        }
+    } else if (tid < 64 && (tid & 1) == 0) {
+        // z: pair (z[c], z[c+1]) goes to every column slot of block 8
+        const int c = tid;
+        const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 1]);
+        const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
+        for (int g8 = 0; g8 < 8; ++g8) fr[((kb * 5 + 4) * 32 + g8 * 4 + t4) * 4 + reg] = pair;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Apply
+// Apply.  Tiles are handed out per slab through an atomic counter: CTA g starts on its home slab
+// g*slabs/G and moves to the next slab that still has tiles when one runs dry, so the CTAs of a
+// slab share its tail and early finishers help elsewhere.  Each output tile depends only on its
+// own Q rows and the slab's S | z, so the result does not depend on who computes it.
 // ---------------------------------------------------------------------------------------------
 template <int PHI, int CW>
 __global__ void __launch_bounds__(StreamApplyCfg<CW>::THREADS, 1)
-stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const float* __restrict__ state,
-                    __nv_bfloat16* __restrict__ Y, uint32_t* __restrict__ status, int N,
-                    int tiles_per_slab, long long W, float eps)
+stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* __restrict__ frags,
+                    __nv_bfloat16* __restrict__ Y, int* __restrict__ tile_counters,
+                    uint32_t* __restrict__ status, int N, int tiles_per_slab, int slabs, float eps)
 {
     using C = StreamApplyCfg<CW>;
     extern __shared__ unsigned char smem_raw[];
@@ -268,11 +328,9 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const float* __r
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
     uint64_t* empty = full + C::STAGES;
+    int2* meta = reinterpret_cast<int2*>(empty + C::STAGES);  // (slab, tile) of each stage; slab < 0 ends
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const long long G = gridDim.x, g = blockIdx.x;
-    const long long u0 = unit_begin(g, W, G), u1 = unit_begin(g + 1, W, G);
-    const int n_units = static_cast<int>(u1 - u0);
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -284,29 +342,70 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const float* __r
     __syncthreads();
 
     if (warp == C::CONSUMER_WARPS) {
+        // ---------------- producer warp (lane 0 issues; all lanes help to find work) ----------------
+        uint64_t policy = 0;
         if (lane == 0) {
             prefetch_tmap(&tmap_q);
-            const uint64_t policy = policy_evict_first();
-            int issued = 0;
-            for (int it = 0; it < n_units; ++it) {
-                const int s = it % C::STAGES;
-                const uint32_t ph = (it / C::STAGES) & 1;
-                if (!mbar_wait(&empty[s], ph ^ 1)) {
-                    report_wait_expired(status);
-                    break;
+            policy = policy_evict_first();
+        }
+        int slab = static_cast<int>((static_cast<long long>(blockIdx.x) * slabs) / gridDim.x);
+        int it = 0, issued = 0;
+        bool ok = true;
+        while (true) {
+            int tile = 0;
+            if (lane == 0) tile = atomicAdd(&tile_counters[slab], 1);
+            tile = __shfl_sync(0xffffffffu, tile, 0);
+            if (tile >= tiles_per_slab) {
+                // Next slab, in cyclic order, whose counter has not run past its tiles.
+                int found = -1;
+                for (int base = 0; base < slabs && found < 0; base += 32) {
+                    const int off = base + lane;
+                    const int cand = (slab + 1 + off) % slabs;
+                    const bool has = off < slabs &&
+                                     *reinterpret_cast<volatile int*>(&tile_counters[cand]) < tiles_per_slab;
+                    const unsigned m = __ballot_sync(0xffffffffu, has);
+                    if (m != 0u) found = (slab + 1 + base + __ffs(m) - 1) % slabs;
                 }
-                const long long u = u0 + it;
-                const int slab = static_cast<int>(u / tiles_per_slab);
-                const int tile = static_cast<int>(u % tiles_per_slab);
-                mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                tma_load_3d(smem + s * C::STAGE_BYTES, &tmap_q, 0, tile * C::TILE, slab, &full[s], policy);
-                ++issued;
+                if (found < 0) break;
+                slab = found;
+                continue;
             }
-            drain_loads<C::STAGES>(full, issued);
+            const int s = it % C::STAGES;
+            if (lane == 0) {
+                ok = mbar_wait(&empty[s], ((it / C::STAGES) & 1) ^ 1);
+                if (ok) {
+                    meta[s] = make_int2(slab, tile);
+                    mbar_expect_tx(&full[s], C::STAGE_BYTES);
+                    tma_load_3d(smem + s * C::STAGE_BYTES, &tmap_q, 0, tile * C::TILE, slab, &full[s], policy);
+                    ++issued;
+                } else {
+                    report_wait_expired(status);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            ++it;
+        }
+        if (lane == 0) {
+            int first = 0;
+            if (ok) {
+                // End marker in the next stage (consumers leave when they see it).  Its stage held
+                // load number issued - STAGES, which the consumers have released by now.
+                const int s = it % C::STAGES;
+                if (mbar_wait(&empty[s], ((it / C::STAGES) & 1) ^ 1)) {
+                    meta[s] = make_int2(-1, 0);
+                    mbar_arrive(&full[s]);
+                    first = issued - C::STAGES + 1;
+                } else {
+                    report_wait_expired(status);
+                }
+            }
+            drain_loads<C::STAGES>(full, first, issued, status);
         }
         return;
     }
 
+    // ---------------- consumers ----------------
     const int g8 = lane >> 2, t4 = lane & 3;
     // A-fragment lane offset in the swizzled Q stage (non-transposed ldmatrix).
     const int sw = lane & 7;
@@ -316,84 +415,75 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const float* __r
 
     uint32_t sfrag[4][9][2];  // [k block][column block][b0, b1], bf16x2
     auto load_state = [&](int slab) {
-        const float* S = state + static_cast<size_t>(slab) * kStreamStateFloats;
-        const float* z = S + 64 * 64;
+        const uint4* fr = reinterpret_cast<const uint4*>(frags + static_cast<size_t>(slab) * kStreamFragWords) + lane;
 #pragma unroll
         for (int kb = 0; kb < 4; ++kb) {
-            const int c = kb * 16 + 2 * t4;
 #pragma unroll
-            for (int nb = 0; nb < 8; ++nb) {
-                // Column slot g8 of block nb carries output channel e: lanes t4 then own channels
-                // 8*t4 .. 8*t4+7 (blocks 0-3) and 32+8*t4 .. (blocks 4-7) of their rows.
-                const int e = 32 * (nb >> 2) + 8 * (g8 >> 1) + 2 * (nb & 3) + (g8 & 1);
-                sfrag[kb][nb][0] = pack_bf16x2(__ldg(S + c * 64 + e), __ldg(S + (c + 1) * 64 + e));
-                sfrag[kb][nb][1] = pack_bf16x2(__ldg(S + (c + 8) * 64 + e), __ldg(S + (c + 9) * 64 + e));
+            for (int nbp = 0; nbp < 5; ++nbp) {
+                const uint4 v = __ldg(fr + (kb * 5 + nbp) * 32);
+                sfrag[kb][2 * nbp][0] = v.x;
+                sfrag[kb][2 * nbp][1] = v.y;
+                if (nbp < 4) {
+                    sfrag[kb][2 * nbp + 1][0] = v.z;
+                    sfrag[kb][2 * nbp + 1][1] = v.w;
+                }
             }
-            sfrag[kb][8][0] = pack_bf16x2(__ldg(z + c), __ldg(z + c + 1));
-            sfrag[kb][8][1] = pack_bf16x2(__ldg(z + c + 8), __ldg(z + c + 9));
         }
     };
 
     int cur_slab = -1;
-    bool failed = false;
-    for (int it = 0; it < n_units; ++it) {
+    for (int it = 0;; ++it) {
         const int s = it % C::STAGES;
-        const uint32_t ph = (it / C::STAGES) & 1;
-        const long long u = u0 + it;
-        const int slab = static_cast<int>(u / tiles_per_slab);
-        const int tile = static_cast<int>(u % tiles_per_slab);
+        if (!mbar_wait(&full[s], (it / C::STAGES) & 1)) {
+            if (lane == 0) report_wait_expired(status);
+            break;
+        }
+        const int2 m = meta[s];
+        const int slab = m.x, tile = m.y;
+        if (slab < 0) break;
         if (slab != cur_slab) {
             load_state(slab);
             cur_slab = slab;
         }
-        if (!failed && !mbar_wait(&full[s], ph)) {
-            if (lane == 0) report_wait_expired(status);
-            failed = true;
-        }
-        if (!failed) {
-            const uint32_t qbase = smem_base + s * C::STAGE_BYTES + q_row;
-            float acc[9][4];
+        const uint32_t qbase = smem_base + s * C::STAGE_BYTES + q_row;
+        float acc[9][4];
 #pragma unroll
-            for (int nb = 0; nb < 9; ++nb)
+        for (int kb = 0; kb < 4; ++kb) {
+            uint32_t a0, a1, a2, a3;
+            ldmatrix_x4(qbase + ((((kb << 1) | q_hi) ^ sw) << 4), a0, a1, a2, a3);
+            a0 = phi_packed_bf16x2<PHI>(a0);
+            a1 = phi_packed_bf16x2<PHI>(a1);
+            a2 = phi_packed_bf16x2<PHI>(a2);
+            a3 = phi_packed_bf16x2<PHI>(a3);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) acc[nb][i] = 0.0f;
-#pragma unroll
-            for (int kb = 0; kb < 4; ++kb) {
-                uint32_t a0, a1, a2, a3;
-                ldmatrix_x4(qbase + ((((kb << 1) | q_hi) ^ sw) << 4), a0, a1, a2, a3);
-                a0 = phi_bf16x2<PHI>(a0);
-                a1 = phi_bf16x2<PHI>(a1);
-                a2 = phi_bf16x2<PHI>(a2);
-                a3 = phi_bf16x2<PHI>(a3);
-#pragma unroll
-                for (int nb = 0; nb < 9; ++nb)
+            for (int nb = 0; nb < 9; ++nb) {
+                if (kb == 0)
+                    mma_bf16_16816_init(acc[nb], a0, a1, a2, a3, sfrag[kb][nb][0], sfrag[kb][nb][1]);
+                else
                     mma_bf16_16816(acc[nb], a0, a1, a2, a3, sfrag[kb][nb][0], sfrag[kb][nb][1]);
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[s]);  // stage is free as soon as the fragments are read
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[s]);  // stage is free as soon as the fragments are read
 
-            const float inv0 = 1.0f / (acc[8][0] + eps);
-            const float inv1 = 1.0f / (acc[8][2] + eps);
-            const long long r0 = static_cast<long long>(tile) * C::TILE + warp * 16 + g8, r1 = r0 + 8;
-            __nv_bfloat16* y0 = Y + (static_cast<size_t>(slab) * N + r0) * 64;
-            __nv_bfloat16* y1 = y0 + 8 * 64;
+        const float inv0 = 1.0f / (acc[8][0] + eps);
+        const float inv1 = 1.0f / (acc[8][2] + eps);
+        const long long r0 = static_cast<long long>(tile) * C::TILE + warp * 16 + g8, r1 = r0 + 8;
+        __nv_bfloat16* y0 = Y + (static_cast<size_t>(slab) * N + r0) * 64;
+        __nv_bfloat16* y1 = y0 + 8 * 64;
 #pragma unroll
-            for (int hi = 0; hi < 2; ++hi) {
-                uint4 v0, v1;
-                v0.x = pack_bf16x2(acc[4 * hi + 0][0] * inv0, acc[4 * hi + 0][1] * inv0);
-                v0.y = pack_bf16x2(acc[4 * hi + 1][0] * inv0, acc[4 * hi + 1][1] * inv0);
-                v0.z = pack_bf16x2(acc[4 * hi + 2][0] * inv0, acc[4 * hi + 2][1] * inv0);
-                v0.w = pack_bf16x2(acc[4 * hi + 3][0] * inv0, acc[4 * hi + 3][1] * inv0);
-                v1.x = pack_bf16x2(acc[4 * hi + 0][2] * inv1, acc[4 * hi + 0][3] * inv1);
-                v1.y = pack_bf16x2(acc[4 * hi + 1][2] * inv1, acc[4 * hi + 1][3] * inv1);
-                v1.z = pack_bf16x2(acc[4 * hi + 2][2] * inv1, acc[4 * hi + 2][3] * inv1);
-                v1.w = pack_bf16x2(acc[4 * hi + 3][2] * inv1, acc[4 * hi + 3][3] * inv1);
-                if (r0 < N) st_stream_16B(y0 + 32 * hi + 8 * t4, v0);
-                if (r1 < N) st_stream_16B(y1 + 32 * hi + 8 * t4, v1);
-            }
-        } else {
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&empty[s]);
+        for (int hi = 0; hi < 2; ++hi) {
+            uint4 v0, v1;
+            v0.x = pack_bf16x2(acc[4 * hi + 0][0] * inv0, acc[4 * hi + 0][1] * inv0);
+            v0.y = pack_bf16x2(acc[4 * hi + 1][0] * inv0, acc[4 * hi + 1][1] * inv0);
+            v0.z = pack_bf16x2(acc[4 * hi + 2][0] * inv0, acc[4 * hi + 2][1] * inv0);
+            v0.w = pack_bf16x2(acc[4 * hi + 3][0] * inv0, acc[4 * hi + 3][1] * inv0);
+            v1.x = pack_bf16x2(acc[4 * hi + 0][2] * inv1, acc[4 * hi + 0][3] * inv1);
+            v1.y = pack_bf16x2(acc[4 * hi + 1][2] * inv1, acc[4 * hi + 1][3] * inv1);
+            v1.z = pack_bf16x2(acc[4 * hi + 2][2] * inv1, acc[4 * hi + 2][3] * inv1);
+            v1.w = pack_bf16x2(acc[4 * hi + 3][2] * inv1, acc[4 * hi + 3][3] * inv1);
+            if (r0 < N) st_stream_16B(y0 + 32 * hi + 8 * t4, v0);
+            if (r1 < N) st_stream_16B(y1 + 32 * hi + 8 * t4, v1);
         }
     }
 }
