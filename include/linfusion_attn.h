@@ -150,6 +150,39 @@ linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host,
 linfusion_status_t linfusion_attn_enable_kernel_timing(linfusion_attn_t* h, int32_t slots);
 linfusion_status_t linfusion_attn_kernel_times(linfusion_attn_t* h, float* ms_sum, int32_t* calls);
 
+/*
+ * The attention without a handle and without any allocation.  (The paper has no counterpart to
+ * this call; it exists for how the library gets embedded.)
+ *
+ * Some hosts cannot let a library allocate device memory: an inference server that hands all of
+ * its device memory to its own arena at start-up, so that a later cudaMalloc from inside a
+ * library either fails or breaks the memory budget it promised; or a latency-bound pipeline that
+ * cannot afford the device-wide synchronization cudaMalloc and cudaFree imply.  create() and the
+ * first forward_host() both allocate, so such callers use this entry point instead.  It runs the
+ * three-launch split path (split-N state, fixed-order reduction, apply; any supported head dim)
+ * and keeps the partial states and the reduced state in a fixed 16 MiB array that is part of the
+ * library's device image: every GPU that loads the library holds those 16 MiB until the process
+ * exits, whether or not this function is ever called.  It calls no cudaMalloc, cudaFree or other
+ * allocating routine, creates no streams or events, and keeps no per-call host state.
+ *
+ * desc: as for create(); flags must be AUTO or SPLIT.  q, k, v, y, cuda_stream: as for forward().
+ * The split of N uses as many chunks as fit in the array; a problem whose state alone does not
+ * fit — 2 * B*H * d*(d+1) * 4 bytes + 512 above 16 MiB, e.g. d = 160 with more than 81 slabs — is
+ * rejected with LINFUSION_ERR_ALLOC and nothing is launched.  Other errors: INVALID_ARG,
+ * UNSUPPORTED, CUDA, as for create() and forward().
+ *
+ * The first call on each device looks up the array's device address and raises the kernels'
+ * shared-memory limits; make that first call before starting any stream capture.
+ * Every call on a device shares the one array, which keeps whatever the last call left in it.
+ * Nothing in it needs clearing between calls (each call writes every element before reading it),
+ * but two calls whose kernels overlap on the GPU — different streams, or several host threads —
+ * race on it and corrupt each other's state: order such calls on one stream, or with events.
+ * Output is bit-identical from call to call for identical inputs on the same device.
+ */
+linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_attn_desc_t* desc, const void* q,
+                                                  const void* k, const void* v, void* y,
+                                                  void* cuda_stream);
+
 /* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);
 

@@ -25,6 +25,7 @@ EXPORTED = [
     "linfusion_attn_set_workspace", "linfusion_attn_status", "linfusion_attn_read_state",
     "linfusion_attn_variant_name", "linfusion_attn_launches_per_forward",
     "linfusion_attn_enable_kernel_timing", "linfusion_attn_kernel_times",
+    "linfusion_attn_forward_noalloc",
 ]
 
 
@@ -83,6 +84,8 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_kernel_times.restype = st
     lib.linfusion_attn_kernel_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
                                                 ctypes.POINTER(ctypes.c_int32)]
+    lib.linfusion_attn_forward_noalloc.restype = st
+    lib.linfusion_attn_forward_noalloc.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -125,6 +128,18 @@ def linfusion_attn_forward_host(handle, q_ptr: int, k_ptr: int, v_ptr: int, y_pt
     rc = load_library().linfusion_attn_forward_host(handle, q_ptr, k_ptr, v_ptr, y_ptr, stream_ptr)
     if rc != OK:
         raise LinFusionError(rc, "linfusion_attn_forward_host")
+
+
+def linfusion_attn_forward_noalloc(desc: Desc, q_ptr: int, k_ptr: int, v_ptr: int, y_ptr: int,
+                                   stream_ptr: int = 0) -> None:
+    """Handle-free forward that allocates nothing: the split-N scratch is a fixed 16 MiB array
+    inside the library's device image.  For hosts that cannot let a library call cudaMalloc.
+    Calls that overlap on the GPU race on that array; problems whose state does not fit raise
+    ``LinFusionError`` with ``ERR_ALLOC``."""
+    rc = load_library().linfusion_attn_forward_noalloc(ctypes.byref(desc), q_ptr, k_ptr, v_ptr,
+                                                       y_ptr, stream_ptr)
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_forward_noalloc")
 
 
 def linfusion_attn_destroy(handle) -> None:

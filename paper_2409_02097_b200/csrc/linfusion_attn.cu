@@ -725,3 +725,134 @@ linfusion_status_t linfusion_attn_destroy(linfusion_attn_t* h)
 }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// Allocation-free forward (see the header): the split-N partials and the reduced state live in a
+// fixed array in device global memory that is part of this library's image, so nothing is ever
+// requested from the CUDA allocator.  Every device that loads the library carries the array
+// until the process exits.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+constexpr size_t kNoAllocScratchBytes = size_t(16) << 20;  // 16 MiB
+constexpr int kNoAllocMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+struct NoAllocDevice {
+    bool ready = false;
+    unsigned char* scratch = nullptr;  // device address of g_noalloc_scratch on this device
+    int sm_count = 0;
+};
+NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+
+// Once per device, with that device current: resolve the array's device address (the symbol's
+// name is only a host-side stand-in and must never be handed to a kernel), read the SM count
+// and raise the kernels' dynamic shared-memory limits.
+linfusion_status_t noalloc_setup(int device, int d, int phi)
+{
+    NoAllocDevice& dev = g_noalloc_dev[device];
+    if (!dev.ready) {
+        cudaDeviceProp prop;
+        if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+        if (prop.major != 10) return LINFUSION_ERR_UNSUPPORTED;
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+        dev.scratch = static_cast<unsigned char*>(ptr);
+        dev.sm_count = prop.multiProcessorCount;
+        dev.ready = true;
+    }
+    cudaError_t e = cudaSuccess;
+#define LF_SET(DV) e = set_attrs_d<DV>(phi)
+    LF_DISPATCH_D(d, LF_SET)
+#undef LF_SET
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
+
+}  // namespace
+
+extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_attn_desc_t* desc,
+                                                             const void* q, const void* k,
+                                                             const void* v, void* y,
+                                                             void* cuda_stream)
+{
+    linfusion_status_t st = validate(desc);
+    if (st != LINFUSION_OK) return st;
+    if (desc->device >= kNoAllocMaxDevices) return LINFUSION_ERR_INVALID_ARG;
+    if ((desc->flags & LINFUSION_VARIANT_MASK) > LINFUSION_VARIANT_SPLIT) return LINFUSION_ERR_UNSUPPORTED;
+    // Capacity first: it depends on the descriptor alone.
+    const size_t per_chunk = static_cast<size_t>(desc->B) * desc->H * desc->d * (desc->d + 1) * 4;
+    const size_t state_bytes = align_up(per_chunk, 256);
+    if (state_bytes + per_chunk + 256 > kNoAllocScratchBytes) return LINFUSION_ERR_ALLOC;
+    if (q == nullptr || k == nullptr || v == nullptr || y == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    const uintptr_t pq = reinterpret_cast<uintptr_t>(q), pk = reinterpret_cast<uintptr_t>(k),
+                    pv = reinterpret_cast<uintptr_t>(v), py = reinterpret_cast<uintptr_t>(y);
+    if (((pq | pk | pv | py) & 15u) != 0) return LINFUSION_ERR_INVALID_ARG;
+    const size_t bytes = static_cast<size_t>(desc->B) * desc->H * desc->N * desc->d * 2;
+    auto overlaps = [&](uintptr_t a) { return a < py + bytes && py < a + bytes; };
+    if (overlaps(pq) || overlaps(pk) || overlaps(pv)) return LINFUSION_ERR_INVALID_ARG;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    if (desc->device >= ndev) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(desc->device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    st = noalloc_setup(desc->device, desc->d, desc->phi);
+    if (st != LINFUSION_OK) return st;
+    const NoAllocDevice& dev = g_noalloc_dev[desc->device];
+
+    // A handle-shaped view on the stack: the three-launch split plan, with as many chunks of N
+    // as the fixed array has room for.  Nothing in the array has to start at zero: every partial
+    // and every state element that is read in this call is written earlier in the same call.
+    linfusion_attn view;
+    view.desc = *desc;
+    view.desc.flags = LINFUSION_VARIANT_SPLIT;
+    st = make_plan(&view.desc, dev.sm_count, &view.plan);
+    if (st != LINFUSION_OK) return st;
+    const size_t room = (kNoAllocScratchBytes - state_bytes - 256) / per_chunk;
+    if (static_cast<size_t>(view.plan.chunks_state) > room) view.plan.chunks_state = static_cast<int>(room);
+    view.sm_count = dev.sm_count;
+    view.ws = dev.scratch;
+    view.owns_ws = false;
+    view.partials = reinterpret_cast<float*>(dev.scratch);
+    view.state = reinterpret_cast<float*>(
+        dev.scratch + align_up(per_chunk * static_cast<size_t>(view.plan.chunks_state), 256));
+    view.frags = nullptr;
+    view.tile_counters = nullptr;
+    view.status = nullptr;
+    view.last_stream = nullptr;
+    for (int i = 0; i < 4; ++i) view.stage[i] = nullptr;
+    view.events = nullptr;
+    view.timing_slots = 0;
+    view.timed_calls = 0;
+
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const __nv_bfloat16* Q = static_cast<const __nv_bfloat16*>(q);
+    const __nv_bfloat16* K = static_cast<const __nv_bfloat16*>(k);
+    const __nv_bfloat16* V = static_cast<const __nv_bfloat16*>(v);
+    __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_LAUNCH(DV)                                                                           \
+    e = view.desc.phi == LINFUSION_PHI_IDENTITY ? launch_split<DV, kPhiIdentity>(&view, Q, K, V, Y, s) \
+                                                : launch_split<DV, kPhiEluPlusOne>(&view, Q, K, V, Y, s)
+    LF_DISPATCH_D(view.desc.d, LF_LAUNCH)
+#undef LF_LAUNCH
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
