@@ -41,6 +41,27 @@ def measured_peak_gbs():
         return 6650.0, "fallback"
 
 
+def recorded_traffic(kernel: str, shape: str):
+    """DRAM bytes per launch from the committed ncu summary, or None when the kernel sources
+    have changed since the counters were taken."""
+    import hashlib
+    try:
+        csrc = os.path.join(ROOT, "paper_2409_02097_b200", "csrc")
+        h = hashlib.sha256()
+        for name in ("common.cuh", "stream_kernels.cuh"):
+            with open(os.path.join(csrc, name), "rb") as f:
+                h.update(f.read())
+        sha = h.hexdigest()[:16]
+        with open(os.path.join(ROOT, "profiles", "dram_traffic.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) == 4 and parts[0] == kernel and parts[1] == shape and parts[3] == sha:
+                    return int(parts[2])
+    except Exception:
+        pass
+    return None
+
+
 class ClockSampler:
     """nvidia-smi clock / throttle-reason samples taken while the benchmark runs (read-only)."""
     FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -265,7 +286,8 @@ def run_cuda(args):
     if dominant is not None:
         roofline = {"bound": "hbm", "kernel": dominant["kernel"], "shape": dominant["shape"],
                     "achieved": dominant["gbs"], "peak": peak, "peak_kind": f"of {peak_kind}",
-                    "unit": "GB/s", "frac": dominant["gbs"] / peak, "traffic": None,
+                    "unit": "GB/s", "frac": dominant["gbs"] / peak,
+                    "traffic": recorded_traffic(dominant["kernel"], dominant["shape"]),
                     "frac_of_nominal_8TBps": dominant["gbs"] / NOMINAL_HBM_GBS}
     step_bytes = sum(s.min_bytes for s in shapes)
     path_gbs = step_bytes * args.steps / (ms * 1e-3) / 1e9
