@@ -15,7 +15,7 @@ using namespace lf;
 namespace {
 
 constexpr int kDefaultSmCount = 148;
-constexpr int kStreamApplyWarps = 10;
+constexpr int kStreamApplyWarps = 11;
 using ApplyCfg = StreamApplyCfg<kStreamApplyWarps>;
 
 enum Variant { kSplit = 1, kStream = 2, kCluster = 3 };

@@ -40,8 +40,8 @@ struct StreamStateCfg {
     static constexpr int TILE = 128;  // tokens per stage
     static constexpr int CONSUMER_WARPS = 8;
     static constexpr int THREADS = 32 * (CONSUMER_WARPS + 1);
-    static constexpr int STAGES = 3;
-    static constexpr int CTAS_PER_SM = 2;
+    static constexpr int STAGES = 2;
+    static constexpr int CTAS_PER_SM = 3;
     static constexpr int TILE_BYTES = TILE * kStreamRowBytes;  // 16 KB per tensor
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;         // K then V
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
@@ -53,7 +53,7 @@ struct StreamApplyCfg {
     static constexpr int TILE = 16 * CW;  // tokens per stage: one m16 block per consumer warp
     static constexpr int THREADS = 32 * (CW + 1);
     static constexpr int STAGE_BYTES = TILE * kStreamRowBytes;
-    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES;
+    static constexpr int STAGES = (198 * 1024) / STAGE_BYTES;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 512;  // + align, barriers, meta
 };
 
