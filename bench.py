@@ -356,6 +356,59 @@ def run_cuda(args):
         dist.destroy_process_group()
 
 
+def run_sweep(args):
+    """Every attention level of the five workload families, every kernel variant that serves it.
+    Shapes smaller than the L2 cache are cycled through enough distinct buffer sets to exceed it;
+    one JSON line per (shape, variant), `effective_gbs` = minimum traffic / time."""
+    import torch
+    from paper_2409_02097_b200 import attn, build, workloads as wl
+
+    build.build_library()
+    torch.cuda.set_device(0)
+    peak, _ = measured_peak_gbs()
+    seen = set()
+    for cfg_idx, cfg in enumerate(wl.CONFIGS):
+        for s in cfg:
+            if s.name in seen:
+                continue
+            seen.add(s.name)
+            sets = max(1, min(64, -(-400_000_000 // s.min_bytes)))
+            bufs = []
+            for r in range(sets):
+                q, k, v = wl.make_qkv(s, seed=wl.BASE_SEED + r, device="cuda:0")
+                bufs.append((q, k, v, torch.empty_like(q)))
+            variants = ["auto", "split"] + (["stream"] if s.d == 64 else []) + \
+                       (["cluster"] if s.N <= 16384 else [])
+            for variant in variants:
+                op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, device=0, variant=variant)
+                steps = max(20, min(args.steps, int(2e10 // s.min_bytes)))
+                for i in range(5):
+                    op.forward(*bufs[i % sets])
+                torch.cuda.synchronize()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for i in range(steps):
+                    op.forward(*bufs[i % sets])
+                e1.record()
+                torch.cuda.synchronize()
+                assert op.status() == attn.OK
+                us = 1e3 * e0.elapsed_time(e1) / steps
+                gbs = s.min_bytes / (us * 1e-6) / 1e9
+                print(json.dumps({
+                    "config": cfg_idx + 1, "shape": s.name, "B": s.B, "H": s.H, "N": s.N, "d": s.d,
+                    "requested": variant, "variant": op.variant, "launches": op.launches_per_forward,
+                    "us_per_forward": us, "tokens_per_s": s.tokens / (us * 1e-6),
+                    "effective_gbs": gbs, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
+                    "frac_of_measured_copy": gbs / peak, "buffer_sets": sets,
+                    "hbm_resident": ("no: cycled through %d buffer sets (%.0f MB) to exceed L2"
+                                     % (sets, sets * s.min_bytes / 1e6)) if sets > 1 else
+                                    "single set, larger than L2",
+                    "roofline_us_at_8TBps": s.min_bytes / 8e12 * 1e6}), flush=True)
+                op.close()
+            del bufs
+            torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -366,8 +419,12 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true",
+                    help="time every shape of the five workload families with every variant")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_cuda(args)
