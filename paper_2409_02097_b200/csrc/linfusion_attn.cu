@@ -66,7 +66,7 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
 
 int largest_cluster(int tiles_kv)
 {
-    int c = 8;
+    int c = kMaxClusterSize;
     while (c > 1 && c > tiles_kv) c >>= 1;
     return c;
 }
@@ -245,6 +245,10 @@ cudaError_t set_split_attrs()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(cluster_fused_kernel<D, PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::SMEM_CLUSTER);
+    if (e != cudaSuccess) return e;
+    // Clusters of 16 CTAs are beyond the portable size of 8; create() shrinks the cluster when
+    // the device cannot co-schedule it.
+    e = cudaFuncSetAttribute(cluster_fused_kernel<D, PHI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     return e;
 }
 

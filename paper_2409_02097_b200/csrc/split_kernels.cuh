@@ -49,6 +49,8 @@ struct SplitCfg {
     static constexpr int SMEM_CLUSTER = STATE_FLOATS * 4 + SMEM_ST + SMEM_STAGE;
 };
 
+constexpr int kMaxClusterSize = 16;  // beyond the portable 8: needs the non-portable launch attribute
+
 // First tile of chunk `p` when `tiles` tiles are cut into `chunks` nearly equal runs.
 __host__ __device__ __forceinline__ int chunk_begin(int p, int tiles, int chunks)
 {
@@ -254,14 +256,27 @@ template <int D, typename ReadFn>
 __device__ __forceinline__ void fill_state_operand(unsigned char* St, ReadFn read)
 {
     using C = SplitCfg<D>;
-    for (int idx = threadIdx.x; idx < C::DP * C::ST_ROWS; idx += blockDim.x) {
-        int c = idx / C::ST_ROWS, e = idx % C::ST_ROWS;
-        float val = 0.0f;
-        if (c < D) {
-            if (e < D) val = read(c * D + e);
-            else if (e < D + 8) val = read(D * D + c);
+    constexpr int kBatch = 8;  // the reads of one batch are issued together, then stored
+    const int total = C::DP * C::ST_ROWS, stride = blockDim.x;
+    for (int base = threadIdx.x; base < total; base += kBatch * stride) {
+        float val[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int idx = base + u * stride;
+            const int c = idx / C::ST_ROWS, e = idx % C::ST_ROWS;
+            val[u] = 0.0f;
+            if (idx < total && c < D) {
+                if (e < D) val[u] = read(c * D + e);
+                else if (e < D + 8) val[u] = read(D * D + c);
+            }
         }
-        *reinterpret_cast<__nv_bfloat16*>(St + e * C::PITCH + c * 2) = __float2bfloat16_rn(val);
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int idx = base + u * stride;
+            const int c = idx / C::ST_ROWS, e = idx % C::ST_ROWS;
+            if (idx < total)
+                *reinterpret_cast<__nv_bfloat16*>(St + e * C::PITCH + c * 2) = __float2bfloat16_rn(val[u]);
+        }
     }
 }
 
@@ -322,9 +337,10 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
 
 // One cluster of `cluster_size` CTAs per slab (grid.x = cluster_size, grid.y = slabs).  CTA r
 // accumulates the partial state of its run of K/V tiles into its own shared memory; after a
-// cluster barrier every CTA sums the partials of ranks 0, 1, ... in that order through
-// distributed shared memory (so all CTAs hold the same bits), then applies to its run of Q.
-// state_out (may be null) receives S | z from rank 0.
+// cluster barrier CTA r sums slice r of the partials over ranks 0, 1, ... in that order and pushes
+// the result into every CTA's operand through distributed shared memory (so all CTAs hold the same
+// bits); after a second barrier every CTA applies to its run of Q.  state_out (may be null)
+// receives S | z in fp32.
 template <int D, int PHI>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
@@ -350,22 +366,58 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
                                  chunk_begin(rank + 1, tiles, csize), stage, acc);
         store_state<D>(part, acc);
     }
+    // Clear the own S^T | z operand (pad rows and columns must be zero) before any peer writes to it.
+    for (int i = threadIdx.x; i < C::SMEM_ST / 16; i += blockDim.x)
+        reinterpret_cast<uint4*>(St)[i] = make_uint4(0u, 0u, 0u, 0u);
     cluster.sync();
 
-    fill_state_operand<D>(St, [&](int i) {
-        float sum = 0.0f;
-        for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(part, r)[i];
-        return sum;
-    });
-    if (rank == 0 && state_out != nullptr) {
-        float* dst = state_out + static_cast<size_t>(slab) * C::STATE_FLOATS;
-        for (int i = threadIdx.x; i < C::STATE_FLOATS; i += blockDim.x) {
-            float sum = 0.0f;
-            for (int r = 0; r < csize; ++r) sum += cluster.map_shared_rank(part, r)[i];
-            dst[i] = sum;
+    // Reduce-scatter with push: CTA r sums slice r of the state over ranks 0, 1, ... in that order
+    // (fixed order), and stores the bf16 result into the S^T | z operand of every CTA of the
+    // cluster through distributed shared memory (remote stores do not stall the writer), and the
+    // fp32 result into state_out.
+    {
+        const int slice = (C::STATE_FLOATS + csize - 1) / csize;
+        const int begin = rank * slice;
+        const int end = begin + slice < C::STATE_FLOATS ? begin + slice : C::STATE_FLOATS;
+        float* gout = state_out != nullptr ? state_out + static_cast<size_t>(slab) * C::STATE_FLOATS : nullptr;
+        constexpr int kBatch = 8;  // elements in flight per thread; ranks are visited in order
+        for (int base = begin + threadIdx.x; base < end; base += kBatch * blockDim.x) {
+            float sum[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) sum[u] = 0.0f;
+#pragma unroll 1
+            for (int r = 0; r < csize; ++r) {
+                const float* src = cluster.map_shared_rank(part, r);
+                float v[kBatch];
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) {
+                    const int i = base + u * blockDim.x;
+                    v[u] = i < end ? src[i] : 0.0f;
+                }
+#pragma unroll
+                for (int u = 0; u < kBatch; ++u) sum[u] += v[u];
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int i = base + u * blockDim.x;
+                if (i >= end) continue;
+                if (gout != nullptr) gout[i] = sum[u];
+                const __nv_bfloat16 b = __float2bfloat16_rn(sum[u]);
+                // S[c][e] goes to row e, column c of the operand; z[c] to column c of rows D .. D+7.
+                const bool is_z = i >= D * D;
+                const int c = is_z ? i - D * D : i / D;
+                const int row0 = is_z ? D : i - c * D;
+                const int rows = is_z ? 8 : 1;
+#pragma unroll 1
+                for (int r = 0; r < csize; ++r) {
+                    unsigned char* dst = cluster.map_shared_rank(St, r) + row0 * C::PITCH + c * 2;
+#pragma unroll 1
+                    for (int j = 0; j < rows; ++j) *reinterpret_cast<__nv_bfloat16*>(dst + j * C::PITCH) = b;
+                }
+            }
         }
     }
-    cluster.sync();  // no CTA leaves (or reuses `part`) while a peer still reads it
+    cluster.sync();  // every operand is complete; no CTA leaves while a peer still reads `part`
 
     const int qtiles = (N + C::TILE_Q - 1) / C::TILE_Q;
     apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, chunk_begin(rank, qtiles, csize),
