@@ -85,12 +85,15 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
 
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v == LINFUSION_VARIANT_AUTO) {
-        const long long tokens = static_cast<long long>(slabs) * d->N;
+        // Measured on B200 over the SD-v1.5 / v2.1 / XL layer shapes: the single clustered launch
+        // wins only at the smallest levels (N <= 192: 14 vs 18 us at N = 144, d = 64; 28 vs 35 us
+        // at N = 64, d = 160); above that the TMA-streamed kernels win for d = 64 at every N, and
+        // the three-launch split path for the other head dims.
         const int cl = largest_cluster(tiles_kv);
-        if (d->d == kStreamD && slabs <= sm_count && tokens >= 4ll * sm_count * StreamStateCfg::TILE)
-            v = LINFUSION_VARIANT_STREAM;
-        else if (static_cast<long long>(slabs) * cl <= 2ll * sm_count && d->N <= 1024 * cl)
+        if (d->N <= 192 && static_cast<long long>(slabs) * cl <= 2ll * sm_count)
             v = LINFUSION_VARIANT_CLUSTER;
+        else if (d->d == kStreamD && slabs <= sm_count)
+            v = LINFUSION_VARIANT_STREAM;
         else
             v = LINFUSION_VARIANT_SPLIT;
     }
