@@ -139,6 +139,30 @@ linfusion_status_t linfusion_attn_status(linfusion_attn_t* h);
 linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host, float* z_host);
 
 /*
+ * Token-sharded (sequence-parallel) use — the distributed inference of Sec. 4.3: every device
+ * owns a run of the tokens of Q, K, V and Y (desc.N is the local token count), and the only
+ * quantity exchanged is the state S | z, whose size does not depend on N.  Per layer:
+ *
+ *   1. linfusion_attn_state(h, k_local, v_local, stream)   S, z of the local K/V tokens
+ *                                                           (split-N kernel + fixed-order reduction)
+ *   2. the caller sums the fp32 buffer returned by linfusion_attn_state_buffer() over all devices,
+ *      in place, on the same stream (e.g. an NCCL all-reduce; the state is additive over token
+ *      shards, Prop. 2)
+ *   3. linfusion_attn_apply(h, q_local, y_local, stream)    Y of the local Q tokens from the
+ *                                                           summed state
+ *
+ * state_buffer: *dev_ptr is the device address of [B*H][d*d S (row = feature c of K, column =
+ * channel e of V), then d z] fp32, *floats its length; it stays valid until the handle is
+ * destroyed or its workspace is replaced.  Handles that resolved to the clustered single-launch
+ * variant cannot be split in two: state() and apply() return UNSUPPORTED for them (create the
+ * handle with LINFUSION_VARIANT_SPLIT or _STREAM).  Other errors as for forward().
+ */
+linfusion_status_t linfusion_attn_state(linfusion_attn_t* h, const void* k, const void* v,
+                                        void* cuda_stream);
+linfusion_status_t linfusion_attn_apply(linfusion_attn_t* h, const void* q, void* y, void* cuda_stream);
+linfusion_status_t linfusion_attn_state_buffer(linfusion_attn_t* h, float** dev_ptr, size_t* floats);
+
+/*
  * Per-kernel timing for benchmarks.  enable(h, slots > 0) creates `slots` sets of CUDA events;
  * from then on every forward() brackets each of its kernels with event records on its stream
  * (set = call index modulo slots).  enable(h, 0) turns it off.  kernel_times() synchronizes the

@@ -26,6 +26,7 @@ EXPORTED = [
     "linfusion_attn_variant_name", "linfusion_attn_launches_per_forward",
     "linfusion_attn_enable_kernel_timing", "linfusion_attn_kernel_times",
     "linfusion_attn_forward_noalloc",
+    "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
 ]
 
 
@@ -86,6 +87,12 @@ def load_library() -> ctypes.CDLL:
                                                 ctypes.POINTER(ctypes.c_int32)]
     lib.linfusion_attn_forward_noalloc.restype = st
     lib.linfusion_attn_forward_noalloc.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp]
+    lib.linfusion_attn_state.restype = st
+    lib.linfusion_attn_state.argtypes = [vp, vp, vp, vp]
+    lib.linfusion_attn_apply.restype = st
+    lib.linfusion_attn_apply.argtypes = [vp, vp, vp, vp]
+    lib.linfusion_attn_state_buffer.restype = st
+    lib.linfusion_attn_state_buffer.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
     _lib = lib
     return lib
 
@@ -215,6 +222,40 @@ class LinFusionAttention:
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_read_state")
         return S, z
+
+    # -- token-sharded use (Sec. 4.3): state of the local K/V, caller's sum, apply to the local Q --
+    def state(self, k, v, stream: Optional[int] = None) -> None:
+        import torch
+        for t, n in ((k, "k"), (v, "v")):
+            self._check(t, n)
+        if stream is None:
+            stream = torch.cuda.current_stream(k.device).cuda_stream
+        rc = self._lib.linfusion_attn_state(self._h, k.data_ptr(), v.data_ptr(), stream)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_state")
+
+    def apply(self, q, y=None, stream: Optional[int] = None):
+        import torch
+        self._check(q, "q")
+        if y is None:
+            y = torch.empty_like(q)
+        else:
+            self._check(y, "y")
+        if stream is None:
+            stream = torch.cuda.current_stream(q.device).cuda_stream
+        rc = self._lib.linfusion_attn_apply(self._h, q.data_ptr(), y.data_ptr(), stream)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_apply")
+        return y
+
+    def state_buffer(self):
+        """(device address, number of floats) of the fp32 S | z buffer: [B*H][d*d + d]."""
+        ptr = ctypes.c_void_p()
+        n = ctypes.c_size_t(0)
+        rc = self._lib.linfusion_attn_state_buffer(self._h, ctypes.byref(ptr), ctypes.byref(n))
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_state_buffer")
+        return int(ptr.value or 0), int(n.value)
 
     def enable_kernel_timing(self, slots: int) -> None:
         rc = self._lib.linfusion_attn_enable_kernel_timing(self._h, int(slots))

@@ -863,3 +863,118 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     }
     return LINFUSION_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Token-sharded (sequence-parallel) use, Sec. 4.3: every device owns a run of the tokens of Q, K, V
+// and Y, builds the state of its own K/V tokens, the devices sum their S | z (the only exchange,
+// d x (d+1) floats per slab whatever N is), and each applies the summed state to its own Q tokens.
+// The library runs the two halves; the sum over devices is the caller's collective on the buffer
+// that linfusion_attn_state_buffer() exposes.
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+template <int D, int PHI>
+cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a,
+                              const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s)
+{
+    using C = SplitCfg<D>;
+    const Plan& p = h->plan;
+    const int N = h->desc.N;
+    if (state_half) {
+        state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
+            a, b, h->partials, N, p.chunks_state);
+        state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
+            h->partials, h->state, C::STATE_FLOATS, p.chunks_state);
+    } else {
+        apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
+            a, h->state, y, N, p.chunks_apply, h->desc.eps);
+    }
+    return cudaGetLastError();
+}
+
+template <int PHI>
+cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a,
+                               const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s)
+{
+    const Plan& p = h->plan;
+    const int N = h->desc.N;
+    const dim3 rgrid((kStreamStateFloats + 255) / 256, p.slabs);
+    if (state_half) {
+        CUtensorMap mk, mv;
+        if (!encode_slab_map(&mk, a, p.slabs, N, StreamStateCfg::TILE) ||
+            !encode_slab_map(&mv, b, p.slabs, N, StreamStateCfg::TILE))
+            return cudaErrorInvalidValue;
+        stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
+            mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans);
+        stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->frags, h->tile_counters,
+                                                  p.tiles_state, p.W_state, p.G_state, p.spans);
+    } else {
+        CUtensorMap mq;
+        if (!encode_slab_map(&mq, a, p.slabs, N, ApplyCfg::TILE)) return cudaErrorInvalidValue;
+        // The state may have been summed over devices since the reduction: rebuild its bf16 image.
+        stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->frags, h->tile_counters);
+        stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
+            mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps);
+    }
+    return cudaGetLastError();
+}
+
+linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, const void* b, void* y,
+                            void* cuda_stream)
+{
+    if (h == nullptr || a == nullptr || (state_half ? b == nullptr : y == nullptr))
+        return LINFUSION_ERR_INVALID_ARG;
+    if (h->plan.variant == kCluster) return LINFUSION_ERR_UNSUPPORTED;
+    const uintptr_t pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b),
+                    py = reinterpret_cast<uintptr_t>(y);
+    if (((pa | pb | py) & 15u) != 0) return LINFUSION_ERR_INVALID_ARG;
+    const size_t bytes = static_cast<size_t>(h->plan.slabs) * h->desc.N * h->desc.d * 2;
+    if (!state_half && pa < py + bytes && py < pa + bytes) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    const __nv_bfloat16* A = static_cast<const __nv_bfloat16*>(a);
+    const __nv_bfloat16* B = static_cast<const __nv_bfloat16*>(b);
+    __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
+    const bool ident = h->desc.phi == LINFUSION_PHI_IDENTITY;
+    cudaError_t e = cudaErrorInvalidValue;
+    if (h->plan.variant == kStream) {
+        e = ident ? launch_stream_half<kPhiIdentity>(h, state_half, A, B, Y, s)
+                  : launch_stream_half<kPhiEluPlusOne>(h, state_half, A, B, Y, s);
+    } else {
+#define LF_HALF(DV)                                                                    \
+    e = ident ? launch_split_half<DV, kPhiIdentity>(h, state_half, A, B, Y, s)         \
+              : launch_split_half<DV, kPhiEluPlusOne>(h, state_half, A, B, Y, s)
+        LF_DISPATCH_D(h->desc.d, LF_HALF)
+#undef LF_HALF
+    }
+    h->last_stream = s;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
+
+}  // namespace
+
+extern "C" linfusion_status_t linfusion_attn_state(linfusion_attn_t* h, const void* k, const void* v,
+                                                   void* cuda_stream)
+{
+    return run_half(h, true, k, v, nullptr, cuda_stream);
+}
+
+extern "C" linfusion_status_t linfusion_attn_apply(linfusion_attn_t* h, const void* q, void* y,
+                                                   void* cuda_stream)
+{
+    return run_half(h, false, q, nullptr, y, cuda_stream);
+}
+
+extern "C" linfusion_status_t linfusion_attn_state_buffer(linfusion_attn_t* h, float** dev_ptr,
+                                                          size_t* floats)
+{
+    if (h == nullptr || dev_ptr == nullptr || floats == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    *dev_ptr = h->state;
+    *floats = static_cast<size_t>(h->plan.slabs) * h->plan.state_floats;
+    return LINFUSION_OK;
+}

@@ -249,6 +249,33 @@ __host__ __device__ __forceinline__ int apply_channel_of(int nb, int g8)
     return 32 * (nb >> 2) + 8 * (g8 >> 1) + 2 * (nb & 3) + (g8 & 1);
 }
 
+// Block blockIdx.x of a (17, slabs) grid of 256 threads holds elements 256*blockIdx.x .. of one
+// slab's fp32 state (S rows 4*blockIdx.x .., or z in block 16) in `sums`; write their share of the
+// fragment image `fr` of that slab.
+__device__ __forceinline__ void emit_state_fragments(const float* sums, uint32_t* fr)
+{
+    const int tid = threadIdx.x;
+    if (blockIdx.x < 16) {
+        // rows c = 4*blockIdx.x + tid/64 of S; even rows pack (S[c][e], S[c+1][e])
+        const int r = tid >> 6, e = tid & 63;
+        if ((r & 1) == 0) {
+            const int c = 4 * blockIdx.x + r;
+            const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 64]);
+            const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
+            const int r32 = e & 31;
+            const int nb = 4 * (e >> 5) + ((r32 & 7) >> 1);
+            const int g8 = 2 * (r32 >> 3) + (r32 & 1);
+            fr[((kb * 5 + (nb >> 1)) * 32 + g8 * 4 + t4) * 4 + (nb & 1) * 2 + reg] = pair;
+        }
+    } else if (tid < 64 && (tid & 1) == 0) {
+        // z: pair (z[c], z[c+1]) goes to every column slot of block 8
+        const int c = tid;
+        const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 1]);
+        const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
+        for (int g8 = 0; g8 < 8; ++g8) fr[((kb * 5 + 4) * 32 + g8 * 4 + t4) * 4 + reg] = pair;
+    }
+}
+
 // grid (17, slabs), 256 threads: state[slab] = sum over the CTAs whose run meets the slab, in
 // increasing CTA index, half 0 then half 1 (fp32, fixed order).  Also writes the bf16 fragment
 // image of S | z for the apply kernel and clears the slab's tile counter for it.
@@ -287,27 +314,24 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
     }
     sums[tid] = sum;
     __syncthreads();
+    emit_state_fragments(sums, frags + static_cast<size_t>(slab) * kStreamFragWords);
+}
 
-    uint32_t* fr = frags + static_cast<size_t>(slab) * kStreamFragWords;
-    if (blockIdx.x < 16) {
-        // rows c = 4*blockIdx.x + tid/64 of S; even rows pack (S[c][e], S[c+1][e])
-        const int r = tid >> 6, e = tid & 63;
-        if ((r & 1) == 0) {
-            const int c = 4 * blockIdx.x + r;
-            const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 64]);
-            const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
-            const int r32 = e & 31;
-            const int nb = 4 * (e >> 5) + ((r32 & 7) >> 1);
-            const int g8 = 2 * (r32 >> 3) + (r32 & 1);
-            fr[((kb * 5 + (nb >> 1)) * 32 + g8 * 4 + t4) * 4 + (nb & 1) * 2 + reg] = pair;
-        }
-    } else if (tid < 64 && (tid & 1) == 0) {
-        // z: pair (z[c], z[c+1]) goes to every column slot of block 8
-        const int c = tid;
-        const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 1]);
-        const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
-        for (int g8 = 0; g8 < 8; ++g8) fr[((kb * 5 + 4) * 32 + g8 * 4 + t4) * 4 + reg] = pair;
-    }
+// grid (17, slabs), 256 threads: rebuild the bf16 fragment image (and clear the tile counters) from
+// an fp32 state that was changed outside the library — the sum over devices of a token-sharded
+// forward (Sec. 4.3).
+__global__ void __launch_bounds__(256)
+stream_pack_kernel(const float* __restrict__ state, uint32_t* __restrict__ frags,
+                   int* __restrict__ tile_counters)
+{
+    __shared__ float sums[256];
+    const int tid = threadIdx.x;
+    const int idx = blockIdx.x * 256 + tid;
+    const int slab = blockIdx.y;
+    if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
+    sums[tid] = idx < kStreamStateFloats ? state[static_cast<size_t>(slab) * kStreamStateFloats + idx] : 0.0f;
+    __syncthreads();
+    emit_state_fragments(sums, frags + static_cast<size_t>(slab) * kStreamFragWords);
 }
 
 // ---------------------------------------------------------------------------------------------
