@@ -201,6 +201,18 @@ struct linfusion_attn {
     cudaEvent_t* events;
     int timing_slots;
     long long timed_calls;
+    struct HostPipe* pipe;  // copy/compute pipeline of the host-buffer entry point (first use)
+};
+
+// forward_host() cuts the slabs into groups and overlaps the upload of group i+1, the kernels of
+// group i and the download of group i-1 on three streams.
+constexpr int kMaxHostGroups = 8;
+struct HostPipe {
+    int groups = 1;
+    linfusion_attn* sub = nullptr;  // handle for one group of slabs (null when groups == 1)
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t entry = nullptr, out = nullptr;
+    cudaEvent_t in[kMaxHostGroups] = {}, done[kMaxHostGroups] = {};
 };
 
 namespace {
@@ -449,6 +461,7 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     h->events = nullptr;
     h->timing_slots = 0;
     h->timed_calls = 0;
+    h->pipe = nullptr;
     st = make_plan(desc, h->sm_count, &h->plan);
     if (st != LINFUSION_OK) {
         delete h;
@@ -638,16 +651,81 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
         }
     }
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
-    // K and V first: they feed the first kernel.
-    if (cudaMemcpyAsync(h->stage[1], k_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(h->stage[2], v_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-        cudaMemcpyAsync(h->stage[0], q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
-        cudaGetLastError();
-        return LINFUSION_ERR_CUDA;
+    if (h->pipe == nullptr) {
+        // First use: decide the grouping, make the group handle, the copy streams and the events.
+        HostPipe* p = new (std::nothrow) HostPipe();
+        if (p == nullptr) return LINFUSION_ERR_ALLOC;
+        const int slabs = h->plan.slabs;
+        for (int g = kMaxHostGroups; g >= 2; --g)
+            if (slabs % g == 0 && bytes / g >= (size_t(32) << 20)) {
+                p->groups = g;
+                break;
+            }
+        bool ok = true;
+        if (p->groups > 1) {
+            linfusion_attn_desc_t d = h->desc;
+            d.B = 1;
+            d.H = slabs / p->groups;
+            d.flags = static_cast<uint32_t>(h->plan.variant);
+            ok = linfusion_attn_create(&d, &p->sub) == LINFUSION_OK;
+            ok = ok && cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) == cudaSuccess;
+            ok = ok && cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) == cudaSuccess;
+            ok = ok && cudaEventCreateWithFlags(&p->entry, cudaEventDisableTiming) == cudaSuccess;
+            ok = ok && cudaEventCreateWithFlags(&p->out, cudaEventDisableTiming) == cudaSuccess;
+            for (int i = 0; ok && i < p->groups; ++i)
+                ok = cudaEventCreateWithFlags(&p->in[i], cudaEventDisableTiming) == cudaSuccess &&
+                     cudaEventCreateWithFlags(&p->done[i], cudaEventDisableTiming) == cudaSuccess;
+        }
+        if (!ok) {
+            cudaGetLastError();
+            p->groups = 1;  // fall back to one group on the caller's stream
+        }
+        h->pipe = p;
     }
-    linfusion_status_t st = linfusion_attn_forward(h, h->stage[0], h->stage[1], h->stage[2], h->stage[3], s);
-    if (st != LINFUSION_OK) return st;
-    if (cudaMemcpyAsync(y_host, h->stage[3], bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+    HostPipe* p = h->pipe;
+    if (p->groups == 1) {
+        // K and V first: they feed the first kernel.
+        if (cudaMemcpyAsync(h->stage[1], k_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(h->stage[2], v_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(h->stage[0], q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+        linfusion_status_t st = linfusion_attn_forward(h, h->stage[0], h->stage[1], h->stage[2], h->stage[3], s);
+        if (st != LINFUSION_OK) return st;
+        if (cudaMemcpyAsync(y_host, h->stage[3], bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+        return LINFUSION_OK;
+    }
+
+    // Uploads run ahead on copy_in, kernels follow on the caller's stream, downloads trail on
+    // copy_out; everything is ordered after the caller's earlier work and before its later work.
+    const size_t gbytes = bytes / p->groups;
+    auto at = [&](const void* base, int i) { return static_cast<const unsigned char*>(base) + i * gbytes; };
+    auto dev = [&](int which, int i) { return static_cast<unsigned char*>(h->stage[which]) + i * gbytes; };
+    bool ok = cudaEventRecord(p->entry, s) == cudaSuccess &&
+              cudaStreamWaitEvent(p->copy_in, p->entry, 0) == cudaSuccess &&
+              cudaStreamWaitEvent(p->copy_out, p->entry, 0) == cudaSuccess;
+    for (int i = 0; ok && i < p->groups; ++i) {
+        ok = cudaMemcpyAsync(dev(1, i), at(k_host, i), gbytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
+             cudaMemcpyAsync(dev(2, i), at(v_host, i), gbytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
+             cudaMemcpyAsync(dev(0, i), at(q_host, i), gbytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
+             cudaEventRecord(p->in[i], p->copy_in) == cudaSuccess &&
+             cudaStreamWaitEvent(s, p->in[i], 0) == cudaSuccess;
+        if (!ok) break;
+        linfusion_status_t st = linfusion_attn_forward(p->sub, dev(0, i), dev(1, i), dev(2, i), dev(3, i), s);
+        if (st != LINFUSION_OK) return st;
+        ok = cudaEventRecord(p->done[i], s) == cudaSuccess &&
+             cudaStreamWaitEvent(p->copy_out, p->done[i], 0) == cudaSuccess &&
+             cudaMemcpyAsync(static_cast<unsigned char*>(y_host) + i * gbytes, dev(3, i), gbytes,
+                             cudaMemcpyDeviceToHost, p->copy_out) == cudaSuccess;
+    }
+    ok = ok && cudaEventRecord(p->out, p->copy_out) == cudaSuccess &&
+         cudaStreamWaitEvent(s, p->out, 0) == cudaSuccess;
+    h->last_stream = s;
+    if (!ok) {
         cudaGetLastError();
         return LINFUSION_ERR_CUDA;
     }
@@ -668,7 +746,9 @@ linfusion_status_t linfusion_attn_status(linfusion_attn_t* h)
         cudaGetLastError();
         return LINFUSION_ERR_CUDA;
     }
-    return word == kStatusOk ? LINFUSION_OK : LINFUSION_ERR_TIMEOUT;
+    if (word != kStatusOk) return LINFUSION_ERR_TIMEOUT;
+    if (h->pipe != nullptr && h->pipe->sub != nullptr) return linfusion_attn_status(h->pipe->sub);
+    return LINFUSION_OK;
 }
 
 linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host, float* z_host)
@@ -723,6 +803,19 @@ linfusion_status_t linfusion_attn_destroy(linfusion_attn_t* h)
         if (h->events != nullptr) {
             for (int i = 0; i < h->timing_slots * 4; ++i) cudaEventDestroy(h->events[i]);
             delete[] h->events;
+        }
+        if (h->pipe != nullptr) {
+            HostPipe* p = h->pipe;
+            if (p->sub != nullptr && linfusion_attn_destroy(p->sub) != LINFUSION_OK) st = LINFUSION_ERR_CUDA;
+            if (p->copy_in != nullptr) cudaStreamDestroy(p->copy_in);
+            if (p->copy_out != nullptr) cudaStreamDestroy(p->copy_out);
+            if (p->entry != nullptr) cudaEventDestroy(p->entry);
+            if (p->out != nullptr) cudaEventDestroy(p->out);
+            for (int i = 0; i < kMaxHostGroups; ++i) {
+                if (p->in[i] != nullptr) cudaEventDestroy(p->in[i]);
+                if (p->done[i] != nullptr) cudaEventDestroy(p->done[i]);
+            }
+            delete p;
         }
     } else {
         st = LINFUSION_ERR_CUDA;
@@ -845,6 +938,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     view.events = nullptr;
     view.timing_slots = 0;
     view.timed_calls = 0;
+    view.pipe = nullptr;
 
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const __nv_bfloat16* Q = static_cast<const __nv_bfloat16*>(q);

@@ -217,3 +217,26 @@ def test_forward_argument_errors_touch_no_memory():
         attn.LinFusionAttention(1, 1, 256, 64, device=torch.cuda.device_count())
     assert e.value.code == attn.ERR_INVALID_ARG
     op.close()
+
+
+def test_forward_host_pipelined_groups():
+    """Large enough for the grouped copy/compute pipeline of forward_host (5 groups of 4 slabs)."""
+    B, H, N, d = 2, 10, 65536, 64
+    q, k, v = wl.make_small(B, H, N, d, seed=19, device="cpu")
+    qp, kp, vp = (t.pin_memory() for t in (q, k, v))
+    yp = torch.full_like(qp, float("nan")).pin_memory()
+    op = attn.LinFusionAttention(B, H, N, d)
+    op.forward_host(qp, kp, vp, yp)
+    torch.cuda.synchronize()
+    first = yp.clone()
+    op.forward_host(qp, kp, vp, yp)          # second call: same bits, buffers reused
+    torch.cuda.synchronize()
+    assert op.status() == attn.OK
+    assert torch.equal(first.view(torch.int16), yp.view(torch.int16))
+    y_dev = op.forward(q.cuda(), k.cuda(), v.cuda())
+    torch.cuda.synchronize()
+    diff = (yp.float() - y_dev.cpu().float()).abs()
+    assert diff.max().item() <= 2e-3                      # same math, different split of N
+    for b, h in [(0, 0), (1, 9), (1, 4)]:
+        assert_parity(yp[b, h], oracle_y(q[b, h], k[b, h], v[b, h]), f"forward_host[{b},{h}]")
+    op.close()
