@@ -56,6 +56,15 @@ typedef enum {
 #define LINFUSION_VARIANT_STREAM 2u  /* three launches, TMA-pipelined persistent kernels (d = 64 only)    */
 #define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N)               */
 #define LINFUSION_VARIANT_MASK 0xFu
+/*
+ * flags: memory layout of Q, K, V and Y.  Default (bit clear): head-major [B, H, N, d].  Bit set:
+ * token-major [B, N, H, d] — the [B, N, C] tensor a UNet block holds, with C = H*d split into
+ * heads in place — so that the caller needs no transpose before or after the attention (a
+ * transpose pass would move twice the attention's own minimum traffic).  Every entry point that
+ * takes a descriptor or a handle follows it; the arithmetic and its order are the same, so Y has
+ * the same bits as in the head-major layout.
+ */
+#define LINFUSION_LAYOUT_TOKEN_MAJOR 0x10u
 
 typedef struct {
     int32_t B;      /* batch                                   > 0 */
@@ -65,7 +74,7 @@ typedef struct {
     int32_t phi;    /* linfusion_phi_t                             */
     float eps;      /* finite, >= 0; added once to phi(Q_i) . z    */
     int32_t device; /* CUDA device ordinal the handle lives on     */
-    uint32_t flags; /* LINFUSION_VARIANT_*                         */
+    uint32_t flags; /* LINFUSION_VARIANT_* | LINFUSION_LAYOUT_*      */
 } linfusion_attn_desc_t;
 
 /*

@@ -101,8 +101,16 @@ def status_string(code: int) -> str:
     return load_library().linfusion_status_string(int(code)).decode()
 
 
-def make_desc(B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto") -> Desc:
+LAYOUT_TOKEN_MAJOR = 0x10   # tensors are [B, N, H, d] instead of [B, H, N, d]
+
+
+def make_desc(B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
+              layout="head_major") -> Desc:
     flags = VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    if layout == "token_major":
+        flags |= LAYOUT_TOKEN_MAJOR
+    elif layout != "head_major":
+        raise ValueError("layout must be 'head_major' or 'token_major'")
     return Desc(int(B), int(H), int(N), int(d), int(phi), float(eps), int(device), flags)
 
 
@@ -156,11 +164,15 @@ def linfusion_attn_destroy(handle) -> None:
 
 
 class LinFusionAttention:
-    """One handle per shape.  ``forward`` takes bf16 CUDA tensors [B, H, N, d]."""
+    """One handle per shape.  ``forward`` takes bf16 CUDA tensors [B, H, N, d] (or [B, N, H, d]
+    with ``layout="token_major"``)."""
 
-    def __init__(self, B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto"):
-        self.desc = make_desc(B, H, N, d, phi, eps, device, variant)
-        self.shape = (int(B), int(H), int(N), int(d))
+    def __init__(self, B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
+                 layout="head_major"):
+        self.desc = make_desc(B, H, N, d, phi, eps, device, variant, layout)
+        # tensors are [B, H, N, d], or [B, N, H, d] in the token-major layout
+        self.shape = (int(B), int(H), int(N), int(d)) if layout == "head_major" else \
+                     (int(B), int(N), int(H), int(d))
         self._lib = load_library()
         self._h = linfusion_attn_create(self.desc)
         self._lent_ws = None
@@ -215,7 +227,7 @@ class LinFusionAttention:
     def read_state(self):
         """(S [B,H,d,d], z [B,H,d]) of the last forward as fp32 numpy arrays."""
         import numpy as np
-        B, H, _, d = self.shape
+        B, H, d = self.desc.B, self.desc.H, self.desc.d
         S = np.empty((B, H, d, d), dtype=np.float32)
         z = np.empty((B, H, d), dtype=np.float32)
         rc = self._lib.linfusion_attn_read_state(self._h, S.ctypes.data, z.ctypes.data)

@@ -22,6 +22,21 @@ constexpr uint32_t kStatusWaitExpired = 1u;
 // an error word instead of a hang.
 constexpr uint32_t kMaxBarrierPolls = 1u << 16;
 
+// Where the rows of one (batch, head) slab sit in a tensor, in elements.  Head-major [B,H,N,d]:
+// batch_stride = H*N*d, head_stride = N*d, row_stride = d.  Token-major [B,N,H,d] (what a UNet
+// holds before it splits heads): batch_stride = N*H*d, head_stride = d, row_stride = H*d.
+struct SlabLayout {
+    long long batch_stride;
+    long long head_stride;
+    int row_stride;
+    int H;
+};
+
+__host__ __device__ __forceinline__ size_t slab_base(const SlabLayout& L, int slab)
+{
+    return static_cast<size_t>(slab / L.H) * L.batch_stride + static_cast<size_t>(slab % L.H) * L.head_stride;
+}
+
 // ---------------------------------------------------------------------------------------------
 // phi (Sec. 2.2: non-negative activation on the K and Q features).  elu(x) + 1:
 // x + 1 for x > 0, exp(x) otherwise; both branches give 1 at 0.  exp(min(x, 0)) is 1 on the
@@ -207,6 +222,18 @@ __device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* tmap, in
         "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
         "[%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(smem_u32(smem_dst)),
         "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(cache_policy)
+        : "memory");
+}
+
+// 4-D variant: coordinates (x, y, z, w) = (channel, token, head, batch), so that head-major and
+// token-major tensors differ only in the strides of the tensor map.
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, int x, int y, int z, int w,
+                                            uint64_t* bar, uint64_t cache_policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3, %4, %5}], [%6], %7;" ::"r"(smem_u32(smem_dst)),
+        "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(w), "r"(smem_u32(bar)), "l"(cache_policy)
         : "memory");
 }
 

@@ -57,7 +57,7 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
     if (!supported_d(d->d)) return LINFUSION_ERR_UNSUPPORTED;
     if (d->phi != LINFUSION_PHI_ELU_PLUS_ONE && d->phi != LINFUSION_PHI_IDENTITY)
         return LINFUSION_ERR_UNSUPPORTED;
-    if ((d->flags & ~LINFUSION_VARIANT_MASK) != 0u) return LINFUSION_ERR_UNSUPPORTED;
+    if ((d->flags & ~(LINFUSION_VARIANT_MASK | LINFUSION_LAYOUT_TOKEN_MAJOR)) != 0u) return LINFUSION_ERR_UNSUPPORTED;
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v > LINFUSION_VARIANT_CLUSTER) return LINFUSION_ERR_UNSUPPORTED;
     if (v == LINFUSION_VARIANT_STREAM && d->d != kStreamD) return LINFUSION_ERR_UNSUPPORTED;
@@ -165,18 +165,37 @@ EncodeTiledFn get_encode_fn()
     return fn;
 }
 
-// bf16 [slabs][N][64] -> boxes of [1][tile_rows][64], 128-byte swizzle, zero fill past N.
-bool encode_slab_map(CUtensorMap* map, const void* base, int slabs, int N, int tile_rows)
+// Element strides of a slab's rows for the layout the descriptor asks for.
+SlabLayout layout_of(const linfusion_attn_desc_t& d)
+{
+    SlabLayout L;
+    L.H = d.H;
+    if ((d.flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u) {  // [B, N, H, d]
+        L.batch_stride = static_cast<long long>(d.N) * d.H * d.d;
+        L.head_stride = d.d;
+        L.row_stride = d.H * d.d;
+    } else {  // [B, H, N, d]
+        L.batch_stride = static_cast<long long>(d.H) * d.N * d.d;
+        L.head_stride = static_cast<long long>(d.N) * d.d;
+        L.row_stride = d.d;
+    }
+    return L;
+}
+
+// bf16 tensor seen as (channel 64, token N, head H, batch B) -> boxes of tile_rows tokens of one
+// (b, h) slab, 128-byte swizzle, zero fill past N.  The layout only changes the strides.
+bool encode_slab_map(CUtensorMap* map, const void* base, const linfusion_attn_desc_t& d, int tile_rows)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (fn == nullptr) return false;
-    cuuint64_t dims[3] = {static_cast<cuuint64_t>(kStreamD), static_cast<cuuint64_t>(N),
-                          static_cast<cuuint64_t>(slabs)};
-    cuuint64_t strides[2] = {static_cast<cuuint64_t>(kStreamRowBytes),
-                             static_cast<cuuint64_t>(N) * kStreamRowBytes};
-    cuuint32_t box[3] = {static_cast<cuuint32_t>(kStreamD), static_cast<cuuint32_t>(tile_rows), 1u};
-    cuuint32_t estr[3] = {1u, 1u, 1u};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box,
+    const SlabLayout L = layout_of(d);
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(kStreamD), static_cast<cuuint64_t>(d.N),
+                          static_cast<cuuint64_t>(d.H), static_cast<cuuint64_t>(d.B)};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(L.row_stride) * 2, static_cast<cuuint64_t>(L.head_stride) * 2,
+                             static_cast<cuuint64_t>(L.batch_stride) * 2};
+    cuuint32_t box[4] = {static_cast<cuuint32_t>(kStreamD), static_cast<cuuint32_t>(tile_rows), 1u, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
@@ -288,13 +307,13 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
     const int N = h->desc.N;
     mark(h, 0, s);
     state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
-        k, v, h->partials, N, p.chunks_state);
+        k, v, h->partials, N, p.chunks_state, layout_of(h->desc));
     mark(h, 1, s);
     state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
         h->partials, h->state, C::STATE_FLOATS, p.chunks_state);
     mark(h, 2, s);
     apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-        q, h->state, y, N, p.chunks_apply, h->desc.eps);
+        q, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc));
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -326,7 +345,7 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
     cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
     mark(h, 0, s);
     cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state,
-                                       h->desc.N, h->desc.eps);
+                                       h->desc.N, h->desc.eps, layout_of(h->desc));
     mark(h, 1, s);
     return e;
 }
@@ -338,19 +357,19 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
     const Plan& p = h->plan;
     const int N = h->desc.N;
     CUtensorMap mq, mk, mv;
-    if (!encode_slab_map(&mk, k, p.slabs, N, StreamStateCfg::TILE) ||
-        !encode_slab_map(&mv, v, p.slabs, N, StreamStateCfg::TILE) ||
-        !encode_slab_map(&mq, q, p.slabs, N, ApplyCfg::TILE))
+    if (!encode_slab_map(&mk, k, h->desc, StreamStateCfg::TILE) ||
+        !encode_slab_map(&mv, v, h->desc, StreamStateCfg::TILE) ||
+        !encode_slab_map(&mq, q, h->desc, ApplyCfg::TILE))
         return cudaErrorInvalidValue;
     mark(h, 0, s);
     stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
-        mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans);
+        mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
     mark(h, 1, s);
     stream_reduce_kernel<<<dim3((kStreamStateFloats + 255) / 256, p.slabs), 256, 0, s>>>(
         h->partials, h->state, h->frags, h->tile_counters, p.tiles_state, p.W_state, p.G_state, p.spans);
     mark(h, 2, s);
     stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-        mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps);
+        mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps, layout_of(h->desc));
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -656,7 +675,9 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
         HostPipe* p = new (std::nothrow) HostPipe();
         if (p == nullptr) return LINFUSION_ERR_ALLOC;
         const int slabs = h->plan.slabs;
-        for (int g = kMaxHostGroups; g >= 2; --g)
+        // Groups are runs of whole slabs, which are contiguous in memory only in the head-major layout.
+        const bool head_major = (h->desc.flags & LINFUSION_LAYOUT_TOKEN_MAJOR) == 0u;
+        for (int g = kMaxHostGroups; head_major && g >= 2; --g)
             if (slabs % g == 0 && bytes / g >= (size_t(32) << 20)) {
                 p->groups = g;
                 break;
@@ -666,7 +687,7 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
             linfusion_attn_desc_t d = h->desc;
             d.B = 1;
             d.H = slabs / p->groups;
-            d.flags = static_cast<uint32_t>(h->plan.variant);
+            d.flags = static_cast<uint32_t>(h->plan.variant);  // head-major only (see the grouping rule above)
             ok = linfusion_attn_create(&d, &p->sub) == LINFUSION_OK;
             ok = ok && cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) == cudaSuccess;
             ok = ok && cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) == cudaSuccess;
@@ -919,7 +940,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     // and every state element that is read in this call is written earlier in the same call.
     linfusion_attn view;
     view.desc = *desc;
-    view.desc.flags = LINFUSION_VARIANT_SPLIT;
+    view.desc.flags = (desc->flags & LINFUSION_LAYOUT_TOKEN_MAJOR) | LINFUSION_VARIANT_SPLIT;
     st = make_plan(&view.desc, dev.sm_count, &view.plan);
     if (st != LINFUSION_OK) return st;
     const size_t room = (kNoAllocScratchBytes - state_bytes - 256) / per_chunk;
@@ -976,12 +997,12 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
     const int N = h->desc.N;
     if (state_half) {
         state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
-            a, b, h->partials, N, p.chunks_state);
+            a, b, h->partials, N, p.chunks_state, layout_of(h->desc));
         state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
             h->partials, h->state, C::STATE_FLOATS, p.chunks_state);
     } else {
         apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-            a, h->state, y, N, p.chunks_apply, h->desc.eps);
+            a, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc));
     }
     return cudaGetLastError();
 }
@@ -995,20 +1016,20 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
     const dim3 rgrid((kStreamStateFloats + 255) / 256, p.slabs);
     if (state_half) {
         CUtensorMap mk, mv;
-        if (!encode_slab_map(&mk, a, p.slabs, N, StreamStateCfg::TILE) ||
-            !encode_slab_map(&mv, b, p.slabs, N, StreamStateCfg::TILE))
+        if (!encode_slab_map(&mk, a, h->desc, StreamStateCfg::TILE) ||
+            !encode_slab_map(&mv, b, h->desc, StreamStateCfg::TILE))
             return cudaErrorInvalidValue;
         stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
-            mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans);
+            mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
         stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->frags, h->tile_counters,
                                                   p.tiles_state, p.W_state, p.G_state, p.spans);
     } else {
         CUtensorMap mq;
-        if (!encode_slab_map(&mq, a, p.slabs, N, ApplyCfg::TILE)) return cudaErrorInvalidValue;
+        if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE)) return cudaErrorInvalidValue;
         // The state may have been summed over devices since the reduction: rebuild its bf16 image.
         stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->frags, h->tile_counters);
         stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-            mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps);
+            mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps, layout_of(h->desc));
     }
     return cudaGetLastError();
 }

@@ -63,7 +63,7 @@ __host__ __device__ __forceinline__ int chunk_begin(int p, int tiles, int chunks
 // ---------------------------------------------------------------------------------------------
 template <int D, int PHI>
 __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict__ Ks,
-                                                 const __nv_bfloat16* __restrict__ Vs, int N,
+                                                 const __nv_bfloat16* __restrict__ Vs, int N, int rs,
                                                  int tile0, int tile1, unsigned char* smem_kv,
                                                  float (&acc)[SplitCfg<D>::NBT][4])
 {
@@ -87,8 +87,8 @@ __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict
             int row = idx / C::CH, ch = idx % C::CH;
             long long j = static_cast<long long>(tile) * C::TILE_KV + row;
             bool ok = (j < N) && (ch * 8 < D);
-            kreg[i] = ok ? ld_stream_16B(Ks + j * D + ch * 8) : zero4;
-            vreg[i] = ok ? ld_stream_16B(Vs + j * D + ch * 8) : zero4;
+            kreg[i] = ok ? ld_stream_16B(Ks + j * rs + ch * 8) : zero4;
+            vreg[i] = ok ? ld_stream_16B(Vs + j * rs + ch * 8) : zero4;
         }
     };
     auto store_tile = [&](int tile) {
@@ -166,7 +166,7 @@ __device__ __forceinline__ void store_state(float* dst, const float (&acc)[Split
 // ---------------------------------------------------------------------------------------------
 template <int D, int PHI>
 __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs,
-                                            __nv_bfloat16* __restrict__ Ys, int N, int tile0,
+                                            __nv_bfloat16* __restrict__ Ys, int N, int rs, int tile0,
                                             int tile1, const unsigned char* St, unsigned char* Qsm,
                                             float eps)
 {
@@ -183,7 +183,7 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
             int row = idx / C::CH, ch = idx % C::CH;
             long long r = static_cast<long long>(tile) * C::TILE_Q + row;
             bool ok = (r < N) && (ch * 8 < D);
-            qreg[i] = ok ? ld_stream_16B(Qs + r * D + ch * 8) : zero4;
+            qreg[i] = ok ? ld_stream_16B(Qs + r * rs + ch * 8) : zero4;
         }
     };
     auto store_tile = [&](int tile) {
@@ -242,8 +242,8 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
 #pragma unroll
         for (int nb = 0; nb < C::NBV; ++nb) {
             int e = nb * 8 + 2 * t;
-            if (r0 < N) st_stream_4B(Ys + r0 * D + e, pack_bf16x2(acc[nb][0] * inv0, acc[nb][1] * inv0));
-            if (r1 < N) st_stream_4B(Ys + r1 * D + e, pack_bf16x2(acc[nb][2] * inv1, acc[nb][3] * inv1));
+            if (r0 < N) st_stream_4B(Ys + r0 * rs + e, pack_bf16x2(acc[nb][0] * inv0, acc[nb][1] * inv0));
+            if (r1 < N) st_stream_4B(Ys + r1 * rs + e, pack_bf16x2(acc[nb][2] * inv1, acc[nb][3] * inv1));
         }
         __syncthreads();
     }
@@ -288,15 +288,15 @@ __device__ __forceinline__ void fill_state_operand(unsigned char* St, ReadFn rea
 template <int D, int PHI>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 state_partial_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
-                     float* __restrict__ partials, int N, int chunks)
+                     float* __restrict__ partials, int N, int chunks, SlabLayout L)
 {
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
     const int slab = blockIdx.y, p = blockIdx.x;
     const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;
-    const size_t slab_off = static_cast<size_t>(slab) * N * D;
+    const size_t slab_off = slab_base(L, slab);
     float acc[C::NBT][4];
-    accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, chunk_begin(p, tiles, chunks),
+    accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
                              chunk_begin(p + 1, tiles, chunks), smem, acc);
     store_state<D>(partials + (static_cast<size_t>(slab) * chunks + p) * C::STATE_FLOATS, acc);
 }
@@ -319,7 +319,7 @@ state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ stat
 template <int D, int PHI>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ state,
-             __nv_bfloat16* __restrict__ Y, int N, int chunks, float eps)
+             __nv_bfloat16* __restrict__ Y, int N, int chunks, float eps, SlabLayout L)
 {
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -330,8 +330,8 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
     const float* st = state + static_cast<size_t>(slab) * C::STATE_FLOATS;
     fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); });
     __syncthreads();
-    const size_t slab_off = static_cast<size_t>(slab) * N * D;
-    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, chunk_begin(p, tiles, chunks),
+    const size_t slab_off = slab_base(L, slab);
+    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
                         chunk_begin(p + 1, tiles, chunks), St, Qsm, eps);
 }
 
@@ -345,7 +345,7 @@ template <int D, int PHI>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                      const __nv_bfloat16* __restrict__ V, __nv_bfloat16* __restrict__ Y,
-                     float* __restrict__ state_out, int N, float eps)
+                     float* __restrict__ state_out, int N, float eps, SlabLayout L)
 {
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -357,12 +357,12 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
     const int rank = static_cast<int>(cluster.block_rank());
     const int csize = static_cast<int>(cluster.num_blocks());
     const int slab = blockIdx.y;
-    const size_t slab_off = static_cast<size_t>(slab) * N * D;
+    const size_t slab_off = slab_base(L, slab);
 
     {
         const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;
         float acc[C::NBT][4];
-        accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, chunk_begin(rank, tiles, csize),
+        accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, L.row_stride, chunk_begin(rank, tiles, csize),
                                  chunk_begin(rank + 1, tiles, csize), stage, acc);
         store_state<D>(part, acc);
     }
@@ -420,7 +420,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
     cluster.sync();  // every operand is complete; no CTA leaves while a peer still reads `part`
 
     const int qtiles = (N + C::TILE_Q - 1) / C::TILE_Q;
-    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, chunk_begin(rank, qtiles, csize),
+    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(rank, qtiles, csize),
                         chunk_begin(rank + 1, qtiles, csize), St, stage, eps);
 }
 

@@ -91,7 +91,7 @@ template <int PHI>
 __global__ void __launch_bounds__(StreamStateCfg::THREADS, StreamStateCfg::CTAS_PER_SM)
 stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, float* __restrict__ partials,
-                    uint32_t* __restrict__ status, int N, int tiles_per_slab, long long W, int spans)
+                    uint32_t* __restrict__ status, int N, int tiles_per_slab, long long W, int spans, int H)
 {
     using C = StreamStateCfg;
     extern __shared__ unsigned char smem_raw[];
@@ -133,8 +133,8 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                 const int tile = static_cast<int>(u % tiles_per_slab);
                 unsigned char* dst = smem + s * C::STAGE_BYTES;
                 mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                tma_load_3d(dst, &tmap_k, 0, tile * C::TILE, slab, &full[s], policy);
-                tma_load_3d(dst + C::TILE_BYTES, &tmap_v, 0, tile * C::TILE, slab, &full[s], policy);
+                tma_load_4d(dst, &tmap_k, 0, tile * C::TILE, slab % H, slab / H, &full[s], policy);
+                tma_load_4d(dst + C::TILE_BYTES, &tmap_v, 0, tile * C::TILE, slab % H, slab / H, &full[s], policy);
                 ++issued;
             }
             drain_loads<C::STAGES>(full, 0, issued, status);
@@ -344,7 +344,7 @@ template <int PHI, int CW>
 __global__ void __launch_bounds__(StreamApplyCfg<CW>::THREADS, 1)
 stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* __restrict__ frags,
                     __nv_bfloat16* __restrict__ Y, int* __restrict__ tile_counters,
-                    uint32_t* __restrict__ status, int N, int tiles_per_slab, int slabs, float eps)
+                    uint32_t* __restrict__ status, int N, int tiles_per_slab, int slabs, float eps, SlabLayout L)
 {
     using C = StreamApplyCfg<CW>;
     extern __shared__ unsigned char smem_raw[];
@@ -400,7 +400,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* 
                 if (ok) {
                     meta[s] = make_int2(slab, tile);
                     mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                    tma_load_3d(smem + s * C::STAGE_BYTES, &tmap_q, 0, tile * C::TILE, slab, &full[s], policy);
+                    tma_load_4d(smem + s * C::STAGE_BYTES, &tmap_q, 0, tile * C::TILE, slab % L.H, slab / L.H, &full[s], policy);
                     ++issued;
                 } else {
                     report_wait_expired(status);
@@ -493,8 +493,8 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* 
         const float inv0 = 1.0f / (acc[8][0] + eps);
         const float inv1 = 1.0f / (acc[8][2] + eps);
         const long long r0 = static_cast<long long>(tile) * C::TILE + warp * 16 + g8, r1 = r0 + 8;
-        __nv_bfloat16* y0 = Y + (static_cast<size_t>(slab) * N + r0) * 64;
-        __nv_bfloat16* y1 = y0 + 8 * 64;
+        __nv_bfloat16* y0 = Y + slab_base(L, slab) + static_cast<size_t>(r0) * L.row_stride;
+        __nv_bfloat16* y1 = y0 + 8 * static_cast<size_t>(L.row_stride);
 #pragma unroll
         for (int hi = 0; hi < 2; ++hi) {
             uint4 v0, v1;

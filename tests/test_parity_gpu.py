@@ -240,3 +240,33 @@ def test_forward_host_pipelined_groups():
     for b, h in [(0, 0), (1, 9), (1, 4)]:
         assert_parity(yp[b, h], oracle_y(q[b, h], k[b, h], v[b, h]), f"forward_host[{b},{h}]")
     op.close()
+
+
+@pytest.mark.parametrize("dims,variant", [((2, 10, 4100, 64), "stream"), ((2, 8, 1000, 40), "split"),
+                                          ((1, 4, 130, 160), "cluster"), ((2, 5, 100, 64), "cluster"),
+                                          ((1, 3, 2049, 80), "auto")], ids=lambda x: str(x))
+def test_token_major_layout_gives_the_same_bits(dims, variant):
+    """[B, N, H, d] tensors (a UNet's [B, N, C] with heads split in place): same arithmetic in the
+    same order as the head-major layout, so the outputs must agree bit for bit."""
+    B, H, N, d = dims
+    q, k, v = wl.make_small(B, H, N, d, seed=23, device="cuda")
+    y_hm, op = run_gpu(q, k, v, variant)
+    resolved = op.variant
+    op.close()
+    tm = lambda t: t.permute(0, 2, 1, 3).contiguous()
+    op = attn.LinFusionAttention(B, H, N, d, eps=EPS, variant=resolved, layout="token_major")
+    y_tm = op.forward(tm(q), tm(k), tm(v))
+    torch.cuda.synchronize()
+    assert op.status() == attn.OK
+    assert y_tm.shape == (B, N, H, d)
+    assert torch.equal(y_tm.permute(0, 2, 1, 3).contiguous().view(torch.int16), y_hm.view(torch.int16))
+    assert_parity(y_tm.permute(0, 2, 1, 3), oracle_y(q, k, v), f"token-major {dims} {variant}")
+    # the allocation-free entry point follows the layout flag too
+    if d != 160 or B * H <= 81:
+        y2 = torch.empty_like(y_tm)
+        desc = attn.make_desc(B, H, N, d, eps=EPS, layout="token_major")
+        attn.linfusion_attn_forward_noalloc(desc, tm(q).data_ptr(), tm(k).data_ptr(), tm(v).data_ptr(),
+                                            y2.data_ptr(), torch.cuda.current_stream().cuda_stream)
+        torch.cuda.synchronize()
+        assert_parity(y2.permute(0, 2, 1, 3), oracle_y(q, k, v), f"token-major noalloc {dims}")
+    op.close()
