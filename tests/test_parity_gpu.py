@@ -255,7 +255,8 @@ def test_token_major_layout_gives_the_same_bits(dims, variant):
     op.close()
     tm = lambda t: t.permute(0, 2, 1, 3).contiguous()
     op = attn.LinFusionAttention(B, H, N, d, eps=EPS, variant=resolved, layout="token_major")
-    y_tm = op.forward(tm(q), tm(k), tm(v))
+    qt, kt, vt = tm(q), tm(k), tm(v)
+    y_tm = op.forward(qt, kt, vt)
     torch.cuda.synchronize()
     assert op.status() == attn.OK
     assert y_tm.shape == (B, N, H, d)
@@ -265,7 +266,7 @@ def test_token_major_layout_gives_the_same_bits(dims, variant):
     if d != 160 or B * H <= 81:
         y2 = torch.empty_like(y_tm)
         desc = attn.make_desc(B, H, N, d, eps=EPS, layout="token_major")
-        attn.linfusion_attn_forward_noalloc(desc, tm(q).data_ptr(), tm(k).data_ptr(), tm(v).data_ptr(),
+        attn.linfusion_attn_forward_noalloc(desc, qt.data_ptr(), kt.data_ptr(), vt.data_ptr(),
                                             y2.data_ptr(), torch.cuda.current_stream().cuda_stream)
         torch.cuda.synchronize()
         assert_parity(y2.permute(0, 2, 1, 3), oracle_y(q, k, v), f"token-major noalloc {dims}")
