@@ -237,8 +237,10 @@ def run_cuda(args):
     layers = []
     for i, s in enumerate(shapes):
         q, k, v = wl.make_qkv(s, seed=wl.BASE_SEED + 100 * rank + i, device=f"cuda:{local_rank}")
+        if args.layout == "token_major":          # [B, N, H, d]: what a UNet holds before splitting heads
+            q, k, v = (t.permute(0, 2, 1, 3).contiguous() for t in (q, k, v))
         y = torch.empty_like(q)
-        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank)
+        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank, layout=args.layout)
         layers.append((s, op, q, k, v, y))
     tokens_per_step = sum(s.tokens for s in shapes)
     launches_per_step = sum(op.launches_per_forward for _, op, *_ in layers)
@@ -346,6 +348,7 @@ def run_cuda(args):
                                   for s in shapes],
                        "variant": [op.variant for _, op, *_ in layers],
                        "l2": "inputs larger than L2 (%.2f GB touched per step)" % (step_bytes / 1e9),
+                       "layout": args.layout,
                        "parallelism": f"independent batches x{world}"},
             "tokens_per_s_per_gpu": value / world,
             "hbm_gbs_whole_path": path_gbs,
@@ -423,6 +426,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layout", default="head_major", choices=["head_major", "token_major"],
+                    help="[B,H,N,d] (default, the benchmark's layout) or [B,N,H,d]")
     ap.add_argument("--sweep", action="store_true",
                     help="time every shape of the five workload families with every variant")
     args = ap.parse_args()
