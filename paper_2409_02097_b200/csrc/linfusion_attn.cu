@@ -195,9 +195,14 @@ bool encode_slab_map(CUtensorMap* map, const void* base, const linfusion_attn_de
                              static_cast<cuuint64_t>(L.batch_stride) * 2};
     cuuint32_t box[4] = {static_cast<cuuint32_t>(kStreamD), static_cast<cuuint32_t>(tile_rows), 1u, 1u};
     cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    // Head-major rows of a slab are contiguous: let L2 fetch 256 bytes per miss.  Token-major rows
+    // are 128-byte segments between other heads' data: fetch only what this CTA will use.
+    const CUtensorMapL2promotion promo = (d.flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u
+                                             ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B
+                                             : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
