@@ -212,21 +212,10 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
     return false;
 }
 
-// 3-D tiled TMA load: box at (x, y, z) = (channel, token, slab) of the tensor map -> shared
-// memory, completion counted in bytes on `bar`.  x * element size must be a multiple of 16 bytes
-// (the kernels here always pass x = 0).
-__device__ __forceinline__ void tma_load_3d(void* smem_dst, const void* tmap, int x, int y, int z,
-                                            uint64_t* bar, uint64_t cache_policy)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
-        "[%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(smem_u32(smem_dst)),
-        "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(smem_u32(bar)), "l"(cache_policy)
-        : "memory");
-}
-
-// 4-D variant: coordinates (x, y, z, w) = (channel, token, head, batch), so that head-major and
-// token-major tensors differ only in the strides of the tensor map.
+// 4-D tiled TMA load: box at (x, y, z, w) = (channel, token, head, batch) of the tensor map ->
+// shared memory, completion counted in bytes on `bar`; head-major and token-major tensors differ
+// only in the strides of the tensor map.  x * element size must be a multiple of 16 bytes (the
+// kernels here always pass x = 0).
 __device__ __forceinline__ void tma_load_4d(void* smem_dst, const void* tmap, int x, int y, int z, int w,
                                             uint64_t* bar, uint64_t cache_policy)
 {
