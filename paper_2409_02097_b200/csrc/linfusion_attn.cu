@@ -92,12 +92,11 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         const int cl = largest_cluster(tiles_kv);
         if (d->N <= 192 && static_cast<long long>(slabs) * cl <= 2ll * sm_count)
             v = LINFUSION_VARIANT_CLUSTER;
-        else if (d->d == kStreamD && slabs <= sm_count)
+        else if (d->d == kStreamD)
             v = LINFUSION_VARIANT_STREAM;
         else
             v = LINFUSION_VARIANT_SPLIT;
     }
-    if (v == LINFUSION_VARIANT_STREAM && slabs > sm_count) return LINFUSION_ERR_UNSUPPORTED;
     p->variant = static_cast<int>(v);
 
     size_t partial_floats = 0;
@@ -117,7 +116,6 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         p->G_state = static_cast<int>(gs < p->W_state ? gs : p->W_state);
         long long ga = sm_count;
         p->G_apply = static_cast<int>(ga < p->W_apply ? ga : p->W_apply);
-        if (p->G_apply < slabs) p->G_apply = slabs;  // every slab is some CTA's home
         int spans = 1;
         for (int g = 0; g < p->G_state; ++g) {
             long long b = unit_begin(g, p->W_state, p->G_state);

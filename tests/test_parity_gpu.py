@@ -81,6 +81,8 @@ EDGE_CASES = [
     (1, 1, 1, 64), (1, 1, 1, 40), (1, 3, 7, 160), (2, 1, 63, 64), (1, 2, 65, 64),
     (1, 1, 127, 64), (1, 1, 129, 64), (1, 5, 191, 64), (1, 1, 193, 64), (3, 1, 1000, 80),
     (1, 7, 333, 40), (1, 1, 4097, 128), (2, 3, 257, 32), (1, 2, 12289, 64), (1, 148, 64, 64),
+    (8, 25, 300, 64),   # more slabs than SMs
+
 ]
 
 
