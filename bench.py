@@ -376,7 +376,7 @@ def run_sweep(args):
     seen = set()
     for cfg_idx, cfg in enumerate(wl.CONFIGS):
         for s in cfg:
-            if s.name in seen:
+            if s.name in seen or (args.only and s.name != args.only):
                 continue
             seen.add(s.name)
             sets = max(1, min(64, -(-400_000_000 // s.min_bytes)))
@@ -430,6 +430,7 @@ def main():
                     help="[B,H,N,d] (default, the benchmark's layout) or [B,N,H,d]")
     ap.add_argument("--sweep", action="store_true",
                     help="time every shape of the five workload families with every variant")
+    ap.add_argument("--only", default="", help="with --sweep: restrict to one shape, e.g. sd15_512_L1")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
