@@ -136,8 +136,13 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     p->partial_bytes = align_up(partial_floats * sizeof(float), 256);
     p->state_off = p->partial_bytes;
     p->frags_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
-    // Stream variant only: bf16 fragment image of S | z and one tile counter per slab.
-    const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM ? static_cast<size_t>(slabs) * kStreamFragWords * 4 : 0;
+    // bf16 operand image of S | z for the apply kernel (stream: MMA fragment order; split: its
+    // shared-memory layout), and for the stream variant one tile counter per slab.
+    const int dp = (d->d + 15) / 16 * 16;
+    const size_t split_image = static_cast<size_t>((d->d + 8 + 15) / 16 * 16) * (((dp / 8) | 1) * 16);
+    const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamFragWords * 4
+                              : v == LINFUSION_VARIANT_SPLIT ? static_cast<size_t>(slabs) * split_image
+                                                             : 0;
     const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM ? align_up(static_cast<size_t>(slabs) * 4, 256) : 0;
     p->counters_off = p->frags_off + align_up(frag_bytes, 256);
     p->status_off = p->counters_off + counter_bytes;
@@ -312,11 +317,13 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
     state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
         k, v, h->partials, N, p.chunks_state, layout_of(h->desc));
     mark(h, 1, s);
+    // h->frags (when the workspace has it) receives the apply kernel's bf16 operand image.
+    unsigned char* image = reinterpret_cast<unsigned char*>(h->frags);
     state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
-        h->partials, h->state, C::STATE_FLOATS, p.chunks_state);
+        h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST);
     mark(h, 2, s);
     apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-        q, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc));
+        q, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc), image);
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -1002,10 +1009,11 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
         state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
             a, b, h->partials, N, p.chunks_state, layout_of(h->desc));
         state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
-            h->partials, h->state, C::STATE_FLOATS, p.chunks_state);
+            h->partials, h->state, C::STATE_FLOATS, p.chunks_state, nullptr, D, C::PITCH, C::SMEM_ST);
     } else {
+        // The fp32 state may have been summed over devices: convert it here, not from an image.
         apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-            a, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc));
+            a, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc), nullptr);
     }
     return cudaGetLastError();
 }

@@ -301,10 +301,13 @@ state_partial_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* _
     store_state<D>(partials + (static_cast<size_t>(slab) * chunks + p) * C::STATE_FLOATS, acc);
 }
 
-// grid (ceil(state_floats / 256), slabs).  Sums `chunks` partials per slab in index order.
+// grid (ceil(state_floats / 256), slabs).  Sums `chunks` partials per slab in index order.  If
+// `st_image` is not null it also receives the bf16 S^T | z operand of the apply kernel, laid out
+// exactly as that kernel holds it in shared memory (`image_bytes` per slab, rows `pitch` bytes
+// apart: row e < d holds S[.][e], rows d .. d+7 hold z; pad bytes stay as the host zeroed them).
 __global__ void __launch_bounds__(256)
 state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state, int state_floats,
-                    int chunks)
+                    int chunks, unsigned char* __restrict__ st_image, int d, int pitch, int image_bytes)
 {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= state_floats) return;
@@ -313,13 +316,26 @@ state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ stat
     float sum = 0.0f;
     for (int p = 0; p < chunks; ++p) sum += src[static_cast<size_t>(p) * state_floats];
     state[static_cast<size_t>(slab) * state_floats + idx] = sum;
+    if (st_image != nullptr) {
+        unsigned char* img = st_image + static_cast<size_t>(slab) * image_bytes;
+        const __nv_bfloat16 b = __float2bfloat16_rn(sum);
+        if (idx < d * d) {
+            const int c = idx / d, e = idx - c * d;
+            *reinterpret_cast<__nv_bfloat16*>(img + e * pitch + c * 2) = b;
+        } else {
+            const int c = idx - d * d;
+            for (int j = 0; j < 8; ++j) *reinterpret_cast<__nv_bfloat16*>(img + (d + j) * pitch + c * 2) = b;
+        }
+    }
 }
 
-// grid (chunks, slabs).
+// grid (chunks, slabs).  `st_image` (may be null) is the operand image written by
+// state_reduce_kernel; without it every CTA converts the fp32 state itself.
 template <int D, int PHI>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ state,
-             __nv_bfloat16* __restrict__ Y, int N, int chunks, float eps, SlabLayout L)
+             __nv_bfloat16* __restrict__ Y, int N, int chunks, float eps, SlabLayout L,
+             const unsigned char* __restrict__ st_image)
 {
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -327,8 +343,15 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
     unsigned char* Qsm = smem + C::SMEM_ST;
     const int slab = blockIdx.y, p = blockIdx.x;
     const int tiles = (N + C::TILE_Q - 1) / C::TILE_Q;
-    const float* st = state + static_cast<size_t>(slab) * C::STATE_FLOATS;
-    fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); });
+    if (st_image != nullptr) {
+        // The reduction kernel left the operand in its shared-memory layout: plain 16-byte copy.
+        const uint4* img = reinterpret_cast<const uint4*>(st_image + static_cast<size_t>(slab) * C::SMEM_ST);
+        for (int i = threadIdx.x; i < C::SMEM_ST / 16; i += blockDim.x)
+            reinterpret_cast<uint4*>(St)[i] = __ldg(img + i);
+    } else {
+        const float* st = state + static_cast<size_t>(slab) * C::STATE_FLOATS;
+        fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); });
+    }
     __syncthreads();
     const size_t slab_off = slab_base(L, slab);
     apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
