@@ -15,8 +15,7 @@ using namespace lf;
 namespace {
 
 constexpr int kDefaultSmCount = 148;
-constexpr int kStreamApplyWarps = 11;
-using ApplyCfg = StreamApplyCfg<kStreamApplyWarps>;
+using ApplyCfg = StreamApplyCfg;
 
 enum Variant { kSplit = 1, kStream = 2, kCluster = 3 };
 
@@ -41,7 +40,7 @@ struct Plan {
     // cluster
     int cluster_size = 0;
     // workspace (bytes, offsets)
-    size_t partial_bytes = 0, state_off = 0, frags_off = 0, counters_off = 0, status_off = 0, total_bytes = 0;
+    size_t partial_bytes = 0, state_off = 0, operand_off = 0, counters_off = 0, status_off = 0, total_bytes = 0;
     int launches = 0;
 };
 
@@ -135,16 +134,16 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     }
     p->partial_bytes = align_up(partial_floats * sizeof(float), 256);
     p->state_off = p->partial_bytes;
-    p->frags_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
-    // bf16 operand image of S | z for the apply kernel (stream: MMA fragment order; split: its
-    // shared-memory layout), and for the stream variant one tile counter per slab.
+    p->operand_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
+    // bf16 operand image of S | z for the apply kernel (in its shared-memory layout), and for the
+    // stream variant one tile counter per slab.
     const int dp = (d->d + 15) / 16 * 16;
     const size_t split_image = static_cast<size_t>((d->d + 8 + 15) / 16 * 16) * (((dp / 8) | 1) * 16);
-    const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamFragWords * 4
+    const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamOperandBytes
                               : v == LINFUSION_VARIANT_SPLIT ? static_cast<size_t>(slabs) * split_image
                                                              : 0;
     const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM ? align_up(static_cast<size_t>(slabs) * 4, 256) : 0;
-    p->counters_off = p->frags_off + align_up(frag_bytes, 256);
+    p->counters_off = p->operand_off + align_up(frag_bytes, 256);
     p->status_off = p->counters_off + counter_bytes;
     p->total_bytes = p->status_off + 256;
     return LINFUSION_OK;
@@ -219,7 +218,7 @@ struct linfusion_attn {
     bool owns_ws;
     float* partials;
     float* state;
-    uint32_t* frags;
+    unsigned char* operand;  // bf16 operand image of S | z for the apply kernels
     int* tile_counters;
     uint32_t* status;
     cudaStream_t last_stream;
@@ -250,7 +249,7 @@ void bind_workspace(linfusion_attn* h, void* ws)
     unsigned char* base = static_cast<unsigned char*>(ws);
     h->partials = reinterpret_cast<float*>(base);
     h->state = reinterpret_cast<float*>(base + h->plan.state_off);
-    h->frags = reinterpret_cast<uint32_t*>(base + h->plan.frags_off);
+    h->operand = base + h->plan.operand_off;
     h->tile_counters = reinterpret_cast<int*>(base + h->plan.counters_off);
     h->status = reinterpret_cast<uint32_t*>(base + h->plan.status_off);
 }
@@ -301,7 +300,7 @@ cudaError_t set_stream_attrs()
     e = cudaFuncSetAttribute(stream_state_kernel<PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              StreamStateCfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(stream_apply_kernel<PHI, kStreamApplyWarps>,
+    e = cudaFuncSetAttribute(stream_apply_kernel<PHI>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg::SMEM_BYTES);
     return e;
 }
@@ -317,8 +316,8 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
     state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
         k, v, h->partials, N, p.chunks_state, layout_of(h->desc));
     mark(h, 1, s);
-    // h->frags (when the workspace has it) receives the apply kernel's bf16 operand image.
-    unsigned char* image = reinterpret_cast<unsigned char*>(h->frags);
+    // h->operand (when the workspace has it) receives the apply kernel's bf16 operand image.
+    unsigned char* image = h->operand;
     state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
         h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST);
     mark(h, 2, s);
@@ -366,20 +365,20 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
 {
     const Plan& p = h->plan;
     const int N = h->desc.N;
-    CUtensorMap mq, mk, mv;
+    CUtensorMap mq, mk, mv, my;
     if (!encode_slab_map(&mk, k, h->desc, StreamStateCfg::TILE) ||
         !encode_slab_map(&mv, v, h->desc, StreamStateCfg::TILE) ||
-        !encode_slab_map(&mq, q, h->desc, ApplyCfg::TILE))
+        !encode_slab_map(&mq, q, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
         return cudaErrorInvalidValue;
     mark(h, 0, s);
     stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
         mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
     mark(h, 1, s);
     stream_reduce_kernel<<<dim3((kStreamStateFloats + 255) / 256, p.slabs), 256, 0, s>>>(
-        h->partials, h->state, h->frags, h->tile_counters, p.tiles_state, p.W_state, p.G_state, p.spans);
+        h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state, p.spans);
     mark(h, 2, s);
-    stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-        mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps, layout_of(h->desc));
+    stream_apply_kernel<PHI><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
+        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, h->desc.eps, h->desc.H);
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -540,7 +539,7 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     }
     h->owns_ws = true;
     bind_workspace(h, ws);
-    if (cudaMemset(h->frags, 0, h->plan.total_bytes - h->plan.frags_off) != cudaSuccess) {
+    if (cudaMemset(h->operand, 0, h->plan.total_bytes - h->plan.operand_off) != cudaSuccess) {
         cudaFree(ws);
         delete h;
         return LINFUSION_ERR_CUDA;
@@ -560,7 +559,7 @@ linfusion_status_t linfusion_attn_set_workspace(linfusion_attn_t* h, void* dev_p
     if (h->owns_ws && h->ws != nullptr) cudaFree(h->ws);
     h->owns_ws = false;
     bind_workspace(h, dev_ptr);
-    if (cudaMemset(h->frags, 0, h->plan.total_bytes - h->plan.frags_off) != cudaSuccess) return LINFUSION_ERR_CUDA;
+    if (cudaMemset(h->operand, 0, h->plan.total_bytes - h->plan.operand_off) != cudaSuccess) return LINFUSION_ERR_CUDA;
     return LINFUSION_OK;
 }
 
@@ -961,7 +960,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     view.partials = reinterpret_cast<float*>(dev.scratch);
     view.state = reinterpret_cast<float*>(
         dev.scratch + align_up(per_chunk * static_cast<size_t>(view.plan.chunks_state), 256));
-    view.frags = nullptr;
+    view.operand = nullptr;
     view.tile_counters = nullptr;
     view.status = nullptr;
     view.last_stream = nullptr;
@@ -1032,15 +1031,16 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
             return cudaErrorInvalidValue;
         stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
             mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
-        stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->frags, h->tile_counters,
+        stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->operand, h->tile_counters,
                                                   p.tiles_state, p.W_state, p.G_state, p.spans);
     } else {
-        CUtensorMap mq;
-        if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE)) return cudaErrorInvalidValue;
+        CUtensorMap mq, my;
+        if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
+            return cudaErrorInvalidValue;
         // The state may have been summed over devices since the reduction: rebuild its bf16 image.
-        stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->frags, h->tile_counters);
-        stream_apply_kernel<PHI, kStreamApplyWarps><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-            mq, h->frags, y, h->tile_counters, h->status, N, p.tiles_apply, p.slabs, h->desc.eps, layout_of(h->desc));
+        stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->operand, h->tile_counters);
+        stream_apply_kernel<PHI><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
+            mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, h->desc.eps, h->desc.H);
     }
     return cudaGetLastError();
 }

@@ -14,18 +14,23 @@
 //                           ldmatrix.trans, phi is applied to the A fragments in registers, and a
 //                           ninth column block of ones produces z.  Each (CTA, slab, half) writes
 //                           its own fp32 partial; nothing is combined with atomics.
-//   stream_reduce_kernel  — sums the partials of a slab in (CTA, half) order; also lays S | z out
-//                           as the bf16 MMA B-fragments the apply kernel loads.
-//   stream_apply_kernel   — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps).  S | z sit in registers as
-//                           bf16 MMA B-fragments (reloaded when the CTA moves to another slab);
-//                           Q tiles are handed out per slab through an atomic counter (the
-//                           result of a tile does not depend on which CTA computes it);
-//                           A = phi(Q) comes from the stage with ldmatrix; the
-//                           columns of S are permuted so that every lane ends up with 8
-//                           contiguous output channels and stores them as one 16-byte vector.
+//   stream_reduce_kernel  — sums the partials of a slab in (CTA, half) order; also lays S^T | z out
+//                           as the bf16, K-major, 128-byte-swizzled B operand the apply kernel
+//                           copies into shared memory.
+//   stream_apply_kernel   — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps) on tcgen05: a 128-row Q tile
+//                           is one MMA tile (M = 128).  Each of the 128 threads of a warpgroup
+//                           reads its row from the stage, applies phi in packed bf16 and writes
+//                           the row to tensor memory as the A operand; one thread of the CTA
+//                           issues D[128 x 80] = A[128 x 64] * B[64 x 80] (B = S^T rows, then z,
+//                           then zero padding, from shared memory); the threads read their row
+//                           of D back, divide by the z column, write the bf16 row over the Q
+//                           row in the stage, and a TMA store sends the tile to Y.  Q tiles are
+//                           handed out per slab through an atomic counter (the result of a tile
+//                           does not depend on which CTA computes it).
 //
-// One extra warp per CTA is the TMA producer.  All mbarrier waits are bounded; a wait that
-// expires records kStatusWaitExpired in the status word and the CTA drains and exits.
+// One extra warp per CTA is the TMA producer (the apply kernel has a store warp and an MMA warp
+// too).  All mbarrier waits are bounded; a wait that expires records kStatusWaitExpired in the
+// status word and the CTA drains and exits.
 #pragma once
 
 #include "common.cuh"
@@ -47,15 +52,26 @@ struct StreamStateCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 };
 
-template <int CW>
 struct StreamApplyCfg {
-    static constexpr int CONSUMER_WARPS = CW;
-    static constexpr int TILE = 16 * CW;  // tokens per stage: one m16 block per consumer warp
-    static constexpr int THREADS = 32 * (CW + 1);
-    static constexpr int STAGE_BYTES = TILE * kStreamRowBytes;
-    static constexpr int STAGES = (198 * 1024) / STAGE_BYTES;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 512;  // + align, barriers, meta
+    static constexpr int TILE = 128;   // tokens per stage = rows of one MMA tile = TMEM lanes
+    static constexpr int GROUPS = 3;   // warpgroups, each working on its own tile
+    static constexpr int CONSUMER_WARPS = 4 * GROUPS;
+    static constexpr int PRODUCER_WARP = CONSUMER_WARPS;
+    static constexpr int STORE_WARP = CONSUMER_WARPS + 1;
+    static constexpr int MMA_WARP = CONSUMER_WARPS + 2;
+    static constexpr int THREADS = 32 * (CONSUMER_WARPS + 3);
+    static constexpr int STAGE_BYTES = TILE * kStreamRowBytes;  // 16 KB: a Q tile, later its Y tile
+    static constexpr int STAGES = 12;
+    static constexpr int B_ROWS = 80;  // N of the MMA: 64 channels of S^T, z, padding to a multiple of 16
+    static constexpr int B_BYTES = B_ROWS * kStreamRowBytes;    // 10 KB
+    static constexpr int TMEM_COLS_PER_GROUP = 128;             // A: 32 columns, D: 80
+    static constexpr int TMEM_COLS = 512;                       // a power of two >= GROUPS * 128
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + B_BYTES + 1024 /*align*/ + 1024 /*barriers, meta*/;
 };
+static_assert(StreamApplyCfg::GROUPS * StreamApplyCfg::TMEM_COLS_PER_GROUP <= StreamApplyCfg::TMEM_COLS, "TMEM budget");
+static_assert(StreamApplyCfg::STAGES >= 2 * StreamApplyCfg::GROUPS + 2, "end markers need released stages");
+// Shared memory beyond half an SM's keeps a second CTA (and its TMEM allocation) off the SM.
+static_assert(StreamApplyCfg::SMEM_BYTES > 116 * 1024, "one apply CTA per SM");
 
 // First unit of CTA g when W units are dealt to G CTAs.
 __host__ __device__ __forceinline__ long long unit_begin(long long g, long long W, long long G)
@@ -237,51 +253,42 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     if (n_units > 0) flush(slab_first, cur_slab);
 }
 
-// Operand image of S | z for the apply kernel: bf16 MMA B-fragments in the order the lanes load
-// them, [k block 4][column-block pair 5][lane 32][4 words] per slab.  Word w of pair p holds
-// register (w & 1) of column block 2p + (w >> 1); block 8 is z, block 9 does not exist.
-constexpr int kStreamFragWords = 4 * 5 * 32 * 4;
-
-// Output channel carried by column slot g8 of column block nb (nb < 8): with this permutation a
-// lane ends up owning channels 8*t4 .. 8*t4+7 (blocks 0-3) and 32+8*t4 .. (blocks 4-7) of its rows.
-__host__ __device__ __forceinline__ int apply_channel_of(int nb, int g8)
-{
-    return 32 * (nb >> 2) + 8 * (g8 >> 1) + 2 * (nb & 3) + (g8 & 1);
-}
+// Operand image of S | z for the apply kernel, per slab: the MMA's B operand in its shared-memory
+// form — 80 rows of 128 bytes, row n < 64 = column n of S (64 bf16 along c), row 64 = z, rows 65-79
+// zero; 16-byte chunk j of row n sits at chunk position j ^ (n & 7) (the 128-byte swizzle).
+constexpr int kStreamOperandBytes = StreamApplyCfg::B_BYTES;
 
 // Block blockIdx.x of a (17, slabs) grid of 256 threads holds elements 256*blockIdx.x .. of one
 // slab's fp32 state (S rows 4*blockIdx.x .., or z in block 16) in `sums`; write their share of the
-// fragment image `fr` of that slab.
-__device__ __forceinline__ void emit_state_fragments(const float* sums, uint32_t* fr)
+// operand image `img` of that slab.
+__device__ __forceinline__ void emit_state_operand(const float* sums, unsigned char* img)
 {
     const int tid = threadIdx.x;
     if (blockIdx.x < 16) {
-        // rows c = 4*blockIdx.x + tid/64 of S; even rows pack (S[c][e], S[c+1][e])
-        const int r = tid >> 6, e = tid & 63;
-        if ((r & 1) == 0) {
-            const int c = 4 * blockIdx.x + r;
-            const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 64]);
-            const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
-            const int r32 = e & 31;
-            const int nb = 4 * (e >> 5) + ((r32 & 7) >> 1);
-            const int g8 = 2 * (r32 >> 3) + (r32 & 1);
-            fr[((kb * 5 + (nb >> 1)) * 32 + g8 * 4 + t4) * 4 + (nb & 1) * 2 + reg] = pair;
+        // S rows c0 .. c0+3 are in sums[r*64 + e]; thread e < 64 writes the four values of column e
+        if (tid < 64) {
+            const int c0 = 4 * blockIdx.x, e = tid;
+            uint2 v;
+            v.x = pack_bf16x2(sums[e], sums[64 + e]);
+            v.y = pack_bf16x2(sums[128 + e], sums[192 + e]);
+            *reinterpret_cast<uint2*>(img + e * 128 + (((c0 >> 3) ^ (e & 7)) << 4) + (c0 & 7) * 2) = v;
         }
-    } else if (tid < 64 && (tid & 1) == 0) {
-        // z: pair (z[c], z[c+1]) goes to every column slot of block 8
-        const int c = tid;
-        const uint32_t pair = pack_bf16x2(sums[tid], sums[tid + 1]);
-        const int kb = c >> 4, reg = (c >> 3) & 1, t4 = (c & 7) >> 1;
-        for (int g8 = 0; g8 < 8; ++g8) fr[((kb * 5 + 4) * 32 + g8 * 4 + t4) * 4 + reg] = pair;
+    } else {
+        // z -> row 64 (64 & 7 = 0: chunks in place), zeros -> rows 65..79
+        if (tid < 32) {
+            *reinterpret_cast<uint32_t*>(img + 64 * 128 + tid * 4) = pack_bf16x2(sums[2 * tid], sums[2 * tid + 1]);
+        } else if (tid < 32 + 120) {
+            reinterpret_cast<uint4*>(img + 65 * 128)[tid - 32] = make_uint4(0u, 0u, 0u, 0u);
+        }
     }
 }
 
 // grid (17, slabs), 256 threads: state[slab] = sum over the CTAs whose run meets the slab, in
-// increasing CTA index, half 0 then half 1 (fp32, fixed order).  Also writes the bf16 fragment
+// increasing CTA index, half 0 then half 1 (fp32, fixed order).  Also writes the bf16 operand
 // image of S | z for the apply kernel and clears the slab's tile counter for it.
 __global__ void __launch_bounds__(256)
 stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
-                     uint32_t* __restrict__ frags, int* __restrict__ tile_counters,
+                     unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
                      int tiles_per_slab, long long W, int G, int spans)
 {
     __shared__ float sums[256];
@@ -314,14 +321,14 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
     }
     sums[tid] = sum;
     __syncthreads();
-    emit_state_fragments(sums, frags + static_cast<size_t>(slab) * kStreamFragWords);
+    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes);
 }
 
-// grid (17, slabs), 256 threads: rebuild the bf16 fragment image (and clear the tile counters) from
+// grid (17, slabs), 256 threads: rebuild the bf16 operand image (and clear the tile counters) from
 // an fp32 state that was changed outside the library — the sum over devices of a token-sharded
 // forward (Sec. 4.3).
 __global__ void __launch_bounds__(256)
-stream_pack_kernel(const float* __restrict__ state, uint32_t* __restrict__ frags,
+stream_pack_kernel(const float* __restrict__ state, unsigned char* __restrict__ operand,
                    int* __restrict__ tile_counters)
 {
     __shared__ float sums[256];
@@ -331,7 +338,7 @@ stream_pack_kernel(const float* __restrict__ state, uint32_t* __restrict__ frags
     if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
     sums[tid] = idx < kStreamStateFloats ? state[static_cast<size_t>(slab) * kStreamStateFloats + idx] : 0.0f;
     __syncthreads();
-    emit_state_fragments(sums, frags + static_cast<size_t>(slab) * kStreamFragWords);
+    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -339,46 +346,72 @@ stream_pack_kernel(const float* __restrict__ state, uint32_t* __restrict__ frags
 // g*slabs/G and moves to the next slab that still has tiles when one runs dry, so the CTAs of a
 // slab share its tail and early finishers help elsewhere.  Each output tile depends only on its
 // own Q rows and the slab's S | z, so the result does not depend on who computes it.
+//
+// Roles in a CTA (one CTA per SM; it owns all 512 TMEM columns):
+//   producer warp — claims tiles, copies the slab's B operand into shared memory when the slab
+//                   changes (after every posted tile has left), loads Q tiles with TMA;
+//   3 warpgroups  — group g takes the tiles posted g-th, (g+3)-th, ...; thread r of a group owns
+//                   row r of the tile = TMEM lane r (a warp may only touch the 32 lanes of its
+//                   quarter, so warp w of the CTA works on rows 32*(w%4) ..);
+//   MMA warp      — one thread issues every tcgen05.mma of the CTA, in posting order;
+//   store warp    — one thread sends finished Y tiles out with TMA, in posting order, and
+//                   releases the stage once the store has read it.
+// Per stage s: full[s] (TMA bytes landed) -> a_ready[g] (4 warps: phi(Q) rows in TMEM) ->
+// mma_done[g] (tcgen05.commit) -> y_ready[s] (4 warps: Y rows in the stage) -> empty[s].
 // ---------------------------------------------------------------------------------------------
-template <int PHI, int CW>
-__global__ void __launch_bounds__(StreamApplyCfg<CW>::THREADS, 1)
-stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* __restrict__ frags,
-                    __nv_bfloat16* __restrict__ Y, int* __restrict__ tile_counters,
-                    uint32_t* __restrict__ status, int N, int tiles_per_slab, int slabs, float eps, SlabLayout L)
+template <int PHI>
+__global__ void __launch_bounds__(StreamApplyCfg::THREADS, 1)
+stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_y,
+                    const unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
+                    uint32_t* __restrict__ status, int tiles_per_slab, int slabs, float eps, int H)
 {
-    using C = StreamApplyCfg<CW>;
+    using C = StreamApplyCfg;
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+    unsigned char* bsm = smem + C::STAGES * C::STAGE_BYTES;  // B operand, on a 1024-byte boundary
+    uint64_t* full = reinterpret_cast<uint64_t*>(bsm + C::B_BYTES);
     uint64_t* empty = full + C::STAGES;
-    int2* meta = reinterpret_cast<int2*>(empty + C::STAGES);  // (slab, tile) of each stage; slab < 0 ends
+    uint64_t* y_ready = empty + C::STAGES;
+    uint64_t* a_ready = y_ready + C::STAGES;  // per group
+    uint64_t* mma_done = a_ready + C::GROUPS;  // per group
+    int2* meta = reinterpret_cast<int2*>(mma_done + C::GROUPS);  // (slab, tile) of each stage; slab < 0 ends
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(meta + C::STAGES);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], C::CONSUMER_WARPS);
+            mbar_init(&empty[s], 1);
+            mbar_init(&y_ready[s], 4);
+        }
+        for (int g = 0; g < C::GROUPS; ++g) {
+            mbar_init(&a_ready[g], 4);
+            mbar_init(&mma_done[g], 1);
         }
         mbar_fence_init();
     }
+    if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tc_fence_before_sync();
     __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == C::CONSUMER_WARPS) {
-        // ---------------- producer warp (lane 0 issues; all lanes help to find work) ----------------
+    if (warp == C::PRODUCER_WARP) {
+        // ---------------- producer warp (lane 0 issues; all lanes help to find work and copy B) ----------------
         uint64_t policy = 0;
         if (lane == 0) {
             prefetch_tmap(&tmap_q);
             policy = policy_evict_first();
         }
         int slab = static_cast<int>((static_cast<long long>(blockIdx.x) * slabs) / gridDim.x);
-        int it = 0, issued = 0;
+        int it = 0, issued = 0, loaded_slab = -1;
         bool ok = true;
+        int next = 0;
+        if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
         while (true) {
-            int tile = 0;
-            if (lane == 0) tile = atomicAdd(&tile_counters[slab], 1);
-            tile = __shfl_sync(0xffffffffu, tile, 0);
+            const int tile = __shfl_sync(0xffffffffu, next, 0);
             if (tile >= tiles_per_slab) {
                 // Next slab, in cyclic order, whose counter has not run past its tiles.
                 int found = -1;
@@ -392,7 +425,27 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* 
                 }
                 if (found < 0) break;
                 slab = found;
+                if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
                 continue;
+            }
+            // Claim the tile after this one now: the atomic's round trip (comparable to the time a
+            // tile takes) overlaps the wait for a free stage and the copy below.
+            if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
+            if (slab != loaded_slab) {
+                // Every tile posted so far must have left (its MMAs, which read B, are then
+                // complete as well) before B is overwritten.
+                if (lane == 0) {
+                    for (int j = it > C::STAGES ? it - C::STAGES : 0; j < it && ok; ++j)
+                        ok = mbar_wait(&empty[j % C::STAGES], (j / C::STAGES) & 1);
+                    if (!ok) report_wait_expired(status);
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+                const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
+                for (int i = lane; i < C::B_BYTES / 16; i += 32) reinterpret_cast<uint4*>(bsm)[i] = __ldg(src + i);
+                fence_proxy_async_smem();
+                __syncwarp();
+                loaded_slab = slab;
             }
             const int s = it % C::STAGES;
             if (lane == 0) {
@@ -400,7 +453,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* 
                 if (ok) {
                     meta[s] = make_int2(slab, tile);
                     mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                    tma_load_4d(smem + s * C::STAGE_BYTES, &tmap_q, 0, tile * C::TILE, slab % L.H, slab / L.H, &full[s], policy);
+                    tma_load_4d(smem + s * C::STAGE_BYTES, &tmap_q, 0, tile * C::TILE, slab % H, slab / H, &full[s], policy);
                     ++issued;
                 } else {
                     report_wait_expired(status);
@@ -413,102 +466,146 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const uint32_t* 
         if (lane == 0) {
             int first = 0;
             if (ok) {
-                // End marker in the next stage (consumers leave when they see it).  Its stage held
-                // load number issued - STAGES, which the consumers have released by now.
-                const int s = it % C::STAGES;
-                if (mbar_wait(&empty[s], ((it / C::STAGES) & 1) ^ 1)) {
-                    meta[s] = make_int2(-1, 0);
-                    mbar_arrive(&full[s]);
-                    first = issued - C::STAGES + 1;
-                } else {
-                    report_wait_expired(status);
+                // One end marker per warpgroup, in consecutive stages (group g reads every third
+                // posting).  Those stages held loads issued - STAGES .., released by now.
+                for (int e = 0; e < C::GROUPS && ok; ++e) {
+                    const int s = it % C::STAGES;
+                    ok = mbar_wait(&empty[s], ((it / C::STAGES) & 1) ^ 1);
+                    if (ok) {
+                        meta[s] = make_int2(-1, 0);
+                        mbar_arrive(&full[s]);
+                        ++it;
+                    } else {
+                        report_wait_expired(status);
+                    }
                 }
+                first = issued - C::STAGES + C::GROUPS;
             }
             drain_loads<C::STAGES>(full, first, issued, status);
         }
-        return;
-    }
-
-    // ---------------- consumers ----------------
-    const int g8 = lane >> 2, t4 = lane & 3;
-    // A-fragment lane offset in the swizzled Q stage (non-transposed ldmatrix).
-    const int sw = lane & 7;
-    const uint32_t q_row = (warp * 16 + (lane & 7) + (((lane >> 3) & 1) << 3)) * 128;
-    const uint32_t q_hi = lane >> 4;  // 16-byte chunk parity inside a 16-channel k block
-    const uint32_t smem_base = smem_u32(smem);
-
-    uint32_t sfrag[4][9][2];  // [k block][column block][b0, b1], bf16x2
-    auto load_state = [&](int slab) {
-        const uint4* fr = reinterpret_cast<const uint4*>(frags + static_cast<size_t>(slab) * kStreamFragWords) + lane;
+    } else if (warp == C::STORE_WARP) {
+        // ---------------- store warp ----------------
+        if (lane == 0) {
+            prefetch_tmap(&tmap_y);
+            const uint64_t policy = policy_evict_first();
+            for (int it = 0;; ++it) {
+                const int s = it % C::STAGES;
+                if (!mbar_wait(&y_ready[s], (it / C::STAGES) & 1)) {
+                    report_wait_expired(status);
+                    break;
+                }
+                const int2 m = meta[s];
+                if (m.x < 0) break;  // the first end marker: every tile posted before it has left
+                tma_store_4d(&tmap_y, smem + s * C::STAGE_BYTES, 0, m.y * C::TILE, m.x % H, m.x / H, policy);
+                tma_store_wait_read();
+                mbar_arrive(&empty[s]);
+            }
+            tma_store_wait_all();
+        }
+    } else if (warp == C::MMA_WARP) {
+        // ---------------- MMA warp ----------------
+        // (tcgen05.mma issued by the leaders of several warpgroups at once lost completions now and
+        // then; with a single issuing thread it has not.)
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16_f32(C::TILE, C::B_ROWS);
+            const uint64_t b_desc = umma_desc_kmajor_sw128(smem_u32(bsm));
+            for (int it = 0;; ++it) {
+                const int s = it % C::STAGES, g = it % C::GROUPS;
+                if (!mbar_wait(&full[s], (it / C::STAGES) & 1)) {
+                    report_wait_expired(status);
+                    break;
+                }
+                if (meta[s].x < 0) break;
+                if (!mbar_wait(&a_ready[g], (it / C::GROUPS) & 1)) {
+                    report_wait_expired(status);
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t a_tmem = tmem_base + g * C::TMEM_COLS_PER_GROUP, d_tmem = a_tmem + 32;
+                // K = 64 as four steps of 16: A advances 8 columns (two bf16 per column), B 32 bytes
 #pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
+                for (int k = 0; k < 4; ++k) umma_bf16_ts(d_tmem, a_tmem + 8 * k, b_desc + 2 * k, idesc, k > 0 ? 1u : 0u);
+                umma_commit(&mma_done[g]);
+            }
+        }
+    } else {
+        // ---------------- consumer warpgroups ----------------
+        const int group = warp >> 2, wq = warp & 3;
+        const int row = wq * 32 + lane;
+        const uint32_t a_tmem = tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + group * C::TMEM_COLS_PER_GROUP;
+        const uint32_t d_tmem = a_tmem + 32;
+        const uint32_t row_base = smem_u32(smem) + row * 128;
+        const uint32_t sw = row & 7;
+        uint32_t tiles_done = 0;
+        for (int it = group;; it += C::GROUPS) {
+            const int s = it % C::STAGES;
+            if (!mbar_wait(&full[s], (it / C::STAGES) & 1)) {
+                if (lane == 0) report_wait_expired(status);
+                break;
+            }
+            const int slab = meta[s].x;
+            __syncwarp();
+            if (slab < 0) {
+                if (lane == 0) mbar_arrive(&y_ready[s]);  // hand the end marker on to the store warp
+                break;
+            }
+            const uint32_t base = row_base + s * C::STAGE_BYTES;
+            {
+                // the row's eight 16-byte chunks; a quarter-warp reads eight different chunk
+                // positions (the swizzle), so the loads are free of bank conflicts
+                uint32_t a[32];
 #pragma unroll
-            for (int nbp = 0; nbp < 5; ++nbp) {
-                const uint4 v = __ldg(fr + (kb * 5 + nbp) * 32);
-                sfrag[kb][2 * nbp][0] = v.x;
-                sfrag[kb][2 * nbp][1] = v.y;
-                if (nbp < 4) {
-                    sfrag[kb][2 * nbp + 1][0] = v.z;
-                    sfrag[kb][2 * nbp + 1][1] = v.w;
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t x0, x1, x2, x3;
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                 : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
+                                 : "r"(base + ((c ^ sw) << 4)));
+                    a[4 * c + 0] = phi_packed_bf16x2<PHI>(x0);
+                    a[4 * c + 1] = phi_packed_bf16x2<PHI>(x1);
+                    a[4 * c + 2] = phi_packed_bf16x2<PHI>(x2);
+                    a[4 * c + 3] = phi_packed_bf16x2<PHI>(x3);
+                }
+                tmem_store_32cols(a_tmem, a);
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&a_ready[group]);
+            const bool ok = mbar_wait(&mma_done[group], tiles_done & 1);
+            ++tiles_done;
+            __syncwarp();
+            if (!ok) {
+                if (lane == 0) report_wait_expired(status);
+                break;
+            }
+            tc_fence_after_sync();
+            const float den = __uint_as_float(tmem_load_1col(d_tmem + 64));  // phi(Q_i) . z
+            const float inv = 1.0f / (den + eps);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t d[32];
+                tmem_load_32cols(d_tmem + 32 * half, d);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t v0 = pack_bf16x2(__uint_as_float(d[8 * c + 0]) * inv, __uint_as_float(d[8 * c + 1]) * inv);
+                    const uint32_t v1 = pack_bf16x2(__uint_as_float(d[8 * c + 2]) * inv, __uint_as_float(d[8 * c + 3]) * inv);
+                    const uint32_t v2 = pack_bf16x2(__uint_as_float(d[8 * c + 4]) * inv, __uint_as_float(d[8 * c + 5]) * inv);
+                    const uint32_t v3 = pack_bf16x2(__uint_as_float(d[8 * c + 6]) * inv, __uint_as_float(d[8 * c + 7]) * inv);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + (((4 * half + c) ^ sw) << 4)),
+                                 "r"(v0), "r"(v1), "r"(v2), "r"(v3)
+                                 : "memory");
                 }
             }
+            tc_fence_before_sync();  // orders the loads of D before the next tile's MMA (through a_ready)
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&y_ready[s]);
         }
-    };
-
-    int cur_slab = -1;
-    for (int it = 0;; ++it) {
-        const int s = it % C::STAGES;
-        if (!mbar_wait(&full[s], (it / C::STAGES) & 1)) {
-            if (lane == 0) report_wait_expired(status);
-            break;
-        }
-        const int2 m = meta[s];
-        const int slab = m.x, tile = m.y;
-        if (slab < 0) break;
-        if (slab != cur_slab) {
-            load_state(slab);
-            cur_slab = slab;
-        }
-        const uint32_t qbase = smem_base + s * C::STAGE_BYTES + q_row;
-        float acc[9][4];
-#pragma unroll
-        for (int kb = 0; kb < 4; ++kb) {
-            uint32_t a0, a1, a2, a3;
-            ldmatrix_x4(qbase + ((((kb << 1) | q_hi) ^ sw) << 4), a0, a1, a2, a3);
-            a0 = phi_packed_bf16x2<PHI>(a0);
-            a1 = phi_packed_bf16x2<PHI>(a1);
-            a2 = phi_packed_bf16x2<PHI>(a2);
-            a3 = phi_packed_bf16x2<PHI>(a3);
-#pragma unroll
-            for (int nb = 0; nb < 9; ++nb) {
-                if (kb == 0)
-                    mma_bf16_16816_init(acc[nb], a0, a1, a2, a3, sfrag[kb][nb][0], sfrag[kb][nb][1]);
-                else
-                    mma_bf16_16816(acc[nb], a0, a1, a2, a3, sfrag[kb][nb][0], sfrag[kb][nb][1]);
-            }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);  // stage is free as soon as the fragments are read
-
-        const float inv0 = 1.0f / (acc[8][0] + eps);
-        const float inv1 = 1.0f / (acc[8][2] + eps);
-        const long long r0 = static_cast<long long>(tile) * C::TILE + warp * 16 + g8, r1 = r0 + 8;
-        __nv_bfloat16* y0 = Y + slab_base(L, slab) + static_cast<size_t>(r0) * L.row_stride;
-        __nv_bfloat16* y1 = y0 + 8 * static_cast<size_t>(L.row_stride);
-#pragma unroll
-        for (int hi = 0; hi < 2; ++hi) {
-            uint4 v0, v1;
-            v0.x = pack_bf16x2(acc[4 * hi + 0][0] * inv0, acc[4 * hi + 0][1] * inv0);
-            v0.y = pack_bf16x2(acc[4 * hi + 1][0] * inv0, acc[4 * hi + 1][1] * inv0);
-            v0.z = pack_bf16x2(acc[4 * hi + 2][0] * inv0, acc[4 * hi + 2][1] * inv0);
-            v0.w = pack_bf16x2(acc[4 * hi + 3][0] * inv0, acc[4 * hi + 3][1] * inv0);
-            v1.x = pack_bf16x2(acc[4 * hi + 0][2] * inv1, acc[4 * hi + 0][3] * inv1);
-            v1.y = pack_bf16x2(acc[4 * hi + 1][2] * inv1, acc[4 * hi + 1][3] * inv1);
-            v1.z = pack_bf16x2(acc[4 * hi + 2][2] * inv1, acc[4 * hi + 2][3] * inv1);
-            v1.w = pack_bf16x2(acc[4 * hi + 3][2] * inv1, acc[4 * hi + 3][3] * inv1);
-            if (r0 < N) st_stream_16B(y0 + 32 * hi + 8 * t4, v0);
-            if (r1 < N) st_stream_16B(y1 + 32 * hi + 8 * t4, v1);
-        }
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
 }
 
