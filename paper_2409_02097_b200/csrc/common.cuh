@@ -307,6 +307,16 @@ __device__ __forceinline__ void tmem_load_32cols(uint32_t taddr, uint32_t (&r)[3
         : "r"(taddr)
         : "memory");
 }
+__device__ __forceinline__ void tmem_load_16cols(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
 __device__ __forceinline__ uint32_t tmem_load_1col(uint32_t taddr)
 {
     uint32_t r;
@@ -329,10 +339,27 @@ __device__ __forceinline__ uint64_t umma_desc_kmajor_sw128(uint32_t smem_addr)
     d |= static_cast<uint64_t>(2) << 61;                      // 128-byte swizzle
     return d;
 }
-// Instruction descriptor of kind::f16 with bf16 A and B (both K-major) and fp32 accumulation, M x N.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int M, int N)
+// The same for an operand stored the other way round (MN-major): 64 values along M (or N) are one
+// 128-byte row, 8 rows along K are one 1024-byte swizzle group.  `sbo` = bytes from one 8-row group
+// to the next along K, `lbo` = bytes from one 64-value block to the next along M/N.  Moving the
+// start by 16 rows (2048 bytes) is one K step.
+__device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, uint32_t lbo, uint32_t sbo)
 {
-    return (1u << 4) /*D fp32*/ | (1u << 7) /*A bf16*/ | (1u << 10) /*B bf16*/ |
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((smem_addr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
+    d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
+// Instruction descriptor of kind::f16 with bf16 A and B and fp32 accumulation, M x N; the operands
+// are K-major unless the flags say MN-major.
+constexpr uint32_t kUmmaAMnMajor = 1u << 15;
+constexpr uint32_t kUmmaBMnMajor = 1u << 16;
+__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int M, int N, uint32_t major_flags = 0u)
+{
+    return (1u << 4) /*D fp32*/ | (1u << 7) /*A bf16*/ | (1u << 10) /*B bf16*/ | major_flags |
            (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
 // D[tmem] (+)= A[tmem] * B[smem]; one thread issues it for the CTA.  A and B are both bf16.
@@ -343,6 +370,16 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
         "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// The same with A from shared memory as well.
+__device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // One arrival on `bar` once every tcgen05.mma this thread has issued so far is complete.

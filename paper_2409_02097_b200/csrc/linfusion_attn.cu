@@ -125,7 +125,7 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
             }
         }
         p->spans = spans;
-        partial_floats = static_cast<size_t>(p->G_state) * spans * 2 * kStreamStateFloats;
+        partial_floats = static_cast<size_t>(p->G_state) * spans * kStreamStateFloats;
         p->launches = 3;
     } else {
         p->cluster_size = largest_cluster(tiles_kv);

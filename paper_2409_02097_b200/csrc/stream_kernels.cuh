@@ -8,13 +8,18 @@
 // and the grid size, so the summation order — and with it every output bit — is fixed.
 //
 //   stream_state_kernel   — per CTA and per slab it touches: partial S_p = sum phi(K_j)^T V_j and
-//                           z_p (Prop. 2, Eq. 5).  Eight consumer warps: warp w owns rows
-//                           16*(w&3).. of the state and the token half (w>>2) of each 128-token
-//                           tile; A = phi(K)^T and B = V come out of the stage with
-//                           ldmatrix.trans, phi is applied to the A fragments in registers, and a
-//                           ninth column block of ones produces z.  Each (CTA, slab, half) writes
-//                           its own fp32 partial; nothing is combined with atomics.
-//   stream_reduce_kernel  — sums the partials of a slab in (CTA, half) order; also lays S^T | z out
+//                           z_p (Prop. 2, Eq. 5) on tcgen05.  A K/V tile of 128 tokens is eight
+//                           MMA steps of 16 tokens: D[128 x 64] += A * B with A = [V^T ; 1 ; 0]
+//                           (the raw V tile plus a constant block whose single row of ones
+//                           yields z) and B = phi(K)^T, both read from shared memory in the
+//                           token-major form TMA delivers (MN-major operands).  Each of 128
+//                           threads of a warpgroup applies phi to its token's K row in place;
+//                           one thread issues the MMAs; the accumulator lives in tensor memory
+//                           and is drained into fp32 registers of three flush warps every 32
+//                           tiles (keeps the tensor core's accumulation chains short).  Each
+//                           (CTA, slab) writes its own fp32 partial; nothing is combined with
+//                           atomics.
+//   stream_reduce_kernel  — sums the partials of a slab in CTA order; also lays S^T | z out
 //                           as the bf16, K-major, 128-byte-swizzled B operand the apply kernel
 //                           copies into shared memory.
 //   stream_apply_kernel   — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps) on tcgen05: a 128-row Q tile
@@ -42,15 +47,24 @@ constexpr int kStreamStateFloats = kStreamD * (kStreamD + 1);  // S [64][64] the
 constexpr int kStreamRowBytes = kStreamD * 2;                  // 128: one swizzle span
 
 struct StreamStateCfg {
-    static constexpr int TILE = 128;  // tokens per stage
-    static constexpr int CONSUMER_WARPS = 8;
-    static constexpr int THREADS = 32 * (CONSUMER_WARPS + 1);
-    static constexpr int STAGES = 2;
-    static constexpr int CTAS_PER_SM = 3;
+    static constexpr int TILE = 128;   // tokens per stage = 8 MMA steps of 16
+    static constexpr int GROUPS = 3;   // warpgroups applying phi, each to its own tile
+    static constexpr int PHI_WARPS = 4 * GROUPS;
+    static constexpr int PRODUCER_WARP = PHI_WARPS;
+    static constexpr int MMA_WARP = PHI_WARPS + 1;
+    static constexpr int FLUSH_WARP0 = PHI_WARPS + 4;  // three warps whose index is 0, 1, 2 mod 4
+    static constexpr int THREADS = 32 * (PHI_WARPS + 7);
+    static constexpr int STAGES = 6;
+    static constexpr int CTAS_PER_SM = 1;
     static constexpr int TILE_BYTES = TILE * kStreamRowBytes;  // 16 KB per tensor
     static constexpr int STAGE_BYTES = 2 * TILE_BYTES;         // K then V
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+    static constexpr int ONES_BYTES = 16 * kStreamRowBytes;    // constant block of A for one MMA step
+    static constexpr int SEGMENT_TILES = 32;                   // tiles accumulated in TMEM before a drain
+    static constexpr int TMEM_COLS = 128;                      // two accumulators of 64 fp32 columns
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + ONES_BYTES + 1024 /*align*/ + 1024 /*barriers*/;
 };
+static_assert(StreamStateCfg::FLUSH_WARP0 % 4 == 0, "flush warps must cover TMEM lane quarters 0, 1, 2");
+static_assert(StreamStateCfg::SMEM_BYTES > 116 * 1024, "one state CTA per SM");
 
 struct StreamApplyCfg {
     static constexpr int TILE = 128;   // tokens per stage = rows of one MMA tile = TMEM lanes
@@ -101,7 +115,17 @@ __device__ __forceinline__ void drain_loads(uint64_t* full, int first, int issue
 }
 
 // ---------------------------------------------------------------------------------------------
-// State: partials[(g * spans + slot) * 2 + half][kStreamStateFloats]
+// State: partials[g * spans + slot][kStreamStateFloats], slot = slab - first slab of CTA g's run.
+//
+// Roles in a CTA (one per SM): producer warp (TMA loads of K and V tiles); 3 warpgroups (thread r
+// of a group rewrites token r's K row as phi(K), zero past N); MMA warp (one thread issues every
+// tcgen05.mma; the stage is released by a commit once the MMAs that read it are complete); three
+// flush warps (TMEM lanes 0..63 = rows of S^T, lane 64 = z).  The run of a CTA is cut into
+// segments of at most SEGMENT_TILES tiles of one slab; segments alternate between two TMEM
+// accumulators, and the flush warps add each finished segment into fp32 registers (round to
+// nearest) and write the partial when the slab ends.
+// Per stage s: full[s] -> k_ready[s] (4 warps) -> empty[s] (commit).  Per accumulator b:
+// acc_done[b] (commit) -> acc_free[b] (3 flush warps).
 // ---------------------------------------------------------------------------------------------
 template <int PHI>
 __global__ void __launch_bounds__(StreamStateCfg::THREADS, StreamStateCfg::CTAS_PER_SM)
@@ -113,24 +137,45 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    uint64_t* full = reinterpret_cast<uint64_t*>(smem + C::STAGES * C::STAGE_BYTES);
+    unsigned char* ones = smem + C::STAGES * C::STAGE_BYTES;  // on a 1024-byte boundary
+    uint64_t* full = reinterpret_cast<uint64_t*>(ones + C::ONES_BYTES);
     uint64_t* empty = full + C::STAGES;
+    uint64_t* k_ready = empty + C::STAGES;
+    uint64_t* acc_done = k_ready + C::STAGES;  // [2]
+    uint64_t* acc_free = acc_done + 2;         // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_free + 2);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long G = gridDim.x, g = blockIdx.x;
     const long long u0 = unit_begin(g, W, G), u1 = unit_begin(g + 1, W, G);
     const int n_units = static_cast<int>(u1 - u0);
+    const int slab_first = static_cast<int>(u0 / tiles_per_slab);
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
             mbar_init(&full[s], 1);
-            mbar_init(&empty[s], C::CONSUMER_WARPS);
+            mbar_init(&empty[s], 1);
+            mbar_init(&k_ready[s], 4);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_done[b], 1);
+            mbar_init(&acc_free[b], 3);
         }
         mbar_fence_init();
     }
+    // Constant block of A (rows 64..127 of [V^T ; 1 ; 0] for 16 tokens): a one at (token t, row 64),
+    // which is the first value of token t's 128-byte row, moved by the swizzle to chunk t & 7.
+    for (int i = tid; i < C::ONES_BYTES / 4; i += C::THREADS) reinterpret_cast<uint32_t*>(ones)[i] = 0u;
     __syncthreads();
+    if (tid < 16) *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = 0x3F80u;  // bf16 1.0
+    fence_proxy_async_smem();
+    if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
 
-    if (warp == C::CONSUMER_WARPS) {
+    if (warp == C::PRODUCER_WARP) {
         // ---------------- producer ----------------
         if (lane == 0) {
             prefetch_tmap(&tmap_k);
@@ -139,8 +184,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
             int issued = 0;
             for (int it = 0; it < n_units; ++it) {
                 const int s = it % C::STAGES;
-                const uint32_t ph = (it / C::STAGES) & 1;
-                if (!mbar_wait(&empty[s], ph ^ 1)) {
+                if (!mbar_wait(&empty[s], ((it / C::STAGES) & 1) ^ 1)) {
                     report_wait_expired(status);
                     break;
                 }
@@ -155,102 +199,136 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
             }
             drain_loads<C::STAGES>(full, 0, issued, status);
         }
-        return;
-    }
-
-    // ---------------- consumers ----------------
-    const int mb = warp & 3, half = warp >> 2;
-    const int g8 = lane >> 2, t4 = lane & 3;
-    float acc[9][4];
+    } else if (warp == C::MMA_WARP) {
+        // ---------------- MMA warp ----------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_bf16_f32(128, 64, kUmmaAMnMajor | kUmmaBMnMajor);
+            const uint32_t ones_addr = smem_u32(ones);
+            int cur_slab = -1, in_segment = 0, segments = 0, buf = 1;
+            for (int it = 0; it < n_units; ++it) {
+                const int s = it % C::STAGES;
+                const int slab = static_cast<int>((u0 + it) / tiles_per_slab);
+                if (slab != cur_slab || in_segment == C::SEGMENT_TILES) {
+                    if (cur_slab >= 0) umma_commit(&acc_done[buf]);  // the segment's accumulator is complete
+                    buf ^= 1;
+                    // this accumulator held the segment before last: its drain must be over
+                    if (segments >= 2 && !mbar_wait(&acc_free[buf], ((segments - 2) >> 1) & 1)) {
+                        report_wait_expired(status);
+                        break;
+                    }
+                    ++segments;
+                    cur_slab = slab;
+                    in_segment = 0;
+                }
+                if (!mbar_wait(&k_ready[s], (it / C::STAGES) & 1)) {
+                    report_wait_expired(status);
+                    break;
+                }
+                tc_fence_after_sync();
+                const uint32_t k_addr = smem_u32(smem + s * C::STAGE_BYTES), v_addr = k_addr + C::TILE_BYTES;
+                const uint32_t d_tmem = tmem_base + buf * 64;
 #pragma unroll
-    for (int nb = 0; nb < 9; ++nb)
-#pragma unroll
-        for (int i = 0; i < 4; ++i) acc[nb][i] = 0.0f;
-
-    // Lane offsets inside a swizzled tile: byte = row*128 + ((chunk ^ (row & 7)) << 4), and
-    // row & 7 == lane & 7 for every row a lane addresses.
-    const int sw = lane & 7;
-    const uint32_t a_lane = (half * 64 + (lane & 7) + ((lane >> 4) << 3)) * 128 +
-                            (((mb * 2 + ((lane >> 3) & 1)) ^ sw) << 4);
-    const uint32_t b_lane = (half * 64 + (lane & 7) + (((lane >> 3) & 1) << 3)) * 128 +
-                            (((lane >> 4) ^ sw) << 4);
-    const uint32_t ones = 0x3F803F80u;
-    const uint32_t smem_base = smem_u32(smem);
-
-    auto flush = [&](int slab_first, int slab) {
-        const int slot = slab - slab_first;
-        float* dst = partials + ((static_cast<size_t>(g) * spans + slot) * 2 + half) * kStreamStateFloats;
-        const int c0 = mb * 16 + g8, c1 = c0 + 8;
-#pragma unroll
-        for (int nb = 0; nb < 8; ++nb) {
-            const int e = nb * 8 + 2 * t4;
-            *reinterpret_cast<float2*>(dst + c0 * 64 + e) = make_float2(acc[nb][0], acc[nb][1]);
-            *reinterpret_cast<float2*>(dst + c1 * 64 + e) = make_float2(acc[nb][2], acc[nb][3]);
+                for (int k = 0; k < C::TILE / 16; ++k) {
+                    // A: 64 rows from the V tile, 64 from the constant block (lbo = their distance);
+                    // 16 tokens = two 8-row groups 1024 bytes apart.
+                    const uint32_t va = v_addr + k * 2048;
+                    const uint64_t a_desc = umma_desc_mnmajor_sw128(va, ones_addr - va, 1024);
+                    const uint64_t b_desc = umma_desc_mnmajor_sw128(k_addr + k * 2048, 0, 1024);
+                    umma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (in_segment == 0 && k == 0) ? 0u : 1u);
+                }
+                ++in_segment;
+                umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
+            }
+            if (cur_slab >= 0) umma_commit(&acc_done[buf]);
         }
-        if (t4 == 0) {
-            dst[64 * 64 + c0] = acc[8][0];
-            dst[64 * 64 + c1] = acc[8][2];
-        }
+    } else if (warp >= C::FLUSH_WARP0 && warp < C::FLUSH_WARP0 + 3) {
+        // ---------------- flush warps ----------------
+        // The same walk over the run as the MMA thread's, segment by segment.
+        const int wq = warp & 3;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(wq * 32) << 16);
+        float acc[64];
 #pragma unroll
-        for (int nb = 0; nb < 9; ++nb)
+        for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
+        int seg = 0;
+        bool ok = true;
+        for (int it = 0; it < n_units && ok;) {
+            const int slab = static_cast<int>((u0 + it) / tiles_per_slab);
+            const long long slab_end = static_cast<long long>(slab + 1) * tiles_per_slab - u0;  // first it of the next slab
+            int len = static_cast<int>(slab_end < n_units ? slab_end : n_units) - it;
+            if (len > C::SEGMENT_TILES) len = C::SEGMENT_TILES;
+            it += len;
+            const int buf = seg & 1;
+            ok = mbar_wait(&acc_done[buf], (seg >> 1) & 1);
+            ++seg;
+            __syncwarp();
+            if (!ok) {
+                if (lane == 0) report_wait_expired(status);
+                break;
+            }
+            tc_fence_after_sync();
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[nb][i] = 0.0f;
-    };
-
-    const int slab_first = static_cast<int>(u0 / tiles_per_slab);
-    int cur_slab = slab_first;
-    bool failed = false;
-    for (int it = 0; it < n_units; ++it) {
-        const int s = it % C::STAGES;
-        const uint32_t ph = (it / C::STAGES) & 1;
-        const long long u = u0 + it;
-        const int slab = static_cast<int>(u / tiles_per_slab);
-        const int tile = static_cast<int>(u % tiles_per_slab);
-        if (slab != cur_slab) {
-            flush(slab_first, cur_slab);
-            cur_slab = slab;
-        }
-        if (!failed && !mbar_wait(&full[s], ph)) {
-            if (lane == 0) report_wait_expired(status);
-            failed = true;
-        }
-        if (!failed) {
-            const uint32_t kbase = smem_base + s * C::STAGE_BYTES;
-            const uint32_t vbase = kbase + C::TILE_BYTES;
-            const int valid = N - tile * C::TILE - half * 64;  // tokens of this warp's half inside N
+            for (int q4 = 0; q4 < 4; ++q4) {
+                uint32_t d[16];
+                tmem_load_16cols(t_lane + buf * 64 + 16 * q4, d);
 #pragma unroll
-            for (int ks = 0; ks < 4; ++ks) {
-                uint32_t a0, a1, a2, a3;
-                ldmatrix_x4_trans(kbase + a_lane + ks * 2048, a0, a1, a2, a3);
-                a0 = phi_packed_bf16x2<PHI>(a0);
-                a1 = phi_packed_bf16x2<PHI>(a1);
-                a2 = phi_packed_bf16x2<PHI>(a2);
-                a3 = phi_packed_bf16x2<PHI>(a3);
-                if (valid < 64) {
-                    // Rows past N were zero-filled by TMA, but phi(0) = 1: clear them explicitly.
-                    // a0/a1 hold tokens j, j+1; a2/a3 hold j+8, j+9 with j = 16*ks + 2*t4.
-                    const int j = ks * 16 + 2 * t4;
-                    const uint32_t m01 = (j < valid ? 0x0000ffffu : 0u) | (j + 1 < valid ? 0xffff0000u : 0u);
-                    const uint32_t m23 = (j + 8 < valid ? 0x0000ffffu : 0u) | (j + 9 < valid ? 0xffff0000u : 0u);
-                    a0 &= m01;
-                    a1 &= m01;
-                    a2 &= m23;
-                    a3 &= m23;
+                for (int c = 0; c < 16; ++c) acc[16 * q4 + c] += __uint_as_float(d[c]);
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&acc_free[buf]);
+            if (it == n_units || it == slab_end) {
+                // the slab's share of this CTA is complete: row e of S^T (lanes 0..63), z (lane 64)
+                float* dst = partials + (static_cast<size_t>(g) * spans + (slab - slab_first)) * kStreamStateFloats;
+                if (wq < 2) {
+                    const int e = wq * 32 + lane;
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) dst[c * 64 + e] = acc[c];
+                } else if (lane == 0) {
+#pragma unroll
+                    for (int c = 0; c < 64; ++c) dst[64 * 64 + c] = acc[c];
                 }
 #pragma unroll
-                for (int nbp = 0; nbp < 4; ++nbp) {
-                    uint32_t b0, b1, b2, b3;
-                    ldmatrix_x4_trans(vbase + ((b_lane + ks * 2048) ^ (nbp << 5)), b0, b1, b2, b3);
-                    mma_bf16_16816(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
-                    mma_bf16_16816(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
-                }
-                mma_bf16_16816(acc[8], a0, a1, a2, a3, ones, ones);
+                for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
             }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[s]);
+    } else if (warp < C::PHI_WARPS) {
+        // ---------------- phi warpgroups ----------------
+        const int group = warp >> 2;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t row_base = smem_u32(smem) + row * 128;
+        const uint32_t sw = row & 7;
+        for (int it = group; it < n_units; it += C::GROUPS) {
+            const int s = it % C::STAGES;
+            if (!mbar_wait(&full[s], (it / C::STAGES) & 1)) {
+                if (lane == 0) report_wait_expired(status);
+                break;
+            }
+            const int tile = static_cast<int>((u0 + it) % tiles_per_slab);
+            const bool valid = tile * C::TILE + row < N;  // a row past N must count for nothing (phi(0) = 1)
+            const uint32_t base = row_base + s * C::STAGE_BYTES;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+                // a quarter-warp touches eight different chunk positions: no bank conflicts
+                uint32_t x0, x1, x2, x3;
+                const uint32_t addr = base + ((c ^ sw) << 4);
+                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(addr));
+                x0 = valid ? phi_packed_bf16x2<PHI>(x0) : 0u;
+                x1 = valid ? phi_packed_bf16x2<PHI>(x1) : 0u;
+                x2 = valid ? phi_packed_bf16x2<PHI>(x2) : 0u;
+                x3 = valid ? phi_packed_bf16x2<PHI>(x3) : 0u;
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x0), "r"(x1), "r"(x2), "r"(x3) : "memory");
+            }
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&k_ready[s]);
+        }
     }
-    if (n_units > 0) flush(slab_first, cur_slab);
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
 }
 
 // Operand image of S | z for the apply kernel, per slab: the MMA's B operand in its shared-memory
@@ -284,7 +362,7 @@ __device__ __forceinline__ void emit_state_operand(const float* sums, unsigned c
 }
 
 // grid (17, slabs), 256 threads: state[slab] = sum over the CTAs whose run meets the slab, in
-// increasing CTA index, half 0 then half 1 (fp32, fixed order).  Also writes the bf16 operand
+// increasing CTA index (fp32, fixed order).  Also writes the bf16 operand
 // image of S | z for the apply kernel and clears the slab's tile counter for it.
 __global__ void __launch_bounds__(256)
 stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
@@ -309,14 +387,10 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
         const int slot0 = slab - static_cast<int>(unit_begin(g0, W, G) / tiles_per_slab);
         const size_t F = kStreamStateFloats;
         const float* src = partials + idx;
-        sum += src[((static_cast<size_t>(g0) * spans + slot0) * 2) * F];
-        sum += src[((static_cast<size_t>(g0) * spans + slot0) * 2 + 1) * F];
+        sum += src[(static_cast<size_t>(g0) * spans + slot0) * F];
         // Every later CTA starts inside this slab: its partial for it is in slot 0.
 #pragma unroll 4
-        for (long long g = g0 + 1; g < g1; ++g) {
-            sum += src[(static_cast<size_t>(g) * spans * 2) * F];
-            sum += src[(static_cast<size_t>(g) * spans * 2 + 1) * F];
-        }
+        for (long long g = g0 + 1; g < g1; ++g) sum += src[(static_cast<size_t>(g) * spans) * F];
         state[static_cast<size_t>(slab) * F + idx] = sum;
     }
     sums[tid] = sum;

@@ -53,9 +53,9 @@ def test_workspace_bytes_is_pure_host_and_monotone():
     a = _ws(attn.make_desc(2, 10, 524288, 64, variant="split"))
     b = _ws(attn.make_desc(2, 10, 2 * 524288, 64, variant="split"))
     assert a == b
-    # stream: G * spans * 2 partials + state + bf16 operand image + tile counters + status word
+    # stream: G * spans partials (one CTA per SM) + state + bf16 operand image + tile counters + status word
     s = _ws(attn.make_desc(2, 10, 524288, 64, variant="stream"))
-    assert s == 444 * 2 * 2 * 4160 * 4 + 20 * 4160 * 4 + 20 * 2560 * 4 + 256 + 256
+    assert s == 148 * 2 * 4160 * 4 + 20 * 4160 * 4 + 20 * 80 * 128 + 256 + 256
     # cluster: no partials in global memory
     c = _ws(attn.make_desc(2, 8, 256, 160, variant="cluster"))
     assert c == (16 * 160 * 161 * 4 + 255) // 256 * 256 + 256
