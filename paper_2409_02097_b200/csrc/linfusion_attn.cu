@@ -85,13 +85,17 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v == LINFUSION_VARIANT_AUTO) {
         // Measured on B200 over the SD-v1.5 / v2.1 / XL layer shapes: the single clustered launch
-        // wins only at the smallest levels (N <= 192: 14 vs 18 us at N = 144, d = 64; 28 vs 35 us
-        // at N = 64, d = 160); above that the TMA-streamed kernels win for d = 64 at every N, and
-        // the three-launch split path for the other head dims.
+        // wins only at the smallest levels (N <= 192: 15 vs 24 us at N = 144, d = 64; 28 vs 35 us
+        // at N = 64, d = 160).  The persistent TMA + tcgen05 kernels (d = 64) pay a few
+        // microseconds of set-up (tensor-memory allocation, one CTA per SM working through its
+        // tiles in turn) and win once every SM has a dozen 128-token tiles (56 vs 70 us at
+        // N = 16384 x 20 slabs; 33 vs 26 us at N = 2304 x 40 slabs); the three-launch split path
+        // takes the rest.
         const int cl = largest_cluster(tiles_kv);
+        const long long stream_tiles = static_cast<long long>(slabs) * ((d->N + StreamStateCfg::TILE - 1) / StreamStateCfg::TILE);
         if (d->N <= 192 && static_cast<long long>(slabs) * cl <= 2ll * sm_count)
             v = LINFUSION_VARIANT_CLUSTER;
-        else if (d->d == kStreamD)
+        else if (d->d == kStreamD && stream_tiles >= 12ll * sm_count)
             v = LINFUSION_VARIANT_STREAM;
         else
             v = LINFUSION_VARIANT_SPLIT;

@@ -99,12 +99,22 @@ def test_edge_shapes_all_variants(dims):
 
 def test_stream_variant_tail_and_slab_crossing():
     """Many slabs, ragged N: every CTA's run crosses slab boundaries and tail tiles are masked."""
-    for (B, H, N) in [(2, 37, 1000), (1, 100, 130), (2, 20, 2500)]:
+    # the last case gives every CTA a run of 60 tiles: more than one tensor-memory segment per slab
+    # and, for the CTAs at the seams, a change of slab in mid-run
+    for (B, H, N) in [(2, 37, 1000), (1, 100, 130), (2, 20, 2500), (1, 3, 378917)]:
         q, k, v = wl.make_small(B, H, N, 64, seed=5, device="cuda")
         ref = oracle_y(q, k, v)
         y, op = run_gpu(q, k, v, "stream")
         assert op.variant == "stream"
         assert_parity(y, ref, f"stream {(B, H, N)}")
+        op.close()
+
+
+def test_auto_policy_follows_the_measured_crossovers():
+    for dims, want in [((2, 10, 16384, 64), "stream"), ((2, 20, 2304, 64), "split"),
+                       ((2, 20, 144, 64), "cluster"), ((2, 8, 4096, 40), "split")]:
+        op = attn.LinFusionAttention(*dims)
+        assert op.variant == want, (dims, op.variant)
         op.close()
 
 
