@@ -304,20 +304,23 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                 break;
             }
             const int tile = static_cast<int>((u0 + it) % tiles_per_slab);
-            const bool valid = tile * C::TILE + row < N;  // a row past N must count for nothing (phi(0) = 1)
             const uint32_t base = row_base + s * C::STAGE_BYTES;
+            if (tile * C::TILE + row < N) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-                // a quarter-warp touches eight different chunk positions: no bank conflicts
-                uint32_t x0, x1, x2, x3;
-                const uint32_t addr = base + ((c ^ sw) << 4);
-                asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(addr));
-                x0 = valid ? phi_packed_bf16x2<PHI>(x0) : 0u;
-                x1 = valid ? phi_packed_bf16x2<PHI>(x1) : 0u;
-                x2 = valid ? phi_packed_bf16x2<PHI>(x2) : 0u;
-                x3 = valid ? phi_packed_bf16x2<PHI>(x3) : 0u;
-                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x0), "r"(x1), "r"(x2), "r"(x3) : "memory");
+                for (int c = 0; c < 8; ++c) {
+                    // a quarter-warp touches eight different chunk positions: no bank conflicts
+                    uint32_t x0, x1, x2, x3;
+                    const uint32_t addr = base + ((c ^ sw) << 4);
+                    asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(addr));
+                    x0 = phi_packed_bf16x2<PHI>(x0);
+                    x1 = phi_packed_bf16x2<PHI>(x1);
+                    x2 = phi_packed_bf16x2<PHI>(x2);
+                    x3 = phi_packed_bf16x2<PHI>(x3);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x0), "r"(x1), "r"(x2), "r"(x3) : "memory");
+                }
             }
+            // else: a row past N.  TMA filled it with zeros and it must count for nothing; phi(0) = 1,
+            // so the zeros are left as they are.  (Only the last tile of a slab has such rows.)
             fence_proxy_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(&k_ready[s]);
