@@ -17,11 +17,13 @@ constexpr int kPhiIdentity = 1;
 constexpr uint32_t kStatusOk = 0u;
 constexpr uint32_t kStatusWaitExpired = 1u;
 
-// Upper bound on polls of one mbarrier wait.  Each failed try_wait already blocks for a
-// hardware-defined interval (about 4 us measured), so this is roughly a quarter of a second: far
-// beyond any legitimate wait here (microseconds), so that a lost transaction ends the kernel with
-// an error word instead of a hang.
-constexpr uint32_t kMaxBarrierPolls = 1u << 16;
+// Upper bound on the time one mbarrier wait may take, in nanoseconds of the global timer: far beyond
+// any legitimate wait here (microseconds, or the length of a kernel for the waits that span one),
+// so that a lost transaction ends the kernel with an error word instead of a hang.
+constexpr unsigned long long kMaxBarrierWaitNs = 250ull * 1000ull * 1000ull;
+// How long one try_wait may keep the thread suspended (it wakes as soon as the phase completes):
+// long, so that a waiting warp issues next to no instructions.
+constexpr uint32_t kBarrierSuspendHintNs = 1000u * 1000u;
 
 // Where the rows of one (batch, head) slab sit in a tensor, in elements.  Head-major [B,H,N,d]:
 // batch_stride = H*N*d, head_stride = N*d, row_stride = d.  Token-major [B,N,H,d] (what a UNet
@@ -192,24 +194,38 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// Returns true once the phase with the given parity has completed, false if the poll budget
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint32_t addr, uint32_t parity)
+{
+    uint32_t done;
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t"
+        "}"
+        : "=r"(done)
+        : "r"(addr), "r"(parity), "r"(kBarrierSuspendHintNs)
+        : "memory");
+    return done != 0u;
+}
+
+// Returns true once the phase with the given parity has completed, false if the time budget
 // ran out (the caller records the failure and leaves).
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity)
 {
-    uint32_t addr = smem_u32(bar);
-    for (uint32_t it = 0; it < kMaxBarrierPolls; ++it) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t"
-            ".reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t"
-            "}"
-            : "=r"(done)
-            : "r"(addr), "r"(parity)
-            : "memory");
-        if (done) return true;
-    }
+    const uint32_t addr = smem_u32(bar);
+    if (mbar_try_wait(addr, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    do {
+        if (mbar_try_wait(addr, parity)) return true;
+    } while (global_timer_ns() - t0 < kMaxBarrierWaitNs);
     return false;
 }
 
