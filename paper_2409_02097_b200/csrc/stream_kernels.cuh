@@ -1,7 +1,7 @@
 // Persistent, TMA-pipelined kernels for head dim 64 (the SD-v2.1 / SD-XL shapes), where the
 // operator is bound by HBM bandwidth: every byte of Q, K, V is read once through
-// cp.async.bulk.tensor into 128-byte-swizzled shared-memory stages, and Y is written once with
-// 16-byte stores.
+// cp.async.bulk.tensor into 128-byte-swizzled shared-memory stages, Y is written once with TMA
+// stores, and both contractions run on tcgen05 with their accumulators in tensor memory.
 //
 // Work is cut into units of one token tile of one slab, numbered slab-major; CTA g of G owns
 // the contiguous run of units [g*W/G, (g+1)*W/G).  That split is a pure function of the shape
