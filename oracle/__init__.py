@@ -51,6 +51,9 @@ def _load():
         lib.oracle_apply.restype = None
         lib.oracle_apply.argtypes = [dp, dp, dp, ctypes.c_long, ctypes.c_long, ctypes.c_int,
                                      ctypes.c_double, ctypes.c_int, dp]
+        lib.oracle_apply_unnormalized.restype = None
+        lib.oracle_apply_unnormalized.argtypes = [dp, dp, ctypes.c_long, ctypes.c_long, ctypes.c_int,
+                                                  ctypes.c_int, dp]
         lib.oracle_linear.restype = ctypes.c_int
         lib.oracle_linear.argtypes = [dp, dp, dp, ctypes.c_long, ctypes.c_long, ctypes.c_int,
                                       ctypes.c_double, ctypes.c_int, dp]
@@ -114,6 +117,23 @@ def apply(q, S, z, eps: float, phi_kind: int = PHI_ELU_PLUS_ONE) -> np.ndarray:
     y = np.empty_like(q)
     _load().oracle_apply(_ptr(q), _ptr(S), _ptr(z), slabs, n, d, float(eps), phi_kind, _ptr(y))
     return y
+
+
+def apply_unnormalized(q, S, phi_kind: int = PHI_ELU_PLUS_ONE) -> np.ndarray:
+    """Y_i = phi(Q_i) S: Prop. 2 without Eq. 5's division (the Tab. 2 ablation)."""
+    q, S = _f64(q), _f64(S)
+    slabs, n, d = _slabs_n_d(q)
+    if S.shape != q.shape[:-2] + (d, d):
+        raise ValueError("S does not match q")
+    y = np.empty_like(q)
+    _load().oracle_apply_unnormalized(_ptr(q), _ptr(S), slabs, n, d, phi_kind, _ptr(y))
+    return y
+
+
+def linear_unnormalized(q, k, v, phi_kind: int = PHI_ELU_PLUS_ONE) -> np.ndarray:
+    """State, then the apply without the normalizer."""
+    S, _ = state(k, v, phi_kind)
+    return apply_unnormalized(q, S, phi_kind)
 
 
 def linear(q, k, v, eps: float, phi_kind: int = PHI_ELU_PLUS_ONE) -> np.ndarray:

@@ -102,6 +102,26 @@ void oracle_apply(const double* q, const double* S, const double* z, long slabs,
     }
 }
 
+/* Apply without the normalizer: Y_i = phi(Q_i) S, i.e. Y = f'(X) g'(X)^T X of Prop. 2 before
+ * Eq. 5's division is put on top (the "without normalization" rows of the ablation in Tab. 2). */
+void oracle_apply_unnormalized(const double* q, const double* S, long slabs, long n, int d,
+                               int phi_kind, double* y)
+{
+    long rows = slabs * n;
+#pragma omp parallel for schedule(static)
+    for (long r = 0; r < rows; ++r) {
+        long s = r / n;
+        const double* qi = q + (size_t)r * d;
+        const double* Ss = S + (size_t)s * d * d;
+        double* yi = y + (size_t)r * d;
+        for (int e = 0; e < d; ++e) yi[e] = 0.0;
+        for (int c = 0; c < d; ++c) {
+            double p = oracle_phi(qi[c], phi_kind);
+            for (int e = 0; e < d; ++e) yi[e] += p * Ss[(size_t)c * d + e];
+        }
+    }
+}
+
 /* The whole path in its linear form.  Returns 0, or -1 if scratch memory cannot be had. */
 int oracle_linear(const double* q, const double* k, const double* v, long slabs, long n,
                   int d, double eps, int phi_kind, double* y)

@@ -243,3 +243,49 @@ def test_slabs_are_independent():
 
 def test_threads_reported():
     assert oracle.num_threads() >= 1
+
+
+# ---- the un-normalized operator (Prop. 2 without Eq. 5's division; Tab. 2 ablation) -------------
+
+def _phi_closed_form(x):
+    return np.where(x > 0, x + 1.0, np.exp(np.minimum(x, 0.0)))
+
+
+def test_unnormalized_hand_worked_case(golden_dir):
+    env = {"e": math.e, "__builtins__": {}}
+    with open(os.path.join(golden_dir, "hand_worked_cases.json")) as f:
+        cases = json.load(f)["unnormalized_cases"]
+    assert cases
+    for case in cases:
+        q, k, v = (np.array(case[n], dtype=np.float64) for n in ("q", "k", "v"))
+        want = np.array([[eval(x, env) for x in row] for row in case["y_expr"]])
+        np.testing.assert_allclose(oracle.linear_unnormalized(q, k, v), want, rtol=1e-14, atol=0)
+
+
+def test_unnormalized_equals_attention_matrix_form():
+    """Y = (phi(Q) phi(K)^T) V with the n x n weights written out (Eq. 4 with the mask dropped)."""
+    rng = np.random.default_rng(77)
+    q, k, v = (rng.standard_normal((3, 37, 5)) for _ in range(3))
+    w = _phi_closed_form(q) @ np.swapaxes(_phi_closed_form(k), -1, -2)   # [3, 37, 37]
+    np.testing.assert_allclose(oracle.linear_unnormalized(q, k, v), w @ v, rtol=1e-12, atol=1e-12)
+
+
+def test_unnormalized_times_reciprocal_denominator_is_the_normalized_output():
+    rng = np.random.default_rng(78)
+    q, k, v = (rng.standard_normal((2, 50, 8)) for _ in range(3))
+    eps = 1e-3
+    S, z = oracle.state(k, v)
+    den = _phi_closed_form(q) @ z[..., None] + eps                          # [2, 50, 1]
+    np.testing.assert_allclose(oracle.apply_unnormalized(q, S) / den, oracle.apply(q, S, z, eps),
+                               rtol=1e-12, atol=1e-14)
+
+
+def test_unnormalized_is_not_the_normalized_operator():
+    """A plausible mistake (dividing anyway) must fail: with V = const the rows are not V."""
+    rng = np.random.default_rng(79)
+    q, k = (rng.standard_normal((1, 20, 4)) for _ in range(2))
+    v = np.ones((1, 20, 4))
+    y = oracle.linear_unnormalized(q, k, v)
+    w = _phi_closed_form(q) @ np.swapaxes(_phi_closed_form(k), -1, -2)
+    np.testing.assert_allclose(y[..., 0], w.sum(-1), rtol=1e-12)            # row sums of the weights
+    assert np.abs(y - 1.0).min() > 1.0
