@@ -66,6 +66,14 @@ typedef enum {
  */
 #define LINFUSION_LAYOUT_TOKEN_MAJOR 0x10u
 
+/*
+ * flags: the operator without its normalizer.  Bit set: Y_i = phi(Q_i) S, i.e. Y = f'(X) g'(X)^T X of
+ * Prop. 2 before the division of Eq. 5 is applied (the "without normalization" rows of the
+ * ablation in Tab. 2).  eps is then unused; z is still accumulated and read_state() returns it.
+ * |Y| grows with N in this form (the paper's reason for the normalizer); outputs are still bf16.
+ */
+#define LINFUSION_FLAG_UNNORMALIZED 0x20u
+
 typedef struct {
     int32_t B;      /* batch                                   > 0 */
     int32_t H;      /* heads                                   > 0 */

@@ -102,11 +102,14 @@ def status_string(code: int) -> str:
 
 
 LAYOUT_TOKEN_MAJOR = 0x10   # tensors are [B, N, H, d] instead of [B, H, N, d]
+FLAG_UNNORMALIZED = 0x20    # Y_i = phi(Q_i) S, without the division by phi(Q_i) . z + eps
 
 
 def make_desc(B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
-              layout="head_major") -> Desc:
+              layout="head_major", normalize=True) -> Desc:
     flags = VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    if not normalize:
+        flags |= FLAG_UNNORMALIZED
     if layout == "token_major":
         flags |= LAYOUT_TOKEN_MAJOR
     elif layout != "head_major":
@@ -168,8 +171,8 @@ class LinFusionAttention:
     with ``layout="token_major"``)."""
 
     def __init__(self, B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
-                 layout="head_major"):
-        self.desc = make_desc(B, H, N, d, phi, eps, device, variant, layout)
+                 layout="head_major", normalize=True):
+        self.desc = make_desc(B, H, N, d, phi, eps, device, variant, layout, normalize)
         # tensors are [B, H, N, d], or [B, N, H, d] in the token-major layout
         self.shape = (int(B), int(H), int(N), int(d)) if layout == "head_major" else \
                      (int(B), int(N), int(H), int(d))

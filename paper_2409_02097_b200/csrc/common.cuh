@@ -59,6 +59,14 @@ __device__ __forceinline__ float phi(float x)
     return fmaxf(x, 0.0f) + ex2_approx(fminf(x, 0.0f) * 1.4426950408889634f);
 }
 
+// Row scale of the apply step: 1 / (phi(Q_i) . z + eps) (Eq. 5), or 1 for the operator without
+// its normalizer, which the host requests by passing a negative eps.
+constexpr float kEpsUnnormalized = -1.0f;
+__device__ __forceinline__ float row_scale(float den, float eps)
+{
+    return eps < 0.0f ? 1.0f : 1.0f / (den + eps);
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
 

@@ -56,7 +56,8 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
     if (!supported_d(d->d)) return LINFUSION_ERR_UNSUPPORTED;
     if (d->phi != LINFUSION_PHI_ELU_PLUS_ONE && d->phi != LINFUSION_PHI_IDENTITY)
         return LINFUSION_ERR_UNSUPPORTED;
-    if ((d->flags & ~(LINFUSION_VARIANT_MASK | LINFUSION_LAYOUT_TOKEN_MAJOR)) != 0u) return LINFUSION_ERR_UNSUPPORTED;
+    if ((d->flags & ~(LINFUSION_VARIANT_MASK | LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED)) != 0u)
+        return LINFUSION_ERR_UNSUPPORTED;
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v > LINFUSION_VARIANT_CLUSTER) return LINFUSION_ERR_UNSUPPORTED;
     if (v == LINFUSION_VARIANT_STREAM && d->d != kStreamD) return LINFUSION_ERR_UNSUPPORTED;
@@ -169,6 +170,12 @@ EncodeTiledFn get_encode_fn()
             fn = reinterpret_cast<EncodeTiledFn>(p);
     }
     return fn;
+}
+
+// eps as the apply kernels take it: negative selects the operator without its normalizer.
+float kernel_eps(const linfusion_attn_desc_t& d)
+{
+    return (d.flags & LINFUSION_FLAG_UNNORMALIZED) != 0u ? kEpsUnnormalized : d.eps;
 }
 
 // Element strides of a slab's rows for the layout the descriptor asks for.
@@ -326,7 +333,7 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
         h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST);
     mark(h, 2, s);
     apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-        q, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc), image);
+        q, h->state, y, N, p.chunks_apply, kernel_eps(h->desc), layout_of(h->desc), image);
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -358,7 +365,7 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
     cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
     mark(h, 0, s);
     cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state,
-                                       h->desc.N, h->desc.eps, layout_of(h->desc));
+                                       h->desc.N, kernel_eps(h->desc), layout_of(h->desc));
     mark(h, 1, s);
     return e;
 }
@@ -382,7 +389,7 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
         h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state, p.spans);
     mark(h, 2, s);
     stream_apply_kernel<PHI><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, h->desc.eps, h->desc.H);
+        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, kernel_eps(h->desc), h->desc.H);
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -700,7 +707,7 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
             linfusion_attn_desc_t d = h->desc;
             d.B = 1;
             d.H = slabs / p->groups;
-            d.flags = static_cast<uint32_t>(h->plan.variant);  // head-major only (see the grouping rule above)
+            d.flags = static_cast<uint32_t>(h->plan.variant) | (h->desc.flags & LINFUSION_FLAG_UNNORMALIZED);  // head-major only (see the grouping rule above)
             ok = linfusion_attn_create(&d, &p->sub) == LINFUSION_OK;
             ok = ok && cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) == cudaSuccess;
             ok = ok && cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) == cudaSuccess;
@@ -953,7 +960,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     // and every state element that is read in this call is written earlier in the same call.
     linfusion_attn view;
     view.desc = *desc;
-    view.desc.flags = (desc->flags & LINFUSION_LAYOUT_TOKEN_MAJOR) | LINFUSION_VARIANT_SPLIT;
+    view.desc.flags = (desc->flags & (LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED)) | LINFUSION_VARIANT_SPLIT;
     st = make_plan(&view.desc, dev.sm_count, &view.plan);
     if (st != LINFUSION_OK) return st;
     const size_t room = (kNoAllocScratchBytes - state_bytes - 256) / per_chunk;
@@ -1016,7 +1023,7 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
     } else {
         // The fp32 state may have been summed over devices: convert it here, not from an image.
         apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-            a, h->state, y, N, p.chunks_apply, h->desc.eps, layout_of(h->desc), nullptr);
+            a, h->state, y, N, p.chunks_apply, kernel_eps(h->desc), layout_of(h->desc), nullptr);
     }
     return cudaGetLastError();
 }
@@ -1044,7 +1051,7 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
         // The state may have been summed over devices since the reduction: rebuild its bf16 image.
         stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->operand, h->tile_counters);
         stream_apply_kernel<PHI><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-            mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, h->desc.eps, h->desc.H);
+            mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, kernel_eps(h->desc), h->desc.H);
     }
     return cudaGetLastError();
 }

@@ -236,8 +236,8 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
             }
         }
         // Every column of the z block holds phi(Q_i) . z for its row.
-        const float inv0 = 1.0f / (acc[C::NBV][0] + eps);
-        const float inv1 = 1.0f / (acc[C::NBV][2] + eps);
+        const float inv0 = row_scale(acc[C::NBV][0], eps);
+        const float inv1 = row_scale(acc[C::NBV][2], eps);
         const long long r0 = static_cast<long long>(tile) * C::TILE_Q + warp * 16 + g, r1 = r0 + 8;
 #pragma unroll
         for (int nb = 0; nb < C::NBV; ++nb) {

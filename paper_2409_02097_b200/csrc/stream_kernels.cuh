@@ -656,7 +656,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             }
             tc_fence_after_sync();
             const float den = __uint_as_float(tmem_load_1col(d_tmem + 64));  // phi(Q_i) . z
-            const float inv = 1.0f / (den + eps);
+            const float inv = row_scale(den, eps);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t d[32];
