@@ -284,6 +284,17 @@ __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bu
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // ---------------------------------------------------------------------------------------------
+// Programmatic dependent launch.  A kernel launched with the programmatic-stream-serialization
+// attribute may be scheduled while the kernel before it in the stream is still running, once every
+// CTA of that kernel has called pdl_launch_dependents() (or has exited).  Its CTAs land on SMs as the
+// earlier kernel's CTAs leave, run their set-up, and block in pdl_wait() until the earlier kernel has
+// completed and its writes are visible: nothing that depends on earlier work in the stream may be
+// touched before pdl_wait().  Without the attribute both calls do nothing.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------------------------
 // tcgen05: tensor memory (TMEM) and the 5th-generation MMA.  A TMEM address is (lane << 16) |
 // column; warp w of a CTA may touch lanes 32*(w%4) .. 32*(w%4)+31 only.
 // ---------------------------------------------------------------------------------------------

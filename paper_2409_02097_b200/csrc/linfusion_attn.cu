@@ -370,6 +370,26 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
     return e;
 }
 
+// Launch with the programmatic-stream-serialization attribute (see pdl_wait() in common.cuh): the
+// kernel's CTAs may be placed, and run their set-up, while the kernel before it drains.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                           Args... args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <int PHI>
 cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                           const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
@@ -381,15 +401,22 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
         !encode_slab_map(&mv, v, h->desc, StreamStateCfg::TILE) ||
         !encode_slab_map(&mq, q, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
         return cudaErrorInvalidValue;
+    cudaError_t e;
     mark(h, 0, s);
-    stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
-        mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
+    e = launch_chained(stream_state_kernel<PHI>, dim3(p.G_state), dim3(StreamStateCfg::THREADS),
+                       StreamStateCfg::SMEM_BYTES, s, mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state,
+                       p.spans, h->desc.H);
+    if (e != cudaSuccess) return e;
     mark(h, 1, s);
-    stream_reduce_kernel<<<dim3((kStreamStateFloats + 255) / 256, p.slabs), 256, 0, s>>>(
-        h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state, p.spans);
+    e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
+                       h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
+                       p.spans);
+    if (e != cudaSuccess) return e;
     mark(h, 2, s);
-    stream_apply_kernel<PHI><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, kernel_eps(h->desc), h->desc.H);
+    e = launch_chained(stream_apply_kernel<PHI>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
+                       mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs,
+                       kernel_eps(h->desc), h->desc.H);
+    if (e != cudaSuccess) return e;
     mark(h, 3, s);
     return cudaGetLastError();
 }

@@ -174,6 +174,10 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Set-up done (barriers, tensor memory): let the next kernel in the stream be scheduled behind
+    // this one, and wait for the one before it to be complete before touching global memory.
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == C::PRODUCER_WARP) {
         // ---------------- producer ----------------
@@ -376,6 +380,8 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
     const int tid = threadIdx.x;
     const int idx = blockIdx.x * 256 + tid;
     const int slab = blockIdx.y;
+    pdl_launch_dependents();
+    pdl_wait();
     if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
     float sum = 0.0f;
     if (idx < kStreamStateFloats) {
@@ -412,6 +418,8 @@ stream_pack_kernel(const float* __restrict__ state, unsigned char* __restrict__ 
     const int tid = threadIdx.x;
     const int idx = blockIdx.x * 256 + tid;
     const int slab = blockIdx.y;
+    pdl_launch_dependents();
+    pdl_wait();
     if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
     sums[tid] = idx < kStreamStateFloats ? state[static_cast<size_t>(slab) * kStreamStateFloats + idx] : 0.0f;
     __syncthreads();
@@ -474,6 +482,10 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Set-up done (barriers, tensor memory): let the next kernel in the stream be scheduled behind
+    // this one, and wait for the one before it to be complete before touching global memory.
+    pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == C::PRODUCER_WARP) {
         // ---------------- producer warp (lane 0 issues; all lanes help to find work and copy B) ----------------
