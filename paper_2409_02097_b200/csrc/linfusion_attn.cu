@@ -316,6 +316,26 @@ cudaError_t set_stream_attrs()
     return e;
 }
 
+// Launch with the programmatic-stream-serialization attribute (see pdl_wait() in common.cuh): the
+// kernel's CTAs may be placed, and run their set-up, while the kernel before it drains.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                           Args... args)
+{
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 template <int D, int PHI>
 cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                          const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
@@ -323,17 +343,21 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
     using C = SplitCfg<D>;
     const Plan& p = h->plan;
     const int N = h->desc.N;
+    cudaError_t e;
     mark(h, 0, s);
-    state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
-        k, v, h->partials, N, p.chunks_state, layout_of(h->desc));
+    e = launch_chained(state_partial_kernel<D, PHI>, dim3(p.chunks_state, p.slabs), dim3(C::NT), C::SMEM_KV, s, k, v,
+                       h->partials, N, p.chunks_state, layout_of(h->desc));
+    if (e != cudaSuccess) return e;
     mark(h, 1, s);
     // h->operand (when the workspace has it) receives the apply kernel's bf16 operand image.
     unsigned char* image = h->operand;
-    state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
-        h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST);
+    e = launch_chained(state_reduce_kernel, dim3((C::STATE_FLOATS + 255) / 256, p.slabs), dim3(256), 0, s,
+                       h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST);
+    if (e != cudaSuccess) return e;
     mark(h, 2, s);
-    apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-        q, h->state, y, N, p.chunks_apply, kernel_eps(h->desc), layout_of(h->desc), image);
+    e = launch_chained(apply_kernel<D, PHI>, dim3(p.chunks_apply, p.slabs), dim3(C::NT), C::SMEM_APPLY, s, q,
+                       h->state, y, N, p.chunks_apply, kernel_eps(h->desc), layout_of(h->desc), image);
+    if (e != cudaSuccess) return e;
     mark(h, 3, s);
     return cudaGetLastError();
 }
@@ -361,33 +385,16 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
                            const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see launch_chained()
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.numAttrs = 2;
     mark(h, 0, s);
     cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state,
                                        h->desc.N, kernel_eps(h->desc), layout_of(h->desc));
     mark(h, 1, s);
     return e;
-}
-
-// Launch with the programmatic-stream-serialization attribute (see pdl_wait() in common.cuh): the
-// kernel's CTAs may be placed, and run their set-up, while the kernel before it drains.
-template <typename... KArgs, typename... Args>
-cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
-                           Args... args)
-{
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
-    cfg.gridDim = grid;
-    cfg.blockDim = block;
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = s;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
 template <int PHI>

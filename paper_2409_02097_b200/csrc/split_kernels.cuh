@@ -290,6 +290,10 @@ __global__ void __launch_bounds__(SplitCfg<D>::NT)
 state_partial_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
                      float* __restrict__ partials, int N, int chunks, SlabLayout L)
 {
+    // Programmatic dependent launch: the next kernel of the stream may be scheduled behind this
+    // one; nothing in global memory is touched before the kernel ahead has completed.
+    pdl_launch_dependents();
+    pdl_wait();
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
     const int slab = blockIdx.y, p = blockIdx.x;
@@ -309,6 +313,10 @@ __global__ void __launch_bounds__(256)
 state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state, int state_floats,
                     int chunks, unsigned char* __restrict__ st_image, int d, int pitch, int image_bytes)
 {
+    // Programmatic dependent launch: the next kernel of the stream may be scheduled behind this
+    // one; nothing in global memory is touched before the kernel ahead has completed.
+    pdl_launch_dependents();
+    pdl_wait();
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= state_floats) return;
     const int slab = blockIdx.y;
@@ -337,6 +345,10 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
              __nv_bfloat16* __restrict__ Y, int N, int chunks, float eps, SlabLayout L,
              const unsigned char* __restrict__ st_image)
 {
+    // Programmatic dependent launch: the next kernel of the stream may be scheduled behind this
+    // one; nothing in global memory is touched before the kernel ahead has completed.
+    pdl_launch_dependents();
+    pdl_wait();
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* St = smem;
@@ -370,6 +382,10 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
                      const __nv_bfloat16* __restrict__ V, __nv_bfloat16* __restrict__ Y,
                      float* __restrict__ state_out, int N, float eps, SlabLayout L)
 {
+    // Programmatic dependent launch: the next kernel of the stream may be scheduled behind this
+    // one; nothing in global memory is touched before the kernel ahead has completed.
+    pdl_launch_dependents();
+    pdl_wait();
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
     float* part = reinterpret_cast<float*>(smem);
