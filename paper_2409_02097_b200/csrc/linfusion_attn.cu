@@ -85,18 +85,16 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
 
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v == LINFUSION_VARIANT_AUTO) {
-        // Measured on B200 over the SD-v1.5 / v2.1 / XL layer shapes: the single clustered launch
-        // wins only at the smallest levels (N <= 192: 15 vs 24 us at N = 144, d = 64; 28 vs 35 us
-        // at N = 64, d = 160).  The persistent TMA + tcgen05 kernels (d = 64) pay a few
-        // microseconds of set-up (tensor-memory allocation, one CTA per SM working through its
-        // tiles in turn) and win once every SM has a dozen 128-token tiles (56 vs 70 us at
-        // N = 16384 x 20 slabs; 33 vs 26 us at N = 2304 x 40 slabs); the three-launch split path
-        // takes the rest.
-        const int cl = largest_cluster(tiles_kv);
+        // Measured on B200 over the SD-v1.5 / v2.1 / XL layer shapes, forwards back to back.  The
+        // persistent TMA + tcgen05 kernels (d = 64) pay a few microseconds of set-up (tensor-memory
+        // allocation, one CTA per SM working through its tiles in turn) and win once every SM has
+        // about eight 128-token tiles (37 vs 41 us at N = 4096 x 40 slabs, 50 vs 70 us at
+        // N = 16384 x 20; 31 vs 29 us at N = 9216 x 10).  Below that the three chained launches of
+        // the split path are the fastest at every shape measured, the smallest levels included
+        // (12.9 us at N = 144, d = 64, against 14.4 us for the single clustered launch; 21.9 vs 27 us
+        // at N = 64, d = 160), so the cluster kernel is only run on request.
         const long long stream_tiles = static_cast<long long>(slabs) * ((d->N + StreamStateCfg::TILE - 1) / StreamStateCfg::TILE);
-        if (d->N <= 192 && static_cast<long long>(slabs) * cl <= 2ll * sm_count)
-            v = LINFUSION_VARIANT_CLUSTER;
-        else if (d->d == kStreamD && stream_tiles >= 12ll * sm_count)
+        if (d->d == kStreamD && stream_tiles >= 8ll * sm_count)
             v = LINFUSION_VARIANT_STREAM;
         else
             v = LINFUSION_VARIANT_SPLIT;
@@ -385,11 +383,8 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
                            const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[2];
+    cudaLaunchAttribute attr[1];
     cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
-    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see launch_chained()
-    attr[1].val.programmaticStreamSerializationAllowed = 1;
-    cfg.numAttrs = 2;
     mark(h, 0, s);
     cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state,
                                        h->desc.N, kernel_eps(h->desc), layout_of(h->desc));

@@ -382,10 +382,6 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
                      const __nv_bfloat16* __restrict__ V, __nv_bfloat16* __restrict__ Y,
                      float* __restrict__ state_out, int N, float eps, SlabLayout L)
 {
-    // Programmatic dependent launch: the next kernel of the stream may be scheduled behind this
-    // one; nothing in global memory is touched before the kernel ahead has completed.
-    pdl_launch_dependents();
-    pdl_wait();
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
     float* part = reinterpret_cast<float*>(smem);
