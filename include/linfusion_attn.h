@@ -194,6 +194,14 @@ linfusion_status_t linfusion_attn_state_buffer(linfusion_attn_t* h, float** dev_
  */
 linfusion_status_t linfusion_attn_enable_kernel_timing(linfusion_attn_t* h, int32_t slots);
 linfusion_status_t linfusion_attn_kernel_times(linfusion_attn_t* h, float* ms_sum, int32_t* calls);
+/*
+ * Sample the timing: only every `stride`-th forward (the first one after enable() included) is
+ * bracketed with events; the others are enqueued exactly as without timing.  An event record between
+ * two kernels keeps the second from being scheduled behind the first (the kernels of a forward
+ * are chained by programmatic dependent launch), so timing every call slows the calls it times;
+ * a stride keeps most of a timed region undisturbed.  Default 1.  Errors: INVALID_ARG (stride < 1).
+ */
+linfusion_status_t linfusion_attn_set_kernel_timing_stride(linfusion_attn_t* h, int32_t stride);
 
 /*
  * The attention without a handle and without any allocation.  (The paper has no counterpart to

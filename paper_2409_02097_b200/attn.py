@@ -25,6 +25,7 @@ EXPORTED = [
     "linfusion_attn_set_workspace", "linfusion_attn_status", "linfusion_attn_read_state",
     "linfusion_attn_variant_name", "linfusion_attn_launches_per_forward",
     "linfusion_attn_enable_kernel_timing", "linfusion_attn_kernel_times",
+    "linfusion_attn_set_kernel_timing_stride",
     "linfusion_attn_forward_noalloc",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
 ]
@@ -82,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_launches_per_forward.argtypes = [vp]
     lib.linfusion_attn_enable_kernel_timing.restype = st
     lib.linfusion_attn_enable_kernel_timing.argtypes = [vp, ctypes.c_int32]
+    lib.linfusion_attn_set_kernel_timing_stride.restype = st
+    lib.linfusion_attn_set_kernel_timing_stride.argtypes = [vp, ctypes.c_int32]
     lib.linfusion_attn_kernel_times.restype = st
     lib.linfusion_attn_kernel_times.argtypes = [vp, ctypes.POINTER(ctypes.c_float),
                                                 ctypes.POINTER(ctypes.c_int32)]
@@ -276,6 +279,11 @@ class LinFusionAttention:
         rc = self._lib.linfusion_attn_enable_kernel_timing(self._h, int(slots))
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_enable_kernel_timing")
+
+    def set_kernel_timing_stride(self, stride: int) -> None:
+        rc = self._lib.linfusion_attn_set_kernel_timing_stride(self._h, int(stride))
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_set_kernel_timing_stride")
 
     def kernel_times(self):
         """([ms_state, ms_reduce, ms_apply] summed, calls) since the last call of this method."""

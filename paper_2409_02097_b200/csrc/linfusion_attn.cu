@@ -236,6 +236,9 @@ struct linfusion_attn {
     cudaEvent_t* events;
     int timing_slots;
     long long timed_calls;
+    int timing_stride;        // every timing_stride-th forward is bracketed with events
+    long long forward_calls;  // forwards since timing was enabled
+    bool sample_now;          // the forward being enqueued is one of them
     struct HostPipe* pipe;  // copy/compute pipeline of the host-buffer entry point (first use)
 };
 
@@ -280,7 +283,7 @@ struct DeviceGuard {
 // Record timing event `i` (0..3) of the current forward, when kernel timing is enabled.
 inline void mark(const linfusion_attn* h, int i, cudaStream_t s)
 {
-    if (h->events != nullptr)
+    if (h->sample_now)
         cudaEventRecord(h->events[(h->timed_calls % h->timing_slots) * 4 + i], s);
 }
 
@@ -529,6 +532,9 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     h->events = nullptr;
     h->timing_slots = 0;
     h->timed_calls = 0;
+    h->timing_stride = 1;
+    h->forward_calls = 0;
+    h->sample_now = false;
     h->pipe = nullptr;
     st = make_plan(desc, h->sm_count, &h->plan);
     if (st != LINFUSION_OK) {
@@ -623,6 +629,7 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
     const __nv_bfloat16* V = static_cast<const __nv_bfloat16*>(v);
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
 
+    h->sample_now = h->events != nullptr && h->forward_calls % h->timing_stride == 0;
     cudaError_t e = cudaErrorInvalidValue;
     if (h->plan.variant == kStream) {
         e = h->desc.phi == LINFUSION_PHI_IDENTITY ? launch_stream<kPhiIdentity>(h, Q, K, V, Y, s)
@@ -633,7 +640,9 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
 #undef LF_LAUNCH
     }
     h->last_stream = s;
-    if (h->events != nullptr) ++h->timed_calls;
+    if (h->events != nullptr) ++h->forward_calls;
+    if (h->sample_now) ++h->timed_calls;
+    h->sample_now = false;
     if (e != cudaSuccess) {
         cudaGetLastError();
         return LINFUSION_ERR_CUDA;
@@ -654,6 +663,8 @@ linfusion_status_t linfusion_attn_enable_kernel_timing(linfusion_attn_t* h, int3
     }
     h->timing_slots = 0;
     h->timed_calls = 0;
+    h->forward_calls = 0;
+    h->sample_now = false;
     if (slots == 0) return LINFUSION_OK;
     cudaEvent_t* ev = new (std::nothrow) cudaEvent_t[slots * 4];
     if (ev == nullptr) return LINFUSION_ERR_ALLOC;
@@ -667,6 +678,13 @@ linfusion_status_t linfusion_attn_enable_kernel_timing(linfusion_attn_t* h, int3
     }
     h->events = ev;
     h->timing_slots = slots;
+    return LINFUSION_OK;
+}
+
+linfusion_status_t linfusion_attn_set_kernel_timing_stride(linfusion_attn_t* h, int32_t stride)
+{
+    if (h == nullptr || stride < 1) return LINFUSION_ERR_INVALID_ARG;
+    h->timing_stride = stride;
     return LINFUSION_OK;
 }
 
@@ -1008,6 +1026,9 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     view.events = nullptr;
     view.timing_slots = 0;
     view.timed_calls = 0;
+    view.timing_stride = 1;
+    view.forward_calls = 0;
+    view.sample_now = false;
     view.pipe = nullptr;
 
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);

@@ -283,3 +283,21 @@ def test_token_major_layout_gives_the_same_bits(dims, variant):
         torch.cuda.synchronize()
         assert_parity(y2.permute(0, 2, 1, 3), oracle_y(q, k, v), f"token-major noalloc {dims}")
     op.close()
+
+
+def test_kernel_timing_stride_samples_every_nth_forward():
+    shape = wl.find_shape("sdxl_2048_L1")
+    q, k, v = wl.make_qkv(shape, seed=3, device="cuda")
+    y, op = run_gpu(q, k, v, "stream")
+    op.enable_kernel_timing(16)
+    op.set_kernel_timing_stride(4)
+    outs = [op.forward(q, k, v).clone() for _ in range(10)]
+    sums, calls = op.kernel_times()
+    assert calls == 3                      # forwards 0, 4 and 8
+    assert all(t > 0 for t in sums)
+    op.enable_kernel_timing(0)
+    for o in outs:                         # timed or not, chained or not: the same bits
+        assert torch.equal(o.view(torch.int16), y.view(torch.int16))
+    with pytest.raises(attn.LinFusionError):
+        op.set_kernel_timing_stride(0)
+    op.close()
