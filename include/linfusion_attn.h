@@ -61,8 +61,10 @@ typedef enum {
  * token-major [B, N, H, d] — the [B, N, C] tensor a UNet block holds, with C = H*d split into
  * heads in place — so that the caller needs no transpose before or after the attention (a
  * transpose pass would move twice the attention's own minimum traffic).  Every entry point that
- * takes a descriptor or a handle follows it; the arithmetic and its order are the same, so Y has
- * the same bits as in the head-major layout.
+ * takes a descriptor or a handle follows it.  The split and cluster variants do the same arithmetic
+ * in the same order in both layouts (same bits); the stream variant uses another fixed split of N
+ * in this layout (the same number of CTAs on every slab, which keeps the heads of a token in step),
+ * so its last bits may differ from the head-major result, reproducibly.
  */
 #define LINFUSION_LAYOUT_TOKEN_MAJOR 0x10u
 

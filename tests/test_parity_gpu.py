@@ -258,8 +258,10 @@ def test_forward_host_pipelined_groups():
                                           ((1, 4, 130, 160), "cluster"), ((2, 5, 100, 64), "cluster"),
                                           ((1, 3, 2049, 80), "auto")], ids=lambda x: str(x))
 def test_token_major_layout_gives_the_same_bits(dims, variant):
-    """[B, N, H, d] tensors (a UNet's [B, N, C] with heads split in place): same arithmetic in the
-    same order as the head-major layout, so the outputs must agree bit for bit."""
+    """[B, N, H, d] tensors (a UNet's [B, N, C] with heads split in place).  The split and cluster
+    variants do the same arithmetic in the same order as in the head-major layout, so their outputs
+    must agree bit for bit; the stream variant deals its CTAs to the slabs differently in this
+    layout (another fixed split of N), so there only the last bits may differ."""
     B, H, N, d = dims
     q, k, v = wl.make_small(B, H, N, d, seed=23, device="cuda")
     y_hm, op = run_gpu(q, k, v, variant)
@@ -272,7 +274,15 @@ def test_token_major_layout_gives_the_same_bits(dims, variant):
     torch.cuda.synchronize()
     assert op.status() == attn.OK
     assert y_tm.shape == (B, N, H, d)
-    assert torch.equal(y_tm.permute(0, 2, 1, 3).contiguous().view(torch.int16), y_hm.view(torch.int16))
+    y_back = y_tm.permute(0, 2, 1, 3).contiguous()
+    if resolved == "stream":
+        diff = (y_back.float() - y_hm.float()).abs()
+        assert (diff <= 2.0 ** -7 * y_hm.float().abs() + 1e-30).all()      # at most one bf16 ulp apart
+        y_again = op.forward(qt, kt, vt)                                       # and reproducible
+        torch.cuda.synchronize()
+        assert torch.equal(y_again.view(torch.int16), y_tm.view(torch.int16))
+    else:
+        assert torch.equal(y_back.view(torch.int16), y_hm.view(torch.int16))
     assert_parity(y_tm.permute(0, 2, 1, 3), oracle_y(q, k, v), f"token-major {dims} {variant}")
     # the allocation-free entry point follows the layout flag too
     if d != 160 or B * H <= 81:
