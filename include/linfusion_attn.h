@@ -75,6 +75,15 @@ typedef enum {
  * |Y| grows with N in this form (the paper's reason for the normalizer); outputs are still bf16.
  */
 #define LINFUSION_FLAG_UNNORMALIZED 0x20u
+/*
+ * flags: storage type of Q, K, V and Y.  Default (bit clear): bf16.  Bit set: fp16 (IEEE half), the
+ * precision the paper's implementation runs in.  Accumulation is fp32 either way.  With fp16 the
+ * state S | z, whose entries grow with N, is handed to the apply step's tensor-core operand scaled
+ * by 2^-ceil(log2 N) so that it fits the format (the scale cancels in Eq. 5's quotient; eps is
+ * scaled with it); read_state() returns the unscaled fp32 state.  The un-normalized operator's
+ * output itself grows like sqrt(N) and must fit fp16's range (65504) in that case.
+ */
+#define LINFUSION_DTYPE_FP16 0x40u
 
 typedef struct {
     int32_t B;      /* batch                                   > 0 */

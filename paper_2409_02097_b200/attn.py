@@ -106,13 +106,18 @@ def status_string(code: int) -> str:
 
 LAYOUT_TOKEN_MAJOR = 0x10   # tensors are [B, N, H, d] instead of [B, H, N, d]
 FLAG_UNNORMALIZED = 0x20    # Y_i = phi(Q_i) S, without the division by phi(Q_i) . z + eps
+DTYPE_FP16 = 0x40           # Q, K, V, Y are fp16 instead of bf16
 
 
 def make_desc(B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
-              layout="head_major", normalize=True) -> Desc:
+              layout="head_major", normalize=True, dtype="bf16") -> Desc:
     flags = VARIANTS[variant] if isinstance(variant, str) else int(variant)
     if not normalize:
         flags |= FLAG_UNNORMALIZED
+    if dtype == "fp16":
+        flags |= DTYPE_FP16
+    elif dtype != "bf16":
+        raise ValueError("dtype must be 'bf16' or 'fp16'")
     if layout == "token_major":
         flags |= LAYOUT_TOKEN_MAJOR
     elif layout != "head_major":
@@ -174,8 +179,9 @@ class LinFusionAttention:
     with ``layout="token_major"``)."""
 
     def __init__(self, B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
-                 layout="head_major", normalize=True):
-        self.desc = make_desc(B, H, N, d, phi, eps, device, variant, layout, normalize)
+                 layout="head_major", normalize=True, dtype="bf16"):
+        self.desc = make_desc(B, H, N, d, phi, eps, device, variant, layout, normalize, dtype)
+        self.dtype = dtype
         # tensors are [B, H, N, d], or [B, N, H, d] in the token-major layout
         self.shape = (int(B), int(H), int(N), int(d)) if layout == "head_major" else \
                      (int(B), int(N), int(H), int(d))
@@ -195,8 +201,9 @@ class LinFusionAttention:
     # -- calls ------------------------------------------------------------------------------
     def _check(self, t, name):
         import torch
-        if tuple(t.shape) != self.shape or t.dtype != torch.bfloat16 or not t.is_contiguous():
-            raise ValueError(f"{name}: expected contiguous bf16 tensor of shape {self.shape}")
+        want = torch.float16 if self.dtype == "fp16" else torch.bfloat16
+        if tuple(t.shape) != self.shape or t.dtype != want or not t.is_contiguous():
+            raise ValueError(f"{name}: expected contiguous {self.dtype} tensor of shape {self.shape}")
 
     def forward(self, q, k, v, y=None, stream: Optional[int] = None):
         import torch

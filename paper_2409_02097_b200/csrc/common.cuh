@@ -13,6 +13,14 @@ namespace lf {
 constexpr int kPhiEluPlusOne = 0;
 constexpr int kPhiIdentity = 1;
 
+// Storage type of Q, K, V, Y (and of the MMA operands).  Kernels are instantiated on one integer
+// KIND = phi | (dtype << 1); pointers to 16-bit data are typed __nv_bfloat16 whatever the dtype.
+constexpr int kDtypeBf16 = 0;
+constexpr int kDtypeFp16 = 1;
+__host__ __device__ constexpr int make_kind(int phi, int dtype) { return phi | (dtype << 1); }
+__host__ __device__ constexpr int kind_phi(int kind) { return kind & 1; }
+__host__ __device__ constexpr int kind_dtype(int kind) { return kind >> 1; }
+
 // Status word values written by kernels (0 = fine).
 constexpr uint32_t kStatusOk = 0u;
 constexpr uint32_t kStatusWaitExpired = 1u;
@@ -52,19 +60,26 @@ __device__ __forceinline__ float ex2_approx(float x)
     return y;
 }
 
-template <int PHI>
+template <int KIND>
 __device__ __forceinline__ float phi(float x)
 {
-    if (PHI == kPhiIdentity) return x;
+    if (kind_phi(KIND) == kPhiIdentity) return x;
     return fmaxf(x, 0.0f) + ex2_approx(fminf(x, 0.0f) * 1.4426950408889634f);
 }
 
-// Row scale of the apply step: 1 / (phi(Q_i) . z + eps) (Eq. 5), or 1 for the operator without
-// its normalizer, which the host requests by passing a negative eps.
+// Row scale of the apply step: 1 / (phi(Q_i) . z + eps) (Eq. 5), or `unnormalized_scale` for the
+// operator without its normalizer, which the host requests by passing a negative eps.  (With fp16
+// operands S | z are held scaled by a power of two s so that z fits the format; the scale cancels
+// in the quotient when eps is scaled too, and unnormalized_scale = 1/s undoes it otherwise.)
 constexpr float kEpsUnnormalized = -1.0f;
-__device__ __forceinline__ float row_scale(float den, float eps)
+struct ApplyScales {
+    float eps;           // eps * operand, or kEpsUnnormalized
+    float unnormalized;  // 1 / operand
+    float operand;       // the power of two s that S | z are multiplied by when they become an MMA operand
+};
+__device__ __forceinline__ float row_scale(float den, const ApplyScales& sc)
 {
-    return eps < 0.0f ? 1.0f : 1.0f / (den + eps);
+    return sc.eps < 0.0f ? sc.unnormalized : 1.0f / (den + sc.eps);
 }
 
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
@@ -77,27 +92,84 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
     return r;
 }
-
-template <int PHI>
-__device__ __forceinline__ uint32_t phi_bf16x2(uint32_t p)
+__device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi)
 {
-    return pack_bf16x2(phi<PHI>(bf16_lo(p)), phi<PHI>(bf16_hi(p)));
+    uint32_t r;
+    asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
 }
 
-// The same activation on a packed bf16 pair, entirely in bf16x2 arithmetic (6 instructions per
-// pair instead of 13 through fp32).  log2(e) is split into a bf16 head and tail so that
-// t = min(x,0) * log2(e) is the correctly rounded bf16 product (one fused rounding); rounding t
-// to bf16 adds a relative error of about |x| * 2^-9 to exp(x), and the bf16 exponential
-// instruction rounds its result toward zero (measured mean -0.27 % on the negative side, where
-// the fp32 route has none) — both of the order of the bf16 rounding the MMA operand gets anyway.
-template <int PHI>
-__device__ __forceinline__ uint32_t phi_packed_bf16x2(uint32_t p)
+// Packed pair of the kernel's storage type <-> two floats.
+template <int KIND>
+__device__ __forceinline__ uint32_t pack_pair(float lo, float hi)
 {
-    if (PHI == kPhiIdentity) return p;
+    return kind_dtype(KIND) == kDtypeFp16 ? pack_f16x2(lo, hi) : pack_bf16x2(lo, hi);
+}
+template <int KIND>
+__device__ __forceinline__ float pair_lo(uint32_t p)
+{
+    if (kind_dtype(KIND) == kDtypeFp16) {
+        float f;
+        asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tcvt.f32.f16 %0, l;\n\t}" : "=f"(f) : "r"(p));
+        return f;
+    }
+    return bf16_lo(p);
+}
+template <int KIND>
+__device__ __forceinline__ float pair_hi(uint32_t p)
+{
+    if (kind_dtype(KIND) == kDtypeFp16) {
+        float f;
+        asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %1;\n\tcvt.f32.f16 %0, h;\n\t}" : "=f"(f) : "r"(p));
+        return f;
+    }
+    return bf16_hi(p);
+}
+// The pair (1, 1).
+template <int KIND>
+__device__ __forceinline__ constexpr uint32_t ones_pair()
+{
+    return kind_dtype(KIND) == kDtypeFp16 ? 0x3C003C00u : 0x3F803F80u;
+}
+// One float -> the 16-bit storage type, by a run-time dtype (kernels that are not instantiated per kind).
+__device__ __forceinline__ uint16_t to_storage16(float x, int dtype)
+{
+    const uint32_t p = dtype == kDtypeFp16 ? pack_f16x2(x, 0.0f) : pack_bf16x2(x, 0.0f);
+    return static_cast<uint16_t>(p & 0xffffu);
+}
+
+template <int KIND>
+__device__ __forceinline__ uint32_t phi_pair(uint32_t p)
+{
+    return pack_pair<KIND>(phi<KIND>(pair_lo<KIND>(p)), phi<KIND>(pair_hi<KIND>(p)));
+}
+
+// The same activation on a packed pair, entirely in packed 16-bit arithmetic (6 PTX instructions per
+// pair instead of 13 through fp32).  log2(e) is split into a head and a tail of the format so that
+// t = min(x,0) * log2(e) is the correctly rounded product (one fused rounding).  bf16: rounding t
+// adds a relative error of about |x| * 2^-9 to exp(x), and the bf16 exponential instruction rounds
+// its result toward zero (measured mean -0.27 % on the negative side, where the fp32 route has
+// none) — both of the order of the bf16 rounding the MMA operand gets anyway.  fp16 has three more
+// mantissa bits and the same structure.
+template <int KIND>
+__device__ __forceinline__ uint32_t phi_packed_pair(uint32_t p)
+{
+    if (kind_phi(KIND) == kPhiIdentity) return p;
     const uint32_t zero = 0u;
+    uint32_t m, u, t, e, r;
+    if (kind_dtype(KIND) == kDtypeFp16) {
+        const uint32_t log2e_hi = 0x3DC53DC5u;  // fp16 pair 1.4423828125
+        const uint32_t log2e_lo = 0x0D1E0D1Eu;  // fp16 pair log2(e) - 1.4423828125 = 3.1233e-4
+        asm("min.f16x2 %0, %1, %2;" : "=r"(m) : "r"(p), "r"(zero));
+        asm("mul.rn.f16x2 %0, %1, %2;" : "=r"(u) : "r"(m), "r"(log2e_lo));
+        asm("fma.rn.f16x2 %0, %1, %2, %3;" : "=r"(t) : "r"(m), "r"(log2e_hi), "r"(u));
+        asm("ex2.approx.f16x2 %0, %1;" : "=r"(e) : "r"(t));
+        asm("max.f16x2 %0, %1, %2;" : "=r"(r) : "r"(p), "r"(zero));
+        asm("add.rn.f16x2 %0, %1, %2;" : "=r"(r) : "r"(r), "r"(e));
+        return r;
+    }
     const uint32_t log2e_hi = 0x3FB93FB9u;  // bf16 pair 1.4453125
     const uint32_t log2e_lo = 0xBB2CBB2Cu;  // bf16 pair log2(e) - 1.4453125 = -0.0026245
-    uint32_t m, u, t, e, r;
     asm("min.bf16x2 %0, %1, %2;" : "=r"(m) : "r"(p), "r"(zero));
     asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(u) : "r"(m), "r"(log2e_lo));
     asm("fma.rn.bf16x2 %0, %1, %2, %3;" : "=r"(t) : "r"(m), "r"(log2e_hi), "r"(u));
@@ -131,26 +203,23 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, u
                  : "r"(addr));
 }
 
-// D(16x8, fp32) += A(16x16, bf16, row) * B(16x8, bf16, col)
-__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                               uint32_t a3, uint32_t b0, uint32_t b1)
+// D(16x8, fp32) += A(16x16, row) * B(16x8, col), operands bf16 or fp16 by KIND
+template <int KIND>
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1)
 {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// D(16x8, fp32) = A * B (accumulator starts at zero; saves clearing the registers first)
-__device__ __forceinline__ void mma_bf16_16816_init(float (&c)[4], uint32_t a0, uint32_t a1,
-                                                    uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
-{
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
-        "{%10,%10,%10,%10};"
-        : "=f"(c[0]), "=f"(c[1]), "=f"(c[2]), "=f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "f"(0.0f));
+    if (kind_dtype(KIND) == kDtypeFp16)
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+            "{%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+            "{%0,%1,%2,%3};"
+            : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -388,17 +457,18 @@ __device__ __forceinline__ uint64_t umma_desc_mnmajor_sw128(uint32_t smem_addr, 
     d |= static_cast<uint64_t>(2) << 61;
     return d;
 }
-// Instruction descriptor of kind::f16 with bf16 A and B and fp32 accumulation, M x N; the operands
+// Instruction descriptor of kind::f16 with bf16 or fp16 A and B and fp32 accumulation, M x N; the operands
 // are K-major unless the flags say MN-major.
 constexpr uint32_t kUmmaAMnMajor = 1u << 15;
 constexpr uint32_t kUmmaBMnMajor = 1u << 16;
-__host__ __device__ constexpr uint32_t umma_idesc_bf16_f32(int M, int N, uint32_t major_flags = 0u)
+__host__ __device__ constexpr uint32_t umma_idesc_f32acc(int dtype, int M, int N, uint32_t major_flags = 0u)
 {
-    return (1u << 4) /*D fp32*/ | (1u << 7) /*A bf16*/ | (1u << 10) /*B bf16*/ | major_flags |
+    // A and B formats: 0 = fp16, 1 = bf16 (both operands always have the same type)
+    return (1u << 4) /*D fp32*/ | ((dtype == kDtypeFp16 ? 0u : 1u) << 7) | ((dtype == kDtypeFp16 ? 0u : 1u) << 10) | major_flags |
            (static_cast<uint32_t>(N >> 3) << 17) | (static_cast<uint32_t>(M >> 4) << 24);
 }
-// D[tmem] (+)= A[tmem] * B[smem]; one thread issues it for the CTA.  A and B are both bf16.
-__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+// D[tmem] (+)= A[tmem] * B[smem]; one thread issues it for the CTA.  A and B have the same 16-bit type.
+__device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                              uint32_t accumulate)
 {
     asm volatile(
@@ -408,7 +478,7 @@ __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, u
         : "memory");
 }
 // The same with A from shared memory as well.
-__device__ __forceinline__ void umma_bf16_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                              uint32_t accumulate)
 {
     asm volatile(

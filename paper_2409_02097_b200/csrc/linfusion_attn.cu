@@ -56,7 +56,8 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
     if (!supported_d(d->d)) return LINFUSION_ERR_UNSUPPORTED;
     if (d->phi != LINFUSION_PHI_ELU_PLUS_ONE && d->phi != LINFUSION_PHI_IDENTITY)
         return LINFUSION_ERR_UNSUPPORTED;
-    if ((d->flags & ~(LINFUSION_VARIANT_MASK | LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED)) != 0u)
+    if ((d->flags & ~(LINFUSION_VARIANT_MASK | LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED |
+                      LINFUSION_DTYPE_FP16)) != 0u)
         return LINFUSION_ERR_UNSUPPORTED;
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v > LINFUSION_VARIANT_CLUSTER) return LINFUSION_ERR_UNSUPPORTED;
@@ -178,11 +179,44 @@ EncodeTiledFn get_encode_fn()
     return fn;
 }
 
-// eps as the apply kernels take it: negative selects the operator without its normalizer.
-float kernel_eps(const linfusion_attn_desc_t& d)
+// KIND the kernels are instantiated on: phi and the 16-bit storage type.
+int kind_of(const linfusion_attn_desc_t& d)
 {
-    return (d.flags & LINFUSION_FLAG_UNNORMALIZED) != 0u ? kEpsUnnormalized : d.eps;
+    return make_kind(d.phi == LINFUSION_PHI_IDENTITY ? kPhiIdentity : kPhiEluPlusOne,
+                     (d.flags & LINFUSION_DTYPE_FP16) != 0u ? kDtypeFp16 : kDtypeBf16);
 }
+int dtype_of(const linfusion_attn_desc_t& d) { return kind_dtype(kind_of(d)); }
+
+// Power of two that S | z are multiplied by when they become the apply kernel's MMA operand.  bf16
+// has fp32's range: 1.  fp16 tops out at 65504 and z ~ N, so 2^-ceil(log2 N): z stays below ~8,
+// S at its natural 1/sqrt(N) relative size.  The scale cancels in the quotient of Eq. 5.
+float operand_scale(const linfusion_attn_desc_t& d)
+{
+    if (dtype_of(d) != kDtypeFp16) return 1.0f;
+    int k = 0;
+    while ((1ll << k) < d.N) ++k;
+    return std::ldexp(1.0f, -k);
+}
+
+// What the apply kernels take besides the tensors: a negative eps selects the operator without
+// its normalizer (whose result must have the operand scale taken out again).
+ApplyScales apply_scales(const linfusion_attn_desc_t& d)
+{
+    ApplyScales sc;
+    sc.operand = operand_scale(d);
+    sc.unnormalized = 1.0f / sc.operand;
+    sc.eps = (d.flags & LINFUSION_FLAG_UNNORMALIZED) != 0u ? kEpsUnnormalized : d.eps * sc.operand;
+    return sc;
+}
+
+#define LF_DISPATCH_KIND(kval, CALL) \
+    switch (kval) {                  \
+        case 0: CALL(0); break;      \
+        case 1: CALL(1); break;      \
+        case 2: CALL(2); break;      \
+        case 3: CALL(3); break;      \
+        default: break;              \
+    }
 
 // Element strides of a slab's rows for the layout the descriptor asks for.
 SlabLayout layout_of(const linfusion_attn_desc_t& d)
@@ -361,11 +395,12 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
     // h->operand (when the workspace has it) receives the apply kernel's bf16 operand image.
     unsigned char* image = h->operand;
     e = launch_chained(state_reduce_kernel, dim3((C::STATE_FLOATS + 255) / 256, p.slabs), dim3(256), 0, s,
-                       h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST);
+                       h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST,
+                       dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 2, s);
     e = launch_chained(apply_kernel<D, PHI>, dim3(p.chunks_apply, p.slabs), dim3(C::NT), C::SMEM_APPLY, s, q,
-                       h->state, y, N, p.chunks_apply, kernel_eps(h->desc), layout_of(h->desc), image);
+                       h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), image);
     if (e != cudaSuccess) return e;
     mark(h, 3, s);
     return cudaGetLastError();
@@ -398,7 +433,7 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
     cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
     mark(h, 0, s);
     cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state,
-                                       h->desc.N, kernel_eps(h->desc), layout_of(h->desc));
+                                       h->desc.N, apply_scales(h->desc), layout_of(h->desc));
     mark(h, 1, s);
     return e;
 }
@@ -423,34 +458,42 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
     mark(h, 1, s);
     e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
                        h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
-                       p.spans);
+                       p.spans, dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 2, s);
     e = launch_chained(stream_apply_kernel<PHI>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
                        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs,
-                       kernel_eps(h->desc), h->desc.H);
+                       apply_scales(h->desc), h->desc.H);
     if (e != cudaSuccess) return e;
     mark(h, 3, s);
     return cudaGetLastError();
 }
 
 template <int D>
-cudaError_t set_attrs_d(int phi)
+cudaError_t set_attrs_d(int kind)
 {
-    return phi == LINFUSION_PHI_IDENTITY ? set_split_attrs<D, kPhiIdentity>()
-                                         : set_split_attrs<D, kPhiEluPlusOne>();
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV) e = set_split_attrs<D, KV>()
+    LF_DISPATCH_KIND(kind, LF_K)
+#undef LF_K
+    return e;
 }
 
 template <int D>
 cudaError_t launch_d(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                      const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
-    const bool ident = h->desc.phi == LINFUSION_PHI_IDENTITY;
-    if (h->plan.variant == kCluster)
-        return ident ? launch_cluster<D, kPhiIdentity>(h, q, k, v, y, s)
-                     : launch_cluster<D, kPhiEluPlusOne>(h, q, k, v, y, s);
-    return ident ? launch_split<D, kPhiIdentity>(h, q, k, v, y, s)
-                 : launch_split<D, kPhiEluPlusOne>(h, q, k, v, y, s);
+    cudaError_t e = cudaErrorInvalidValue;
+    if (h->plan.variant == kCluster) {
+#define LF_K(KV) e = launch_cluster<D, KV>(h, q, k, v, y, s)
+        LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
+    } else {
+#define LF_K(KV) e = launch_split<D, KV>(h, q, k, v, y, s)
+        LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
+    }
+    return e;
 }
 
 #define LF_DISPATCH_D(dval, CALL)   \
@@ -465,15 +508,16 @@ cudaError_t launch_d(const linfusion_attn* h, const __nv_bfloat16* q, const __nv
     }
 
 template <int D>
-bool cluster_fits(int phi, int cluster_size, int slabs)
+bool cluster_fits(int kind, int cluster_size, int slabs)
 {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     cluster_config<D>(&cfg, attr, cluster_size, slabs, nullptr);
     int n = 0;
-    cudaError_t e = phi == LINFUSION_PHI_IDENTITY
-                        ? cudaOccupancyMaxActiveClusters(&n, cluster_fused_kernel<D, kPhiIdentity>, &cfg)
-                        : cudaOccupancyMaxActiveClusters(&n, cluster_fused_kernel<D, kPhiEluPlusOne>, &cfg);
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV) e = cudaOccupancyMaxActiveClusters(&n, cluster_fused_kernel<D, KV>, &cfg)
+    LF_DISPATCH_KIND(kind, LF_K)
+#undef LF_K
     if (e != cudaSuccess) {
         cudaGetLastError();
         return false;
@@ -551,12 +595,14 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     }
 
     cudaError_t e = cudaSuccess;
-#define LF_SET(DV) e = set_attrs_d<DV>(desc->phi)
+#define LF_SET(DV) e = set_attrs_d<DV>(kind_of(*desc))
     LF_DISPATCH_D(desc->d, LF_SET)
 #undef LF_SET
-    if (e == cudaSuccess && desc->d == kStreamD)
-        e = desc->phi == LINFUSION_PHI_IDENTITY ? set_stream_attrs<kPhiIdentity>()
-                                                : set_stream_attrs<kPhiEluPlusOne>();
+    if (e == cudaSuccess && desc->d == kStreamD) {
+#define LF_K(KV) e = set_stream_attrs<KV>()
+        LF_DISPATCH_KIND(kind_of(*desc), LF_K)
+#undef LF_K
+    }
     if (e != cudaSuccess) {
         cudaGetLastError();
         delete h;
@@ -568,7 +614,7 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
         bool fits = false;
         const bool forced = (desc->flags & LINFUSION_VARIANT_MASK) == LINFUSION_VARIANT_CLUSTER;
         while (true) {
-#define LF_FIT(DV) fits = cluster_fits<DV>(desc->phi, h->plan.cluster_size, h->plan.slabs)
+#define LF_FIT(DV) fits = cluster_fits<DV>(kind_of(*desc), h->plan.cluster_size, h->plan.slabs)
             LF_DISPATCH_D(desc->d, LF_FIT)
 #undef LF_FIT
             if (fits || h->plan.cluster_size == 1) break;
@@ -640,8 +686,9 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
     h->sample_now = h->events != nullptr && h->forward_calls % h->timing_stride == 0;
     cudaError_t e = cudaErrorInvalidValue;
     if (h->plan.variant == kStream) {
-        e = h->desc.phi == LINFUSION_PHI_IDENTITY ? launch_stream<kPhiIdentity>(h, Q, K, V, Y, s)
-                                                  : launch_stream<kPhiEluPlusOne>(h, Q, K, V, Y, s);
+#define LF_K(KV) e = launch_stream<KV>(h, Q, K, V, Y, s)
+        LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
     } else {
 #define LF_LAUNCH(DV) e = launch_d<DV>(h, Q, K, V, Y, s)
         LF_DISPATCH_D(h->desc.d, LF_LAUNCH)
@@ -762,7 +809,8 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
             linfusion_attn_desc_t d = h->desc;
             d.B = 1;
             d.H = slabs / p->groups;
-            d.flags = static_cast<uint32_t>(h->plan.variant) | (h->desc.flags & LINFUSION_FLAG_UNNORMALIZED);  // head-major only (see the grouping rule above)
+            d.flags = static_cast<uint32_t>(h->plan.variant) |
+                      (h->desc.flags & (LINFUSION_FLAG_UNNORMALIZED | LINFUSION_DTYPE_FP16));  // head-major only (see the grouping rule above)
             ok = linfusion_attn_create(&d, &p->sub) == LINFUSION_OK;
             ok = ok && cudaStreamCreateWithFlags(&p->copy_in, cudaStreamNonBlocking) == cudaSuccess;
             ok = ok && cudaStreamCreateWithFlags(&p->copy_out, cudaStreamNonBlocking) == cudaSuccess;
@@ -945,7 +993,7 @@ NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
 // Once per device, with that device current: resolve the array's device address (the symbol's
 // name is only a host-side stand-in and must never be handed to a kernel), read the SM count
 // and raise the kernels' dynamic shared-memory limits.
-linfusion_status_t noalloc_setup(int device, int d, int phi)
+linfusion_status_t noalloc_setup(int device, int d, int kind)
 {
     NoAllocDevice& dev = g_noalloc_dev[device];
     if (!dev.ready) {
@@ -965,7 +1013,7 @@ linfusion_status_t noalloc_setup(int device, int d, int phi)
         dev.ready = true;
     }
     cudaError_t e = cudaSuccess;
-#define LF_SET(DV) e = set_attrs_d<DV>(phi)
+#define LF_SET(DV) e = set_attrs_d<DV>(kind)
     LF_DISPATCH_D(d, LF_SET)
 #undef LF_SET
     if (e != cudaSuccess) {
@@ -1006,7 +1054,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     if (desc->device >= ndev) return LINFUSION_ERR_INVALID_ARG;
     DeviceGuard guard(desc->device);
     if (!guard.ok) return LINFUSION_ERR_CUDA;
-    st = noalloc_setup(desc->device, desc->d, desc->phi);
+    st = noalloc_setup(desc->device, desc->d, kind_of(*desc));
     if (st != LINFUSION_OK) return st;
     const NoAllocDevice& dev = g_noalloc_dev[desc->device];
 
@@ -1015,7 +1063,8 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     // and every state element that is read in this call is written earlier in the same call.
     linfusion_attn view;
     view.desc = *desc;
-    view.desc.flags = (desc->flags & (LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED)) | LINFUSION_VARIANT_SPLIT;
+    view.desc.flags = (desc->flags & (LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED | LINFUSION_DTYPE_FP16)) |
+                      LINFUSION_VARIANT_SPLIT;
     st = make_plan(&view.desc, dev.sm_count, &view.plan);
     if (st != LINFUSION_OK) return st;
     const size_t room = (kNoAllocScratchBytes - state_bytes - 256) / per_chunk;
@@ -1045,9 +1094,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     const __nv_bfloat16* V = static_cast<const __nv_bfloat16*>(v);
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
     cudaError_t e = cudaErrorInvalidValue;
-#define LF_LAUNCH(DV)                                                                           \
-    e = view.desc.phi == LINFUSION_PHI_IDENTITY ? launch_split<DV, kPhiIdentity>(&view, Q, K, V, Y, s) \
-                                                : launch_split<DV, kPhiEluPlusOne>(&view, Q, K, V, Y, s)
+#define LF_LAUNCH(DV) e = launch_d<DV>(&view, Q, K, V, Y, s)
     LF_DISPATCH_D(view.desc.d, LF_LAUNCH)
 #undef LF_LAUNCH
     if (e != cudaSuccess) {
@@ -1077,11 +1124,12 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
         state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
             a, b, h->partials, N, p.chunks_state, layout_of(h->desc));
         state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
-            h->partials, h->state, C::STATE_FLOATS, p.chunks_state, nullptr, D, C::PITCH, C::SMEM_ST);
+            h->partials, h->state, C::STATE_FLOATS, p.chunks_state, nullptr, D, C::PITCH, C::SMEM_ST,
+            dtype_of(h->desc), operand_scale(h->desc));
     } else {
         // The fp32 state may have been summed over devices: convert it here, not from an image.
         apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-            a, h->state, y, N, p.chunks_apply, kernel_eps(h->desc), layout_of(h->desc), nullptr);
+            a, h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), nullptr);
     }
     return cudaGetLastError();
 }
@@ -1101,17 +1149,30 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
         stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
             mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
         stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->operand, h->tile_counters,
-                                                  p.tiles_state, p.W_state, p.G_state, p.spans);
+                                                  p.tiles_state, p.W_state, p.G_state, p.spans,
+                                                  dtype_of(h->desc), operand_scale(h->desc));
     } else {
         CUtensorMap mq, my;
         if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
             return cudaErrorInvalidValue;
         // The state may have been summed over devices since the reduction: rebuild its bf16 image.
-        stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->operand, h->tile_counters);
+        stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->operand, h->tile_counters, dtype_of(h->desc),
+                                                operand_scale(h->desc));
         stream_apply_kernel<PHI><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-            mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, kernel_eps(h->desc), h->desc.H);
+            mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, apply_scales(h->desc), h->desc.H);
     }
     return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t split_half_d(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a, const __nv_bfloat16* b,
+                         __nv_bfloat16* y, cudaStream_t s)
+{
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV) e = launch_split_half<D, KV>(h, state_half, a, b, y, s)
+    LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
+    return e;
 }
 
 linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, const void* b, void* y,
@@ -1131,15 +1192,13 @@ linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, c
     const __nv_bfloat16* A = static_cast<const __nv_bfloat16*>(a);
     const __nv_bfloat16* B = static_cast<const __nv_bfloat16*>(b);
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
-    const bool ident = h->desc.phi == LINFUSION_PHI_IDENTITY;
     cudaError_t e = cudaErrorInvalidValue;
     if (h->plan.variant == kStream) {
-        e = ident ? launch_stream_half<kPhiIdentity>(h, state_half, A, B, Y, s)
-                  : launch_stream_half<kPhiEluPlusOne>(h, state_half, A, B, Y, s);
+#define LF_K(KV) e = launch_stream_half<KV>(h, state_half, A, B, Y, s)
+        LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
     } else {
-#define LF_HALF(DV)                                                                    \
-    e = ident ? launch_split_half<DV, kPhiIdentity>(h, state_half, A, B, Y, s)         \
-              : launch_split_half<DV, kPhiEluPlusOne>(h, state_half, A, B, Y, s)
+#define LF_HALF(DV) e = split_half_d<DV>(h, state_half, A, B, Y, s)
         LF_DISPATCH_D(h->desc.d, LF_HALF)
 #undef LF_HALF
     }

@@ -100,10 +100,10 @@ __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict
             bool ok = (j < N) && (ch * 8 < D);
             uint4 pk = zero4;  // rows past N and pad channels contribute nothing (not phi(0) = 1)
             if (ok) {
-                pk.x = phi_bf16x2<PHI>(kreg[i].x);
-                pk.y = phi_bf16x2<PHI>(kreg[i].y);
-                pk.z = phi_bf16x2<PHI>(kreg[i].z);
-                pk.w = phi_bf16x2<PHI>(kreg[i].w);
+                pk.x = phi_pair<PHI>(kreg[i].x);
+                pk.y = phi_pair<PHI>(kreg[i].y);
+                pk.z = phi_pair<PHI>(kreg[i].z);
+                pk.w = phi_pair<PHI>(kreg[i].w);
             }
             *reinterpret_cast<uint4*>(Ksm + row * C::PITCH + ch * 16) = pk;
             *reinterpret_cast<uint4*>(Vsm + row * C::PITCH + ch * 16) = vreg[i];
@@ -117,7 +117,7 @@ __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict
     const uint32_t a_off = ((lane & 7) + ((lane >> 4) << 3)) * C::PITCH +
                            (warp * 16 + ((lane >> 3) & 1) * 8) * 2;
     const uint32_t b_off = ((lane & 7) + (((lane >> 3) & 1) << 3)) * C::PITCH + ((lane >> 4) * 8) * 2;
-    const uint32_t ones = 0x3F803F80u;  // bf16 (1, 1)
+    const uint32_t ones = ones_pair<PHI>();
 
     if (tile0 < tile1) load_tile(tile0);
     for (int tile = tile0; tile < tile1; ++tile) {
@@ -132,10 +132,10 @@ __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict
             for (int nbp = 0; nbp < (C::NBV + 1) / 2; ++nbp) {
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4_trans(vsm_base + ks * 16 * C::PITCH + b_off + nbp * 32, b0, b1, b2, b3);
-                mma_bf16_16816(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
-                if (2 * nbp + 1 < C::NBV) mma_bf16_16816(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
+                mma_16816<PHI>(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
+                if (2 * nbp + 1 < C::NBV) mma_16816<PHI>(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
             }
-            mma_bf16_16816(acc[C::NBV], a0, a1, a2, a3, ones, ones);
+            mma_16816<PHI>(acc[C::NBV], a0, a1, a2, a3, ones, ones);
         }
         __syncthreads();
     }
@@ -168,7 +168,7 @@ template <int D, int PHI>
 __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs,
                                             __nv_bfloat16* __restrict__ Ys, int N, int rs, int tile0,
                                             int tile1, const unsigned char* St, unsigned char* Qsm,
-                                            float eps)
+                                            ApplyScales sc)
 {
     using C = SplitCfg<D>;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -195,10 +195,10 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
             bool ok = (r < N) && (ch * 8 < D);
             uint4 pq = zero4;
             if (ok) {
-                pq.x = phi_bf16x2<PHI>(qreg[i].x);
-                pq.y = phi_bf16x2<PHI>(qreg[i].y);
-                pq.z = phi_bf16x2<PHI>(qreg[i].z);
-                pq.w = phi_bf16x2<PHI>(qreg[i].w);
+                pq.x = phi_pair<PHI>(qreg[i].x);
+                pq.y = phi_pair<PHI>(qreg[i].y);
+                pq.z = phi_pair<PHI>(qreg[i].z);
+                pq.w = phi_pair<PHI>(qreg[i].w);
             }
             *reinterpret_cast<uint4*>(Qsm + row * C::PITCH + ch * 16) = pq;
         }
@@ -231,29 +231,29 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
             for (int nbp = 0; nbp < (C::NBT + 1) / 2; ++nbp) {
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4(s_base + nbp * 16 * C::PITCH + kb * 32, b0, b1, b2, b3);
-                mma_bf16_16816(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
-                if (2 * nbp + 1 < C::NBT) mma_bf16_16816(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
+                mma_16816<PHI>(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
+                if (2 * nbp + 1 < C::NBT) mma_16816<PHI>(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
             }
         }
         // Every column of the z block holds phi(Q_i) . z for its row.
-        const float inv0 = row_scale(acc[C::NBV][0], eps);
-        const float inv1 = row_scale(acc[C::NBV][2], eps);
+        const float inv0 = row_scale(acc[C::NBV][0], sc);
+        const float inv1 = row_scale(acc[C::NBV][2], sc);
         const long long r0 = static_cast<long long>(tile) * C::TILE_Q + warp * 16 + g, r1 = r0 + 8;
 #pragma unroll
         for (int nb = 0; nb < C::NBV; ++nb) {
             int e = nb * 8 + 2 * t;
-            if (r0 < N) st_stream_4B(Ys + r0 * rs + e, pack_bf16x2(acc[nb][0] * inv0, acc[nb][1] * inv0));
-            if (r1 < N) st_stream_4B(Ys + r1 * rs + e, pack_bf16x2(acc[nb][2] * inv1, acc[nb][3] * inv1));
+            if (r0 < N) st_stream_4B(Ys + r0 * rs + e, pack_pair<PHI>(acc[nb][0] * inv0, acc[nb][1] * inv0));
+            if (r1 < N) st_stream_4B(Ys + r1 * rs + e, pack_pair<PHI>(acc[nb][2] * inv1, acc[nb][3] * inv1));
         }
         __syncthreads();
     }
 }
 
-// Fill the shared S^T | z operand (bf16, rows = output channel e, then 8 rows of z, then zero
+// Fill the shared S^T | z operand (16-bit storage type, scaled; rows = output channel e, then 8 rows of z, then zero
 // rows; columns = feature c padded with zeros) from fp32 S [D][D], z [D].  `read(idx)` returns
 // element idx of that fp32 state.
 template <int D, typename ReadFn>
-__device__ __forceinline__ void fill_state_operand(unsigned char* St, ReadFn read)
+__device__ __forceinline__ void fill_state_operand(unsigned char* St, ReadFn read, int dtype, float scale)
 {
     using C = SplitCfg<D>;
     constexpr int kBatch = 8;  // the reads of one batch are issued together, then stored
@@ -275,7 +275,7 @@ __device__ __forceinline__ void fill_state_operand(unsigned char* St, ReadFn rea
             const int idx = base + u * stride;
             const int c = idx / C::ST_ROWS, e = idx % C::ST_ROWS;
             if (idx < total)
-                *reinterpret_cast<__nv_bfloat16*>(St + e * C::PITCH + c * 2) = __float2bfloat16_rn(val[u]);
+                *reinterpret_cast<uint16_t*>(St + e * C::PITCH + c * 2) = to_storage16(val[u] * scale, dtype);
         }
     }
 }
@@ -306,12 +306,14 @@ state_partial_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* _
 }
 
 // grid (ceil(state_floats / 256), slabs).  Sums `chunks` partials per slab in index order.  If
-// `st_image` is not null it also receives the bf16 S^T | z operand of the apply kernel, laid out
+// `st_image` is not null it also receives the S^T | z operand of the apply kernel (16-bit storage
+// type `dtype`, values times `operand_scale`), laid out
 // exactly as that kernel holds it in shared memory (`image_bytes` per slab, rows `pitch` bytes
 // apart: row e < d holds S[.][e], rows d .. d+7 hold z; pad bytes stay as the host zeroed them).
 __global__ void __launch_bounds__(256)
 state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state, int state_floats,
-                    int chunks, unsigned char* __restrict__ st_image, int d, int pitch, int image_bytes)
+                    int chunks, unsigned char* __restrict__ st_image, int d, int pitch, int image_bytes,
+                    int dtype, float operand_scale)
 {
     // Programmatic dependent launch: the next kernel of the stream may be scheduled behind this
     // one; nothing in global memory is touched before the kernel ahead has completed.
@@ -326,13 +328,13 @@ state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ stat
     state[static_cast<size_t>(slab) * state_floats + idx] = sum;
     if (st_image != nullptr) {
         unsigned char* img = st_image + static_cast<size_t>(slab) * image_bytes;
-        const __nv_bfloat16 b = __float2bfloat16_rn(sum);
+        const uint16_t b = to_storage16(sum * operand_scale, dtype);
         if (idx < d * d) {
             const int c = idx / d, e = idx - c * d;
-            *reinterpret_cast<__nv_bfloat16*>(img + e * pitch + c * 2) = b;
+            *reinterpret_cast<uint16_t*>(img + e * pitch + c * 2) = b;
         } else {
             const int c = idx - d * d;
-            for (int j = 0; j < 8; ++j) *reinterpret_cast<__nv_bfloat16*>(img + (d + j) * pitch + c * 2) = b;
+            for (int j = 0; j < 8; ++j) *reinterpret_cast<uint16_t*>(img + (d + j) * pitch + c * 2) = b;
         }
     }
 }
@@ -342,7 +344,7 @@ state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ stat
 template <int D, int PHI>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ state,
-             __nv_bfloat16* __restrict__ Y, int N, int chunks, float eps, SlabLayout L,
+             __nv_bfloat16* __restrict__ Y, int N, int chunks, ApplyScales sc, SlabLayout L,
              const unsigned char* __restrict__ st_image)
 {
     // Programmatic dependent launch: the next kernel of the stream may be scheduled behind this
@@ -362,12 +364,12 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
             reinterpret_cast<uint4*>(St)[i] = __ldg(img + i);
     } else {
         const float* st = state + static_cast<size_t>(slab) * C::STATE_FLOATS;
-        fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); });
+        fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); }, kind_dtype(PHI), sc.operand);
     }
     __syncthreads();
     const size_t slab_off = slab_base(L, slab);
     apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
-                        chunk_begin(p + 1, tiles, chunks), St, Qsm, eps);
+                        chunk_begin(p + 1, tiles, chunks), St, Qsm, sc);
 }
 
 // One cluster of `cluster_size` CTAs per slab (grid.x = cluster_size, grid.y = slabs).  CTA r
@@ -380,7 +382,7 @@ template <int D, int PHI>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                      const __nv_bfloat16* __restrict__ V, __nv_bfloat16* __restrict__ Y,
-                     float* __restrict__ state_out, int N, float eps, SlabLayout L)
+                     float* __restrict__ state_out, int N, ApplyScales sc, SlabLayout L)
 {
     using C = SplitCfg<D>;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -437,7 +439,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
                 const int i = base + u * blockDim.x;
                 if (i >= end) continue;
                 if (gout != nullptr) gout[i] = sum[u];
-                const __nv_bfloat16 b = __float2bfloat16_rn(sum[u]);
+                const uint16_t b = to_storage16(sum[u] * sc.operand, kind_dtype(PHI));
                 // S[c][e] goes to row e, column c of the operand; z[c] to column c of rows D .. D+7.
                 const bool is_z = i >= D * D;
                 const int c = is_z ? i - D * D : i / D;
@@ -447,7 +449,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
                 for (int r = 0; r < csize; ++r) {
                     unsigned char* dst = cluster.map_shared_rank(St, r) + row0 * C::PITCH + c * 2;
 #pragma unroll 1
-                    for (int j = 0; j < rows; ++j) *reinterpret_cast<__nv_bfloat16*>(dst + j * C::PITCH) = b;
+                    for (int j = 0; j < rows; ++j) *reinterpret_cast<uint16_t*>(dst + j * C::PITCH) = b;
                 }
             }
         }
@@ -456,7 +458,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
 
     const int qtiles = (N + C::TILE_Q - 1) / C::TILE_Q;
     apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(rank, qtiles, csize),
-                        chunk_begin(rank + 1, qtiles, csize), St, stage, eps);
+                        chunk_begin(rank + 1, qtiles, csize), St, stage, sc);
 }
 
 }  // namespace lf

@@ -167,7 +167,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     // which is the first value of token t's 128-byte row, moved by the swizzle to chunk t & 7.
     for (int i = tid; i < C::ONES_BYTES / 4; i += C::THREADS) reinterpret_cast<uint32_t*>(ones)[i] = 0u;
     __syncthreads();
-    if (tid < 16) *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = 0x3F80u;  // bf16 1.0
+    if (tid < 16) *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = static_cast<uint16_t>(ones_pair<PHI>() & 0xffffu);
     fence_proxy_async_smem();
     if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
     tc_fence_before_sync();
@@ -206,7 +206,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     } else if (warp == C::MMA_WARP) {
         // ---------------- MMA warp ----------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16_f32(128, 64, kUmmaAMnMajor | kUmmaBMnMajor);
+            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(PHI), 128, 64, kUmmaAMnMajor | kUmmaBMnMajor);
             const uint32_t ones_addr = smem_u32(ones);
             int cur_slab = -1, in_segment = 0, segments = 0, buf = 1;
             for (int it = 0; it < n_units; ++it) {
@@ -238,7 +238,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     const uint32_t va = v_addr + k * 2048;
                     const uint64_t a_desc = umma_desc_mnmajor_sw128(va, ones_addr - va, 1024);
                     const uint64_t b_desc = umma_desc_mnmajor_sw128(k_addr + k * 2048, 0, 1024);
-                    umma_bf16_ss(d_tmem, a_desc, b_desc, idesc, (in_segment == 0 && k == 0) ? 0u : 1u);
+                    umma_ss(d_tmem, a_desc, b_desc, idesc, (in_segment == 0 && k == 0) ? 0u : 1u);
                 }
                 ++in_segment;
                 umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
@@ -316,10 +316,10 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     uint32_t x0, x1, x2, x3;
                     const uint32_t addr = base + ((c ^ sw) << 4);
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(addr));
-                    x0 = phi_packed_bf16x2<PHI>(x0);
-                    x1 = phi_packed_bf16x2<PHI>(x1);
-                    x2 = phi_packed_bf16x2<PHI>(x2);
-                    x3 = phi_packed_bf16x2<PHI>(x3);
+                    x0 = phi_packed_pair<PHI>(x0);
+                    x1 = phi_packed_pair<PHI>(x1);
+                    x2 = phi_packed_pair<PHI>(x2);
+                    x3 = phi_packed_pair<PHI>(x3);
                     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x0), "r"(x1), "r"(x2), "r"(x3) : "memory");
                 }
             }
@@ -346,7 +346,7 @@ constexpr int kStreamOperandBytes = StreamApplyCfg::B_BYTES;
 // Block blockIdx.x of a (17, slabs) grid of 256 threads holds elements 256*blockIdx.x .. of one
 // slab's fp32 state (S rows 4*blockIdx.x .., or z in block 16) in `sums`; write their share of the
 // operand image `img` of that slab.
-__device__ __forceinline__ void emit_state_operand(const float* sums, unsigned char* img)
+__device__ __forceinline__ void emit_state_operand(const float* sums, unsigned char* img, int dtype, float scale)
 {
     const int tid = threadIdx.x;
     if (blockIdx.x < 16) {
@@ -354,14 +354,17 @@ __device__ __forceinline__ void emit_state_operand(const float* sums, unsigned c
         if (tid < 64) {
             const int c0 = 4 * blockIdx.x, e = tid;
             uint2 v;
-            v.x = pack_bf16x2(sums[e], sums[64 + e]);
-            v.y = pack_bf16x2(sums[128 + e], sums[192 + e]);
+            v.x = to_storage16(sums[e] * scale, dtype) | (static_cast<uint32_t>(to_storage16(sums[64 + e] * scale, dtype)) << 16);
+            v.y = to_storage16(sums[128 + e] * scale, dtype) |
+                  (static_cast<uint32_t>(to_storage16(sums[192 + e] * scale, dtype)) << 16);
             *reinterpret_cast<uint2*>(img + e * 128 + (((c0 >> 3) ^ (e & 7)) << 4) + (c0 & 7) * 2) = v;
         }
     } else {
         // z -> row 64 (64 & 7 = 0: chunks in place), zeros -> rows 65..79
         if (tid < 32) {
-            *reinterpret_cast<uint32_t*>(img + 64 * 128 + tid * 4) = pack_bf16x2(sums[2 * tid], sums[2 * tid + 1]);
+            *reinterpret_cast<uint32_t*>(img + 64 * 128 + tid * 4) =
+                to_storage16(sums[2 * tid] * scale, dtype) |
+                (static_cast<uint32_t>(to_storage16(sums[2 * tid + 1] * scale, dtype)) << 16);
         } else if (tid < 32 + 120) {
             reinterpret_cast<uint4*>(img + 65 * 128)[tid - 32] = make_uint4(0u, 0u, 0u, 0u);
         }
@@ -374,7 +377,7 @@ __device__ __forceinline__ void emit_state_operand(const float* sums, unsigned c
 __global__ void __launch_bounds__(256)
 stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
                      unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
-                     int tiles_per_slab, long long W, int G, int spans)
+                     int tiles_per_slab, long long W, int G, int spans, int dtype, float operand_scale)
 {
     __shared__ float sums[256];
     const int tid = threadIdx.x;
@@ -404,7 +407,7 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
     }
     sums[tid] = sum;
     __syncthreads();
-    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes);
+    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes, dtype, operand_scale);
 }
 
 // grid (17, slabs), 256 threads: rebuild the bf16 operand image (and clear the tile counters) from
@@ -412,7 +415,7 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
 // forward (Sec. 4.3).
 __global__ void __launch_bounds__(256)
 stream_pack_kernel(const float* __restrict__ state, unsigned char* __restrict__ operand,
-                   int* __restrict__ tile_counters)
+                   int* __restrict__ tile_counters, int dtype, float operand_scale)
 {
     __shared__ float sums[256];
     const int tid = threadIdx.x;
@@ -423,7 +426,7 @@ stream_pack_kernel(const float* __restrict__ state, unsigned char* __restrict__ 
     if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
     sums[tid] = idx < kStreamStateFloats ? state[static_cast<size_t>(slab) * kStreamStateFloats + idx] : 0.0f;
     __syncthreads();
-    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes);
+    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes, dtype, operand_scale);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -448,7 +451,7 @@ template <int PHI>
 __global__ void __launch_bounds__(StreamApplyCfg::THREADS, 1)
 stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_y,
                     const unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
-                    uint32_t* __restrict__ status, int tiles_per_slab, int slabs, float eps, int H)
+                    uint32_t* __restrict__ status, int tiles_per_slab, int slabs, ApplyScales sc, int H)
 {
     using C = StreamApplyCfg;
     extern __shared__ unsigned char smem_raw[];
@@ -596,7 +599,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         // (tcgen05.mma issued by the leaders of several warpgroups at once lost completions now and
         // then; with a single issuing thread it has not.)
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_bf16_f32(C::TILE, C::B_ROWS);
+            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(PHI), C::TILE, C::B_ROWS);
             const uint64_t b_desc = umma_desc_kmajor_sw128(smem_u32(bsm));
             for (int it = 0;; ++it) {
                 const int s = it % C::STAGES, g = it % C::GROUPS;
@@ -613,7 +616,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 const uint32_t a_tmem = tmem_base + g * C::TMEM_COLS_PER_GROUP, d_tmem = a_tmem + 32;
                 // K = 64 as four steps of 16: A advances 8 columns (two bf16 per column), B 32 bytes
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_bf16_ts(d_tmem, a_tmem + 8 * k, b_desc + 2 * k, idesc, k > 0 ? 1u : 0u);
+                for (int k = 0; k < 4; ++k) umma_ts(d_tmem, a_tmem + 8 * k, b_desc + 2 * k, idesc, k > 0 ? 1u : 0u);
                 umma_commit(&mma_done[g]);
             }
         }
@@ -649,10 +652,10 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                                  : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
                                  : "r"(base + ((c ^ sw) << 4)));
-                    a[4 * c + 0] = phi_packed_bf16x2<PHI>(x0);
-                    a[4 * c + 1] = phi_packed_bf16x2<PHI>(x1);
-                    a[4 * c + 2] = phi_packed_bf16x2<PHI>(x2);
-                    a[4 * c + 3] = phi_packed_bf16x2<PHI>(x3);
+                    a[4 * c + 0] = phi_packed_pair<PHI>(x0);
+                    a[4 * c + 1] = phi_packed_pair<PHI>(x1);
+                    a[4 * c + 2] = phi_packed_pair<PHI>(x2);
+                    a[4 * c + 3] = phi_packed_pair<PHI>(x3);
                 }
                 tmem_store_32cols(a_tmem, a);
             }
@@ -668,17 +671,17 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             }
             tc_fence_after_sync();
             const float den = __uint_as_float(tmem_load_1col(d_tmem + 64));  // phi(Q_i) . z
-            const float inv = row_scale(den, eps);
+            const float inv = row_scale(den, sc);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t d[32];
                 tmem_load_32cols(d_tmem + 32 * half, d);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint32_t v0 = pack_bf16x2(__uint_as_float(d[8 * c + 0]) * inv, __uint_as_float(d[8 * c + 1]) * inv);
-                    const uint32_t v1 = pack_bf16x2(__uint_as_float(d[8 * c + 2]) * inv, __uint_as_float(d[8 * c + 3]) * inv);
-                    const uint32_t v2 = pack_bf16x2(__uint_as_float(d[8 * c + 4]) * inv, __uint_as_float(d[8 * c + 5]) * inv);
-                    const uint32_t v3 = pack_bf16x2(__uint_as_float(d[8 * c + 6]) * inv, __uint_as_float(d[8 * c + 7]) * inv);
+                    const uint32_t v0 = pack_pair<PHI>(__uint_as_float(d[8 * c + 0]) * inv, __uint_as_float(d[8 * c + 1]) * inv);
+                    const uint32_t v1 = pack_pair<PHI>(__uint_as_float(d[8 * c + 2]) * inv, __uint_as_float(d[8 * c + 3]) * inv);
+                    const uint32_t v2 = pack_pair<PHI>(__uint_as_float(d[8 * c + 4]) * inv, __uint_as_float(d[8 * c + 5]) * inv);
+                    const uint32_t v3 = pack_pair<PHI>(__uint_as_float(d[8 * c + 6]) * inv, __uint_as_float(d[8 * c + 7]) * inv);
                     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + (((4 * half + c) ^ sw) << 4)),
                                  "r"(v0), "r"(v1), "r"(v2), "r"(v3)
                                  : "memory");

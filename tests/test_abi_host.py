@@ -80,7 +80,7 @@ def test_invalid_descriptors(kw):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(d=48), dict(d=7), dict(d=256), dict(phi=7), dict(variant=9), dict(variant=0x40),
+    dict(d=48), dict(d=7), dict(d=256), dict(phi=7), dict(variant=9), dict(variant=0x80),
     dict(d=40, variant="stream"),
 ])
 def test_unsupported_descriptors(kw):
