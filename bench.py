@@ -240,8 +240,11 @@ def run_cuda(args):
         q, k, v = wl.make_qkv(s, seed=wl.BASE_SEED + 100 * rank + i, device=f"cuda:{local_rank}")
         if args.layout == "token_major":          # [B, N, H, d]: what a UNet holds before splitting heads
             q, k, v = (t.permute(0, 2, 1, 3).contiguous() for t in (q, k, v))
+        if args.dtype == "fp16":
+            q, k, v = (t.half() for t in (q, k, v))
         y = torch.empty_like(q)
-        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank, layout=args.layout)
+        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank, layout=args.layout,
+                                     dtype=args.dtype)
         layers.append((s, op, q, k, v, y))
     tokens_per_step = sum(s.tokens for s in shapes)
     launches_per_step = sum(op.launches_per_forward for _, op, *_ in layers)
@@ -347,7 +350,7 @@ def run_cuda(args):
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": args.dtype, "data": "synthetic",
             "config": {"workload": args.workload,
                        "shapes": [{"name": s.name, "B": s.B, "H": s.H, "N": s.N, "d": s.d}
                                   for s in shapes],
@@ -435,6 +438,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layout", default="head_major", choices=["head_major", "token_major"],
                     help="[B,H,N,d] (default, the benchmark's layout) or [B,N,H,d]")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"],
+                    help="storage type of Q, K, V, Y (the headline number is bf16)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every shape of the five workload families with every variant")
     ap.add_argument("--only", default="", help="with --sweep: restrict to one shape, e.g. sd15_512_L1")
