@@ -14,7 +14,7 @@
  * already non-negative).  eps is this library's guard on the denominator; the paper has none.
  *
  * Unless a function says otherwise, tensor arguments are DEVICE pointers to dense row-major
- * bf16 [B, H, N, d] (token rows of d contiguous channels, one slab of N rows per (b, h)),
+ * bf16 (or fp16: LINFUSION_DTYPE_FP16) [B, H, N, d] (token rows of d contiguous channels, one slab of N rows per (b, h)),
  * 16-byte aligned.  Y must not overlap Q, K or V.  The caller owns Q, K, V, Y and the stream.
  * The handle owns an fp32 workspace on its device unless the caller lends one (set_workspace).
  *
@@ -72,7 +72,7 @@ typedef enum {
  * flags: the operator without its normalizer.  Bit set: Y_i = phi(Q_i) S, i.e. Y = f'(X) g'(X)^T X of
  * Prop. 2 before the division of Eq. 5 is applied (the "without normalization" rows of the
  * ablation in Tab. 2).  eps is then unused; z is still accumulated and read_state() returns it.
- * |Y| grows with N in this form (the paper's reason for the normalizer); outputs are still bf16.
+ * |Y| grows with N in this form (the paper's reason for the normalizer); outputs are still 16-bit.
  */
 #define LINFUSION_FLAG_UNNORMALIZED 0x20u
 /*
@@ -107,8 +107,8 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
 
 /*
  * Enqueue Y = norm-linear-attention(Q, K, V) on `cuda_stream` (a cudaStream_t / CUstream;
- * NULL is the legacy default stream).  q, k, v: const bf16 [B,H,N,d] device memory;
- * y: bf16 [B,H,N,d] device memory, written in full, rounded to nearest even from fp32.
+ * NULL is the legacy default stream).  q, k, v: const bf16 (or fp16) [B,H,N,d] device memory;
+ * y: the same type, [B,H,N,d] device memory, written in full, rounded to nearest even from fp32.
  * Steps: split-N state reduction (S_p, z_p per chunk p of the tokens; Prop. 2 and Eq. 5),
  * fixed-order reduction to (S, z), apply — or all three in one clustered launch for small N.
  * Errors: INVALID_ARG (null handle or pointer, pointer not 16-byte aligned, y overlapping an

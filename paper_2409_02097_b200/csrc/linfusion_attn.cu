@@ -147,7 +147,7 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     p->partial_bytes = align_up(partial_floats * sizeof(float), 256);
     p->state_off = p->partial_bytes;
     p->operand_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
-    // bf16 operand image of S | z for the apply kernel (in its shared-memory layout), and for the
+    // 16-bit operand image of S | z for the apply kernel (in its shared-memory layout), and for the
     // stream variant one tile counter per slab.
     const int dp = (d->d + 15) / 16 * 16;
     const size_t split_image = static_cast<size_t>((d->d + 8 + 15) / 16 * 16) * (((dp / 8) | 1) * 16);
@@ -235,7 +235,7 @@ SlabLayout layout_of(const linfusion_attn_desc_t& d)
     return L;
 }
 
-// bf16 tensor seen as (channel 64, token N, head H, batch B) -> boxes of tile_rows tokens of one
+// 16-bit (bf16 or fp16) tensor seen as (channel 64, token N, head H, batch B) -> boxes of tile_rows tokens of one
 // (b, h) slab, 128-byte swizzle, zero fill past N.  The layout only changes the strides.
 bool encode_slab_map(CUtensorMap* map, const void* base, const linfusion_attn_desc_t& d, int tile_rows)
 {
@@ -269,7 +269,7 @@ struct linfusion_attn {
     bool owns_ws;
     float* partials;
     float* state;
-    unsigned char* operand;  // bf16 operand image of S | z for the apply kernels
+    unsigned char* operand;  // 16-bit operand image of S | z for the apply kernels
     int* tile_counters;
     uint32_t* status;
     cudaStream_t last_stream;
@@ -329,32 +329,32 @@ inline void mark(const linfusion_attn* h, int i, cudaStream_t s)
         cudaEventRecord(h->events[(h->timed_calls % h->timing_slots) * 4 + i], s);
 }
 
-template <int D, int PHI>
+template <int D, int KIND>
 cudaError_t set_split_attrs()
 {
     using C = SplitCfg<D>;
     cudaError_t e;
-    e = cudaFuncSetAttribute(state_partial_kernel<D, PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+    e = cudaFuncSetAttribute(state_partial_kernel<D, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(apply_kernel<D, PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY);
+    e = cudaFuncSetAttribute(apply_kernel<D, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(cluster_fused_kernel<D, PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(cluster_fused_kernel<D, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::SMEM_CLUSTER);
     if (e != cudaSuccess) return e;
     // Clusters of 16 CTAs are beyond the portable size of 8; create() shrinks the cluster when
     // the device cannot co-schedule it.
-    e = cudaFuncSetAttribute(cluster_fused_kernel<D, PHI>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    e = cudaFuncSetAttribute(cluster_fused_kernel<D, KIND>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     return e;
 }
 
-template <int PHI>
+template <int KIND>
 cudaError_t set_stream_attrs()
 {
     cudaError_t e;
-    e = cudaFuncSetAttribute(stream_state_kernel<PHI>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(stream_state_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              StreamStateCfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(stream_apply_kernel<PHI>,
+    e = cudaFuncSetAttribute(stream_apply_kernel<KIND>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg::SMEM_BYTES);
     return e;
 }
@@ -379,7 +379,7 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-template <int D, int PHI>
+template <int D, int KIND>
 cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                          const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
@@ -388,18 +388,18 @@ cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const 
     const int N = h->desc.N;
     cudaError_t e;
     mark(h, 0, s);
-    e = launch_chained(state_partial_kernel<D, PHI>, dim3(p.chunks_state, p.slabs), dim3(C::NT), C::SMEM_KV, s, k, v,
+    e = launch_chained(state_partial_kernel<D, KIND>, dim3(p.chunks_state, p.slabs), dim3(C::NT), C::SMEM_KV, s, k, v,
                        h->partials, N, p.chunks_state, layout_of(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 1, s);
-    // h->operand (when the workspace has it) receives the apply kernel's bf16 operand image.
+    // h->operand (when the workspace has it) receives the apply kernel's 16-bit operand image.
     unsigned char* image = h->operand;
     e = launch_chained(state_reduce_kernel, dim3((C::STATE_FLOATS + 255) / 256, p.slabs), dim3(256), 0, s,
                        h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST,
                        dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 2, s);
-    e = launch_chained(apply_kernel<D, PHI>, dim3(p.chunks_apply, p.slabs), dim3(C::NT), C::SMEM_APPLY, s, q,
+    e = launch_chained(apply_kernel<D, KIND>, dim3(p.chunks_apply, p.slabs), dim3(C::NT), C::SMEM_APPLY, s, q,
                        h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), image);
     if (e != cudaSuccess) return e;
     mark(h, 3, s);
@@ -424,7 +424,7 @@ void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int clus
     cfg->numAttrs = 1;
 }
 
-template <int D, int PHI>
+template <int D, int KIND>
 cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                            const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
@@ -432,13 +432,13 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
     cudaLaunchAttribute attr[1];
     cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
     mark(h, 0, s);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, PHI>, q, k, v, y, h->state,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, KIND>, q, k, v, y, h->state,
                                        h->desc.N, apply_scales(h->desc), layout_of(h->desc));
     mark(h, 1, s);
     return e;
 }
 
-template <int PHI>
+template <int KIND>
 cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                           const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
@@ -451,7 +451,7 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
         return cudaErrorInvalidValue;
     cudaError_t e;
     mark(h, 0, s);
-    e = launch_chained(stream_state_kernel<PHI>, dim3(p.G_state), dim3(StreamStateCfg::THREADS),
+    e = launch_chained(stream_state_kernel<KIND>, dim3(p.G_state), dim3(StreamStateCfg::THREADS),
                        StreamStateCfg::SMEM_BYTES, s, mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state,
                        p.spans, h->desc.H);
     if (e != cudaSuccess) return e;
@@ -461,7 +461,7 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
                        p.spans, dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 2, s);
-    e = launch_chained(stream_apply_kernel<PHI>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
+    e = launch_chained(stream_apply_kernel<KIND>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
                        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs,
                        apply_scales(h->desc), h->desc.H);
     if (e != cudaSuccess) return e;
@@ -1113,7 +1113,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-template <int D, int PHI>
+template <int D, int KIND>
 cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a,
                               const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s)
 {
@@ -1121,20 +1121,20 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
     const Plan& p = h->plan;
     const int N = h->desc.N;
     if (state_half) {
-        state_partial_kernel<D, PHI><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
+        state_partial_kernel<D, KIND><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
             a, b, h->partials, N, p.chunks_state, layout_of(h->desc));
         state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
             h->partials, h->state, C::STATE_FLOATS, p.chunks_state, nullptr, D, C::PITCH, C::SMEM_ST,
             dtype_of(h->desc), operand_scale(h->desc));
     } else {
         // The fp32 state may have been summed over devices: convert it here, not from an image.
-        apply_kernel<D, PHI><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
+        apply_kernel<D, KIND><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
             a, h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), nullptr);
     }
     return cudaGetLastError();
 }
 
-template <int PHI>
+template <int KIND>
 cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a,
                                const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s)
 {
@@ -1146,7 +1146,7 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
         if (!encode_slab_map(&mk, a, h->desc, StreamStateCfg::TILE) ||
             !encode_slab_map(&mv, b, h->desc, StreamStateCfg::TILE))
             return cudaErrorInvalidValue;
-        stream_state_kernel<PHI><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
+        stream_state_kernel<KIND><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
             mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
         stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->operand, h->tile_counters,
                                                   p.tiles_state, p.W_state, p.G_state, p.spans,
@@ -1155,10 +1155,10 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
         CUtensorMap mq, my;
         if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
             return cudaErrorInvalidValue;
-        // The state may have been summed over devices since the reduction: rebuild its bf16 image.
+        // The state may have been summed over devices since the reduction: rebuild its 16-bit image.
         stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->operand, h->tile_counters, dtype_of(h->desc),
                                                 operand_scale(h->desc));
-        stream_apply_kernel<PHI><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
+        stream_apply_kernel<KIND><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
             mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, apply_scales(h->desc), h->desc.H);
     }
     return cudaGetLastError();

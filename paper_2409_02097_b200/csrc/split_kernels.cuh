@@ -11,7 +11,7 @@
 // MMA roles.  State: D[c][e] += A[c][j] B[j][e] with A = phi(K)^T and B = V, the contraction
 // running over tokens j; one warp owns one 16-row block of c and every column block of e,
 // plus one extra column block fed with ones, which yields z.  Apply: D[i][e] += A[i][c] B[c][e]
-// with A = phi(Q) and B = S (held transposed, as bf16), one warp per 16 tokens, plus one
+// with A = phi(Q) and B = S (held transposed, in the 16-bit storage type), one warp per 16 tokens, plus one
 // extra column block holding z in every column, which yields the denominator.
 #pragma once
 
@@ -61,7 +61,7 @@ __host__ __device__ __forceinline__ int chunk_begin(int p, int tiles, int chunks
 // State accumulation over K/V tiles [tile0, tile1) of one slab.  acc[nb][.] holds this warp's
 // 16 x 8 block (rows c = 16*warp + ..., columns 8*nb + ...), acc[NBV] the z block.
 // ---------------------------------------------------------------------------------------------
-template <int D, int PHI>
+template <int D, int KIND>
 __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict__ Ks,
                                                  const __nv_bfloat16* __restrict__ Vs, int N, int rs,
                                                  int tile0, int tile1, unsigned char* smem_kv,
@@ -100,10 +100,10 @@ __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict
             bool ok = (j < N) && (ch * 8 < D);
             uint4 pk = zero4;  // rows past N and pad channels contribute nothing (not phi(0) = 1)
             if (ok) {
-                pk.x = phi_pair<PHI>(kreg[i].x);
-                pk.y = phi_pair<PHI>(kreg[i].y);
-                pk.z = phi_pair<PHI>(kreg[i].z);
-                pk.w = phi_pair<PHI>(kreg[i].w);
+                pk.x = phi_pair<KIND>(kreg[i].x);
+                pk.y = phi_pair<KIND>(kreg[i].y);
+                pk.z = phi_pair<KIND>(kreg[i].z);
+                pk.w = phi_pair<KIND>(kreg[i].w);
             }
             *reinterpret_cast<uint4*>(Ksm + row * C::PITCH + ch * 16) = pk;
             *reinterpret_cast<uint4*>(Vsm + row * C::PITCH + ch * 16) = vreg[i];
@@ -117,7 +117,7 @@ __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict
     const uint32_t a_off = ((lane & 7) + ((lane >> 4) << 3)) * C::PITCH +
                            (warp * 16 + ((lane >> 3) & 1) * 8) * 2;
     const uint32_t b_off = ((lane & 7) + (((lane >> 3) & 1) << 3)) * C::PITCH + ((lane >> 4) * 8) * 2;
-    const uint32_t ones = ones_pair<PHI>();
+    const uint32_t ones = ones_pair<KIND>();
 
     if (tile0 < tile1) load_tile(tile0);
     for (int tile = tile0; tile < tile1; ++tile) {
@@ -132,10 +132,10 @@ __device__ __forceinline__ void accumulate_state(const __nv_bfloat16* __restrict
             for (int nbp = 0; nbp < (C::NBV + 1) / 2; ++nbp) {
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4_trans(vsm_base + ks * 16 * C::PITCH + b_off + nbp * 32, b0, b1, b2, b3);
-                mma_16816<PHI>(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
-                if (2 * nbp + 1 < C::NBV) mma_16816<PHI>(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
+                mma_16816<KIND>(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
+                if (2 * nbp + 1 < C::NBV) mma_16816<KIND>(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
             }
-            mma_16816<PHI>(acc[C::NBV], a0, a1, a2, a3, ones, ones);
+            mma_16816<KIND>(acc[C::NBV], a0, a1, a2, a3, ones, ones);
         }
         __syncthreads();
     }
@@ -162,9 +162,10 @@ __device__ __forceinline__ void store_state(float* dst, const float (&acc)[Split
 }
 
 // ---------------------------------------------------------------------------------------------
-// Apply over Q tiles [tile0, tile1) of one slab, with S^T | z resident in shared memory as bf16.
+// Apply over Q tiles [tile0, tile1) of one slab, with S^T | z resident in shared memory in the
+// 16-bit storage type.
 // ---------------------------------------------------------------------------------------------
-template <int D, int PHI>
+template <int D, int KIND>
 __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs,
                                             __nv_bfloat16* __restrict__ Ys, int N, int rs, int tile0,
                                             int tile1, const unsigned char* St, unsigned char* Qsm,
@@ -195,10 +196,10 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
             bool ok = (r < N) && (ch * 8 < D);
             uint4 pq = zero4;
             if (ok) {
-                pq.x = phi_pair<PHI>(qreg[i].x);
-                pq.y = phi_pair<PHI>(qreg[i].y);
-                pq.z = phi_pair<PHI>(qreg[i].z);
-                pq.w = phi_pair<PHI>(qreg[i].w);
+                pq.x = phi_pair<KIND>(qreg[i].x);
+                pq.y = phi_pair<KIND>(qreg[i].y);
+                pq.z = phi_pair<KIND>(qreg[i].z);
+                pq.w = phi_pair<KIND>(qreg[i].w);
             }
             *reinterpret_cast<uint4*>(Qsm + row * C::PITCH + ch * 16) = pq;
         }
@@ -231,8 +232,8 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
             for (int nbp = 0; nbp < (C::NBT + 1) / 2; ++nbp) {
                 uint32_t b0, b1, b2, b3;
                 ldmatrix_x4(s_base + nbp * 16 * C::PITCH + kb * 32, b0, b1, b2, b3);
-                mma_16816<PHI>(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
-                if (2 * nbp + 1 < C::NBT) mma_16816<PHI>(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
+                mma_16816<KIND>(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
+                if (2 * nbp + 1 < C::NBT) mma_16816<KIND>(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
             }
         }
         // Every column of the z block holds phi(Q_i) . z for its row.
@@ -242,8 +243,8 @@ __device__ __forceinline__ void apply_tiles(const __nv_bfloat16* __restrict__ Qs
 #pragma unroll
         for (int nb = 0; nb < C::NBV; ++nb) {
             int e = nb * 8 + 2 * t;
-            if (r0 < N) st_stream_4B(Ys + r0 * rs + e, pack_pair<PHI>(acc[nb][0] * inv0, acc[nb][1] * inv0));
-            if (r1 < N) st_stream_4B(Ys + r1 * rs + e, pack_pair<PHI>(acc[nb][2] * inv1, acc[nb][3] * inv1));
+            if (r0 < N) st_stream_4B(Ys + r0 * rs + e, pack_pair<KIND>(acc[nb][0] * inv0, acc[nb][1] * inv0));
+            if (r1 < N) st_stream_4B(Ys + r1 * rs + e, pack_pair<KIND>(acc[nb][2] * inv1, acc[nb][3] * inv1));
         }
         __syncthreads();
     }
@@ -285,7 +286,7 @@ __device__ __forceinline__ void fill_state_operand(unsigned char* St, ReadFn rea
 // ---------------------------------------------------------------------------------------------
 
 // grid (chunks, slabs).  partials: [slab][chunk][D*(D+1)] fp32.
-template <int D, int PHI>
+template <int D, int KIND>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 state_partial_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* __restrict__ V,
                      float* __restrict__ partials, int N, int chunks, SlabLayout L)
@@ -300,7 +301,7 @@ state_partial_kernel(const __nv_bfloat16* __restrict__ K, const __nv_bfloat16* _
     const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;
     const size_t slab_off = slab_base(L, slab);
     float acc[C::NBT][4];
-    accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
+    accumulate_state<D, KIND>(K + slab_off, V + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
                              chunk_begin(p + 1, tiles, chunks), smem, acc);
     store_state<D>(partials + (static_cast<size_t>(slab) * chunks + p) * C::STATE_FLOATS, acc);
 }
@@ -341,7 +342,7 @@ state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ stat
 
 // grid (chunks, slabs).  `st_image` (may be null) is the operand image written by
 // state_reduce_kernel; without it every CTA converts the fp32 state itself.
-template <int D, int PHI>
+template <int D, int KIND>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ state,
              __nv_bfloat16* __restrict__ Y, int N, int chunks, ApplyScales sc, SlabLayout L,
@@ -364,11 +365,11 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
             reinterpret_cast<uint4*>(St)[i] = __ldg(img + i);
     } else {
         const float* st = state + static_cast<size_t>(slab) * C::STATE_FLOATS;
-        fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); }, kind_dtype(PHI), sc.operand);
+        fill_state_operand<D>(St, [&](int i) { return __ldg(st + i); }, kind_dtype(KIND), sc.operand);
     }
     __syncthreads();
     const size_t slab_off = slab_base(L, slab);
-    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
+    apply_tiles<D, KIND>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(p, tiles, chunks),
                         chunk_begin(p + 1, tiles, chunks), St, Qsm, sc);
 }
 
@@ -378,7 +379,7 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
 // the result into every CTA's operand through distributed shared memory (so all CTAs hold the same
 // bits); after a second barrier every CTA applies to its run of Q.  state_out (may be null)
 // receives S | z in fp32.
-template <int D, int PHI>
+template <int D, int KIND>
 __global__ void __launch_bounds__(SplitCfg<D>::NT)
 cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* __restrict__ K,
                      const __nv_bfloat16* __restrict__ V, __nv_bfloat16* __restrict__ Y,
@@ -399,7 +400,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
     {
         const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;
         float acc[C::NBT][4];
-        accumulate_state<D, PHI>(K + slab_off, V + slab_off, N, L.row_stride, chunk_begin(rank, tiles, csize),
+        accumulate_state<D, KIND>(K + slab_off, V + slab_off, N, L.row_stride, chunk_begin(rank, tiles, csize),
                                  chunk_begin(rank + 1, tiles, csize), stage, acc);
         store_state<D>(part, acc);
     }
@@ -409,7 +410,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
     cluster.sync();
 
     // Reduce-scatter with push: CTA r sums slice r of the state over ranks 0, 1, ... in that order
-    // (fixed order), and stores the bf16 result into the S^T | z operand of every CTA of the
+    // (fixed order), and stores the 16-bit result into the S^T | z operand of every CTA of the
     // cluster through distributed shared memory (remote stores do not stall the writer), and the
     // fp32 result into state_out.
     {
@@ -439,7 +440,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
                 const int i = base + u * blockDim.x;
                 if (i >= end) continue;
                 if (gout != nullptr) gout[i] = sum[u];
-                const uint16_t b = to_storage16(sum[u] * sc.operand, kind_dtype(PHI));
+                const uint16_t b = to_storage16(sum[u] * sc.operand, kind_dtype(KIND));
                 // S[c][e] goes to row e, column c of the operand; z[c] to column c of rows D .. D+7.
                 const bool is_z = i >= D * D;
                 const int c = is_z ? i - D * D : i / D;
@@ -457,7 +458,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
     cluster.sync();  // every operand is complete; no CTA leaves while a peer still reads `part`
 
     const int qtiles = (N + C::TILE_Q - 1) / C::TILE_Q;
-    apply_tiles<D, PHI>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(rank, qtiles, csize),
+    apply_tiles<D, KIND>(Q + slab_off, Y + slab_off, N, L.row_stride, chunk_begin(rank, qtiles, csize),
                         chunk_begin(rank + 1, qtiles, csize), St, stage, sc);
 }
 

@@ -20,15 +20,15 @@
 //                           (CTA, slab) writes its own fp32 partial; nothing is combined with
 //                           atomics.
 //   stream_reduce_kernel  — sums the partials of a slab in CTA order; also lays S^T | z out
-//                           as the bf16, K-major, 128-byte-swizzled B operand the apply kernel
+//                           as the 16-bit, K-major, 128-byte-swizzled B operand the apply kernel
 //                           copies into shared memory.
 //   stream_apply_kernel   — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps) on tcgen05: a 128-row Q tile
 //                           is one MMA tile (M = 128).  Each of the 128 threads of a warpgroup
-//                           reads its row from the stage, applies phi in packed bf16 and writes
+//                           reads its row from the stage, applies phi in packed 16-bit arithmetic and writes
 //                           the row to tensor memory as the A operand; one thread of the CTA
 //                           issues D[128 x 80] = A[128 x 64] * B[64 x 80] (B = S^T rows, then z,
 //                           then zero padding, from shared memory); the threads read their row
-//                           of D back, divide by the z column, write the bf16 row over the Q
+//                           of D back, divide by the z column, write the 16-bit row over the Q
 //                           row in the stage, and a TMA store sends the tile to Y.  Q tiles are
 //                           handed out per slab through an atomic counter (the result of a tile
 //                           does not depend on which CTA computes it).
@@ -127,7 +127,7 @@ __device__ __forceinline__ void drain_loads(uint64_t* full, int first, int issue
 // Per stage s: full[s] -> k_ready[s] (4 warps) -> empty[s] (commit).  Per accumulator b:
 // acc_done[b] (commit) -> acc_free[b] (3 flush warps).
 // ---------------------------------------------------------------------------------------------
-template <int PHI>
+template <int KIND>
 __global__ void __launch_bounds__(StreamStateCfg::THREADS, StreamStateCfg::CTAS_PER_SM)
 stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, float* __restrict__ partials,
@@ -167,7 +167,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     // which is the first value of token t's 128-byte row, moved by the swizzle to chunk t & 7.
     for (int i = tid; i < C::ONES_BYTES / 4; i += C::THREADS) reinterpret_cast<uint32_t*>(ones)[i] = 0u;
     __syncthreads();
-    if (tid < 16) *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = static_cast<uint16_t>(ones_pair<PHI>() & 0xffffu);
+    if (tid < 16) *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = static_cast<uint16_t>(ones_pair<KIND>() & 0xffffu);
     fence_proxy_async_smem();
     if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
     tc_fence_before_sync();
@@ -206,7 +206,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     } else if (warp == C::MMA_WARP) {
         // ---------------- MMA warp ----------------
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(PHI), 128, 64, kUmmaAMnMajor | kUmmaBMnMajor);
+            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), 128, 64, kUmmaAMnMajor | kUmmaBMnMajor);
             const uint32_t ones_addr = smem_u32(ones);
             int cur_slab = -1, in_segment = 0, segments = 0, buf = 1;
             for (int it = 0; it < n_units; ++it) {
@@ -316,10 +316,10 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     uint32_t x0, x1, x2, x3;
                     const uint32_t addr = base + ((c ^ sw) << 4);
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3) : "r"(addr));
-                    x0 = phi_packed_pair<PHI>(x0);
-                    x1 = phi_packed_pair<PHI>(x1);
-                    x2 = phi_packed_pair<PHI>(x2);
-                    x3 = phi_packed_pair<PHI>(x3);
+                    x0 = phi_packed_pair<KIND>(x0);
+                    x1 = phi_packed_pair<KIND>(x1);
+                    x2 = phi_packed_pair<KIND>(x2);
+                    x3 = phi_packed_pair<KIND>(x3);
                     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x0), "r"(x1), "r"(x2), "r"(x3) : "memory");
                 }
             }
@@ -339,7 +339,7 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
 }
 
 // Operand image of S | z for the apply kernel, per slab: the MMA's B operand in its shared-memory
-// form — 80 rows of 128 bytes, row n < 64 = column n of S (64 bf16 along c), row 64 = z, rows 65-79
+// form — 80 rows of 128 bytes, row n < 64 = column n of S (64 values of the storage type along c), row 64 = z, rows 65-79
 // zero; 16-byte chunk j of row n sits at chunk position j ^ (n & 7) (the 128-byte swizzle).
 constexpr int kStreamOperandBytes = StreamApplyCfg::B_BYTES;
 
@@ -372,7 +372,7 @@ __device__ __forceinline__ void emit_state_operand(const float* sums, unsigned c
 }
 
 // grid (17, slabs), 256 threads: state[slab] = sum over the CTAs whose run meets the slab, in
-// increasing CTA index (fp32, fixed order).  Also writes the bf16 operand
+// increasing CTA index (fp32, fixed order).  Also writes the 16-bit operand
 // image of S | z for the apply kernel and clears the slab's tile counter for it.
 __global__ void __launch_bounds__(256)
 stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
@@ -410,7 +410,7 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
     emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes, dtype, operand_scale);
 }
 
-// grid (17, slabs), 256 threads: rebuild the bf16 operand image (and clear the tile counters) from
+// grid (17, slabs), 256 threads: rebuild the 16-bit operand image (and clear the tile counters) from
 // an fp32 state that was changed outside the library — the sum over devices of a token-sharded
 // forward (Sec. 4.3).
 __global__ void __launch_bounds__(256)
@@ -447,7 +447,7 @@ stream_pack_kernel(const float* __restrict__ state, unsigned char* __restrict__ 
 // Per stage s: full[s] (TMA bytes landed) -> a_ready[g] (4 warps: phi(Q) rows in TMEM) ->
 // mma_done[g] (tcgen05.commit) -> y_ready[s] (4 warps: Y rows in the stage) -> empty[s].
 // ---------------------------------------------------------------------------------------------
-template <int PHI>
+template <int KIND>
 __global__ void __launch_bounds__(StreamApplyCfg::THREADS, 1)
 stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_y,
                     const unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
@@ -599,7 +599,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         // (tcgen05.mma issued by the leaders of several warpgroups at once lost completions now and
         // then; with a single issuing thread it has not.)
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(PHI), C::TILE, C::B_ROWS);
+            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), C::TILE, C::B_ROWS);
             const uint64_t b_desc = umma_desc_kmajor_sw128(smem_u32(bsm));
             for (int it = 0;; ++it) {
                 const int s = it % C::STAGES, g = it % C::GROUPS;
@@ -614,7 +614,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 }
                 tc_fence_after_sync();
                 const uint32_t a_tmem = tmem_base + g * C::TMEM_COLS_PER_GROUP, d_tmem = a_tmem + 32;
-                // K = 64 as four steps of 16: A advances 8 columns (two bf16 per column), B 32 bytes
+                // K = 64 as four steps of 16: A advances 8 columns (two 16-bit values per column), B 32 bytes
 #pragma unroll
                 for (int k = 0; k < 4; ++k) umma_ts(d_tmem, a_tmem + 8 * k, b_desc + 2 * k, idesc, k > 0 ? 1u : 0u);
                 umma_commit(&mma_done[g]);
@@ -652,10 +652,10 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
                                  : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
                                  : "r"(base + ((c ^ sw) << 4)));
-                    a[4 * c + 0] = phi_packed_pair<PHI>(x0);
-                    a[4 * c + 1] = phi_packed_pair<PHI>(x1);
-                    a[4 * c + 2] = phi_packed_pair<PHI>(x2);
-                    a[4 * c + 3] = phi_packed_pair<PHI>(x3);
+                    a[4 * c + 0] = phi_packed_pair<KIND>(x0);
+                    a[4 * c + 1] = phi_packed_pair<KIND>(x1);
+                    a[4 * c + 2] = phi_packed_pair<KIND>(x2);
+                    a[4 * c + 3] = phi_packed_pair<KIND>(x3);
                 }
                 tmem_store_32cols(a_tmem, a);
             }
@@ -678,10 +678,10 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 tmem_load_32cols(d_tmem + 32 * half, d);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    const uint32_t v0 = pack_pair<PHI>(__uint_as_float(d[8 * c + 0]) * inv, __uint_as_float(d[8 * c + 1]) * inv);
-                    const uint32_t v1 = pack_pair<PHI>(__uint_as_float(d[8 * c + 2]) * inv, __uint_as_float(d[8 * c + 3]) * inv);
-                    const uint32_t v2 = pack_pair<PHI>(__uint_as_float(d[8 * c + 4]) * inv, __uint_as_float(d[8 * c + 5]) * inv);
-                    const uint32_t v3 = pack_pair<PHI>(__uint_as_float(d[8 * c + 6]) * inv, __uint_as_float(d[8 * c + 7]) * inv);
+                    const uint32_t v0 = pack_pair<KIND>(__uint_as_float(d[8 * c + 0]) * inv, __uint_as_float(d[8 * c + 1]) * inv);
+                    const uint32_t v1 = pack_pair<KIND>(__uint_as_float(d[8 * c + 2]) * inv, __uint_as_float(d[8 * c + 3]) * inv);
+                    const uint32_t v2 = pack_pair<KIND>(__uint_as_float(d[8 * c + 4]) * inv, __uint_as_float(d[8 * c + 5]) * inv);
+                    const uint32_t v3 = pack_pair<KIND>(__uint_as_float(d[8 * c + 6]) * inv, __uint_as_float(d[8 * c + 7]) * inv);
                     asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(base + (((4 * half + c) ^ sw) << 4)),
                                  "r"(v0), "r"(v1), "r"(v2), "r"(v3)
                                  : "memory");
