@@ -192,6 +192,29 @@ linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host,
 linfusion_status_t linfusion_attn_state(linfusion_attn_t* h, const void* k, const void* v,
                                         void* cuda_stream);
 linfusion_status_t linfusion_attn_apply(linfusion_attn_t* h, const void* q, void* y, void* cuda_stream);
+
+/*
+ * Steps 2 and 3 in one: the apply half that sums the devices' states itself (Sec. 4.3's exchange of
+ * the c' x c quantity, done by the kernel that needs it instead of a separate collective).
+ * peer_states is a HOST array of n_peers (1 .. LINFUSION_MAX_PEERS) DEVICE addresses, entry r the
+ * state_buffer() of rank r's handle (this rank's own included), each readable from this handle's
+ * device: the caller maps peers' buffers (peer access, CUDA IPC or symmetric memory) and passes
+ * the same list, in the same order, on every rank.  A small kernel adds the n states element by
+ * element in list order with plain loads (over NVLink for peers' entries; 4*B*H*d*(d+1) bytes
+ * from each) into this handle's 16-bit operand image, and the apply kernel follows on the same
+ * stream.  Same list => same summation order => the same bits of S | z on every rank.  Nobody's
+ * state buffer is written, so ranks may run this concurrently; read_state() keeps returning the
+ * local, unsummed state.
+ * Synchronization is the caller's: every rank's linfusion_attn_state() must have completed, and
+ * no rank may start its next linfusion_attn_state() on these handles before all ranks' apply_peers
+ * kernels have read its buffer (e.g. a stream-ordered barrier on either side).
+ * Errors: INVALID_ARG (null / misaligned pointers, n_peers out of range), UNSUPPORTED (cluster
+ * handle), CUDA.
+ */
+#define LINFUSION_MAX_PEERS 16
+linfusion_status_t linfusion_attn_apply_peers(linfusion_attn_t* h, const void* q, void* y,
+                                              const float* const* peer_states, int32_t n_peers,
+                                              void* cuda_stream);
 linfusion_status_t linfusion_attn_state_buffer(linfusion_attn_t* h, float** dev_ptr, size_t* floats);
 
 /*

@@ -28,6 +28,7 @@ EXPORTED = [
     "linfusion_attn_set_kernel_timing_stride",
     "linfusion_attn_forward_noalloc",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
+    "linfusion_attn_apply_peers",
 ]
 
 
@@ -94,6 +95,8 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_state.argtypes = [vp, vp, vp, vp]
     lib.linfusion_attn_apply.restype = st
     lib.linfusion_attn_apply.argtypes = [vp, vp, vp, vp]
+    lib.linfusion_attn_apply_peers.restype = st
+    lib.linfusion_attn_apply_peers.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32, vp]
     lib.linfusion_attn_state_buffer.restype = st
     lib.linfusion_attn_state_buffer.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
     _lib = lib
@@ -271,6 +274,25 @@ class LinFusionAttention:
         rc = self._lib.linfusion_attn_apply(self._h, q.data_ptr(), y.data_ptr(), stream)
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_apply")
+        return y
+
+    def apply_peers(self, q, peer_state_ptrs, y=None, stream: Optional[int] = None):
+        """Apply with the sum over devices done by the library: ``peer_state_ptrs`` lists the
+        device addresses of every rank's state buffer (``state_buffer()[0]``, this rank's own
+        included), readable from this device, in the same order on every rank."""
+        import torch
+        self._check(q, "q")
+        if y is None:
+            y = torch.empty_like(q)
+        else:
+            self._check(y, "y")
+        if stream is None:
+            stream = torch.cuda.current_stream(q.device).cuda_stream
+        ptrs = (ctypes.c_void_p * len(peer_state_ptrs))(*[int(p) for p in peer_state_ptrs])
+        rc = self._lib.linfusion_attn_apply_peers(self._h, q.data_ptr(), y.data_ptr(), ptrs,
+                                                  len(peer_state_ptrs), stream)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_apply_peers")
         return y
 
     def state_buffer(self):

@@ -82,6 +82,21 @@ __device__ __forceinline__ float row_scale(float den, const ApplyScales& sc)
     return sc.eps < 0.0f ? sc.unnormalized : 1.0f / (den + sc.eps);
 }
 
+// The fp32 states S | z of the devices of a token-sharded forward (Sec. 4.3), as device addresses
+// this GPU can load from (its own buffer, and peers' buffers mapped over NVLink).  Kernels sum them
+// in index order with plain loads, so every device that is given the same list gets the same bits.
+constexpr int kMaxPeers = 16;
+struct PeerStates {
+    const float* p[kMaxPeers];
+    int n;
+};
+__device__ __forceinline__ float peer_sum(const PeerStates& ps, size_t i)
+{
+    float sum = 0.0f;
+    for (int r = 0; r < ps.n; ++r) sum += ps.p[r][i];
+    return sum;
+}
+
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
 

@@ -1115,7 +1115,7 @@ namespace {
 
 template <int D, int KIND>
 cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a,
-                              const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s)
+                              const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s, const PeerStates* peers)
 {
     using C = SplitCfg<D>;
     const Plan& p = h->plan;
@@ -1126,6 +1126,12 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
         state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
             h->partials, h->state, C::STATE_FLOATS, p.chunks_state, nullptr, D, C::PITCH, C::SMEM_ST,
             dtype_of(h->desc), operand_scale(h->desc));
+    } else if (peers != nullptr) {
+        // Sum the devices' states into the operand image, then apply from the image.
+        peer_sum_image_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
+            *peers, C::STATE_FLOATS, h->operand, D, C::PITCH, C::SMEM_ST, dtype_of(h->desc), operand_scale(h->desc));
+        apply_kernel<D, KIND><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
+            a, h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), h->operand);
     } else {
         // The fp32 state may have been summed over devices: convert it here, not from an image.
         apply_kernel<D, KIND><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
@@ -1136,7 +1142,7 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
 
 template <int KIND>
 cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a,
-                               const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s)
+                               const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s, const PeerStates* peers)
 {
     const Plan& p = h->plan;
     const int N = h->desc.N;
@@ -1155,9 +1161,13 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
         CUtensorMap mq, my;
         if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
             return cudaErrorInvalidValue;
-        // The state may have been summed over devices since the reduction: rebuild its 16-bit image.
-        stream_pack_kernel<<<rgrid, 256, 0, s>>>(h->state, h->operand, h->tile_counters, dtype_of(h->desc),
-                                                operand_scale(h->desc));
+        // The state may have been summed over devices since the reduction, or is summed over the
+        // devices' buffers here: rebuild its 16-bit image.
+        PeerStates own;
+        own.p[0] = h->state;
+        own.n = 1;
+        stream_pack_kernel<<<rgrid, 256, 0, s>>>(peers != nullptr ? *peers : own, h->operand, h->tile_counters,
+                                                dtype_of(h->desc), operand_scale(h->desc));
         stream_apply_kernel<KIND><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
             mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, apply_scales(h->desc), h->desc.H);
     }
@@ -1166,17 +1176,17 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
 
 template <int D>
 cudaError_t split_half_d(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a, const __nv_bfloat16* b,
-                         __nv_bfloat16* y, cudaStream_t s)
+                         __nv_bfloat16* y, cudaStream_t s, const PeerStates* peers)
 {
     cudaError_t e = cudaErrorInvalidValue;
-#define LF_K(KV) e = launch_split_half<D, KV>(h, state_half, a, b, y, s)
+#define LF_K(KV) e = launch_split_half<D, KV>(h, state_half, a, b, y, s, peers)
     LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
     return e;
 }
 
 linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, const void* b, void* y,
-                            void* cuda_stream)
+                            void* cuda_stream, const PeerStates* peers = nullptr)
 {
     if (h == nullptr || a == nullptr || (state_half ? b == nullptr : y == nullptr))
         return LINFUSION_ERR_INVALID_ARG;
@@ -1194,11 +1204,11 @@ linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, c
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
     cudaError_t e = cudaErrorInvalidValue;
     if (h->plan.variant == kStream) {
-#define LF_K(KV) e = launch_stream_half<KV>(h, state_half, A, B, Y, s)
+#define LF_K(KV) e = launch_stream_half<KV>(h, state_half, A, B, Y, s, peers)
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
     } else {
-#define LF_HALF(DV) e = split_half_d<DV>(h, state_half, A, B, Y, s)
+#define LF_HALF(DV) e = split_half_d<DV>(h, state_half, A, B, Y, s, peers)
         LF_DISPATCH_D(h->desc.d, LF_HALF)
 #undef LF_HALF
     }
@@ -1222,6 +1232,22 @@ extern "C" linfusion_status_t linfusion_attn_apply(linfusion_attn_t* h, const vo
                                                    void* cuda_stream)
 {
     return run_half(h, false, q, nullptr, y, cuda_stream);
+}
+
+extern "C" linfusion_status_t linfusion_attn_apply_peers(linfusion_attn_t* h, const void* q, void* y,
+                                                         const float* const* peer_states, int32_t n_peers,
+                                                         void* cuda_stream)
+{
+    if (h == nullptr || peer_states == nullptr || n_peers < 1 || n_peers > kMaxPeers) return LINFUSION_ERR_INVALID_ARG;
+    PeerStates ps;
+    ps.n = n_peers;
+    for (int r = 0; r < kMaxPeers; ++r) ps.p[r] = nullptr;
+    for (int r = 0; r < n_peers; ++r) {
+        if (peer_states[r] == nullptr || (reinterpret_cast<uintptr_t>(peer_states[r]) & 3u) != 0)
+            return LINFUSION_ERR_INVALID_ARG;
+        ps.p[r] = peer_states[r];
+    }
+    return run_half(h, false, q, nullptr, y, cuda_stream, &ps);
 }
 
 extern "C" linfusion_status_t linfusion_attn_state_buffer(linfusion_attn_t* h, float** dev_ptr,

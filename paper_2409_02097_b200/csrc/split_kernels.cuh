@@ -340,6 +340,30 @@ state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ stat
     }
 }
 
+// grid (ceil(state_floats / 256), slabs): the apply kernel's operand image from the sum, in index
+// order, of the fp32 states of the devices of a token-sharded forward (Sec. 4.3; loads from peers'
+// memory when the list holds peers' buffers).  Same image layout as state_reduce_kernel writes.
+__global__ void __launch_bounds__(256)
+peer_sum_image_kernel(PeerStates states, int state_floats, unsigned char* __restrict__ st_image, int d,
+                      int pitch, int image_bytes, int dtype, float operand_scale)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= state_floats) return;
+    const int slab = blockIdx.y;
+    const float sum = peer_sum(states, static_cast<size_t>(slab) * state_floats + idx);
+    unsigned char* img = st_image + static_cast<size_t>(slab) * image_bytes;
+    const uint16_t b = to_storage16(sum * operand_scale, dtype);
+    if (idx < d * d) {
+        const int c = idx / d, e = idx - c * d;
+        *reinterpret_cast<uint16_t*>(img + e * pitch + c * 2) = b;
+    } else {
+        const int c = idx - d * d;
+        for (int j = 0; j < 8; ++j) *reinterpret_cast<uint16_t*>(img + (d + j) * pitch + c * 2) = b;
+    }
+}
+
 // grid (chunks, slabs).  `st_image` (may be null) is the operand image written by
 // state_reduce_kernel; without it every CTA converts the fp32 state itself.
 template <int D, int KIND>

@@ -411,10 +411,11 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
 }
 
 // grid (17, slabs), 256 threads: rebuild the 16-bit operand image (and clear the tile counters) from
-// an fp32 state that was changed outside the library — the sum over devices of a token-sharded
-// forward (Sec. 4.3).
+// fp32 states that were changed or live outside the reduction — the state after a sum over devices
+// of a token-sharded forward (Sec. 4.3), or the devices' states themselves, which are then summed
+// here in index order (loads from peers' memory when the list holds peers' buffers).
 __global__ void __launch_bounds__(256)
-stream_pack_kernel(const float* __restrict__ state, unsigned char* __restrict__ operand,
+stream_pack_kernel(PeerStates states, unsigned char* __restrict__ operand,
                    int* __restrict__ tile_counters, int dtype, float operand_scale)
 {
     __shared__ float sums[256];
@@ -424,7 +425,7 @@ stream_pack_kernel(const float* __restrict__ state, unsigned char* __restrict__ 
     pdl_launch_dependents();
     pdl_wait();
     if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
-    sums[tid] = idx < kStreamStateFloats ? state[static_cast<size_t>(slab) * kStreamStateFloats + idx] : 0.0f;
+    sums[tid] = idx < kStreamStateFloats ? peer_sum(states, static_cast<size_t>(slab) * kStreamStateFloats + idx) : 0.0f;
     __syncthreads();
     emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes, dtype, operand_scale);
 }

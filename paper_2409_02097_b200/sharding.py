@@ -71,5 +71,20 @@ class TokenShardedAttention:
 
         return sharded_forward(state_fn, lambda q_: self.op.apply(q_, y), allreduce_sum, q, k, v)
 
+    def forward_peers(self, q, k, v, peer_state_ptrs, barrier: Callable[[], None], y=None):
+        """The same layer with the cross-device sum done by the apply step itself instead of an
+        all-reduce: ``peer_state_ptrs`` lists, in rank order, device addresses of every rank's
+        state buffer that this device can load from (this rank's own is
+        ``self.op.state_buffer()[0]``; peers' come from whatever maps their memory here — peer
+        access within a process, CUDA IPC or symmetric memory across processes).  ``barrier()``
+        must return only when every rank's state kernel has completed (it is called between the
+        two halves, and once more after the apply so that no rank overwrites a state that a peer
+        is still reading)."""
+        self.op.state(k, v)
+        barrier()
+        out = self.op.apply_peers(q, peer_state_ptrs, y)
+        barrier()
+        return out
+
     def close(self):
         self.op.close()

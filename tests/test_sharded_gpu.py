@@ -40,6 +40,44 @@ def test_two_token_shards_summed_state(dims, variant):
     assert_parity(y, ref, f"sharded {dims} {variant}")
 
 
+@pytest.mark.parametrize("dims,variant,world", [((2, 5, 9000, 64), "stream", 2), ((1, 4, 3001, 64), "split", 3),
+                                                ((1, 2, 700, 160), "split", 2), ((1, 3, 20000, 64), "stream", 8)],
+                         ids=lambda x: str(x))
+def test_apply_sums_the_shards_states_itself(dims, variant, world):
+    """apply_peers on one GPU: the shards' handles stand in for the ranks, their state buffers for
+    the peers' memory.  Every shard is given the same list, so every shard sums in the same order."""
+    B, H, N, d = dims
+    q, k, v = wl.make_small(B, H, N, d, seed=79, device="cuda")
+    ref = oracle_y(q, k, v)
+    ops, cuts = [], []
+    for r in range(world):
+        b, e = sharding.token_shard(N, r, world)
+        op = attn.LinFusionAttention(B, H, e - b, d, eps=EPS, variant=variant)
+        op.state(k[:, :, b:e].contiguous(), v[:, :, b:e].contiguous())
+        ops.append(op)
+        cuts.append((b, e))
+    torch.cuda.synchronize()                                    # the stand-in for the cross-rank barrier
+    ptrs = [op.state_buffer()[0] for op in ops]
+    y = torch.empty_like(q)
+    for op, (b, e) in zip(ops, cuts):
+        y[:, :, b:e] = op.apply_peers(q[:, :, b:e].contiguous(), ptrs)
+    torch.cuda.synchronize()
+    assert_parity(y, ref, f"apply_peers {dims} {variant} x{world}")
+    # the local states were left alone, and their sum is the whole sequence's state
+    S_sum = sum(op.read_state()[0] for op in ops)
+    full = attn.LinFusionAttention(B, H, N, d, eps=EPS, variant=variant)
+    full.forward(q, k, v)
+    S_full, _ = full.read_state()
+    assert np.linalg.norm(S_sum - S_full) <= 1e-5 * np.linalg.norm(S_full)
+    with pytest.raises(attn.LinFusionError):
+        ops[0].apply_peers(q[:, :, cuts[0][0]:cuts[0][1]].contiguous(), [])
+    with pytest.raises(attn.LinFusionError):
+        ops[0].apply_peers(q[:, :, cuts[0][0]:cuts[0][1]].contiguous(), ptrs * 9)
+    for op in ops + [full]:
+        assert op.status() == attn.OK
+        op.close()
+
+
 def test_single_rank_sharded_forward_equals_forward_bits():
     """World size 1: state + apply is the same computation as forward."""
     B, H, N, d = 2, 4, 5000, 64
