@@ -365,8 +365,7 @@ template <typename... KArgs, typename... Args>
 cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
                            Args... args)
 {
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
+    cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
@@ -411,7 +410,7 @@ void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int clus
                     cudaStream_t s)
 {
     using C = SplitCfg<D>;
-    memset(cfg, 0, sizeof(*cfg));
+    *cfg = cudaLaunchConfig_t{};
     cfg->gridDim = dim3(cluster_size, slabs, 1);
     cfg->blockDim = dim3(C::NT, 1, 1);
     cfg->dynamicSmemBytes = C::SMEM_CLUSTER;
