@@ -304,7 +304,7 @@ def test_kernel_timing_stride_samples_every_nth_forward():
     outs = [op.forward(q, k, v).clone() for _ in range(10)]
     sums, calls = op.kernel_times()
     assert calls == 3                      # forwards 0, 4 and 8
-    assert op.launches_per_forward == 2 and all(t > 0 for t in sums[:2]) and sums[2] == 0
+    assert all(t > 0 for t in sums)
     op.enable_kernel_timing(0)
     for o in outs:                         # timed or not, chained or not: the same bits
         assert torch.equal(o.view(torch.int16), y.view(torch.int16))
