@@ -283,7 +283,7 @@ def run_cuda(args):
     # Per-kernel durations recorded inside the timed region.
     peak, peak_kind = measured_peak_gbs()
     kernels = []
-    names = ["stream_state_kernel", "stream_apply_kernel"]   # launch order of the stream path
+    names = ["stream_state_kernel", "stream_reduce_kernel", "stream_apply_kernel"]
     for s, op, *_ in layers:
         sums, calls = op.kernel_times()
         op.enable_kernel_timing(0)
@@ -291,7 +291,7 @@ def run_cuda(args):
             if calls == 0:
                 continue
             avg_ms = total / calls
-            algo = 2 * s.B * s.N * s.C * 2
+            algo = 2 * s.B * s.N * s.C * 2 if name != "stream_reduce_kernel" else 0
             kernels.append({"kernel": name, "shape": s.name, "avg_ms": avg_ms,
                             "algorithmic_bytes": algo,
                             "gbs": (algo / (avg_ms * 1e-3) / 1e9) if avg_ms > 0 else None})

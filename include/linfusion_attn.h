@@ -53,7 +53,7 @@ typedef enum {
 /* flags: kernel-variant selection.  0 lets the library choose from (N, d, B*H). */
 #define LINFUSION_VARIANT_AUTO 0u
 #define LINFUSION_VARIANT_SPLIT 1u   /* three launches: split-N state, reduction, apply (any supported d) */
-#define LINFUSION_VARIANT_STREAM 2u  /* two launches, persistent TMA + tcgen05 kernels (d = 64 only)       */
+#define LINFUSION_VARIANT_STREAM 2u  /* three launches, TMA-pipelined persistent kernels (d = 64 only)    */
 #define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N)               */
 #define LINFUSION_VARIANT_MASK 0xFu
 /*
@@ -222,9 +222,8 @@ linfusion_status_t linfusion_attn_state_buffer(linfusion_attn_t* h, float** dev_
  * from then on every forward() brackets each of its kernels with event records on its stream
  * (set = call index modulo slots).  enable(h, 0) turns it off.  kernel_times() synchronizes the
  * handle's last stream and returns, for the calls recorded since the last kernel_times()
- * (at most `slots`), the summed milliseconds of each kernel in launch order — split path:
- * ms_sum[0] the state kernel, ms_sum[1] the reduction, ms_sum[2] the apply; stream path (its
- * state kernel includes the reduction): ms_sum[0] state, ms_sum[1] apply; cluster: ms_sum[0] —
+ * (at most `slots`), the summed milliseconds of each kernel in launch order — ms_sum[0] the
+ * state kernel (or the single clustered kernel), ms_sum[1] the reduction, ms_sum[2] the apply —
  * and the number of calls summed.  Errors: INVALID_ARG, ALLOC, CUDA.
  */
 linfusion_status_t linfusion_attn_enable_kernel_timing(linfusion_attn_t* h, int32_t slots);

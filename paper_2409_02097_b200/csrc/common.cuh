@@ -364,13 +364,6 @@ __device__ __forceinline__ void tma_store_4d(const void* tmap, const void* smem_
 __device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// Barrier among `threads` threads of the CTA (a multiple of 32; whole warps), on hardware barrier `id`
-// (1..15; 0 is __syncthreads()).
-__device__ __forceinline__ void named_barrier_sync(int id, int threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
-
 // Generic-proxy writes to shared memory made visible to the async proxy (TMA stores, tcgen05.mma).
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 

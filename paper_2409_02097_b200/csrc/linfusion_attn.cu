@@ -138,7 +138,7 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         }
         p->spans = spans;
         partial_floats = static_cast<size_t>(p->G_state) * spans * kStreamStateFloats;
-        p->launches = 2;  // state (with its second stage), apply
+        p->launches = 3;
     } else {
         p->cluster_size = largest_cluster(tiles_kv);
         partial_floats = 0;
@@ -148,14 +148,13 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     p->state_off = p->partial_bytes;
     p->operand_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
     // 16-bit operand image of S | z for the apply kernel (in its shared-memory layout), and for the
-    // stream variant two counters per slab: the apply kernel's tile counter, and the count of
-    // partials delivered (the state kernel's second stage runs where it reaches its total).
+    // stream variant one tile counter per slab.
     const int dp = (d->d + 15) / 16 * 16;
     const size_t split_image = static_cast<size_t>((d->d + 8 + 15) / 16 * 16) * (((dp / 8) | 1) * 16);
     const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamOperandBytes
                               : v == LINFUSION_VARIANT_SPLIT ? static_cast<size_t>(slabs) * split_image
                                                              : 0;
-    const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM ? align_up(static_cast<size_t>(slabs) * 2 * 4, 256) : 0;
+    const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM ? align_up(static_cast<size_t>(slabs) * 4, 256) : 0;
     p->counters_off = p->operand_off + align_up(frag_bytes, 256);
     p->status_off = p->counters_off + counter_bytes;
     p->total_bytes = p->status_off + 256;
@@ -453,15 +452,19 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
     mark(h, 0, s);
     e = launch_chained(stream_state_kernel<KIND>, dim3(p.G_state), dim3(StreamStateCfg::THREADS),
                        StreamStateCfg::SMEM_BYTES, s, mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state,
-                       p.spans, h->desc.H, h->state, h->operand, h->tile_counters + p.slabs, h->tile_counters,
-                       dtype_of(h->desc), operand_scale(h->desc));
+                       p.spans, h->desc.H);
     if (e != cudaSuccess) return e;
     mark(h, 1, s);
+    e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
+                       h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
+                       p.spans, dtype_of(h->desc), operand_scale(h->desc));
+    if (e != cudaSuccess) return e;
+    mark(h, 2, s);
     e = launch_chained(stream_apply_kernel<KIND>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
                        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs,
                        apply_scales(h->desc), h->desc.H);
     if (e != cudaSuccess) return e;
-    mark(h, 2, s);
+    mark(h, 3, s);
     return cudaGetLastError();
 }
 
@@ -1149,8 +1152,10 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
             !encode_slab_map(&mv, b, h->desc, StreamStateCfg::TILE))
             return cudaErrorInvalidValue;
         stream_state_kernel<KIND><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
-            mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H, h->state, h->operand,
-            h->tile_counters + p.slabs, h->tile_counters, dtype_of(h->desc), operand_scale(h->desc));
+            mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
+        stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->operand, h->tile_counters,
+                                                  p.tiles_state, p.W_state, p.G_state, p.spans,
+                                                  dtype_of(h->desc), operand_scale(h->desc));
     } else {
         CUtensorMap mq, my;
         if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))

@@ -19,10 +19,9 @@
 //                           tiles (keeps the tensor core's accumulation chains short).  Each
 //                           (CTA, slab) writes its own fp32 partial; nothing is combined with
 //                           atomics.
-//                           The CTA that delivers a slab's last partial (an atomic count per slab)
-//                           sums the slab's partials in CTA order — fixed order, whoever does it —
-//                           and lays S^T | z out as the 16-bit, K-major, 128-byte-swizzled B operand
-//                           the apply kernel copies into shared memory: no reduction kernel.
+//   stream_reduce_kernel  — sums the partials of a slab in CTA order; also lays S^T | z out
+//                           as the 16-bit, K-major, 128-byte-swizzled B operand the apply kernel
+//                           copies into shared memory.
 //   stream_apply_kernel   — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps) on tcgen05: a 128-row Q tile
 //                           is one MMA tile (M = 128).  Each of the 128 threads of a warpgroup
 //                           reads its row from the stage, applies phi in packed 16-bit arithmetic and writes
@@ -115,66 +114,6 @@ __device__ __forceinline__ void drain_loads(uint64_t* full, int first, int issue
         }
 }
 
-// The CTAs whose runs meet slab `slab`: g0 is the one whose run contains the slab's first unit, g1
-// the first whose run starts at or after its end; slot0 is the slab's slot in CTA g0's partials
-// (every later CTA starts inside the slab: slot 0).
-__device__ __forceinline__ void slab_contributors(int slab, int tiles_per_slab, long long W, long long G,
-                                                  long long& g0, long long& g1, int& slot0)
-{
-    const long long lo = static_cast<long long>(slab) * tiles_per_slab, hi = lo + tiles_per_slab;
-    g0 = (lo * G) / W;
-    while (g0 + 1 < G && unit_begin(g0 + 1, W, G) <= lo) ++g0;
-    while (g0 > 0 && unit_begin(g0, W, G) > lo) --g0;
-    g1 = (hi * G) / W;
-    while (g1 < G && unit_begin(g1, W, G) < hi) ++g1;
-    while (g1 > 0 && unit_begin(g1 - 1, W, G) >= hi) --g1;
-    slot0 = slab - static_cast<int>(unit_begin(g0, W, G) / tiles_per_slab);
-}
-
-// Second stage of the state reduction for one slab, run by the NT threads (t = 0 .. NT-1) of the CTA
-// that delivered the slab's last partial: state[slab] = sum of the partials in increasing CTA index
-// (fp32, fixed order, whoever runs this), and the 16-bit operand image of S | z for the apply kernel
-// (layout: see kStreamOperandBytes below).  The partials were written by other CTAs: loads bypass L1.
-template <int NT>
-__device__ __forceinline__ void reduce_slab(const float* __restrict__ partials, float* __restrict__ state_slab,
-                                            unsigned char* __restrict__ img, int slab, int tiles_per_slab,
-                                            long long W, long long G, int spans, int dtype, float scale, int t)
-{
-    long long g0, g1;
-    int slot0;
-    slab_contributors(slab, tiles_per_slab, W, G, g0, g1, slot0);
-    const size_t F = kStreamStateFloats;
-    const float* first = partials + (static_cast<size_t>(g0) * spans + slot0) * F;
-    auto sum_at = [&](int idx) {
-        float sum = __ldcg(first + idx);
-        for (long long g = g0 + 1; g < g1; ++g) sum += __ldcg(partials + (static_cast<size_t>(g) * spans) * F + idx);
-        return sum;
-    };
-    // S: four consecutive features c0 .. c0+3 of channel e are one 8-byte piece of image row e
-    for (int u = t; u < 16 * 64; u += NT) {
-        const int c0 = 4 * (u >> 6), e = u & 63;
-        float v[4];
-#pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            v[r] = sum_at((c0 + r) * 64 + e);
-            state_slab[(c0 + r) * 64 + e] = v[r];
-        }
-        uint2 w;
-        w.x = to_storage16(v[0] * scale, dtype) | (static_cast<uint32_t>(to_storage16(v[1] * scale, dtype)) << 16);
-        w.y = to_storage16(v[2] * scale, dtype) | (static_cast<uint32_t>(to_storage16(v[3] * scale, dtype)) << 16);
-        *reinterpret_cast<uint2*>(img + e * 128 + (((c0 >> 3) ^ (e & 7)) << 4) + (c0 & 7) * 2) = w;
-    }
-    // z -> row 64 (64 & 7 = 0: chunks in place); rows 65..79 are zero
-    for (int u = t; u < 32; u += NT) {
-        const float a = sum_at(64 * 64 + 2 * u), b = sum_at(64 * 64 + 2 * u + 1);
-        state_slab[64 * 64 + 2 * u] = a;
-        state_slab[64 * 64 + 2 * u + 1] = b;
-        *reinterpret_cast<uint32_t*>(img + 64 * 128 + u * 4) =
-            to_storage16(a * scale, dtype) | (static_cast<uint32_t>(to_storage16(b * scale, dtype)) << 16);
-    }
-    for (int u = t; u < 120; u += NT) reinterpret_cast<uint4*>(img + 65 * 128)[u] = make_uint4(0u, 0u, 0u, 0u);
-}
-
 // ---------------------------------------------------------------------------------------------
 // State: partials[g * spans + slot][kStreamStateFloats], slot = slab - first slab of CTA g's run.
 //
@@ -192,9 +131,7 @@ template <int KIND>
 __global__ void __launch_bounds__(StreamStateCfg::THREADS, StreamStateCfg::CTAS_PER_SM)
 stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, float* __restrict__ partials,
-                    uint32_t* __restrict__ status, int N, int tiles_per_slab, long long W, int spans, int H,
-                    float* __restrict__ state, unsigned char* __restrict__ operand, int* __restrict__ slab_done,
-                    int* __restrict__ tile_counters, int dtype, float operand_scale)
+                    uint32_t* __restrict__ status, int N, int tiles_per_slab, long long W, int spans, int H)
 {
     using C = StreamStateCfg;
     extern __shared__ unsigned char smem_raw[];
@@ -356,29 +293,6 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                 }
 #pragma unroll
                 for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
-                // Second stage, by whichever CTA delivers the slab's last partial: make this partial
-                // visible, count it, and if every contributor has been counted sum them all.
-                __threadfence();
-                named_barrier_sync(1, 96);
-                int* last_flag = reinterpret_cast<int*>(tmem_slot + 1);
-                if (wq == 0 && lane == 0) {
-                    long long g0, g1;
-                    int slot0;
-                    slab_contributors(slab, tiles_per_slab, W, G, g0, g1, slot0);
-                    *last_flag = atomicAdd(&slab_done[slab], 1) + 1 == static_cast<int>(g1 - g0) ? 1 : 0;
-                }
-                named_barrier_sync(1, 96);
-                if (*last_flag != 0) {
-                    __threadfence();
-                    reduce_slab<96>(partials, state + static_cast<size_t>(slab) * kStreamStateFloats,
-                                    operand + static_cast<size_t>(slab) * StreamApplyCfg::B_BYTES, slab, tiles_per_slab,
-                                    W, G, spans, dtype, operand_scale, wq * 32 + lane);
-                    if (wq == 0 && lane == 0) {
-                        slab_done[slab] = 0;        // ready for the next forward
-                        tile_counters[slab] = 0;    // the apply kernel's tile counter of this slab
-                    }
-                }
-                named_barrier_sync(1, 96);          // last_flag may be rewritten only after all have read it
             }
         }
     } else if (warp < C::PHI_WARPS) {
@@ -455,6 +369,45 @@ __device__ __forceinline__ void emit_state_operand(const float* sums, unsigned c
             reinterpret_cast<uint4*>(img + 65 * 128)[tid - 32] = make_uint4(0u, 0u, 0u, 0u);
         }
     }
+}
+
+// grid (17, slabs), 256 threads: state[slab] = sum over the CTAs whose run meets the slab, in
+// increasing CTA index (fp32, fixed order).  Also writes the 16-bit operand
+// image of S | z for the apply kernel and clears the slab's tile counter for it.
+__global__ void __launch_bounds__(256)
+stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
+                     unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
+                     int tiles_per_slab, long long W, int G, int spans, int dtype, float operand_scale)
+{
+    __shared__ float sums[256];
+    const int tid = threadIdx.x;
+    const int idx = blockIdx.x * 256 + tid;
+    const int slab = blockIdx.y;
+    pdl_launch_dependents();
+    pdl_wait();
+    if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
+    float sum = 0.0f;
+    if (idx < kStreamStateFloats) {
+        const long long lo = static_cast<long long>(slab) * tiles_per_slab, hi = lo + tiles_per_slab;
+        // g0: the CTA whose run contains unit `lo`; g1: the first CTA whose run starts at or after `hi`.
+        long long g0 = (lo * G) / W;
+        while (g0 + 1 < G && unit_begin(g0 + 1, W, G) <= lo) ++g0;
+        while (g0 > 0 && unit_begin(g0, W, G) > lo) --g0;
+        long long g1 = (hi * G) / W;
+        while (g1 < G && unit_begin(g1, W, G) < hi) ++g1;
+        while (g1 > 0 && unit_begin(g1 - 1, W, G) >= hi) --g1;
+        const int slot0 = slab - static_cast<int>(unit_begin(g0, W, G) / tiles_per_slab);
+        const size_t F = kStreamStateFloats;
+        const float* src = partials + idx;
+        sum += src[(static_cast<size_t>(g0) * spans + slot0) * F];
+        // Every later CTA starts inside this slab: its partial for it is in slot 0.
+#pragma unroll 4
+        for (long long g = g0 + 1; g < g1; ++g) sum += src[(static_cast<size_t>(g) * spans) * F];
+        state[static_cast<size_t>(slab) * F + idx] = sum;
+    }
+    sums[tid] = sum;
+    __syncthreads();
+    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes, dtype, operand_scale);
 }
 
 // grid (17, slabs), 256 threads: rebuild the 16-bit operand image (and clear the tile counters) from
