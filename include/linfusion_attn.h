@@ -163,6 +163,17 @@ linfusion_status_t linfusion_attn_set_workspace(linfusion_attn_t* h, void* dev_p
 linfusion_status_t linfusion_attn_status(linfusion_attn_t* h);
 
 /*
+ * Self-test of the failure reporting (the paper has no counterpart): runs a one-warp kernel that
+ * waits on a barrier nothing will ever complete, exactly as the attention kernels wait, on the
+ * handle's last stream.  The wait must give up after its time bound (a quarter of a second), the
+ * kernel must end normally and the device status word must be set.  Returns TIMEOUT when all of
+ * that happened (the expected result), OK if the wait claimed to have succeeded, or CUDA; the
+ * status word is cleared again, so the handle and the context stay usable.  *waited_ms (may be NULL)
+ * receives the kernel's duration.
+ */
+linfusion_status_t linfusion_attn_selftest_wait(linfusion_attn_t* h, float* waited_ms);
+
+/*
  * Copy the reduced state of the last forward to HOST buffers (fp32): S [B*H][d][d] (row =
  * feature c of K, column = channel e of V) and z [B*H][d].  Synchronizes the handle's last
  * stream.  Either pointer may be NULL.  This is the c' x c quantity that the paper's

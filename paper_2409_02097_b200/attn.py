@@ -28,7 +28,7 @@ EXPORTED = [
     "linfusion_attn_set_kernel_timing_stride",
     "linfusion_attn_forward_noalloc",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
-    "linfusion_attn_apply_peers",
+    "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait",
 ]
 
 
@@ -95,6 +95,8 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_state.argtypes = [vp, vp, vp, vp]
     lib.linfusion_attn_apply.restype = st
     lib.linfusion_attn_apply.argtypes = [vp, vp, vp, vp]
+    lib.linfusion_attn_selftest_wait.restype = st
+    lib.linfusion_attn_selftest_wait.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.linfusion_attn_apply_peers.restype = st
     lib.linfusion_attn_apply_peers.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32, vp]
     lib.linfusion_attn_state_buffer.restype = st
@@ -308,6 +310,12 @@ class LinFusionAttention:
         rc = self._lib.linfusion_attn_enable_kernel_timing(self._h, int(slots))
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_enable_kernel_timing")
+
+    def selftest_wait(self):
+        """(status code, milliseconds) of the bounded-wait self-test; ERR_TIMEOUT is the expected code."""
+        ms = ctypes.c_float(0.0)
+        rc = self._lib.linfusion_attn_selftest_wait(self._h, ctypes.byref(ms))
+        return int(rc), float(ms.value)
 
     def set_kernel_timing_stride(self, stride: int) -> None:
         rc = self._lib.linfusion_attn_set_kernel_timing_stride(self._h, int(stride))

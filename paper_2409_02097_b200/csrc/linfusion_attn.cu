@@ -894,6 +894,36 @@ linfusion_status_t linfusion_attn_status(linfusion_attn_t* h)
     return LINFUSION_OK;
 }
 
+linfusion_status_t linfusion_attn_selftest_wait(linfusion_attn_t* h, float* waited_ms)
+{
+    if (h == nullptr || h->status == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    cudaStream_t s = h->last_stream;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        if (e0 != nullptr) cudaEventDestroy(e0);
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    cudaEventRecord(e0, s);
+    wait_selftest_kernel<<<1, 32, 0, s>>>(h->status);
+    cudaEventRecord(e1, s);
+    uint32_t word = 0;
+    float ms = 0.0f;
+    bool ok = cudaStreamSynchronize(s) == cudaSuccess && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess &&
+              cudaMemcpy(&word, h->status, sizeof(word), cudaMemcpyDeviceToHost) == cudaSuccess &&
+              cudaMemset(h->status, 0, sizeof(word)) == cudaSuccess;  // the handle stays usable
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (!ok) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    if (waited_ms != nullptr) *waited_ms = ms;
+    return word != kStatusOk ? LINFUSION_ERR_TIMEOUT : LINFUSION_OK;
+}
+
 linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host, float* z_host)
 {
     if (h == nullptr) return LINFUSION_ERR_INVALID_ARG;

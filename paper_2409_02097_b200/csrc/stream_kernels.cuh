@@ -98,6 +98,21 @@ __device__ __forceinline__ void report_wait_expired(uint32_t* status)
     atomicExch(status, kStatusWaitExpired);
 }
 
+// One warp waits on an mbarrier that nothing ever arrives on: the bounded wait must give up after
+// kMaxBarrierWaitNs and leave the error word behind, and the kernel must end normally.  Run by the
+// library's self-test of its failure reporting, never on the attention path.
+__global__ void __launch_bounds__(32)
+wait_selftest_kernel(uint32_t* __restrict__ status)
+{
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        mbar_fence_init();
+    }
+    __syncwarp();
+    if (!mbar_wait(&bar, 0) && threadIdx.x == 0) report_wait_expired(status);
+}
+
 // Before the producer leaves: a bounded wait for every bulk copy it still has in flight, so
 // that no copy lands in shared memory after the CTA has gone.
 // Loads [first, issued) are waited for; a load whose stage has been armed again since (its phase

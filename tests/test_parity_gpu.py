@@ -311,3 +311,20 @@ def test_kernel_timing_stride_samples_every_nth_forward():
     with pytest.raises(attn.LinFusionError):
         op.set_kernel_timing_stride(0)
     op.close()
+
+
+def test_a_wait_that_cannot_complete_gives_up_and_is_reported():
+    """Failure reporting without a fault: a bounded wait on a barrier nothing arrives on runs out,
+    the kernel returns normally, the status word says so, and the handle keeps working."""
+    shape = wl.find_shape("sdxl_2048_L2")
+    q, k, v = wl.make_qkv(shape, seed=4, device="cuda")
+    y0, op = run_gpu(q, k, v, "stream")
+    rc, ms = op.selftest_wait()
+    assert rc == attn.ERR_TIMEOUT
+    assert 200.0 <= ms <= 2000.0, ms          # the bound is a quarter of a second
+    assert op.status() == attn.OK              # cleared again
+    y1 = op.forward(q, k, v)
+    torch.cuda.synchronize()
+    assert op.status() == attn.OK
+    assert torch.equal(y0.view(torch.int16), y1.view(torch.int16))
+    op.close()
