@@ -3,9 +3,9 @@
 // cp.async.bulk.tensor into 128-byte-swizzled shared-memory stages, Y is written once with TMA
 // stores, and both contractions run on tcgen05 with their accumulators in tensor memory.
 //
-// Work is cut into units of one token tile of one slab, numbered slab-major; CTA g of G owns
-// the contiguous run of units [g*W/G, (g+1)*W/G).  That split is a pure function of the shape
-// and the grid size, so the summation order — and with it every output bit — is fixed.
+// The state kernel's work is cut into units of one token tile of one slab, numbered slab-major;
+// CTA g of G owns the contiguous run of units [g*W/G, (g+1)*W/G).  That split is a pure function of
+// the shape and the grid size, so the summation order — and with it every output bit — is fixed.
 //
 //   stream_state_kernel   — per CTA and per slab it touches: partial S_p = sum phi(K_j)^T V_j and
 //                           z_p (Prop. 2, Eq. 5) on tcgen05.  A K/V tile of 128 tokens is eight
@@ -24,8 +24,9 @@
 //                           copies into shared memory.
 //   stream_apply_kernel   — Y_i = phi(Q_i) S / (phi(Q_i) . z + eps) on tcgen05: a 128-row Q tile
 //                           is one MMA tile (M = 128).  Each of the 128 threads of a warpgroup
-//                           reads its row from the stage, applies phi in packed 16-bit arithmetic and writes
-//                           the row to tensor memory as the A operand; one thread of the CTA
+//                           reads its row from the stage, applies phi in packed 16-bit
+//                           arithmetic and writes the row to tensor memory as the A operand; one
+//                           thread of the CTA
 //                           issues D[128 x 80] = A[128 x 64] * B[64 x 80] (B = S^T rows, then z,
 //                           then zero padding, from shared memory); the threads read their row
 //                           of D back, divide by the z column, write the 16-bit row over the Q
@@ -182,7 +183,8 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     // which is the first value of token t's 128-byte row, moved by the swizzle to chunk t & 7.
     for (int i = tid; i < C::ONES_BYTES / 4; i += C::THREADS) reinterpret_cast<uint32_t*>(ones)[i] = 0u;
     __syncthreads();
-    if (tid < 16) *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = static_cast<uint16_t>(ones_pair<KIND>() & 0xffffu);
+    if (tid < 16)
+        *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = static_cast<uint16_t>(ones_pair<KIND>() & 0xffffu);
     fence_proxy_async_smem();
     if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
     tc_fence_before_sync();
@@ -335,7 +337,8 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     x1 = phi_packed_pair<KIND>(x1);
                     x2 = phi_packed_pair<KIND>(x2);
                     x3 = phi_packed_pair<KIND>(x3);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x0), "r"(x1), "r"(x2), "r"(x3) : "memory");
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(x0), "r"(x1), "r"(x2), "r"(x3)
+                                 : "memory");
                 }
             }
             // else: a row past N.  TMA filled it with zeros and it must count for nothing; phi(0) = 1,
