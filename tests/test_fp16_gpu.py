@@ -93,3 +93,42 @@ def test_fp16_rejects_bf16_tensors():
     with pytest.raises(ValueError):
         op.forward(x, x, x)
     op.close()
+
+
+def test_fp16_host_buffers_no_alloc_and_peer_sum():
+    B, H, N, d = 1, 4, 9000, 64
+    q, k, v = make_fp16(B, H, N, d, seed=53)
+    ref = oracle.linear(to_f64(q), to_f64(k), to_f64(v), EPS)
+    # host-buffer forward
+    op = attn.LinFusionAttention(B, H, N, d, eps=EPS, dtype="fp16")
+    qh, kh, vh = q.cpu(), k.cpu(), v.cpu()
+    yh = torch.empty_like(qh)
+    op.forward_host(qh, kh, vh, yh)
+    torch.cuda.synchronize()
+    assert_parity(yh, ref, "fp16 forward_host")
+    op.close()
+    # allocation-free entry point
+    y = torch.empty_like(q)
+    desc = attn.make_desc(B, H, N, d, eps=EPS, dtype="fp16")
+    attn.linfusion_attn_forward_noalloc(desc, q.data_ptr(), k.data_ptr(), v.data_ptr(), y.data_ptr(),
+                                        torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    assert_parity(y, ref, "fp16 forward_noalloc")
+    # token shards whose states the apply step sums itself (the operand scale follows the shard's N)
+    from paper_2409_02097_b200 import sharding
+    ops, cuts = [], []
+    for r in range(3):
+        b, e = sharding.token_shard(N, r, 3)
+        o = attn.LinFusionAttention(B, H, e - b, d, eps=EPS, variant="stream", dtype="fp16")
+        o.state(k[:, :, b:e].contiguous(), v[:, :, b:e].contiguous())
+        ops.append(o)
+        cuts.append((b, e))
+    torch.cuda.synchronize()
+    ptrs = [o.state_buffer()[0] for o in ops]
+    y2 = torch.empty_like(q)
+    for o, (b, e) in zip(ops, cuts):
+        y2[:, :, b:e] = o.apply_peers(q[:, :, b:e].contiguous(), ptrs)
+    torch.cuda.synchronize()
+    assert_parity(y2, ref, "fp16 apply_peers")
+    for o in ops:
+        o.close()
