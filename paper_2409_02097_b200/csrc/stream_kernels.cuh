@@ -192,15 +192,18 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // Set-up done (barriers, tensor memory): let the next kernel in the stream be scheduled behind
-    // this one, and wait for the one before it to be complete before touching global memory.
+    // this one, and wait for the one before it to be complete before touching global memory.  (The
+    // tensor maps are kernel parameters: fetching them does not depend on earlier work.)
+    if (warp == C::PRODUCER_WARP && lane == 0) {
+        prefetch_tmap(&tmap_k);
+        prefetch_tmap(&tmap_v);
+    }
     pdl_launch_dependents();
     pdl_wait();
 
     if (warp == C::PRODUCER_WARP) {
         // ---------------- producer ----------------
         if (lane == 0) {
-            prefetch_tmap(&tmap_k);
-            prefetch_tmap(&tmap_v);
             const uint64_t policy = policy_evict_first();
             int issued = 0;
             for (int it = 0; it < n_units; ++it) {
@@ -482,7 +485,8 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     uint64_t* y_ready = empty + C::STAGES;
     uint64_t* a_ready = y_ready + C::STAGES;  // per group
     uint64_t* mma_done = a_ready + C::GROUPS;  // per group
-    int2* meta = reinterpret_cast<int2*>(mma_done + C::GROUPS);  // (slab, tile) of each stage; slab < 0 ends
+    uint64_t* b_ready = mma_done + C::GROUPS;  // the operand of the slab now being posted is in shared memory
+    int2* meta = reinterpret_cast<int2*>(b_ready + 1);  // (slab, tile) of each stage; slab < 0 ends
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(meta + C::STAGES);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -497,6 +501,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             mbar_init(&a_ready[g], 4);
             mbar_init(&mma_done[g], 1);
         }
+        mbar_init(b_ready, 1);
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
@@ -505,17 +510,17 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     // Set-up done (barriers, tensor memory): let the next kernel in the stream be scheduled behind
-    // this one, and wait for the one before it to be complete before touching global memory.
+    // this one, and wait for the one before it to be complete before touching global memory.  (The
+    // tensor maps are kernel parameters: fetching them does not depend on earlier work.)
+    if (warp == C::PRODUCER_WARP && lane == 0) prefetch_tmap(&tmap_q);
+    if (warp == C::STORE_WARP && lane == 0) prefetch_tmap(&tmap_y);
     pdl_launch_dependents();
     pdl_wait();
 
     if (warp == C::PRODUCER_WARP) {
         // ---------------- producer warp (lane 0 issues; all lanes help to find work and copy B) ----------------
         uint64_t policy = 0;
-        if (lane == 0) {
-            prefetch_tmap(&tmap_q);
-            policy = policy_evict_first();
-        }
+        if (lane == 0) policy = policy_evict_first();
         int slab = static_cast<int>((static_cast<long long>(blockIdx.x) * slabs) / gridDim.x);
         int it = 0, issued = 0, loaded_slab = -1;
         bool ok = true;
@@ -542,7 +547,8 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             // Claim the tile after this one now: the atomic's round trip (comparable to the time a
             // tile takes) overlaps the wait for a free stage and the copy below.
             if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
-            if (slab != loaded_slab) {
+            const bool new_slab = slab != loaded_slab;
+            if (new_slab) {
                 // Every tile posted so far must have left (its MMAs, which read B, are then
                 // complete as well) before B is overwritten.
                 if (lane == 0) {
@@ -552,11 +558,6 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 }
                 ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                 if (!ok) break;
-                const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
-                for (int i = lane; i < C::B_BYTES / 16; i += 32) reinterpret_cast<uint4*>(bsm)[i] = __ldg(src + i);
-                fence_proxy_async_smem();
-                __syncwarp();
-                loaded_slab = slab;
             }
             const int s = it % C::STAGES;
             if (lane == 0) {
@@ -573,6 +574,16 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
             ++it;
+            if (new_slab) {
+                // The slab's operand, copied while the tile above is on its way; the MMA thread
+                // waits for b_ready before the first MMA of a slab.
+                const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
+                for (int i = lane; i < C::B_BYTES / 16; i += 32) reinterpret_cast<uint4*>(bsm)[i] = __ldg(src + i);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(b_ready);
+                loaded_slab = slab;
+            }
         }
         if (lane == 0) {
             int first = 0;
@@ -597,7 +608,6 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     } else if (warp == C::STORE_WARP) {
         // ---------------- store warp ----------------
         if (lane == 0) {
-            prefetch_tmap(&tmap_y);
             const uint64_t policy = policy_evict_first();
             for (int it = 0;; ++it) {
                 const int s = it % C::STAGES;
@@ -620,13 +630,24 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), C::TILE, C::B_ROWS);
             const uint64_t b_desc = umma_desc_kmajor_sw128(smem_u32(bsm));
+            int cur_slab = -1;
+            uint32_t operands_seen = 0;
             for (int it = 0;; ++it) {
                 const int s = it % C::STAGES, g = it % C::GROUPS;
                 if (!mbar_wait(&full[s], (it / C::STAGES) & 1)) {
                     report_wait_expired(status);
                     break;
                 }
-                if (meta[s].x < 0) break;
+                const int slab = meta[s].x;
+                if (slab < 0) break;
+                if (slab != cur_slab) {
+                    if (!mbar_wait(b_ready, operands_seen & 1)) {
+                        report_wait_expired(status);
+                        break;
+                    }
+                    ++operands_seen;
+                    cur_slab = slab;
+                }
                 if (!mbar_wait(&a_ready[g], (it / C::GROUPS) & 1)) {
                     report_wait_expired(status);
                     break;
