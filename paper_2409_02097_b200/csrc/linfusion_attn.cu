@@ -457,7 +457,7 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
     mark(h, 1, s);
     e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
                        h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
-                       p.spans, dtype_of(h->desc), operand_scale(h->desc), p.G_apply);
+                       p.spans, dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 2, s);
     e = launch_chained(stream_apply_kernel<KIND>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
@@ -1185,7 +1185,7 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
             mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
         stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->operand, h->tile_counters,
                                                   p.tiles_state, p.W_state, p.G_state, p.spans,
-                                                  dtype_of(h->desc), operand_scale(h->desc), p.G_apply);
+                                                  dtype_of(h->desc), operand_scale(h->desc));
     } else {
         CUtensorMap mq, my;
         if (!encode_slab_map(&mq, a, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
@@ -1196,7 +1196,7 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
         own.p[0] = h->state;
         own.n = 1;
         stream_pack_kernel<<<rgrid, 256, 0, s>>>(peers != nullptr ? *peers : own, h->operand, h->tile_counters,
-                                                dtype_of(h->desc), operand_scale(h->desc), p.G_apply);
+                                                dtype_of(h->desc), operand_scale(h->desc));
         stream_apply_kernel<KIND><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
             mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, apply_scales(h->desc), h->desc.H);
     }

@@ -88,15 +88,6 @@ static_assert(StreamApplyCfg::STAGES >= 2 * StreamApplyCfg::GROUPS + 2, "end mar
 // Shared memory beyond half an SM's keeps a second CTA (and its TMEM allocation) off the SM.
 static_assert(StreamApplyCfg::SMEM_BYTES > 116 * 1024, "one apply CTA per SM");
 
-// Apply kernel: CTA g of G starts on its home slab floor(g * slabs / G).  The CTAs whose home is slab
-// s are g = apply_first_cta(s) .. apply_first_cta(s + 1) - 1; the r-th of them takes tile r of the
-// slab without asking (the slab's tile counter starts at their number), the rest is handed out
-// through the counters.
-__host__ __device__ __forceinline__ int apply_first_cta(int slab, int slabs, int G)
-{
-    return static_cast<int>((static_cast<long long>(slab) * G + slabs - 1) / slabs);
-}
-
 // First unit of CTA g when W units are dealt to G CTAs.
 __host__ __device__ __forceinline__ long long unit_begin(long long g, long long W, long long G)
 {
@@ -200,18 +191,15 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    // Set-up done (barriers, tensor memory): wait for the kernel before this one in the stream to be
-    // complete before touching global memory, and let the next one be scheduled behind this one.
-    // (The tensor maps are kernel parameters: fetching them does not depend on earlier work.)
+    // Set-up done (barriers, tensor memory): let the next kernel in the stream be scheduled behind
+    // this one, and wait for the one before it to be complete before touching global memory.  (The
+    // tensor maps are kernel parameters: fetching them does not depend on earlier work.)
     if (warp == C::PRODUCER_WARP && lane == 0) {
         prefetch_tmap(&tmap_k);
         prefetch_tmap(&tmap_v);
     }
-    // The wait comes first here: the kernels chained behind this one (reduction, apply) may then
-    // rely on everything that precedes this forward in the stream being complete as soon as they
-    // run at all — the apply kernel reads its first Q tile before its own wait.
-    pdl_wait();
     pdl_launch_dependents();
+    pdl_wait();
 
     if (warp == C::PRODUCER_WARP) {
         // ---------------- producer ----------------
@@ -410,8 +398,7 @@ __device__ __forceinline__ void emit_state_operand(const float* sums, unsigned c
 __global__ void __launch_bounds__(256)
 stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
                      unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
-                     int tiles_per_slab, long long W, int G, int spans, int dtype, float operand_scale,
-                     int apply_ctas)
+                     int tiles_per_slab, long long W, int G, int spans, int dtype, float operand_scale)
 {
     __shared__ float sums[256];
     const int tid = threadIdx.x;
@@ -419,8 +406,7 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
     const int slab = blockIdx.y;
     pdl_launch_dependents();
     pdl_wait();
-    if (blockIdx.x == 0 && tid == 0)  // tiles 0 .. (home CTAs - 1) are taken without asking
-        tile_counters[slab] = apply_first_cta(slab + 1, gridDim.y, apply_ctas) - apply_first_cta(slab, gridDim.y, apply_ctas);
+    if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
     float sum = 0.0f;
     if (idx < kStreamStateFloats) {
         const long long lo = static_cast<long long>(slab) * tiles_per_slab, hi = lo + tiles_per_slab;
@@ -451,7 +437,7 @@ stream_reduce_kernel(const float* __restrict__ partials, float* __restrict__ sta
 // here in index order (loads from peers' memory when the list holds peers' buffers).
 __global__ void __launch_bounds__(256)
 stream_pack_kernel(PeerStates states, unsigned char* __restrict__ operand,
-                   int* __restrict__ tile_counters, int dtype, float operand_scale, int apply_ctas)
+                   int* __restrict__ tile_counters, int dtype, float operand_scale)
 {
     __shared__ float sums[256];
     const int tid = threadIdx.x;
@@ -459,8 +445,7 @@ stream_pack_kernel(PeerStates states, unsigned char* __restrict__ operand,
     const int slab = blockIdx.y;
     pdl_launch_dependents();
     pdl_wait();
-    if (blockIdx.x == 0 && tid == 0)  // tiles 0 .. (home CTAs - 1) are taken without asking
-        tile_counters[slab] = apply_first_cta(slab + 1, gridDim.y, apply_ctas) - apply_first_cta(slab, gridDim.y, apply_ctas);
+    if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
     sums[tid] = idx < kStreamStateFloats ? peer_sum(states, static_cast<size_t>(slab) * kStreamStateFloats + idx) : 0.0f;
     __syncthreads();
     emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes, dtype, operand_scale);
@@ -527,21 +512,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     // Set-up done (barriers, tensor memory): let the next kernel in the stream be scheduled behind
     // this one, and wait for the one before it to be complete before touching global memory.  (The
     // tensor maps are kernel parameters: fetching them does not depend on earlier work.)
-    // The CTA's first tile is fixed (tile `rank` of its home slab, see apply_first_cta) and Q is an
-    // input of the forward: when this kernel runs as part of a forward, the state kernel ahead of it
-    // has waited for everything earlier in the stream before letting anything be scheduled behind
-    // it, so Q may be fetched now, while the reduction kernel is still at work.
-    const int home = static_cast<int>((static_cast<long long>(blockIdx.x) * slabs) / gridDim.x);
-    const int rank = static_cast<int>(blockIdx.x) - apply_first_cta(home, slabs, gridDim.x);
-    const bool early_tile = rank < tiles_per_slab;
-    if (warp == C::PRODUCER_WARP && lane == 0) {
-        prefetch_tmap(&tmap_q);
-        if (early_tile) {
-            meta[0] = make_int2(home, rank);
-            mbar_expect_tx(&full[0], C::STAGE_BYTES);
-            tma_load_4d(smem, &tmap_q, 0, rank * C::TILE, home % H, home / H, &full[0], policy_evict_first());
-        }
-    }
+    if (warp == C::PRODUCER_WARP && lane == 0) prefetch_tmap(&tmap_q);
     if (warp == C::STORE_WARP && lane == 0) prefetch_tmap(&tmap_y);
     pdl_launch_dependents();
     pdl_wait();
@@ -550,19 +521,9 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         // ---------------- producer warp (lane 0 issues; all lanes help to find work and copy B) ----------------
         uint64_t policy = 0;
         if (lane == 0) policy = policy_evict_first();
-        int slab = home;
+        int slab = static_cast<int>((static_cast<long long>(blockIdx.x) * slabs) / gridDim.x);
         int it = 0, issued = 0, loaded_slab = -1;
         bool ok = true;
-        if (early_tile) {
-            // stage 0 holds the first tile already; its slab's operand is still to come
-            const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
-            for (int i = lane; i < C::B_BYTES / 16; i += 32) reinterpret_cast<uint4*>(bsm)[i] = __ldg(src + i);
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(b_ready);
-            loaded_slab = slab;
-            it = issued = 1;
-        }
         int next = 0;
         if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
         while (true) {
