@@ -89,8 +89,8 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // Measured on B200 over the SD-v1.5 / v2.1 / XL layer shapes, forwards back to back.  The
         // persistent TMA + tcgen05 kernels (d = 64) pay a few microseconds of set-up (tensor-memory
         // allocation, one CTA per SM working through its tiles in turn) and win once every SM has
-        // about eight 128-token tiles (37 vs 41 us at N = 4096 x 40 slabs, 50 vs 70 us at
-        // N = 16384 x 20; 31 vs 29 us at N = 9216 x 10).  Below that the three chained launches of
+        // about eight 128-token tiles (35 vs 41 us at N = 4096 x 40 slabs, 47 vs 70 us at
+        // N = 16384 x 20; 29 vs 29 us at N = 9216 x 10, 24 vs 22 us at N = 2304 x 10).  Below that the three chained launches of
         // the split path are the fastest at every shape measured, the smallest levels included
         // (12.9 us at N = 144, d = 64, against 14.4 us for the single clustered launch; 21.9 vs 27 us
         // at N = 64, d = 160), so the cluster kernel is only run on request.
