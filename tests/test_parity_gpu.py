@@ -328,3 +328,33 @@ def test_a_wait_that_cannot_complete_gives_up_and_is_reported():
     assert op.status() == attn.OK
     assert torch.equal(y0.view(torch.int16), y1.view(torch.int16))
     op.close()
+
+
+def test_forwards_of_several_handles_replay_from_a_cuda_graph():
+    """A UNet level's handles captured once and replayed: forward() only enqueues kernels on the
+    given stream (no allocation, no synchronization), chained launches included."""
+    shapes = [wl.find_shape("sdxl_2048_L1"), wl.find_shape("sd15_512_L2")]
+    layers = []
+    for i, s in enumerate(shapes):
+        q, k, v = wl.make_qkv(s, seed=60 + i, device="cuda")
+        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=EPS)
+        layers.append((op, q, k, v, op.forward(q, k, v).clone(), torch.empty_like(q)))
+    torch.cuda.synchronize()
+    st = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(st):
+        for op, q, k, v, _, y in layers:                       # warm-up on the capture stream
+            op.forward(q, k, v, y, stream=st.cuda_stream)
+        st.synchronize()
+        with torch.cuda.graph(graph, stream=st):
+            for op, q, k, v, _, y in layers:
+                op.forward(q, k, v, y, stream=st.cuda_stream)
+    for *_, y in layers:
+        y.zero_()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    for op, q, k, v, ref, y in layers:
+        assert torch.equal(y.view(torch.int16), ref.view(torch.int16)), op.variant
+        assert op.status() == attn.OK
+        op.close()
