@@ -393,11 +393,16 @@ def run_sweep(args):
             bufs = []
             for r in range(sets):
                 q, k, v = wl.make_qkv(s, seed=wl.BASE_SEED + r, device="cuda:0")
+                if args.layout == "token_major":
+                    q, k, v = (t.permute(0, 2, 1, 3).contiguous() for t in (q, k, v))
+                if args.dtype == "fp16":
+                    q, k, v = (t.half() for t in (q, k, v))
                 bufs.append((q, k, v, torch.empty_like(q)))
             variants = ["auto", "split"] + (["stream"] if s.d == 64 else []) + \
                        (["cluster"] if s.N <= 16384 else [])
             for variant in variants:
-                op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, device=0, variant=variant)
+                op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, device=0, variant=variant, layout=args.layout,
+                                             dtype=args.dtype)
                 steps = max(20, min(args.steps, int(2e10 // s.min_bytes)))
                 for i in range(5):
                     op.forward(*bufs[i % sets])
@@ -414,6 +419,7 @@ def run_sweep(args):
                 print(json.dumps({
                     "config": cfg_idx + 1, "shape": s.name, "B": s.B, "H": s.H, "N": s.N, "d": s.d,
                     "requested": variant, "variant": op.variant, "launches": op.launches_per_forward,
+                    "layout": args.layout, "dtype": args.dtype,
                     "us_per_forward": us, "tokens_per_s": s.tokens / (us * 1e-6),
                     "effective_gbs": gbs, "frac_of_nominal_8TBps": gbs / NOMINAL_HBM_GBS,
                     "frac_of_measured_copy": gbs / peak, "buffer_sets": sets,
