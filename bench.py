@@ -9,8 +9,16 @@ One step = one forward of each attention level of the 16384x8192 SD-XL workload
 stage of the path (split-N state, fixed-order reduction, apply) over one batch.  Prints ONE JSON
 line: tokens/s over all GPUs with inputs resident in HBM, the same through the host-buffer entry
 point (copies inside the timed region), the roofline of the slowest kernel, and the oracle timed
-on a bounded sample as a CPU baseline.  With N > 1 (torchrun) every rank runs the same per-GPU
-workload on its own seeded batch: independent units, no data-path collective (weak scaling).
+on a bounded sample as a CPU baseline.
+
+With N > 1 there is one rank per GPU (started by torchrun, or by this script itself when it is run
+plainly with --gpus N).  Default there is the token-sharded forward of Sec. 4.3: every rank owns
+the N tokens of the two levels as its run of a sequence of world x N tokens, builds the state of its
+own K/V tokens, the ranks sum their states (one all-reduce of B*H*d*(d+1) fp32 per level, whatever
+N is) and every rank applies the sum to its own Q tokens: per-GPU work is fixed, the exchange is
+the constant-size one the paper points out (weak scaling).  `--parallelism replicas` runs
+independent batches instead (no data-path collective); `--parallelism token_sharded_peers` lets the
+apply step read the peers' states itself over NVLink (symmetric memory, plain loads).
 """
 from __future__ import annotations
 
@@ -80,7 +88,8 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
-    def stop(self, t0: float, t1: float):
+    def stop(self, windows):
+        """`windows`: name -> (t0, t1) in time.time() seconds; returns name -> summary."""
         if self.proc is not None:
             self.proc.terminate()
             try:
@@ -104,10 +113,14 @@ class ClockSampler:
             os.unlink(self.file.name)
         except Exception:
             pass
+        return {name: self._summarize(rows, t0, t1, name) for name, (t0, t1) in windows.items()}
+
+    @staticmethod
+    def _summarize(rows, t0, t1, name):
         if not rows:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
         inside = [r for r in rows if t0 - 0.05 <= r[0] <= t1 + 0.05]
-        window = "timed_region"
+        window = name + "_region"
         if len(inside) < 3:
             # Too short a region for the sampler: use the samples taken under load in this run.
             pmax = max(r[3] for r in rows)
@@ -202,15 +215,43 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def launcher_command(argv, gpus):
+    """The command that starts one rank per GPU on this node for `python bench.py <argv>`."""
+    return [sys.executable, "-m", "torch.distributed.run", "--standalone", "--nnodes=1",
+            f"--nproc-per-node={gpus}", "--local-addr", "127.0.0.1",
+            os.path.join(ROOT, "bench.py")] + list(argv)
+
+
+def maybe_relaunch(args, argv):
+    """`python bench.py --gpus N` with N > 1 outside torchrun: start the N ranks ourselves.
+    Returns True when this process was replaced by (and has waited for) the launcher."""
+    if args.gpus <= 1 or "WORLD_SIZE" in os.environ:
+        return False
+    rc = subprocess.call(launcher_command(argv, args.gpus))
+    if rc != 0:
+        raise SystemExit(rc)
+    return True
+
+
 def run_cuda(args):
     import torch
-    from paper_2409_02097_b200 import attn, build, workloads as wl
+    from paper_2409_02097_b200 import attn, build, sharding, workloads as wl
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the attention has no CPU path")
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if torch.cuda.device_count() < (int(os.environ.get("LOCAL_WORLD_SIZE", world))):
+        raise SystemExit(f"bench.py: --gpus {args.gpus} needs {world} CUDA devices on this node, "
+                         f"{torch.cuda.device_count()} visible")
+    parallelism = args.parallelism
+    if parallelism == "auto":
+        parallelism = "token_sharded" if world > 1 else "single"
+    if parallelism != "single" and (args.layout != "head_major"):
+        raise SystemExit("bench.py: the token-sharded modes time the head-major layout")
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
@@ -236,6 +277,8 @@ def run_cuda(args):
         shapes = [wl.AttnShape(s.name + "_eighth", s.B, s.H, s.N // 8, s.d) for s in shapes]
     eps = 1e-6
     layers = []
+    sharded = parallelism in ("token_sharded", "token_sharded_peers")
+    symm = None
     for i, s in enumerate(shapes):
         q, k, v = wl.make_qkv(s, seed=wl.BASE_SEED + 100 * rank + i, device=f"cuda:{local_rank}")
         if args.layout == "token_major":          # [B, N, H, d]: what a UNet holds before splitting heads
@@ -243,25 +286,51 @@ def run_cuda(args):
         if args.dtype == "fp16":
             q, k, v = (t.half() for t in (q, k, v))
         y = torch.empty_like(q)
-        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank, layout=args.layout,
-                                     dtype=args.dtype)
-        layers.append((s, op, q, k, v, y))
+        if sharded:
+            # This rank's run of a sequence of world * N tokens (its own seeded tokens).
+            sh = sharding.TokenShardedAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank,
+                                                variant="stream", dtype=args.dtype,
+                                                symmetric=(parallelism == "token_sharded_peers"))
+            layers.append((s, sh.op, q, k, v, y, sh))
+        else:
+            op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=eps, device=local_rank, layout=args.layout,
+                                         dtype=args.dtype)
+            layers.append((s, op, q, k, v, y, None))
     tokens_per_step = sum(s.tokens for s in shapes)
-    launches_per_step = sum(op.launches_per_forward for _, op, *_ in layers)
+    launches_per_step = sum((4 if sh is not None else op.launches_per_forward) for _, op, *_, sh in layers)
+
+    # The all-reduce (or the peers' barrier) of every KERNEL_TIMING_STRIDE-th step is bracketed
+    # with events so that the exchange's share of the step can be reported.
+    exchange_events = []
+    step_index = [0]
 
     def step():
-        for _, op, q, k, v, y in layers:
-            op.forward(q, k, v, y)
+        sample = sharded and step_index[0] % KERNEL_TIMING_STRIDE == 0
+        step_index[0] += 1
+        for _, op, q, k, v, y, sh in layers:
+            if sh is None:
+                op.forward(q, k, v, y)
+            else:
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if sample else None
+                if parallelism == "token_sharded":
+                    sh.forward(q, k, v, y, events=ev)
+                else:
+                    sh.forward_symmetric(q, k, v, y, events=ev)
+                if ev is not None:
+                    exchange_events.append((_.name, ev))
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     for _ in range(max(args.warmup, 3)):
         step()
+    exchange_events.clear()
+    step_index[0] = 0
     # Per-kernel durations: CUDA events around each kernel of every KERNEL_TIMING_STRIDE-th step of
     # the timed region (an event record between two kernels undoes their chained launch, so timing
     # every step would slow the steps it measures).
-    for _, op, *_ in layers:
-        op.enable_kernel_timing(min(args.steps, 4096))
-        op.set_kernel_timing_stride(KERNEL_TIMING_STRIDE)
+    if not sharded:
+        for _, op, *_ in layers:
+            op.enable_kernel_timing(min(args.steps, 4096))
+            op.set_kernel_timing_stride(KERNEL_TIMING_STRIDE)
     barrier()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0 = time.time()
@@ -279,14 +348,73 @@ def run_cuda(args):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
         ms = float(t.item())
     value = world * tokens_per_step * args.steps / (ms * 1e-3)
+    exchange = None
+    if sharded:
+        state_bytes = sum(s.B * s.H * s.d * (s.d + 1) * 4 for s in shapes)
+        exchange = {"kind": "nccl all_reduce (sum) of S|z" if parallelism == "token_sharded"
+                            else "peers' S|z read by the apply step (symmetric memory, plain loads)",
+                    "bytes_per_step_per_rank": state_bytes, "independent_of_N": True}
+        if exchange_events:
+            n_sampled = len(exchange_events) // len(shapes)
+            ex_ms = sum(ev[1].elapsed_time(ev[2]) for _, ev in exchange_events) / n_sampled
+            exchange["ms_per_step"] = ex_ms
+            exchange["share_of_step"] = ex_ms / (ms / args.steps)
+            exchange["sampled_steps"] = n_sampled
+
+    kernel_times_taken = {}
+    if not sharded:
+        for s_, op, *_ in layers:
+            kernel_times_taken[s_.name] = op.kernel_times()
+    # A second, longer region of back-to-back steps: the board reaches its power limit within a
+    # few hundred milliseconds and the SM clock settles below its maximum, so the burst above and
+    # the steady state differ.  Timed the same way; its clock samples come from inside its window.
+    sustained = None
+    if args.sustained_seconds > 0:
+        n_sus = max(args.steps, int(args.sustained_seconds / max(ms / args.steps * 1e-3, 1e-6)) + 1)
+        if not sharded:
+            for _, op, *_ in layers:
+                op.enable_kernel_timing(0)          # undisturbed chained launches
+        barrier()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ts0 = time.time()
+        s0.record()
+        for _ in range(n_sus):
+            step()
+        s1.record()
+        barrier()
+        ts1 = time.time()
+        ms_sus = s0.elapsed_time(s1)
+        if dist is not None:
+            t = torch.tensor([ms_sus], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms_sus = float(t.item())
+        step_bytes_ = sum(s.min_bytes for s in shapes)
+        sustained = {"steps": n_sus, "ms_per_step": ms_sus / n_sus, "seconds": ms_sus * 1e-3,
+                     "value": world * tokens_per_step * n_sus / (ms_sus * 1e-3), "unit": UNIT,
+                     "hbm_gbs_whole_path": step_bytes_ * n_sus / (ms_sus * 1e-3) / 1e9,
+                     "hbm_frac_of_nominal_8TBps": step_bytes_ * n_sus / (ms_sus * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                     "window": (ts0, ts1)}
 
     # Per-kernel durations recorded inside the timed region.
     peak, peak_kind = measured_peak_gbs()
     kernels = []
     names = ["stream_state_kernel", "stream_reduce_kernel", "stream_apply_kernel"]
+    if sharded:
+        # The two halves, each bracketed as a whole on the sampled steps (state kernel + reduction;
+        # operand packing + apply kernel).
+        for s in shapes:
+            evs = [ev for name, ev in exchange_events if name == s.name]
+            for label, i in (("stream_state_kernel+stream_reduce_kernel", 0), ("stream_pack_kernel+stream_apply_kernel", 2)):
+                if not evs:
+                    continue
+                avg_ms = sum(ev[i].elapsed_time(ev[i + 1]) for ev in evs) / len(evs)
+                algo = 2 * s.B * s.N * s.C * 2
+                kernels.append({"kernel": label, "shape": s.name, "avg_ms": avg_ms, "algorithmic_bytes": algo,
+                                "gbs": algo / (avg_ms * 1e-3) / 1e9})
     for s, op, *_ in layers:
-        sums, calls = op.kernel_times()
-        op.enable_kernel_timing(0)
+        if sharded or kernel_times_taken.get(s.name) is None:
+            continue
+        sums, calls = kernel_times_taken[s.name]
         for name, total in zip(names, sums):
             if calls == 0:
                 continue
@@ -308,9 +436,9 @@ def run_cuda(args):
 
     # End to end through the host-buffer entry point: H2D of Q, K, V and D2H of Y every step.
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not sharded:
         host = []
-        for s, op, q, k, v, y in layers:
+        for s, op, q, k, v, y, _ in layers:
             hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
             hy = torch.empty_like(hq).pin_memory()
             host.append((op, hq, hk, hv, hy))
@@ -339,7 +467,23 @@ def run_cuda(args):
                "ms_per_step": ms_e2e / k_e2e}
         del host
 
-    clocks = sampler.stop(t0, t1) if sampler is not None else None
+    clocks = None
+    if sampler is not None:
+        # The timed region is often shorter than the sampler's period; the sustained region follows
+        # it directly, so the two together are the window the clock record describes.
+        windows = {"timed": (t0, t1)}
+        if sustained is not None:
+            windows["sustained"] = sustained["window"]
+            windows["timed"] = (t0, sustained["window"][1])
+        rec = sampler.stop(windows)
+        clocks = rec["timed"]
+        if sustained is not None:
+            sc = rec["sustained"]
+            sustained.update({"sm_mhz_median": sc["sm_mhz"], "sm_max_mhz": sc["sm_max_mhz"], "reasons": sc["reasons"],
+                              "clock_samples": sc["samples"], "power_w_max": sc.get("power_w_max"),
+                              "ms_per_step_x_sm_mhz": (sustained["ms_per_step"] * sc["sm_mhz"]) if sc["sm_mhz"] else None})
+    if sustained is not None:
+        sustained.pop("window", None)
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -357,11 +501,18 @@ def run_cuda(args):
                        "variant": [op.variant for _, op, *_ in layers],
                        "l2": "inputs larger than L2 (%.2f GB touched per step)" % (step_bytes / 1e9),
                        "layout": args.layout,
-                       "parallelism": f"independent batches x{world}"},
+                       "parallelism": {"single": "one GPU",
+                                       "replicas": f"independent batches x{world} (no data-path collective)",
+                                       "token_sharded": f"token-sharded x{world}: each rank owns N tokens of a "
+                                                        f"{world}xN-token sequence; one all-reduce of S|z per level",
+                                       "token_sharded_peers": f"token-sharded x{world}: the apply step sums the "
+                                                              f"peers' S|z itself over NVLink"}[parallelism],
+                       "exchange": exchange},
             "tokens_per_s_per_gpu": value / world,
             "hbm_gbs_whole_path": path_gbs,
             "hbm_frac_of_nominal_8TBps": path_gbs / NOMINAL_HBM_GBS,
             "hbm_frac_of_measured_copy": path_gbs / peak,
+            "sustained": sustained,
             "roofline": roofline, "kernels": kernels,
             "kernel_timing": f"CUDA events around each kernel of every {KERNEL_TIMING_STRIDE}th step of the timed region",
             "cpu_baseline": cpu_baseline, "e2e": e2e,
@@ -432,7 +583,7 @@ def run_sweep(args):
             torch.cuda.empty_cache()
 
 
-def main():
+def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=300)
@@ -440,6 +591,11 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "sdxl_16k_eighth"])
     ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--sustained-seconds", type=float, default=2.5,
+                    help="length of the second, back-to-back region timed after the --steps region (0: none)")
+    ap.add_argument("--parallelism", default="auto",
+                    choices=["auto", "single", "replicas", "token_sharded", "token_sharded_peers"],
+                    help="auto: token_sharded when --gpus > 1")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layout", default="head_major", choices=["head_major", "token_major"],
@@ -449,9 +605,12 @@ def main():
     ap.add_argument("--sweep", action="store_true",
                     help="time every shape of the five workload families with every variant")
     ap.add_argument("--only", default="", help="with --sweep: restrict to one shape, e.g. sd15_512_L1")
-    args = ap.parse_args()
+    argv = sys.argv[1:] if argv is None else argv
+    args = ap.parse_args(argv)
     if args.sweep:
         run_sweep(args)
+    elif maybe_relaunch(args, argv):
+        return
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -87,7 +87,7 @@ typedef enum {
 
 typedef struct {
     int32_t B;      /* batch                                   > 0 */
-    int32_t H;      /* heads                                   > 0 */
+    int32_t H;      /* heads                                   > 0; B*H <= 65535 (one grid row per slab) */
     int32_t N;      /* tokens per slab                         > 0 */
     int32_t d;      /* head dim: one of 32, 40, 64, 80, 128, 160   */
     int32_t phi;    /* linfusion_phi_t                             */
@@ -101,7 +101,9 @@ typedef struct {
  * Validates the descriptor, checks that `device` is compute capability 10.x, fixes the
  * split of N and allocates the workspace (cudaMalloc) on that device.
  * Errors: INVALID_ARG (null pointers, sizes <= 0, eps negative or not finite),
- * UNSUPPORTED (d, phi, variant, device architecture), ALLOC, CUDA.  *out is NULL on error.
+ * UNSUPPORTED (d, phi, variant, unknown flag bits, B*H > 65535, device architecture), ALLOC, CUDA.
+ * *out is NULL on error.  create() and set_workspace() return only when the workspace has been
+ * cleared, so a forward() may follow at once on any stream.
  */
 linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linfusion_attn_t** out);
 
@@ -219,6 +221,9 @@ linfusion_status_t linfusion_attn_apply(linfusion_attn_t* h, const void* q, void
  * Synchronization is the caller's: every rank's linfusion_attn_state() must have completed, and
  * no rank may start its next linfusion_attn_state() on these handles before all ranks' apply_peers
  * kernels have read its buffer (e.g. a stream-ordered barrier on either side).
+ * With fp16 storage the operand scale 2^-ceil(log2 N) is derived from the LOCAL token count, while
+ * the summed z is about 1.2 * N_local * n_peers: the scaled z stays below 1.2 * n_peers (well
+ * inside fp16's 65504 for any n_peers <= LINFUSION_MAX_PEERS), S keeps its relative size.
  * Errors: INVALID_ARG (null / misaligned pointers, n_peers out of range), UNSUPPORTED (cluster
  * handle), CUDA.
  */
@@ -260,17 +265,24 @@ linfusion_status_t linfusion_attn_set_kernel_timing_stride(linfusion_attn_t* h, 
  * three-launch split path (split-N state, fixed-order reduction, apply; any supported head dim)
  * and keeps the partial states and the reduced state in a fixed 16 MiB array that is part of the
  * library's device image: every GPU that loads the library holds those 16 MiB until the process
- * exits, whether or not this function is ever called.  It calls no cudaMalloc, cudaFree or other
- * allocating routine, creates no streams or events, and keeps no per-call host state.
+ * exits.  (With CUDA's default lazy module loading the driver commits the library's device image,
+ * these 16 MiB included, when the library is first used on a device — the first call of this
+ * function, if nothing else came before; with CUDA_MODULE_LOADING=EAGER, when the library is
+ * loaded.  A host that gives all remaining device memory to its arena must make that first call,
+ * or load eagerly, before it does so.)  It calls no cudaMalloc, cudaFree or other allocating
+ * routine, creates no streams or events, and keeps no per-call host state.
  *
  * desc: as for create(); flags must be AUTO or SPLIT.  q, k, v, y, cuda_stream: as for forward().
  * The split of N uses as many chunks as fit in the array; a problem whose state alone does not
  * fit — 2 * B*H * d*(d+1) * 4 bytes + 512 above 16 MiB, e.g. d = 160 with more than 81 slabs — is
  * rejected with LINFUSION_ERR_ALLOC and nothing is launched.  Other errors: INVALID_ARG,
- * UNSUPPORTED, CUDA, as for create() and forward().
+ * UNSUPPORTED (as for create(), B*H > 65535 included), CUDA, as for create() and forward().
  *
- * The first call on each device looks up the array's device address and raises the kernels'
- * shared-memory limits; make that first call before starting any stream capture.
+ * The first call on each device looks up the array's device address, and the first call for each
+ * (device, head dim, phi, storage type) raises the two kernels' shared-memory limits; later calls
+ * make no CUDA call besides the three launches.  Make those first calls before starting any
+ * stream capture.  First calls from several host threads at once are safe (the set-up is
+ * serialized); the array's contents are what concurrent calls race on, see below.
  * Every call on a device shares the one array, which keeps whatever the last call left in it.
  * Nothing in it needs clearing between calls (each call writes every element before reading it),
  * but two calls whose kernels overlap on the GPU — different streams, or several host threads —
@@ -280,6 +292,18 @@ linfusion_status_t linfusion_attn_set_kernel_timing_stride(linfusion_attn_t* h, 
 linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_attn_desc_t* desc, const void* q,
                                                   const void* k, const void* v, void* y,
                                                   void* cuda_stream);
+
+/*
+ * Where forward_noalloc() would put a problem in its fixed array, without touching a device (the
+ * paper has no counterpart): *chunks = partial states per slab that the split of N uses on a GPU
+ * with `sm_count` SMs (<= 0: 148), cut down to what leaves room for the state; *state_offset = byte
+ * offset of the reduced state (the partials start at 0); *bytes_used = end of the state;
+ * *capacity = size of the array.  Any output pointer may be NULL.  bytes_used <= capacity whenever
+ * OK is returned.  Errors: INVALID_ARG, UNSUPPORTED, ALLOC (does not fit), as forward_noalloc().
+ */
+linfusion_status_t linfusion_attn_noalloc_layout(const linfusion_attn_desc_t* desc, int sm_count,
+                                                 int32_t* chunks, size_t* state_offset,
+                                                 size_t* bytes_used, size_t* capacity);
 
 /* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);

@@ -26,7 +26,7 @@ EXPORTED = [
     "linfusion_attn_variant_name", "linfusion_attn_launches_per_forward",
     "linfusion_attn_enable_kernel_timing", "linfusion_attn_kernel_times",
     "linfusion_attn_set_kernel_timing_stride",
-    "linfusion_attn_forward_noalloc",
+    "linfusion_attn_forward_noalloc", "linfusion_attn_noalloc_layout",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
     "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait",
 ]
@@ -91,6 +91,10 @@ def load_library() -> ctypes.CDLL:
                                                 ctypes.POINTER(ctypes.c_int32)]
     lib.linfusion_attn_forward_noalloc.restype = st
     lib.linfusion_attn_forward_noalloc.argtypes = [ctypes.POINTER(Desc), vp, vp, vp, vp, vp]
+    lib.linfusion_attn_noalloc_layout.restype = st
+    lib.linfusion_attn_noalloc_layout.argtypes = [ctypes.POINTER(Desc), ctypes.c_int,
+                                                  ctypes.POINTER(ctypes.c_int32)] + \
+                                                 [ctypes.POINTER(ctypes.c_size_t)] * 3
     lib.linfusion_attn_state.restype = st
     lib.linfusion_attn_state.argtypes = [vp, vp, vp, vp]
     lib.linfusion_attn_apply.restype = st
@@ -171,6 +175,18 @@ def linfusion_attn_forward_noalloc(desc: Desc, q_ptr: int, k_ptr: int, v_ptr: in
                                                        y_ptr, stream_ptr)
     if rc != OK:
         raise LinFusionError(rc, "linfusion_attn_forward_noalloc")
+
+
+def linfusion_attn_noalloc_layout(desc: Desc, sm_count: int = 0):
+    """(chunks, state_offset, bytes_used, capacity) of a problem in the allocation-free entry
+    point's fixed array; raises ``LinFusionError`` (``ERR_ALLOC``) when it does not fit."""
+    chunks = ctypes.c_int32(0)
+    off, used, cap = ctypes.c_size_t(0), ctypes.c_size_t(0), ctypes.c_size_t(0)
+    rc = load_library().linfusion_attn_noalloc_layout(ctypes.byref(desc), int(sm_count), ctypes.byref(chunks),
+                                                      ctypes.byref(off), ctypes.byref(used), ctypes.byref(cap))
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_noalloc_layout")
+    return int(chunks.value), int(off.value), int(used.value), int(cap.value)
 
 
 def linfusion_attn_destroy(handle) -> None:

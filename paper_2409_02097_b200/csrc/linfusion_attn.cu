@@ -2,9 +2,11 @@
 // fixed split of N, workspace layout, tensor-map encoding and kernel launches.
 #include "../../include/linfusion_attn.h"
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "split_kernels.cuh"
@@ -306,6 +308,20 @@ void bind_workspace(linfusion_attn* h, void* ws)
     h->operand = base + h->plan.operand_off;
     h->tile_counters = reinterpret_cast<int*>(base + h->plan.counters_off);
     h->status = reinterpret_cast<uint32_t*>(base + h->plan.status_off);
+}
+
+// Zero the operand image, the tile counters and the status word, and return only when that is done:
+// a forward enqueued right afterwards on any stream (non-blocking side streams included, which the
+// legacy default stream does not order against) must find them cleared and must not be overtaken
+// by the clear.
+bool clear_workspace_tail(linfusion_attn* h)
+{
+    if (cudaMemsetAsync(h->operand, 0, h->plan.total_bytes - h->plan.operand_off, nullptr) != cudaSuccess ||
+        cudaStreamSynchronize(nullptr) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return true;
 }
 
 struct DeviceGuard {
@@ -638,7 +654,7 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     }
     h->owns_ws = true;
     bind_workspace(h, ws);
-    if (cudaMemset(h->operand, 0, h->plan.total_bytes - h->plan.operand_off) != cudaSuccess) {
+    if (!clear_workspace_tail(h)) {
         cudaFree(ws);
         delete h;
         return LINFUSION_ERR_CUDA;
@@ -658,7 +674,7 @@ linfusion_status_t linfusion_attn_set_workspace(linfusion_attn_t* h, void* dev_p
     if (h->owns_ws && h->ws != nullptr) cudaFree(h->ws);
     h->owns_ws = false;
     bind_workspace(h, dev_ptr);
-    if (cudaMemset(h->operand, 0, h->plan.total_bytes - h->plan.operand_off) != cudaSuccess) return LINFUSION_ERR_CUDA;
+    if (!clear_workspace_tail(h)) return LINFUSION_ERR_CUDA;
     return LINFUSION_OK;
 }
 
@@ -1013,19 +1029,61 @@ constexpr int kNoAllocMaxDevices = 64;
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
 
 struct NoAllocDevice {
-    bool ready = false;
+    std::atomic<bool> ready{false};
     unsigned char* scratch = nullptr;  // device address of g_noalloc_scratch on this device
     int sm_count = 0;
+    std::atomic<uint32_t> configured{0};  // bit (d index * 4 + kind): shared-memory limits raised
 };
 NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
+std::mutex g_noalloc_mutex;  // serializes the set-up below (first calls from several host threads)
 
-// Once per device, with that device current: resolve the array's device address (the symbol's
-// name is only a host-side stand-in and must never be handed to a kernel), read the SM count
-// and raise the kernels' dynamic shared-memory limits.
+int d_index(int d)
+{
+    switch (d) {
+        case 32: return 0;
+        case 40: return 1;
+        case 64: return 2;
+        case 80: return 3;
+        case 128: return 4;
+        case 160: return 5;
+        default: return -1;
+    }
+}
+
+// The two kernels this entry point launches per (head dim, kind); the cluster kernel is not among them.
+template <int D>
+cudaError_t set_noalloc_attrs_d(int kind)
+{
+    using C = SplitCfg<D>;
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV)                                                                                                    \
+    e = cudaFuncSetAttribute(state_partial_kernel<D, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV); \
+    if (e == cudaSuccess)                                                                                           \
+    e = cudaFuncSetAttribute(apply_kernel<D, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY)
+    LF_DISPATCH_KIND(kind, LF_K)
+#undef LF_K
+    return e;
+}
+
+// With `device` current.  Once per device: resolve the array's device address (the symbol's name
+// is only a host-side stand-in and must never be handed to a kernel) and read the SM count.  Once
+// per (device, head dim, kind): raise the two kernels' dynamic shared-memory limits.  Later calls
+// find both done and make no CUDA call here.  Safe for first calls made by several host threads
+// at once: the set-up runs under a mutex and is published with release / acquire.
 linfusion_status_t noalloc_setup(int device, int d, int kind)
 {
     NoAllocDevice& dev = g_noalloc_dev[device];
-    if (!dev.ready) {
+    const uint32_t bit = 1u << (d_index(d) * 4 + kind);
+    if (dev.ready.load(std::memory_order_acquire) && (dev.configured.load(std::memory_order_acquire) & bit) != 0u)
+        return LINFUSION_OK;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!dev.ready.load(std::memory_order_relaxed)) {
+        int ndev = 0;
+        if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+        if (device >= ndev) return LINFUSION_ERR_INVALID_ARG;
         cudaDeviceProp prop;
         if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) {
             cudaGetLastError();
@@ -1039,34 +1097,76 @@ linfusion_status_t noalloc_setup(int device, int d, int kind)
         }
         dev.scratch = static_cast<unsigned char*>(ptr);
         dev.sm_count = prop.multiProcessorCount;
-        dev.ready = true;
+        dev.ready.store(true, std::memory_order_release);
     }
-    cudaError_t e = cudaSuccess;
-#define LF_SET(DV) e = set_attrs_d<DV>(kind)
-    LF_DISPATCH_D(d, LF_SET)
+    if ((dev.configured.load(std::memory_order_relaxed) & bit) == 0u) {
+        cudaError_t e = cudaErrorInvalidValue;
+#define LF_SET(DV) e = set_noalloc_attrs_d<DV>(kind)
+        LF_DISPATCH_D(d, LF_SET)
 #undef LF_SET
-    if (e != cudaSuccess) {
-        cudaGetLastError();
-        return LINFUSION_ERR_CUDA;
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+        dev.configured.fetch_or(bit, std::memory_order_release);
     }
     return LINFUSION_OK;
 }
 
+// Where a problem's partial states and reduced state sit in the fixed array: `chunks` partials of
+// per_chunk bytes from offset 0, the state at the next 256-byte boundary.  The split of N is the
+// split path's plan for `sm_count` SMs, cut down to as many chunks as leave room for the state.
+// ALLOC when not even one chunk and the state fit.  Pure host arithmetic.
+linfusion_status_t noalloc_layout(const linfusion_attn_desc_t* desc, int sm_count, Plan* plan, size_t* state_off,
+                                  size_t* bytes_used)
+{
+    linfusion_status_t st = validate(desc);
+    if (st != LINFUSION_OK) return st;
+    if ((desc->flags & LINFUSION_VARIANT_MASK) > LINFUSION_VARIANT_SPLIT) return LINFUSION_ERR_UNSUPPORTED;
+    const size_t per_chunk = static_cast<size_t>(desc->B) * desc->H * desc->d * (desc->d + 1) * 4;
+    const size_t state_bytes = align_up(per_chunk, 256);
+    if (state_bytes + per_chunk + 256 > kNoAllocScratchBytes) return LINFUSION_ERR_ALLOC;
+    linfusion_attn_desc_t d = *desc;
+    d.flags = (desc->flags & (LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED | LINFUSION_DTYPE_FP16)) |
+              LINFUSION_VARIANT_SPLIT;
+    st = make_plan(&d, sm_count, plan);
+    if (st != LINFUSION_OK) return st;
+    const size_t room = (kNoAllocScratchBytes - state_bytes - 256) / per_chunk;
+    if (static_cast<size_t>(plan->chunks_state) > room) plan->chunks_state = static_cast<int>(room);
+    *state_off = align_up(per_chunk * static_cast<size_t>(plan->chunks_state), 256);
+    *bytes_used = *state_off + per_chunk;
+    return LINFUSION_OK;
+}
+
 }  // namespace
+
+extern "C" linfusion_status_t linfusion_attn_noalloc_layout(const linfusion_attn_desc_t* desc, int sm_count,
+                                                            int32_t* chunks, size_t* state_offset,
+                                                            size_t* bytes_used, size_t* capacity)
+{
+    Plan plan;
+    size_t off = 0, used = 0;
+    linfusion_status_t st = noalloc_layout(desc, sm_count, &plan, &off, &used);
+    if (capacity != nullptr) *capacity = kNoAllocScratchBytes;
+    if (st != LINFUSION_OK) return st;
+    if (chunks != nullptr) *chunks = plan.chunks_state;
+    if (state_offset != nullptr) *state_offset = off;
+    if (bytes_used != nullptr) *bytes_used = used;
+    return LINFUSION_OK;
+}
 
 extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_attn_desc_t* desc,
                                                              const void* q, const void* k,
                                                              const void* v, void* y,
                                                              void* cuda_stream)
 {
-    linfusion_status_t st = validate(desc);
+    // Descriptor and capacity first: they depend on the descriptor alone (the chunk count is
+    // settled below, once the device's SM count is known).
+    linfusion_attn view;
+    size_t state_off = 0, bytes_used = 0;
+    linfusion_status_t st = noalloc_layout(desc, 0, &view.plan, &state_off, &bytes_used);
     if (st != LINFUSION_OK) return st;
     if (desc->device >= kNoAllocMaxDevices) return LINFUSION_ERR_INVALID_ARG;
-    if ((desc->flags & LINFUSION_VARIANT_MASK) > LINFUSION_VARIANT_SPLIT) return LINFUSION_ERR_UNSUPPORTED;
-    // Capacity first: it depends on the descriptor alone.
-    const size_t per_chunk = static_cast<size_t>(desc->B) * desc->H * desc->d * (desc->d + 1) * 4;
-    const size_t state_bytes = align_up(per_chunk, 256);
-    if (state_bytes + per_chunk + 256 > kNoAllocScratchBytes) return LINFUSION_ERR_ALLOC;
     if (q == nullptr || k == nullptr || v == nullptr || y == nullptr) return LINFUSION_ERR_INVALID_ARG;
     const uintptr_t pq = reinterpret_cast<uintptr_t>(q), pk = reinterpret_cast<uintptr_t>(k),
                     pv = reinterpret_cast<uintptr_t>(v), py = reinterpret_cast<uintptr_t>(y);
@@ -1075,14 +1175,14 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     auto overlaps = [&](uintptr_t a) { return a < py + bytes && py < a + bytes; };
     if (overlaps(pq) || overlaps(pk) || overlaps(pv)) return LINFUSION_ERR_INVALID_ARG;
 
-    int ndev = 0;
-    if (cudaGetDeviceCount(&ndev) != cudaSuccess) {
-        cudaGetLastError();
-        return LINFUSION_ERR_CUDA;
-    }
-    if (desc->device >= ndev) return LINFUSION_ERR_INVALID_ARG;
+    // (A device ordinal the process does not have fails in cudaSetDevice here, or in the first
+    // call's set-up, which asks for the device count.)
     DeviceGuard guard(desc->device);
-    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    if (!guard.ok) {
+        cudaGetLastError();
+        return g_noalloc_dev[desc->device].ready.load(std::memory_order_acquire) ? LINFUSION_ERR_CUDA
+                                                                                 : LINFUSION_ERR_INVALID_ARG;
+    }
     st = noalloc_setup(desc->device, desc->d, kind_of(*desc));
     if (st != LINFUSION_OK) return st;
     const NoAllocDevice& dev = g_noalloc_dev[desc->device];
@@ -1090,20 +1190,17 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     // A handle-shaped view on the stack: the three-launch split plan, with as many chunks of N
     // as the fixed array has room for.  Nothing in the array has to start at zero: every partial
     // and every state element that is read in this call is written earlier in the same call.
-    linfusion_attn view;
     view.desc = *desc;
     view.desc.flags = (desc->flags & (LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED | LINFUSION_DTYPE_FP16)) |
                       LINFUSION_VARIANT_SPLIT;
-    st = make_plan(&view.desc, dev.sm_count, &view.plan);
+    st = noalloc_layout(desc, dev.sm_count, &view.plan, &state_off, &bytes_used);
     if (st != LINFUSION_OK) return st;
-    const size_t room = (kNoAllocScratchBytes - state_bytes - 256) / per_chunk;
-    if (static_cast<size_t>(view.plan.chunks_state) > room) view.plan.chunks_state = static_cast<int>(room);
+    if (bytes_used > kNoAllocScratchBytes) return LINFUSION_ERR_ALLOC;  // cannot happen; the array is never overrun
     view.sm_count = dev.sm_count;
     view.ws = dev.scratch;
     view.owns_ws = false;
     view.partials = reinterpret_cast<float*>(dev.scratch);
-    view.state = reinterpret_cast<float*>(
-        dev.scratch + align_up(per_chunk * static_cast<size_t>(view.plan.chunks_state), 256));
+    view.state = reinterpret_cast<float*>(dev.scratch + state_off);
     view.operand = nullptr;
     view.tile_counters = nullptr;
     view.status = nullptr;

@@ -125,3 +125,37 @@ def test_binding_has_no_fallback(monkeypatch):
     monkeypatch.setattr(attn, "LIB_PATH", os.path.join(ROOT, "does_not_exist.so"))
     with pytest.raises(ImportError):
         attn.load_library()
+
+
+def test_noalloc_layout_never_leaves_the_array():
+    """Host arithmetic of the allocation-free entry point: over a sweep of descriptors and SM
+    counts the partial states and the reduced state stay inside the fixed array, the state starts
+    on a 256-byte boundary behind the last partial, and what cannot fit is refused."""
+    fits = refused = clamped = 0
+    for d in (32, 40, 64, 80, 128, 160):
+        for slabs in (1, 2, 7, 16, 40, 64, 81, 82, 200, 1000, 4000, 65535):
+            for N in (1, 63, 64, 65, 4096, 524288):
+                for sm in (0, 1, 74, 148, 400):
+                    desc = attn.make_desc(1, slabs, N, d)
+                    per_chunk = slabs * d * (d + 1) * 4
+                    try:
+                        chunks, off, used, cap = attn.linfusion_attn_noalloc_layout(desc, sm)
+                    except attn.LinFusionError as e:
+                        assert e.code == attn.ERR_ALLOC
+                        assert 2 * per_chunk + 256 > (16 << 20) - 256, (d, slabs)
+                        refused += 1
+                        continue
+                    fits += 1
+                    assert cap == 16 << 20
+                    assert 1 <= chunks <= max(1, -(-N // 64))
+                    assert off % 256 == 0 and off >= chunks * per_chunk
+                    assert used == off + per_chunk and used <= cap
+                    planned = min(max(1, -(-2 * (sm or 148) // slabs)), -(-N // 64))
+                    clamped += chunks < planned
+    assert fits > 500 and refused > 50 and clamped > 20
+    with pytest.raises(attn.LinFusionError) as e:
+        attn.linfusion_attn_noalloc_layout(attn.make_desc(1, 4, 64, 64, variant="cluster"))
+    assert e.value.code == attn.ERR_UNSUPPORTED
+    with pytest.raises(attn.LinFusionError) as e:
+        attn.linfusion_attn_noalloc_layout(attn.make_desc(1, 70000, 64, 64))
+    assert e.value.code == attn.ERR_UNSUPPORTED
