@@ -227,6 +227,11 @@ def maybe_relaunch(args, argv):
     Returns True when this process was replaced by (and has waited for) the launcher."""
     if args.gpus <= 1 or "WORLD_SIZE" in os.environ:
         return False
+    if args.impl == "cuda":
+        import torch
+        if torch.cuda.device_count() < args.gpus:
+            raise SystemExit(f"bench.py: --gpus {args.gpus} needs {args.gpus} CUDA devices on this node, "
+                             f"{torch.cuda.device_count()} visible")
     rc = subprocess.call(launcher_command(argv, args.gpus))
     if rc != 0:
         raise SystemExit(rc)
@@ -240,10 +245,10 @@ def run_cuda(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the attention has no CPU path")
     if world != args.gpus:
         raise SystemExit(f"bench.py: --gpus {args.gpus} but the launcher started {world} rank(s)")
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention has no CPU path")
     if torch.cuda.device_count() < (int(os.environ.get("LOCAL_WORLD_SIZE", world))):
         raise SystemExit(f"bench.py: --gpus {args.gpus} needs {world} CUDA devices on this node, "
                          f"{torch.cuda.device_count()} visible")
@@ -275,6 +280,10 @@ def run_cuda(args):
         # Same layers at one eighth of the tokens: small enough for a multi-pass profiler capture,
         # still several times the L2 capacity.  Not a benchmark workload.
         shapes = [wl.AttnShape(s.name + "_eighth", s.B, s.H, s.N // 8, s.d) for s in shapes]
+    elif args.workload == "sdxl_16k_L2":
+        # The smaller of the two levels alone, full size (2.7 GB on the device): for profiler
+        # captures of DRAM counters over whole launches.  Not a benchmark workload.
+        shapes = shapes[1:]
     eps = 1e-6
     layers = []
     sharded = parallelism in ("token_sharded", "token_sharded_peers")
@@ -589,7 +598,7 @@ def main(argv=None):
     ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
-    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "sdxl_16k_eighth"])
+    ap.add_argument("--workload", default=WORKLOAD, choices=[WORKLOAD, "sdxl_16k_eighth", "sdxl_16k_L2"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--sustained-seconds", type=float, default=2.5,
                     help="length of the second, back-to-back region timed after the --steps region (0: none)")

@@ -70,7 +70,8 @@ class TokenShardedAttention:
             import torch.distributed as dist
             import torch.distributed._symmetric_memory as symm_mem
             self._ws = symm_mem.empty(nbytes + 256, dtype=torch.uint8, device=dev)
-            self._symm = symm_mem.rendezvous(self._ws, dist.group.WORLD if group is None else group)
+            pg = group if group is not None else dist.distributed_c10d._get_default_group()
+            self._symm = symm_mem.rendezvous(self._ws, pg.group_name)
         else:
             self._ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
         off = (-self._ws.data_ptr()) % 256
