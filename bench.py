@@ -558,7 +558,7 @@ def run_sweep(args):
                 if args.dtype == "fp16":
                     q, k, v = (t.half() for t in (q, k, v))
                 bufs.append((q, k, v, torch.empty_like(q)))
-            variants = ["auto", "split"] + (["stream"] if s.d == 64 else []) + \
+            variants = ["auto", "split"] + (["stream", "fused"] if s.d == 64 else []) + \
                        (["cluster"] if s.N <= 16384 else [])
             for variant in variants:
                 op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, device=0, variant=variant, layout=args.layout,

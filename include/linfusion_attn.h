@@ -55,6 +55,7 @@ typedef enum {
 #define LINFUSION_VARIANT_SPLIT 1u   /* three launches: split-N state, reduction, apply (any supported d) */
 #define LINFUSION_VARIANT_STREAM 2u  /* three launches, TMA-pipelined persistent kernels (d = 64 only)    */
 #define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N)               */
+#define LINFUSION_VARIANT_FUSED 4u   /* one launch, persistent TMA + tcgen05 kernel with per-slab counters (d = 64) */
 #define LINFUSION_VARIANT_MASK 0xFu
 /*
  * flags: memory layout of Q, K, V and Y.  Default (bit clear): head-major [B, H, N, d].  Bit set:
@@ -112,7 +113,7 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
  * NULL is the legacy default stream).  q, k, v: const bf16 (or fp16) [B,H,N,d] device memory;
  * y: the same type, [B,H,N,d] device memory, written in full, rounded to nearest even from fp32.
  * Steps: split-N state reduction (S_p, z_p per chunk p of the tokens; Prop. 2 and Eq. 5),
- * fixed-order reduction to (S, z), apply — or all three in one clustered launch for small N.
+ * fixed-order reduction to (S, z), apply — or all three in one launch (CLUSTER, FUSED).
  * Errors: INVALID_ARG (null handle or pointer, pointer not 16-byte aligned, y overlapping an
  * input), CUDA (launch or tensor-map encoding failed).  A bounded device-side wait that
  * expired is reported by status(), not here.
@@ -174,6 +175,14 @@ linfusion_status_t linfusion_attn_status(linfusion_attn_t* h);
  * receives the kernel's duration.
  */
 linfusion_status_t linfusion_attn_selftest_wait(linfusion_attn_t* h, float* waited_ms);
+/*
+ * The same self-test for the other kind of bounded wait: the single-launch variant
+ * (LINFUSION_VARIANT_FUSED) lets the CTAs that apply a slab wait, by polling a counter in global
+ * memory, until every CTA that contributes a partial state of that slab (Prop. 2's sum over tokens,
+ * split over CTAs) has delivered it.  This runs one warp that polls a counter nothing advances.
+ * Results as for selftest_wait().
+ */
+linfusion_status_t linfusion_attn_selftest_counter_wait(linfusion_attn_t* h, float* waited_ms);
 
 /*
  * Copy the reduced state of the last forward to HOST buffers (fp32): S [B*H][d][d] (row =
@@ -198,9 +207,10 @@ linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host,
  *
  * state_buffer: *dev_ptr is the device address of [B*H][d*d S (row = feature c of K, column =
  * channel e of V), then d z] fp32, *floats its length; it stays valid until the handle is
- * destroyed or its workspace is replaced.  Handles that resolved to the clustered single-launch
- * variant cannot be split in two: state() and apply() return UNSUPPORTED for them (create the
- * handle with LINFUSION_VARIANT_SPLIT or _STREAM).  Other errors as for forward().
+ * destroyed or its workspace is replaced.  Handles that resolved to a single-launch variant
+ * (CLUSTER, FUSED; AUTO picks FUSED for many small slabs of head dim 64) cannot be split in two:
+ * state() and apply() return UNSUPPORTED for them (create the handle with LINFUSION_VARIANT_SPLIT
+ * or _STREAM).  Other errors as for forward().
  */
 linfusion_status_t linfusion_attn_state(linfusion_attn_t* h, const void* k, const void* v,
                                         void* cuda_stream);

@@ -15,9 +15,9 @@ LIB_PATH = os.path.join(_PKG, "liblinfusion_attn.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(6)
 PHI_ELU_PLUS_ONE, PHI_IDENTITY = 0, 1
-VARIANT_AUTO, VARIANT_SPLIT, VARIANT_STREAM, VARIANT_CLUSTER = 0, 1, 2, 3
+VARIANT_AUTO, VARIANT_SPLIT, VARIANT_STREAM, VARIANT_CLUSTER, VARIANT_FUSED = 0, 1, 2, 3, 4
 VARIANTS = {"auto": VARIANT_AUTO, "split": VARIANT_SPLIT, "stream": VARIANT_STREAM,
-            "cluster": VARIANT_CLUSTER}
+            "cluster": VARIANT_CLUSTER, "fused": VARIANT_FUSED}
 
 EXPORTED = [
     "linfusion_attn_create", "linfusion_attn_forward", "linfusion_attn_forward_host",
@@ -28,7 +28,7 @@ EXPORTED = [
     "linfusion_attn_set_kernel_timing_stride",
     "linfusion_attn_forward_noalloc", "linfusion_attn_noalloc_layout",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
-    "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait",
+    "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait", "linfusion_attn_selftest_counter_wait",
 ]
 
 
@@ -101,6 +101,8 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_apply.argtypes = [vp, vp, vp, vp]
     lib.linfusion_attn_selftest_wait.restype = st
     lib.linfusion_attn_selftest_wait.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.linfusion_attn_selftest_counter_wait.restype = st
+    lib.linfusion_attn_selftest_counter_wait.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.linfusion_attn_apply_peers.restype = st
     lib.linfusion_attn_apply_peers.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32, vp]
     lib.linfusion_attn_state_buffer.restype = st
@@ -331,6 +333,12 @@ class LinFusionAttention:
         """(status code, milliseconds) of the bounded-wait self-test; ERR_TIMEOUT is the expected code."""
         ms = ctypes.c_float(0.0)
         rc = self._lib.linfusion_attn_selftest_wait(self._h, ctypes.byref(ms))
+        return int(rc), float(ms.value)
+
+    def selftest_counter_wait(self):
+        """The same for the bounded poll of a global counter (the single-launch variant's wait)."""
+        ms = ctypes.c_float(0.0)
+        rc = self._lib.linfusion_attn_selftest_counter_wait(self._h, ctypes.byref(ms))
         return int(rc), float(ms.value)
 
     def set_kernel_timing_stride(self, stride: int) -> None:

@@ -8,7 +8,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "liblinfusion_attn.so")
 _SOURCES = ["linfusion_attn.cu"]
-_HEADERS = ["common.cuh", "split_kernels.cuh", "stream_kernels.cuh"]
+_HEADERS = ["common.cuh", "split_kernels.cuh", "stream_kernels.cuh", "fused_kernels.cuh"]
 
 
 def _newest_source_mtime() -> float:

@@ -11,6 +11,7 @@
 
 #include "split_kernels.cuh"
 #include "stream_kernels.cuh"
+#include "fused_kernels.cuh"
 
 using namespace lf;
 
@@ -19,7 +20,7 @@ namespace {
 constexpr int kDefaultSmCount = 148;
 using ApplyCfg = StreamApplyCfg;
 
-enum Variant { kSplit = 1, kStream = 2, kCluster = 3 };
+enum Variant { kSplit = 1, kStream = 2, kCluster = 3, kFused = 4 };
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -41,6 +42,8 @@ struct Plan {
     int G_state = 0, G_apply = 0, spans = 0;
     // cluster
     int cluster_size = 0;
+    // fused
+    int fused_split = 0, fused_whole = 0;
     // workspace (bytes, offsets)
     size_t partial_bytes = 0, state_off = 0, operand_off = 0, counters_off = 0, status_off = 0, total_bytes = 0;
     int launches = 0;
@@ -62,8 +65,8 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
                       LINFUSION_DTYPE_FP16)) != 0u)
         return LINFUSION_ERR_UNSUPPORTED;
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
-    if (v > LINFUSION_VARIANT_CLUSTER) return LINFUSION_ERR_UNSUPPORTED;
-    if (v == LINFUSION_VARIANT_STREAM && d->d != kStreamD) return LINFUSION_ERR_UNSUPPORTED;
+    if (v > LINFUSION_VARIANT_FUSED) return LINFUSION_ERR_UNSUPPORTED;
+    if ((v == LINFUSION_VARIANT_STREAM || v == LINFUSION_VARIANT_FUSED) && d->d != kStreamD) return LINFUSION_ERR_UNSUPPORTED;
     return LINFUSION_OK;
 }
 
@@ -97,8 +100,17 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // (12.9 us at N = 144, d = 64, against 14.4 us for the single clustered launch; 21.9 vs 27 us
         // at N = 64, d = 160), so the cluster kernel is only run on request.
         const long long stream_tiles = static_cast<long long>(slabs) * ((d->N + StreamStateCfg::TILE - 1) / StreamStateCfg::TILE);
+        // The single persistent launch wins where no state has to cross CTAs: slabs of at most eight
+        // 128-token tiles, enough of them to occupy a quarter of the SMs, each handled whole by one
+        // CTA (10.9 vs 12.9 us at N = 144 x 40 slabs, 15.2 vs 18.6 us at N = 576 x 40).  Where slabs
+        // are shared between CTAs its exchange through global memory costs more than two kernel
+        // boundaries (32 vs 22 us at N = 2304 x 20, 106 vs 47 us at N = 16384 x 20), so it is not
+        // chosen there.
+        const int fused_tiles = (d->N + FusedCfg::TILE - 1) / FusedCfg::TILE;
         if (d->d == kStreamD && stream_tiles >= 8ll * sm_count)
             v = LINFUSION_VARIANT_STREAM;
+        else if (d->d == kStreamD && fused_tiles <= 8 && 4 * slabs >= sm_count && stream_tiles < 4ll * sm_count)
+            v = LINFUSION_VARIANT_FUSED;
         else
             v = LINFUSION_VARIANT_SPLIT;
     }
@@ -141,6 +153,40 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         p->spans = spans;
         partial_floats = static_cast<size_t>(p->G_state) * spans * kStreamStateFloats;
         p->launches = 3;
+    } else if (v == LINFUSION_VARIANT_FUSED) {
+        // One persistent launch.  Two waves of slabs once every CTA has a couple of tiles in each
+        // (the exchange of one wave's states then hides behind the other wave's streaming); at
+        // most 32 CTAs per slab (the reducer warp keeps one contributor per lane).
+        const int tiles = (d->N + FusedCfg::TILE - 1) / FusedCfg::TILE;
+        p->tiles_state = p->tiles_apply = tiles;
+        p->W_state = p->W_apply = static_cast<long long>(slabs) * tiles;
+        const bool two = slabs >= 2 && p->W_state >= 4ll * sm_count;
+        p->fused_split = two ? (slabs + 1) / 2 : slabs;
+        // Small slabs are dealt whole, one CTA per slab or more slabs per CTA: nothing is exchanged.
+        p->fused_whole = (!two && tiles <= 8 && 4 * slabs >= sm_count) ? 1 : 0;
+        const FusedPlan fp = {tiles, slabs, p->fused_split, p->fused_whole};
+        long long G = sm_count;
+        if (p->fused_whole != 0) {
+            if (G > slabs) G = slabs;
+        } else {
+            if (G > fused_wave_units(fp, 0)) G = fused_wave_units(fp, 0);
+            const long long min_wave_slabs = two ? slabs - p->fused_split : slabs;
+            if (G > 30 * min_wave_slabs) G = 30 * min_wave_slabs;
+        }
+        p->G_state = p->G_apply = static_cast<int>(G);
+        int spans = 1;
+        for (int g = 0; g < p->G_state; ++g) {
+            int touched = 0;
+            for (int w = 0; w < fused_waves(fp); ++w) {
+                long long b, e;
+                fused_run(fp, g, G, w, &b, &e);
+                touched += fused_run_slabs(b, e, tiles);
+            }
+            if (touched > spans) spans = touched;
+        }
+        p->spans = spans;
+        partial_floats = static_cast<size_t>(p->G_state) * spans * kStreamStateFloats;
+        p->launches = 1;
     } else {
         p->cluster_size = largest_cluster(tiles_kv);
         partial_floats = 0;
@@ -156,7 +202,10 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamOperandBytes
                               : v == LINFUSION_VARIANT_SPLIT ? static_cast<size_t>(slabs) * split_image
                                                              : 0;
-    const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM ? align_up(static_cast<size_t>(slabs) * 4, 256) : 0;
+    // Stream: one tile counter per slab.  Fused: two arrival counters per slab, then the control words.
+    const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM  ? align_up(static_cast<size_t>(slabs) * 4, 256)
+                                 : v == LINFUSION_VARIANT_FUSED ? align_up(static_cast<size_t>(slabs) * 8, 256) + 256
+                                                                : 0;
     p->counters_off = p->operand_off + align_up(frag_bytes, 256);
     p->status_off = p->counters_off + counter_bytes;
     p->total_bytes = p->status_off + 256;
@@ -372,6 +421,9 @@ cudaError_t set_stream_attrs()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(stream_apply_kernel<KIND>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, ApplyCfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(stream_fused_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             FusedCfg::SMEM_BYTES);
     return e;
 }
 
@@ -481,6 +533,27 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
                        apply_scales(h->desc), h->desc.H);
     if (e != cudaSuccess) return e;
     mark(h, 3, s);
+    return cudaGetLastError();
+}
+
+template <int KIND>
+cudaError_t launch_fused(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                         const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
+{
+    const Plan& p = h->plan;
+    CUtensorMap mq, mk, mv, my;
+    if (!encode_slab_map(&mk, k, h->desc, FusedCfg::TILE) || !encode_slab_map(&mv, v, h->desc, FusedCfg::TILE) ||
+        !encode_slab_map(&mq, q, h->desc, FusedCfg::TILE) || !encode_slab_map(&my, y, h->desc, FusedCfg::TILE))
+        return cudaErrorInvalidValue;
+    uint32_t* arrive = reinterpret_cast<uint32_t*>(h->tile_counters);
+    uint32_t* ctrl = arrive + align_up(static_cast<size_t>(p.slabs) * 8, 256) / 4;
+    const FusedPlan fp = {p.tiles_state, p.slabs, p.fused_split, p.fused_whole};
+    mark(h, 0, s);
+    cudaError_t e = launch_chained(stream_fused_kernel<KIND>, dim3(p.G_state), dim3(FusedCfg::THREADS),
+                                   FusedCfg::SMEM_BYTES, s, mk, mv, mq, my, h->partials, h->state, arrive, ctrl,
+                                   h->status, h->desc.N, fp, p.spans, h->desc.H, apply_scales(h->desc));
+    if (e != cudaSuccess) return e;
+    mark(h, 1, s);
     return cudaGetLastError();
 }
 
@@ -704,6 +777,10 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
 #define LF_K(KV) e = launch_stream<KV>(h, Q, K, V, Y, s)
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
+    } else if (h->plan.variant == kFused) {
+#define LF_K(KV) e = launch_fused<KV>(h, Q, K, V, Y, s)
+        LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
     } else {
 #define LF_LAUNCH(DV) e = launch_d<DV>(h, Q, K, V, Y, s)
         LF_DISPATCH_D(h->desc.d, LF_LAUNCH)
@@ -910,7 +987,19 @@ linfusion_status_t linfusion_attn_status(linfusion_attn_t* h)
     return LINFUSION_OK;
 }
 
+static linfusion_status_t selftest_wait_impl(linfusion_attn_t* h, float* waited_ms, bool counter);
+
 linfusion_status_t linfusion_attn_selftest_wait(linfusion_attn_t* h, float* waited_ms)
+{
+    return selftest_wait_impl(h, waited_ms, false);
+}
+
+linfusion_status_t linfusion_attn_selftest_counter_wait(linfusion_attn_t* h, float* waited_ms)
+{
+    return selftest_wait_impl(h, waited_ms, true);
+}
+
+static linfusion_status_t selftest_wait_impl(linfusion_attn_t* h, float* waited_ms, bool counter)
 {
     if (h == nullptr || h->status == nullptr) return LINFUSION_ERR_INVALID_ARG;
     DeviceGuard guard(h->desc.device);
@@ -923,7 +1012,10 @@ linfusion_status_t linfusion_attn_selftest_wait(linfusion_attn_t* h, float* wait
         return LINFUSION_ERR_CUDA;
     }
     cudaEventRecord(e0, s);
-    wait_selftest_kernel<<<1, 32, 0, s>>>(h->status);
+    if (counter)  // a word nothing advances: the second word behind the status word (always zero)
+        counter_wait_selftest_kernel<<<1, 32, 0, s>>>(h->status, h->status + 1);
+    else
+        wait_selftest_kernel<<<1, 32, 0, s>>>(h->status);
     cudaEventRecord(e1, s);
     uint32_t word = 0;
     float ms = 0.0f;
@@ -971,6 +1063,7 @@ const char* linfusion_attn_variant_name(const linfusion_attn_t* h)
         case kSplit: return "split";
         case kStream: return "stream";
         case kCluster: return "cluster";
+        case kFused: return "fused";
         default: return "";
     }
 }
@@ -1316,7 +1409,7 @@ linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, c
 {
     if (h == nullptr || a == nullptr || (state_half ? b == nullptr : y == nullptr))
         return LINFUSION_ERR_INVALID_ARG;
-    if (h->plan.variant == kCluster) return LINFUSION_ERR_UNSUPPORTED;
+    if (h->plan.variant == kCluster || h->plan.variant == kFused) return LINFUSION_ERR_UNSUPPORTED;
     const uintptr_t pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b),
                     py = reinterpret_cast<uintptr_t>(y);
     if (((pa | pb | py) & 15u) != 0) return LINFUSION_ERR_INVALID_ARG;

@@ -81,7 +81,7 @@ def test_invalid_descriptors(kw):
 
 @pytest.mark.parametrize("kw", [
     dict(d=48), dict(d=7), dict(d=256), dict(phi=7), dict(variant=9), dict(variant=0x80),
-    dict(d=40, variant="stream"),
+    dict(d=40, variant="stream"), dict(d=40, variant="fused"),
 ])
 def test_unsupported_descriptors(kw):
     args = dict(B=2, H=8, N=4096, d=64, eps=1e-6, device=0)

@@ -30,6 +30,7 @@ def variants_for(shape):
     out = ["auto", "split"]
     if shape.d == 64:
         out.append("stream")
+        out.append("fused")
     if shape.N <= 16384:
         out.append("cluster")
     return out
@@ -114,6 +115,7 @@ EDGE_CASES = [
     (1, 1, 127, 64), (1, 1, 129, 64), (1, 5, 191, 64), (1, 1, 193, 64), (3, 1, 1000, 80),
     (1, 7, 333, 40), (1, 1, 4097, 128), (2, 3, 257, 32), (1, 2, 12289, 64), (1, 148, 64, 64),
     (8, 25, 300, 64),   # more slabs than SMs
+    (3, 100, 100, 64),  # 300 one-tile slabs: the single-launch variant deals whole slabs, two or three per CTA
 
 ]
 
@@ -136,15 +138,17 @@ def test_stream_variant_tail_and_slab_crossing():
     for (B, H, N) in [(2, 37, 1000), (1, 100, 130), (2, 20, 2500), (1, 3, 378917)]:
         q, k, v = wl.make_small(B, H, N, 64, seed=5, device="cuda")
         ref = oracle_y(q, k, v)
-        y, op = run_gpu(q, k, v, "stream")
-        assert op.variant == "stream"
-        assert_parity(y, ref, f"stream {(B, H, N)}")
-        op.close()
+        for variant in ("stream", "fused"):
+            y, op = run_gpu(q, k, v, variant)
+            assert op.variant == variant
+            assert_parity(y, ref, f"{variant} {(B, H, N)}")
+            op.close()
 
 
 def test_auto_policy_follows_the_measured_crossovers():
     for dims, want in [((2, 10, 16384, 64), "stream"), ((2, 20, 4096, 64), "stream"),
-                       ((2, 20, 2304, 64), "split"), ((2, 20, 144, 64), "split"), ((2, 8, 4096, 40), "split")]:
+                       ((2, 20, 2304, 64), "split"), ((2, 20, 144, 64), "fused"), ((2, 20, 576, 64), "fused"),
+                       ((2, 2, 144, 64), "split"), ((2, 8, 4096, 40), "split")]:
         op = attn.LinFusionAttention(*dims)
         assert op.variant == want, (dims, op.variant)
         op.close()
@@ -152,6 +156,8 @@ def test_auto_policy_follows_the_measured_crossovers():
 
 def test_bit_reproducible_run_to_run():
     for shape, variant in [(wl.find_shape("sdxl_2048_L2"), "stream"),
+                           (wl.find_shape("sdxl_2048_L2"), "fused"),
+                           (wl.find_shape("sd21_768_L4"), "fused"),
                            (wl.find_shape("sd15_512_L1"), "split"),
                            (wl.find_shape("sd15_512_L2"), "cluster")]:
         q, k, v = wl.make_qkv(shape, seed=3, device="cuda")
@@ -169,7 +175,7 @@ def test_state_matches_oracle_state():
     shape = wl.find_shape("sd21_768_L2")
     q, k, v = wl.make_qkv(shape, seed=9, device="cuda")
     S, z = oracle.state(to_f64(k), to_f64(v))
-    for variant in ("split", "stream", "cluster"):
+    for variant in ("split", "stream", "cluster", "fused"):
         _, op = run_gpu(q, k, v, variant)
         S_gpu, z_gpu = op.read_state()
         op.close()
@@ -365,11 +371,12 @@ def test_a_wait_that_cannot_complete_gives_up_and_is_reported():
 def test_forwards_of_several_handles_replay_from_a_cuda_graph():
     """A UNet level's handles captured once and replayed: forward() only enqueues kernels on the
     given stream (no allocation, no synchronization), chained launches included."""
-    shapes = [wl.find_shape("sdxl_2048_L1"), wl.find_shape("sd15_512_L2")]
+    shapes = [(wl.find_shape("sdxl_2048_L1"), "auto"), (wl.find_shape("sd15_512_L2"), "auto"),
+              (wl.find_shape("sd21_768_L2"), "fused"), (wl.find_shape("sd21_768_L4"), "fused")]
     layers = []
-    for i, s in enumerate(shapes):
+    for i, (s, variant) in enumerate(shapes):
         q, k, v = wl.make_qkv(s, seed=60 + i, device="cuda")
-        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=EPS)
+        op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, eps=EPS, variant=variant)
         layers.append((op, q, k, v, op.forward(q, k, v).clone(), torch.empty_like(q)))
     torch.cuda.synchronize()
     st = torch.cuda.Stream()
@@ -390,3 +397,38 @@ def test_forwards_of_several_handles_replay_from_a_cuda_graph():
         assert torch.equal(y.view(torch.int16), ref.view(torch.int16)), op.variant
         assert op.status() == attn.OK
         op.close()
+
+
+def test_fused_variant_many_forwards_in_a_row_and_its_bounded_counter_wait():
+    """The single-launch variant keeps per-slab arrival counters that are never reset (an epoch
+    word says where they stood): many forwards in a row, alternating inputs, must keep giving the
+    bits of the first ones; the bounded poll gives up on a counter nothing advances and reports."""
+    shape = wl.find_shape("sd21_768_L3")
+    qa, ka, va = wl.make_qkv(shape, seed=81, device="cuda")
+    qb, kb, vb = wl.make_qkv(shape, seed=82, device="cuda")
+    ya, op = run_gpu(qa, ka, va, "fused")
+    yb = op.forward(qb, kb, vb).clone()
+    assert_parity(ya, oracle_y(qa, ka, va), "fused a")
+    assert_parity(yb, oracle_y(qb, kb, vb), "fused b")
+    y = torch.empty_like(ya)
+    for i in range(300):
+        op.forward(*((qa, ka, va) if i % 2 == 0 else (qb, kb, vb)), y)
+        if i % 50 in (0, 1):
+            torch.cuda.synchronize()
+            assert torch.equal(y.view(torch.int16), (ya if i % 2 == 0 else yb).view(torch.int16)), i
+    assert op.status() == attn.OK
+    S_gpu, z_gpu = op.read_state()
+    S, z = oracle.state(to_f64(kb), to_f64(vb))
+    assert np.abs(z_gpu - z).max() <= 2e-3 * np.abs(z).max()
+    assert np.linalg.norm(S_gpu - S) <= 5e-3 * np.linalg.norm(S)
+    rc, ms = op.selftest_counter_wait()
+    assert rc == attn.ERR_TIMEOUT
+    assert 200.0 <= ms <= 2000.0, ms
+    assert op.status() == attn.OK
+    y2 = op.forward(qa, ka, va)
+    torch.cuda.synchronize()
+    assert torch.equal(y2.view(torch.int16), ya.view(torch.int16))
+    with pytest.raises(attn.LinFusionError) as e:
+        op.state(ka, va)                       # one launch cannot be split in two halves
+    assert e.value.code == attn.ERR_UNSUPPORTED
+    op.close()
