@@ -95,7 +95,22 @@ typedef struct {
     float eps;      /* finite, >= 0; added once to phi(Q_i) . z    */
     int32_t device; /* CUDA device ordinal the handle lives on     */
     uint32_t flags; /* LINFUSION_VARIANT_* | LINFUSION_LAYOUT_*      */
+    int32_t d_qk;   /* feature width d' of Q and K when it differs from d (Prop. 3); 0 = d.
+                       Supported pairs (d', d): (128, 64), (80, 40), (32, 64)              */
 } linfusion_attn_desc_t;
+
+/*
+ * Two widths (Prop. 3).  The proposition lets f' and g' map a token to d' features while the values
+ * keep d channels: Q and K are then [B, H, N, d'] (token-major: [B, N, H, d']), V and Y stay
+ * [B, H, N, d], the state S is d' x d and z has d' entries:
+ *
+ *     S = sum_j phi(K_j)^T V_j  (d' x d),   z = sum_j phi(K_j)  (d'),   Y_i = phi(Q_i) S / (phi(Q_i) . z + eps)
+ *
+ * desc.d is the value width d, desc.d_qk the feature width d' (0: the same as d, the released
+ * model's case).  The three-launch split path and the cluster kernel serve d' != d; the TMA +
+ * tcgen05 variants (STREAM, FUSED) are for d' = d = 64.  Everywhere this header says [.., d] for Q
+ * or K, or d x d for S, or d for z, read d' for the feature side.
+ */
 
 /*
  * Create a handle for one problem shape (Prop. 2's token mixer at fixed B, H, N, d).

@@ -36,7 +36,7 @@ class Desc(ctypes.Structure):
     """Mirror of ``linfusion_attn_desc_t``."""
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32),
                 ("d", ctypes.c_int32), ("phi", ctypes.c_int32), ("eps", ctypes.c_float),
-                ("device", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+                ("device", ctypes.c_int32), ("flags", ctypes.c_uint32), ("d_qk", ctypes.c_int32)]
 
 
 class LinFusionError(RuntimeError):
@@ -121,7 +121,9 @@ DTYPE_FP16 = 0x40           # Q, K, V, Y are fp16 instead of bf16
 
 
 def make_desc(B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
-              layout="head_major", normalize=True, dtype="bf16") -> Desc:
+              layout="head_major", normalize=True, dtype="bf16", d_qk=0) -> Desc:
+    """``d`` is the width of V and Y; ``d_qk`` the feature width d' of Q and K when it differs
+    (Prop. 3), 0 meaning the same."""
     flags = VARIANTS[variant] if isinstance(variant, str) else int(variant)
     if not normalize:
         flags |= FLAG_UNNORMALIZED
@@ -133,7 +135,7 @@ def make_desc(B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="aut
         flags |= LAYOUT_TOKEN_MAJOR
     elif layout != "head_major":
         raise ValueError("layout must be 'head_major' or 'token_major'")
-    return Desc(int(B), int(H), int(N), int(d), int(phi), float(eps), int(device), flags)
+    return Desc(int(B), int(H), int(N), int(d), int(phi), float(eps), int(device), flags, int(d_qk))
 
 
 def linfusion_attn_workspace_bytes(desc: Desc, sm_count: int = 0) -> int:
@@ -199,15 +201,19 @@ def linfusion_attn_destroy(handle) -> None:
 
 class LinFusionAttention:
     """One handle per shape.  ``forward`` takes bf16 CUDA tensors [B, H, N, d] (or [B, N, H, d]
-    with ``layout="token_major"``)."""
+    with ``layout="token_major"``).  With ``d_qk`` (Prop. 3's feature width d') Q and K are
+    [.., d_qk] while V and Y stay [.., d]."""
 
     def __init__(self, B, H, N, d, phi=PHI_ELU_PLUS_ONE, eps=1e-6, device=0, variant="auto",
-                 layout="head_major", normalize=True, dtype="bf16"):
-        self.desc = make_desc(B, H, N, d, phi, eps, device, variant, layout, normalize, dtype)
+                 layout="head_major", normalize=True, dtype="bf16", d_qk=0):
+        self.desc = make_desc(B, H, N, d, phi, eps, device, variant, layout, normalize, dtype, d_qk)
         self.dtype = dtype
-        # tensors are [B, H, N, d], or [B, N, H, d] in the token-major layout
+        dk = int(d_qk) if d_qk else int(d)
+        self.dk = dk
+        # V and Y are [B, H, N, d], or [B, N, H, d] in the token-major layout; Q and K have d' channels
         self.shape = (int(B), int(H), int(N), int(d)) if layout == "head_major" else \
                      (int(B), int(N), int(H), int(d))
+        self.shape_qk = self.shape[:3] + (dk,)
         self._lib = load_library()
         self._h = linfusion_attn_create(self.desc)
         self._lent_ws = None
@@ -225,8 +231,13 @@ class LinFusionAttention:
     def _check(self, t, name):
         import torch
         want = torch.float16 if self.dtype == "fp16" else torch.bfloat16
-        if tuple(t.shape) != self.shape or t.dtype != want or not t.is_contiguous():
-            raise ValueError(f"{name}: expected contiguous {self.dtype} tensor of shape {self.shape}")
+        shape = self.shape_qk if name in ("q", "k") else self.shape
+        if tuple(t.shape) != shape or t.dtype != want or not t.is_contiguous():
+            raise ValueError(f"{name}: expected contiguous {self.dtype} tensor of shape {shape}")
+
+    def _new_y(self, like):
+        import torch
+        return torch.empty(self.shape, dtype=like.dtype, device=like.device)
 
     def forward(self, q, k, v, y=None, stream: Optional[int] = None):
         import torch
@@ -235,7 +246,7 @@ class LinFusionAttention:
             if not t.is_cuda:
                 raise ValueError(f"{n}: expected a CUDA tensor")
         if y is None:
-            y = torch.empty_like(q)
+            y = self._new_y(q)
         else:
             self._check(y, "y")
         if stream is None:
@@ -261,11 +272,11 @@ class LinFusionAttention:
         return int(self._lib.linfusion_attn_status(self._h))
 
     def read_state(self):
-        """(S [B,H,d,d], z [B,H,d]) of the last forward as fp32 numpy arrays."""
+        """(S [B,H,d',d], z [B,H,d']) of the last forward as fp32 numpy arrays."""
         import numpy as np
         B, H, d = self.desc.B, self.desc.H, self.desc.d
-        S = np.empty((B, H, d, d), dtype=np.float32)
-        z = np.empty((B, H, d), dtype=np.float32)
+        S = np.empty((B, H, self.dk, d), dtype=np.float32)
+        z = np.empty((B, H, self.dk), dtype=np.float32)
         rc = self._lib.linfusion_attn_read_state(self._h, S.ctypes.data, z.ctypes.data)
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_read_state")
@@ -286,7 +297,7 @@ class LinFusionAttention:
         import torch
         self._check(q, "q")
         if y is None:
-            y = torch.empty_like(q)
+            y = self._new_y(q)
         else:
             self._check(y, "y")
         if stream is None:
@@ -303,7 +314,7 @@ class LinFusionAttention:
         import torch
         self._check(q, "q")
         if y is None:
-            y = torch.empty_like(q)
+            y = self._new_y(q)
         else:
             self._check(y, "y")
         if stream is None:

@@ -29,6 +29,17 @@ bool supported_d(int d)
     return d == 32 || d == 40 || d == 64 || d == 80 || d == 128 || d == 160;
 }
 
+// Feature width d' of Q and K (Prop. 3); the descriptor's 0 means "same as d".
+int dk_of(const linfusion_attn_desc_t& d) { return d.d_qk > 0 ? d.d_qk : d.d; }
+
+// (d', d) pairs the split and cluster kernels are instantiated for: every supported square case,
+// and the widened / narrowed feature widths below.
+bool supported_widths(int dk, int dv)
+{
+    if (dk == dv) return supported_d(dv);
+    return (dk == 128 && dv == 64) || (dk == 80 && dv == 40) || (dk == 32 && dv == 64);
+}
+
 // Everything that follows from (descriptor, SM count) alone.
 struct Plan {
     int variant = 0;
@@ -58,7 +69,8 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
     if (!std::isfinite(d->eps) || d->eps < 0.0f) return LINFUSION_ERR_INVALID_ARG;
     if (d->device < 0) return LINFUSION_ERR_INVALID_ARG;
     if (static_cast<long long>(d->B) * d->H > 65535) return LINFUSION_ERR_UNSUPPORTED;
-    if (!supported_d(d->d)) return LINFUSION_ERR_UNSUPPORTED;
+    if (d->d_qk < 0) return LINFUSION_ERR_INVALID_ARG;
+    if (!supported_widths(dk_of(*d), d->d)) return LINFUSION_ERR_UNSUPPORTED;
     if (d->phi != LINFUSION_PHI_ELU_PLUS_ONE && d->phi != LINFUSION_PHI_IDENTITY)
         return LINFUSION_ERR_UNSUPPORTED;
     if ((d->flags & ~(LINFUSION_VARIANT_MASK | LINFUSION_LAYOUT_TOKEN_MAJOR | LINFUSION_FLAG_UNNORMALIZED |
@@ -66,7 +78,8 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
         return LINFUSION_ERR_UNSUPPORTED;
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v > LINFUSION_VARIANT_FUSED) return LINFUSION_ERR_UNSUPPORTED;
-    if ((v == LINFUSION_VARIANT_STREAM || v == LINFUSION_VARIANT_FUSED) && d->d != kStreamD) return LINFUSION_ERR_UNSUPPORTED;
+    if ((v == LINFUSION_VARIANT_STREAM || v == LINFUSION_VARIANT_FUSED) && (d->d != kStreamD || dk_of(*d) != kStreamD))
+        return LINFUSION_ERR_UNSUPPORTED;
     return LINFUSION_OK;
 }
 
@@ -85,9 +98,11 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     *p = Plan();
     const int slabs = d->B * d->H;
     p->slabs = slabs;
-    p->state_floats = d->d * (d->d + 1);
+    const int dk = dk_of(*d), dv = d->d;
+    const bool square64 = dk == kStreamD && dv == kStreamD;
+    p->state_floats = dk * (dv + 1);
     const int tiles_kv = (d->N + 63) / 64;
-    const int tiles_q = (d->N + tile_q_of(d->d) - 1) / tile_q_of(d->d);
+    const int tiles_q = (d->N + tile_q_of(dk) - 1) / tile_q_of(dk);
 
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v == LINFUSION_VARIANT_AUTO) {
@@ -107,9 +122,9 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // boundaries (32 vs 22 us at N = 2304 x 20, 106 vs 47 us at N = 16384 x 20), so it is not
         // chosen there.
         const int fused_tiles = (d->N + FusedCfg::TILE - 1) / FusedCfg::TILE;
-        if (d->d == kStreamD && stream_tiles >= 8ll * sm_count)
+        if (square64 && stream_tiles >= 8ll * sm_count)
             v = LINFUSION_VARIANT_STREAM;
-        else if (d->d == kStreamD && fused_tiles <= 8 && 4 * slabs >= sm_count && stream_tiles < 4ll * sm_count)
+        else if (square64 && fused_tiles <= 8 && 4 * slabs >= sm_count && stream_tiles < 4ll * sm_count)
             v = LINFUSION_VARIANT_FUSED;
         else
             v = LINFUSION_VARIANT_SPLIT;
@@ -197,8 +212,8 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     p->operand_off = p->state_off + align_up(static_cast<size_t>(slabs) * p->state_floats * sizeof(float), 256);
     // 16-bit operand image of S | z for the apply kernel (in its shared-memory layout), and for the
     // stream variant one tile counter per slab.
-    const int dp = (d->d + 15) / 16 * 16;
-    const size_t split_image = static_cast<size_t>((d->d + 8 + 15) / 16 * 16) * (((dp / 8) | 1) * 16);
+    const int dkp = (dk + 15) / 16 * 16;
+    const size_t split_image = static_cast<size_t>((dv + 8 + 15) / 16 * 16) * (((dkp / 8) | 1) * 16);
     const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamOperandBytes
                               : v == LINFUSION_VARIANT_SPLIT ? static_cast<size_t>(slabs) * split_image
                                                              : 0;
@@ -269,22 +284,27 @@ ApplyScales apply_scales(const linfusion_attn_desc_t& d)
         default: break;              \
     }
 
-// Element strides of a slab's rows for the layout the descriptor asks for.
-SlabLayout layout_of(const linfusion_attn_desc_t& d)
+// Element strides of a slab's rows, `width` channels each, for the layout the descriptor asks for.
+SlabLayout layout_of(const linfusion_attn_desc_t& d, int width)
 {
     SlabLayout L;
     L.H = d.H;
-    if ((d.flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u) {  // [B, N, H, d]
-        L.batch_stride = static_cast<long long>(d.N) * d.H * d.d;
-        L.head_stride = d.d;
-        L.row_stride = d.H * d.d;
-    } else {  // [B, H, N, d]
-        L.batch_stride = static_cast<long long>(d.H) * d.N * d.d;
-        L.head_stride = static_cast<long long>(d.N) * d.d;
-        L.row_stride = d.d;
+    if ((d.flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u) {  // [B, N, H, width]
+        L.batch_stride = static_cast<long long>(d.N) * d.H * width;
+        L.head_stride = width;
+        L.row_stride = d.H * width;
+    } else {  // [B, H, N, width]
+        L.batch_stride = static_cast<long long>(d.H) * d.N * width;
+        L.head_stride = static_cast<long long>(d.N) * width;
+        L.row_stride = width;
     }
     return L;
 }
+SlabLayout layout_qk(const linfusion_attn_desc_t& d) { return layout_of(d, dk_of(d)); }  // Q and K
+SlabLayout layout_vy(const linfusion_attn_desc_t& d) { return layout_of(d, d.d); }       // V and Y
+// Bytes of Q (or K), and of V (or Y).
+size_t bytes_qk(const linfusion_attn_desc_t& d) { return static_cast<size_t>(d.B) * d.H * d.N * dk_of(d) * 2; }
+size_t bytes_vy(const linfusion_attn_desc_t& d) { return static_cast<size_t>(d.B) * d.H * d.N * d.d * 2; }
 
 // 16-bit (bf16 or fp16) tensor seen as (channel 64, token N, head H, batch B) -> boxes of tile_rows tokens of one
 // (b, h) slab, 128-byte swizzle, zero fill past N.  The layout only changes the strides.
@@ -292,7 +312,7 @@ bool encode_slab_map(CUtensorMap* map, const void* base, const linfusion_attn_de
 {
     EncodeTiledFn fn = get_encode_fn();
     if (fn == nullptr) return false;
-    const SlabLayout L = layout_of(d);
+    const SlabLayout L = layout_vy(d);  // these kernels have d' = d = 64
     cuuint64_t dims[4] = {static_cast<cuuint64_t>(kStreamD), static_cast<cuuint64_t>(d.N),
                           static_cast<cuuint64_t>(d.H), static_cast<cuuint64_t>(d.B)};
     cuuint64_t strides[3] = {static_cast<cuuint64_t>(L.row_stride) * 2, static_cast<cuuint64_t>(L.head_stride) * 2,
@@ -394,21 +414,21 @@ inline void mark(const linfusion_attn* h, int i, cudaStream_t s)
         cudaEventRecord(h->events[(h->timed_calls % h->timing_slots) * 4 + i], s);
 }
 
-template <int D, int KIND>
+template <int DK, int DV, int KIND>
 cudaError_t set_split_attrs()
 {
-    using C = SplitCfg<D>;
+    using C = SplitCfg<DK, DV>;
     cudaError_t e;
-    e = cudaFuncSetAttribute(state_partial_kernel<D, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
+    e = cudaFuncSetAttribute(state_partial_kernel<DK, DV, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(apply_kernel<D, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY);
+    e = cudaFuncSetAttribute(apply_kernel<DK, DV, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(cluster_fused_kernel<D, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(cluster_fused_kernel<DK, DV, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              C::SMEM_CLUSTER);
     if (e != cudaSuccess) return e;
     // Clusters of 16 CTAs are beyond the portable size of 8; create() shrinks the cluster when
     // the device cannot co-schedule it.
-    e = cudaFuncSetAttribute(cluster_fused_kernel<D, KIND>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    e = cudaFuncSetAttribute(cluster_fused_kernel<DK, DV, KIND>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     return e;
 }
 
@@ -446,38 +466,38 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
-template <int D, int KIND>
+template <int DK, int DV, int KIND>
 cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                          const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
-    using C = SplitCfg<D>;
+    using C = SplitCfg<DK, DV>;
     const Plan& p = h->plan;
     const int N = h->desc.N;
     cudaError_t e;
     mark(h, 0, s);
-    e = launch_chained(state_partial_kernel<D, KIND>, dim3(p.chunks_state, p.slabs), dim3(C::NT), C::SMEM_KV, s, k, v,
-                       h->partials, N, p.chunks_state, layout_of(h->desc));
+    e = launch_chained(state_partial_kernel<DK, DV, KIND>, dim3(p.chunks_state, p.slabs), dim3(C::NT), C::SMEM_KV, s, k, v,
+                       h->partials, N, p.chunks_state, layout_qk(h->desc), layout_vy(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 1, s);
     // h->operand (when the workspace has it) receives the apply kernel's 16-bit operand image.
     unsigned char* image = h->operand;
     e = launch_chained(state_reduce_kernel, dim3((C::STATE_FLOATS + 255) / 256, p.slabs), dim3(256), 0, s,
-                       h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, D, C::PITCH, C::SMEM_ST,
+                       h->partials, h->state, C::STATE_FLOATS, p.chunks_state, image, DK, DV, C::PITCHK, C::SMEM_ST,
                        dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 2, s);
-    e = launch_chained(apply_kernel<D, KIND>, dim3(p.chunks_apply, p.slabs), dim3(C::NT), C::SMEM_APPLY, s, q,
-                       h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), image);
+    e = launch_chained(apply_kernel<DK, DV, KIND>, dim3(p.chunks_apply, p.slabs), dim3(C::NT), C::SMEM_APPLY, s, q,
+                       h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_qk(h->desc), layout_vy(h->desc), image);
     if (e != cudaSuccess) return e;
     mark(h, 3, s);
     return cudaGetLastError();
 }
 
-template <int D>
+template <int DK, int DV>
 void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int cluster_size, int slabs,
                     cudaStream_t s)
 {
-    using C = SplitCfg<D>;
+    using C = SplitCfg<DK, DV>;
     *cfg = cudaLaunchConfig_t{};
     cfg->gridDim = dim3(cluster_size, slabs, 1);
     cfg->blockDim = dim3(C::NT, 1, 1);
@@ -491,16 +511,16 @@ void cluster_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, int clus
     cfg->numAttrs = 1;
 }
 
-template <int D, int KIND>
+template <int DK, int DV, int KIND>
 cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                            const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    cluster_config<D>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
+    cluster_config<DK, DV>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
     mark(h, 0, s);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<D, KIND>, q, k, v, y, h->state,
-                                       h->desc.N, apply_scales(h->desc), layout_of(h->desc));
+    cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<DK, DV, KIND>, q, k, v, y, h->state,
+                                       h->desc.N, apply_scales(h->desc), layout_qk(h->desc), layout_vy(h->desc));
     mark(h, 1, s);
     return e;
 }
@@ -557,53 +577,57 @@ cudaError_t launch_fused(const linfusion_attn* h, const __nv_bfloat16* q, const 
     return cudaGetLastError();
 }
 
-template <int D>
+template <int DK, int DV>
 cudaError_t set_attrs_d(int kind)
 {
     cudaError_t e = cudaErrorInvalidValue;
-#define LF_K(KV) e = set_split_attrs<D, KV>()
+#define LF_K(KV) e = set_split_attrs<DK, DV, KV>()
     LF_DISPATCH_KIND(kind, LF_K)
 #undef LF_K
     return e;
 }
 
-template <int D>
+template <int DK, int DV>
 cudaError_t launch_d(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                      const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
     cudaError_t e = cudaErrorInvalidValue;
     if (h->plan.variant == kCluster) {
-#define LF_K(KV) e = launch_cluster<D, KV>(h, q, k, v, y, s)
+#define LF_K(KV) e = launch_cluster<DK, DV, KV>(h, q, k, v, y, s)
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
     } else {
-#define LF_K(KV) e = launch_split<D, KV>(h, q, k, v, y, s)
+#define LF_K(KV) e = launch_split<DK, DV, KV>(h, q, k, v, y, s)
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
     }
     return e;
 }
 
-#define LF_DISPATCH_D(dval, CALL)   \
-    switch (dval) {                 \
-        case 32: CALL(32); break;   \
-        case 40: CALL(40); break;   \
-        case 64: CALL(64); break;   \
-        case 80: CALL(80); break;   \
-        case 128: CALL(128); break; \
-        case 160: CALL(160); break; \
-        default: break;             \
+// CALL(DK, DV) for the descriptor's pair of widths (supported_widths() lists the same pairs).
+#define LF_DISPATCH_D(desc, CALL)               \
+    switch (dk_of(desc) * 1000 + (desc).d) {    \
+        case 32032: CALL(32, 32); break;        \
+        case 40040: CALL(40, 40); break;        \
+        case 64064: CALL(64, 64); break;        \
+        case 80080: CALL(80, 80); break;        \
+        case 128128: CALL(128, 128); break;     \
+        case 160160: CALL(160, 160); break;     \
+        case 128064: CALL(128, 64); break;      \
+        case 80040: CALL(80, 40); break;        \
+        case 32064: CALL(32, 64); break;        \
+        default: break;                         \
     }
 
-template <int D>
+template <int DK, int DV>
 bool cluster_fits(int kind, int cluster_size, int slabs)
 {
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
-    cluster_config<D>(&cfg, attr, cluster_size, slabs, nullptr);
+    cluster_config<DK, DV>(&cfg, attr, cluster_size, slabs, nullptr);
     int n = 0;
     cudaError_t e = cudaErrorInvalidValue;
-#define LF_K(KV) e = cudaOccupancyMaxActiveClusters(&n, cluster_fused_kernel<D, KV>, &cfg)
+#define LF_K(KV) e = cudaOccupancyMaxActiveClusters(&n, cluster_fused_kernel<DK, DV, KV>, &cfg)
     LF_DISPATCH_KIND(kind, LF_K)
 #undef LF_K
     if (e != cudaSuccess) {
@@ -683,10 +707,10 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     }
 
     cudaError_t e = cudaSuccess;
-#define LF_SET(DV) e = set_attrs_d<DV>(kind_of(*desc))
-    LF_DISPATCH_D(desc->d, LF_SET)
+#define LF_SET(DKV, DVV) e = set_attrs_d<DKV, DVV>(kind_of(*desc))
+    LF_DISPATCH_D(*desc, LF_SET)
 #undef LF_SET
-    if (e == cudaSuccess && desc->d == kStreamD) {
+    if (e == cudaSuccess && desc->d == kStreamD && dk_of(*desc) == kStreamD) {
 #define LF_K(KV) e = set_stream_attrs<KV>()
         LF_DISPATCH_KIND(kind_of(*desc), LF_K)
 #undef LF_K
@@ -702,8 +726,8 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
         bool fits = false;
         const bool forced = (desc->flags & LINFUSION_VARIANT_MASK) == LINFUSION_VARIANT_CLUSTER;
         while (true) {
-#define LF_FIT(DV) fits = cluster_fits<DV>(kind_of(*desc), h->plan.cluster_size, h->plan.slabs)
-            LF_DISPATCH_D(desc->d, LF_FIT)
+#define LF_FIT(DKV, DVV) fits = cluster_fits<DKV, DVV>(kind_of(*desc), h->plan.cluster_size, h->plan.slabs)
+            LF_DISPATCH_D(*desc, LF_FIT)
 #undef LF_FIT
             if (fits || h->plan.cluster_size == 1) break;
             h->plan.cluster_size >>= 1;
@@ -759,9 +783,9 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
     const uintptr_t pq = reinterpret_cast<uintptr_t>(q), pk = reinterpret_cast<uintptr_t>(k),
                     pv = reinterpret_cast<uintptr_t>(v), py = reinterpret_cast<uintptr_t>(y);
     if (((pq | pk | pv | py) & 15u) != 0) return LINFUSION_ERR_INVALID_ARG;
-    const size_t bytes = static_cast<size_t>(h->plan.slabs) * h->desc.N * h->desc.d * 2;
-    auto overlaps = [&](uintptr_t a) { return a < py + bytes && py < a + bytes; };
-    if (overlaps(pq) || overlaps(pk) || overlaps(pv)) return LINFUSION_ERR_INVALID_ARG;
+    const size_t nqk = bytes_qk(h->desc), nvy = bytes_vy(h->desc);
+    auto overlaps = [&](uintptr_t a, size_t n) { return a < py + nvy && py < a + n; };
+    if (overlaps(pq, nqk) || overlaps(pk, nqk) || overlaps(pv, nvy)) return LINFUSION_ERR_INVALID_ARG;
 
     DeviceGuard guard(h->desc.device);
     if (!guard.ok) return LINFUSION_ERR_CUDA;
@@ -782,8 +806,8 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
     } else {
-#define LF_LAUNCH(DV) e = launch_d<DV>(h, Q, K, V, Y, s)
-        LF_DISPATCH_D(h->desc.d, LF_LAUNCH)
+#define LF_LAUNCH(DKV, DVV) e = launch_d<DKV, DVV>(h, Q, K, V, Y, s)
+        LF_DISPATCH_D(h->desc, LF_LAUNCH)
 #undef LF_LAUNCH
     }
     h->last_stream = s;
@@ -872,10 +896,13 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
         return LINFUSION_ERR_INVALID_ARG;
     DeviceGuard guard(h->desc.device);
     if (!guard.ok) return LINFUSION_ERR_CUDA;
-    const size_t bytes = static_cast<size_t>(h->plan.slabs) * h->desc.N * h->desc.d * 2;
+    // Staging buffers 0..3 hold Q, K, V, Y: Q and K are d' wide, V and Y d wide.
+    const size_t nqk = bytes_qk(h->desc), nvy = bytes_vy(h->desc);
+    const size_t stage_bytes[4] = {nqk, nqk, nvy, nvy};
+    const size_t bytes = nvy;
     if (h->stage[0] == nullptr) {
         for (int i = 0; i < 4; ++i) {
-            if (cudaMalloc(&h->stage[i], bytes) != cudaSuccess) {
+            if (cudaMalloc(&h->stage[i], stage_bytes[i]) != cudaSuccess) {
                 cudaGetLastError();
                 for (int j = 0; j < i; ++j) cudaFree(h->stage[j]);
                 for (int j = 0; j < 4; ++j) h->stage[j] = nullptr;
@@ -921,15 +948,15 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
     HostPipe* p = h->pipe;
     if (p->groups == 1) {
         // K and V first: they feed the first kernel.
-        if (cudaMemcpyAsync(h->stage[1], k_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-            cudaMemcpyAsync(h->stage[2], v_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess ||
-            cudaMemcpyAsync(h->stage[0], q_host, bytes, cudaMemcpyHostToDevice, s) != cudaSuccess) {
+        if (cudaMemcpyAsync(h->stage[1], k_host, nqk, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(h->stage[2], v_host, nvy, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+            cudaMemcpyAsync(h->stage[0], q_host, nqk, cudaMemcpyHostToDevice, s) != cudaSuccess) {
             cudaGetLastError();
             return LINFUSION_ERR_CUDA;
         }
         linfusion_status_t st = linfusion_attn_forward(h, h->stage[0], h->stage[1], h->stage[2], h->stage[3], s);
         if (st != LINFUSION_OK) return st;
-        if (cudaMemcpyAsync(y_host, h->stage[3], bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
+        if (cudaMemcpyAsync(y_host, h->stage[3], nvy, cudaMemcpyDeviceToHost, s) != cudaSuccess) {
             cudaGetLastError();
             return LINFUSION_ERR_CUDA;
         }
@@ -938,16 +965,18 @@ linfusion_status_t linfusion_attn_forward_host(linfusion_attn_t* h, const void* 
 
     // Uploads run ahead on copy_in, kernels follow on the caller's stream, downloads trail on
     // copy_out; everything is ordered after the caller's earlier work and before its later work.
-    const size_t gbytes = bytes / p->groups;
-    auto at = [&](const void* base, int i) { return static_cast<const unsigned char*>(base) + i * gbytes; };
-    auto dev = [&](int which, int i) { return static_cast<unsigned char*>(h->stage[which]) + i * gbytes; };
+    const size_t gbytes = nvy / p->groups, gbytes_qk = nqk / p->groups;
+    auto at = [&](const void* base, int i, size_t gb) { return static_cast<const unsigned char*>(base) + i * gb; };
+    auto dev = [&](int which, int i) {
+        return static_cast<unsigned char*>(h->stage[which]) + i * (which < 2 ? gbytes_qk : gbytes);
+    };
     bool ok = cudaEventRecord(p->entry, s) == cudaSuccess &&
               cudaStreamWaitEvent(p->copy_in, p->entry, 0) == cudaSuccess &&
               cudaStreamWaitEvent(p->copy_out, p->entry, 0) == cudaSuccess;
     for (int i = 0; ok && i < p->groups; ++i) {
-        ok = cudaMemcpyAsync(dev(1, i), at(k_host, i), gbytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
-             cudaMemcpyAsync(dev(2, i), at(v_host, i), gbytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
-             cudaMemcpyAsync(dev(0, i), at(q_host, i), gbytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
+        ok = cudaMemcpyAsync(dev(1, i), at(k_host, i, gbytes_qk), gbytes_qk, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
+             cudaMemcpyAsync(dev(2, i), at(v_host, i, gbytes), gbytes, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
+             cudaMemcpyAsync(dev(0, i), at(q_host, i, gbytes_qk), gbytes_qk, cudaMemcpyHostToDevice, p->copy_in) == cudaSuccess &&
              cudaEventRecord(p->in[i], p->copy_in) == cudaSuccess &&
              cudaStreamWaitEvent(s, p->in[i], 0) == cudaSuccess;
         if (!ok) break;
@@ -1041,15 +1070,15 @@ linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host,
         cudaGetLastError();
         return LINFUSION_ERR_CUDA;
     }
-    const int d = h->desc.d, sf = h->plan.state_floats;
+    const int dk = dk_of(h->desc), dv = h->desc.d, sf = h->plan.state_floats;
     for (int s = 0; s < h->plan.slabs; ++s) {
         const float* src = h->state + static_cast<size_t>(s) * sf;
         if (S_host != nullptr &&
-            cudaMemcpy(S_host + static_cast<size_t>(s) * d * d, src, sizeof(float) * d * d,
+            cudaMemcpy(S_host + static_cast<size_t>(s) * dk * dv, src, sizeof(float) * dk * dv,
                        cudaMemcpyDeviceToHost) != cudaSuccess)
             return LINFUSION_ERR_CUDA;
         if (z_host != nullptr &&
-            cudaMemcpy(z_host + static_cast<size_t>(s) * d, src + d * d, sizeof(float) * d,
+            cudaMemcpy(z_host + static_cast<size_t>(s) * dk, src + dk * dv, sizeof(float) * dk,
                        cudaMemcpyDeviceToHost) != cudaSuccess)
             return LINFUSION_ERR_CUDA;
     }
@@ -1125,34 +1154,38 @@ struct NoAllocDevice {
     std::atomic<bool> ready{false};
     unsigned char* scratch = nullptr;  // device address of g_noalloc_scratch on this device
     int sm_count = 0;
-    std::atomic<uint32_t> configured{0};  // bit (d index * 4 + kind): shared-memory limits raised
+    std::atomic<uint64_t> configured{0};  // bit (width-pair index * 4 + kind): shared-memory limits raised
 };
 NoAllocDevice g_noalloc_dev[kNoAllocMaxDevices];
 std::mutex g_noalloc_mutex;  // serializes the set-up below (first calls from several host threads)
 
-int d_index(int d)
+// Index of a supported (d', d) pair.
+int width_pair_index(int dk, int dv)
 {
-    switch (d) {
-        case 32: return 0;
-        case 40: return 1;
-        case 64: return 2;
-        case 80: return 3;
-        case 128: return 4;
-        case 160: return 5;
+    switch (dk * 1000 + dv) {
+        case 32032: return 0;
+        case 40040: return 1;
+        case 64064: return 2;
+        case 80080: return 3;
+        case 128128: return 4;
+        case 160160: return 5;
+        case 128064: return 6;
+        case 80040: return 7;
+        case 32064: return 8;
         default: return -1;
     }
 }
 
 // The two kernels this entry point launches per (head dim, kind); the cluster kernel is not among them.
-template <int D>
+template <int DK, int DV>
 cudaError_t set_noalloc_attrs_d(int kind)
 {
-    using C = SplitCfg<D>;
+    using C = SplitCfg<DK, DV>;
     cudaError_t e = cudaErrorInvalidValue;
-#define LF_K(KV)                                                                                                    \
-    e = cudaFuncSetAttribute(state_partial_kernel<D, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV); \
-    if (e == cudaSuccess)                                                                                           \
-    e = cudaFuncSetAttribute(apply_kernel<D, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY)
+#define LF_K(KV)                                                                                                         \
+    e = cudaFuncSetAttribute(state_partial_kernel<DK, DV, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_KV); \
+    if (e == cudaSuccess)                                                                                                \
+    e = cudaFuncSetAttribute(apply_kernel<DK, DV, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_APPLY)
     LF_DISPATCH_KIND(kind, LF_K)
 #undef LF_K
     return e;
@@ -1163,10 +1196,11 @@ cudaError_t set_noalloc_attrs_d(int kind)
 // per (device, head dim, kind): raise the two kernels' dynamic shared-memory limits.  Later calls
 // find both done and make no CUDA call here.  Safe for first calls made by several host threads
 // at once: the set-up runs under a mutex and is published with release / acquire.
-linfusion_status_t noalloc_setup(int device, int d, int kind)
+linfusion_status_t noalloc_setup(const linfusion_attn_desc_t& desc, int kind)
 {
+    const int device = desc.device;
     NoAllocDevice& dev = g_noalloc_dev[device];
-    const uint32_t bit = 1u << (d_index(d) * 4 + kind);
+    const uint64_t bit = uint64_t(1) << (width_pair_index(dk_of(desc), desc.d) * 4 + kind);
     if (dev.ready.load(std::memory_order_acquire) && (dev.configured.load(std::memory_order_acquire) & bit) != 0u)
         return LINFUSION_OK;
     std::lock_guard<std::mutex> lock(g_noalloc_mutex);
@@ -1194,8 +1228,8 @@ linfusion_status_t noalloc_setup(int device, int d, int kind)
     }
     if ((dev.configured.load(std::memory_order_relaxed) & bit) == 0u) {
         cudaError_t e = cudaErrorInvalidValue;
-#define LF_SET(DV) e = set_noalloc_attrs_d<DV>(kind)
-        LF_DISPATCH_D(d, LF_SET)
+#define LF_SET(DKV, DVV) e = set_noalloc_attrs_d<DKV, DVV>(kind)
+        LF_DISPATCH_D(desc, LF_SET)
 #undef LF_SET
         if (e != cudaSuccess) {
             cudaGetLastError();
@@ -1216,7 +1250,7 @@ linfusion_status_t noalloc_layout(const linfusion_attn_desc_t* desc, int sm_coun
     linfusion_status_t st = validate(desc);
     if (st != LINFUSION_OK) return st;
     if ((desc->flags & LINFUSION_VARIANT_MASK) > LINFUSION_VARIANT_SPLIT) return LINFUSION_ERR_UNSUPPORTED;
-    const size_t per_chunk = static_cast<size_t>(desc->B) * desc->H * desc->d * (desc->d + 1) * 4;
+    const size_t per_chunk = static_cast<size_t>(desc->B) * desc->H * dk_of(*desc) * (desc->d + 1) * 4;
     const size_t state_bytes = align_up(per_chunk, 256);
     if (state_bytes + per_chunk + 256 > kNoAllocScratchBytes) return LINFUSION_ERR_ALLOC;
     linfusion_attn_desc_t d = *desc;
@@ -1264,9 +1298,9 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     const uintptr_t pq = reinterpret_cast<uintptr_t>(q), pk = reinterpret_cast<uintptr_t>(k),
                     pv = reinterpret_cast<uintptr_t>(v), py = reinterpret_cast<uintptr_t>(y);
     if (((pq | pk | pv | py) & 15u) != 0) return LINFUSION_ERR_INVALID_ARG;
-    const size_t bytes = static_cast<size_t>(desc->B) * desc->H * desc->N * desc->d * 2;
-    auto overlaps = [&](uintptr_t a) { return a < py + bytes && py < a + bytes; };
-    if (overlaps(pq) || overlaps(pk) || overlaps(pv)) return LINFUSION_ERR_INVALID_ARG;
+    const size_t nqk = bytes_qk(*desc), nvy = bytes_vy(*desc);
+    auto overlaps = [&](uintptr_t a, size_t n) { return a < py + nvy && py < a + n; };
+    if (overlaps(pq, nqk) || overlaps(pk, nqk) || overlaps(pv, nvy)) return LINFUSION_ERR_INVALID_ARG;
 
     // (A device ordinal the process does not have fails in cudaSetDevice here, or in the first
     // call's set-up, which asks for the device count.)
@@ -1276,7 +1310,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
         return g_noalloc_dev[desc->device].ready.load(std::memory_order_acquire) ? LINFUSION_ERR_CUDA
                                                                                  : LINFUSION_ERR_INVALID_ARG;
     }
-    st = noalloc_setup(desc->device, desc->d, kind_of(*desc));
+    st = noalloc_setup(*desc, kind_of(*desc));
     if (st != LINFUSION_OK) return st;
     const NoAllocDevice& dev = g_noalloc_dev[desc->device];
 
@@ -1313,8 +1347,8 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     const __nv_bfloat16* V = static_cast<const __nv_bfloat16*>(v);
     __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(y);
     cudaError_t e = cudaErrorInvalidValue;
-#define LF_LAUNCH(DV) e = launch_d<DV>(&view, Q, K, V, Y, s)
-    LF_DISPATCH_D(view.desc.d, LF_LAUNCH)
+#define LF_LAUNCH(DKV, DVV) e = launch_d<DKV, DVV>(&view, Q, K, V, Y, s)
+    LF_DISPATCH_D(view.desc, LF_LAUNCH)
 #undef LF_LAUNCH
     if (e != cudaSuccess) {
         cudaGetLastError();
@@ -1332,29 +1366,30 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-template <int D, int KIND>
+template <int DK, int DV, int KIND>
 cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a,
                               const __nv_bfloat16* b, __nv_bfloat16* y, cudaStream_t s, const PeerStates* peers)
 {
-    using C = SplitCfg<D>;
+    using C = SplitCfg<DK, DV>;
+    const SlabLayout LK = layout_qk(h->desc), LV = layout_vy(h->desc);
     const Plan& p = h->plan;
     const int N = h->desc.N;
     if (state_half) {
-        state_partial_kernel<D, KIND><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
-            a, b, h->partials, N, p.chunks_state, layout_of(h->desc));
+        state_partial_kernel<DK, DV, KIND><<<dim3(p.chunks_state, p.slabs), C::NT, C::SMEM_KV, s>>>(
+            a, b, h->partials, N, p.chunks_state, LK, LV);
         state_reduce_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
-            h->partials, h->state, C::STATE_FLOATS, p.chunks_state, nullptr, D, C::PITCH, C::SMEM_ST,
+            h->partials, h->state, C::STATE_FLOATS, p.chunks_state, nullptr, DK, DV, C::PITCHK, C::SMEM_ST,
             dtype_of(h->desc), operand_scale(h->desc));
     } else if (peers != nullptr) {
         // Sum the devices' states into the operand image, then apply from the image.
         peer_sum_image_kernel<<<dim3((C::STATE_FLOATS + 255) / 256, p.slabs), 256, 0, s>>>(
-            *peers, C::STATE_FLOATS, h->operand, D, C::PITCH, C::SMEM_ST, dtype_of(h->desc), operand_scale(h->desc));
-        apply_kernel<D, KIND><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-            a, h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), h->operand);
+            *peers, C::STATE_FLOATS, h->operand, DK, DV, C::PITCHK, C::SMEM_ST, dtype_of(h->desc), operand_scale(h->desc));
+        apply_kernel<DK, DV, KIND><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
+            a, h->state, y, N, p.chunks_apply, apply_scales(h->desc), LK, LV, h->operand);
     } else {
         // The fp32 state may have been summed over devices: convert it here, not from an image.
-        apply_kernel<D, KIND><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
-            a, h->state, y, N, p.chunks_apply, apply_scales(h->desc), layout_of(h->desc), nullptr);
+        apply_kernel<DK, DV, KIND><<<dim3(p.chunks_apply, p.slabs), C::NT, C::SMEM_APPLY, s>>>(
+            a, h->state, y, N, p.chunks_apply, apply_scales(h->desc), LK, LV, nullptr);
     }
     return cudaGetLastError();
 }
@@ -1393,12 +1428,12 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
     return cudaGetLastError();
 }
 
-template <int D>
+template <int DK, int DV>
 cudaError_t split_half_d(const linfusion_attn* h, bool state_half, const __nv_bfloat16* a, const __nv_bfloat16* b,
                          __nv_bfloat16* y, cudaStream_t s, const PeerStates* peers)
 {
     cudaError_t e = cudaErrorInvalidValue;
-#define LF_K(KV) e = launch_split_half<D, KV>(h, state_half, a, b, y, s, peers)
+#define LF_K(KV) e = launch_split_half<DK, DV, KV>(h, state_half, a, b, y, s, peers)
     LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
     return e;
@@ -1413,8 +1448,7 @@ linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, c
     const uintptr_t pa = reinterpret_cast<uintptr_t>(a), pb = reinterpret_cast<uintptr_t>(b),
                     py = reinterpret_cast<uintptr_t>(y);
     if (((pa | pb | py) & 15u) != 0) return LINFUSION_ERR_INVALID_ARG;
-    const size_t bytes = static_cast<size_t>(h->plan.slabs) * h->desc.N * h->desc.d * 2;
-    if (!state_half && pa < py + bytes && py < pa + bytes) return LINFUSION_ERR_INVALID_ARG;
+    if (!state_half && pa < py + bytes_vy(h->desc) && py < pa + bytes_qk(h->desc)) return LINFUSION_ERR_INVALID_ARG;
     DeviceGuard guard(h->desc.device);
     if (!guard.ok) return LINFUSION_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
@@ -1427,8 +1461,8 @@ linfusion_status_t run_half(linfusion_attn* h, bool state_half, const void* a, c
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
     } else {
-#define LF_HALF(DV) e = split_half_d<DV>(h, state_half, A, B, Y, s, peers)
-        LF_DISPATCH_D(h->desc.d, LF_HALF)
+#define LF_HALF(DKV, DVV) e = split_half_d<DKV, DVV>(h, state_half, A, B, Y, s, peers)
+        LF_DISPATCH_D(h->desc, LF_HALF)
 #undef LF_HALF
     }
     h->last_stream = s;

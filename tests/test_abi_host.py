@@ -159,3 +159,25 @@ def test_noalloc_layout_never_leaves_the_array():
     with pytest.raises(attn.LinFusionError) as e:
         attn.linfusion_attn_noalloc_layout(attn.make_desc(1, 70000, 64, 64))
     assert e.value.code == attn.ERR_UNSUPPORTED
+
+
+def test_two_widths_in_the_descriptor():
+    """Prop. 3: d_qk = d' is the width of Q and K, d that of V and Y; the state is d' x d."""
+    # state floats follow d' * (d + 1): the cluster variant's workspace is state + status only
+    sq = _ws(attn.make_desc(2, 4, 256, 64, variant="cluster"))
+    wide = _ws(attn.make_desc(2, 4, 256, 64, variant="cluster", d_qk=128))
+    narrow = _ws(attn.make_desc(2, 4, 256, 64, variant="cluster", d_qk=32))
+    assert wide - sq == 8 * (128 - 64) * 65 * 4 and sq - narrow == 8 * (64 - 32) * 65 * 4
+    assert _ws(attn.make_desc(2, 4, 256, 64, variant="split", d_qk=64)) == \
+        _ws(attn.make_desc(2, 4, 256, 64, variant="split"))
+    for kw in (dict(d=64, d_qk=48), dict(d=40, d_qk=128), dict(d=64, d_qk=128, variant="stream"),
+               dict(d=64, d_qk=128, variant="fused")):
+        with pytest.raises(attn.LinFusionError) as e:
+            _ws(attn.make_desc(1, 1, 256, kw["d"], d_qk=kw["d_qk"], variant=kw.get("variant", "auto")))
+        assert e.value.code == attn.ERR_UNSUPPORTED
+    with pytest.raises(attn.LinFusionError) as e:
+        _ws(attn.make_desc(1, 1, 256, 64, d_qk=-8))
+    assert e.value.code == attn.ERR_INVALID_ARG
+    # the allocation-free entry point sizes its array use by d' * (d + 1) too
+    chunks, off, used, cap = attn.linfusion_attn_noalloc_layout(attn.make_desc(2, 8, 4096, 64, d_qk=128), 148)
+    assert used - off == 16 * 128 * 65 * 4 and used <= cap and chunks >= 1
