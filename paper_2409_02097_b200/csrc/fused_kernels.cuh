@@ -433,16 +433,31 @@ stream_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         const float scale = sc.operand;
         bool ok = true;
 
-        // The exchange of visit kx through global memory (steps 2 and 3 above; for a slab that is
-        // local to this CTA but could not take the register shortcut, a plain copy).
-        auto exchange = [&](int kx) {
+        // The exchange of visit kx through global memory, in two halves so that a CTA whose run
+        // meets several slabs delivers its slice of every one of them (first half) before it waits
+        // for anybody else's (second half): a CTA that waited for slab s to be complete before it
+        // contributed its slice of slab s+1 would chain the slabs' exchanges one behind the other
+        // across the grid.  (For a slab that is local to this CTA but could not take the register
+        // shortcut, both halves together are a plain copy.)
+        struct Visit {
+            int slab, P, r, g0, w;
+        };
+        auto visit_of = [&](int kx) {
             int it = 0;
             for (int i = 0; i < kx; ++i) it += walk.left_in_slab(it, tiles_per_slab);
-            const int slab = static_cast<int>(walk.unit(it) / tiles_per_slab);
-            const int w = it < walk.n0 ? 0 : 1;
-            int g0, g1;
-            fused_contributors(plan, slab, w, G, &g0, &g1);
-            const int P = g1 - g0, r = static_cast<int>(g) - g0;
+            Visit v;
+            v.slab = static_cast<int>(walk.unit(it) / tiles_per_slab);
+            v.w = it < walk.n0 ? 0 : 1;
+            int g1;
+            fused_contributors(plan, v.slab, v.w, G, &v.g0, &g1);
+            v.P = g1 - v.g0;
+            v.r = static_cast<int>(g) - v.g0;
+            return v;
+        };
+        // First half (step 2 above): wait for the slab's partials, sum this CTA's slice, deliver it.
+        auto exchange_slice = [&](int kx) {
+            const Visit vis = visit_of(kx);
+            const int slab = vis.slab, w = vis.w, g0 = vis.g0, P = vis.P, r = vis.r;
             // 1. every contributor's partial is written (P = 1: this CTA's own three draining warps)
             int seen = 1;
             if (lane == 0) seen = counter_wait(&arrive[slab], epoch * static_cast<uint32_t>(P * C::FLUSH_ARRIVALS),
@@ -503,12 +518,18 @@ stream_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 }
             }
             __syncwarp();
-            // 3. every slice of every contributor is in (each of the four warps counts once)
-            if (lane == 0) {
-                red_release_gpu_add(&arrive2[slab], 1u);
+            if (lane == 0) red_release_gpu_add(&arrive2[slab], 1u);  // each of the four warps counts once
+            return true;
+        };
+        // Second half (step 3 above): every slice of every contributor is in; build the operand.
+        auto exchange_operand = [&](int kx) {
+            const Visit vis = visit_of(kx);
+            const int slab = vis.slab, P = vis.P;
+            float4* st4 = reinterpret_cast<float4*>(state + static_cast<size_t>(slab) * kStreamStateFloats);
+            int seen = 1;
+            if (lane == 0)
                 seen = counter_wait(&arrive2[slab], epoch * static_cast<uint32_t>(P * C::SLICE_ARRIVALS),
                                     static_cast<uint32_t>(P * C::SLICE_ARRIVALS)) ? 1 : 0;
-            }
             seen = __shfl_sync(0xffffffffu, seen, 0);
             __syncwarp();
             if (seen == 0) return false;
@@ -551,7 +572,7 @@ stream_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         float acc[64];
 #pragma unroll
         for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
-        int aseg = 0, k = 0, k_x = 0;
+        int aseg = 0, k = 0, k_s = 0, k_x = 0;  // visits drained; with their slice delivered; with their operand built
         bool visit_from_tile0 = walk.unit(0) % tiles_per_slab == 0;
         for (int it = 0; it < n_units && ok;) {
             const long long u = walk.unit(it);
@@ -614,7 +635,7 @@ stream_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&b_ready[k & 1]);
-                k_x = k + 1;
+                k_s = k_x = k + 1;
             } else if (drains) {
                 // partial k of this CTA: row e of S^T (lanes 0..63), z (lane 64)
                 float* dst = partials + (static_cast<size_t>(g) * spans + k) * kStreamStateFloats;
@@ -634,13 +655,16 @@ stream_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             visit_from_tile0 = true;  // the next visit starts a new slab (tile 0) unless it opens a wave's run mid-slab
             if (it < n_units) visit_from_tile0 = walk.unit(it) % tiles_per_slab == 0;
             // Wave 0 is drained and wave 1 is streaming: exchange what fits in the two free buffers now.
-            if (it == walk.n0 && walk.n0 < n_units)
-                while (ok && k_x < k && k_x < 2) ok = exchange(k_x++);
+            if (it == walk.n0 && walk.n0 < n_units) {
+                while (ok && k_s < k) ok = exchange_slice(k_s++);
+                while (ok && k_x < k && k_x < 2) ok = exchange_operand(k_x++);
+            }
             // (cleared after the exchange, so that the sums are not kept alive across it)
 #pragma unroll
             for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
         }
-        while (ok && k_x < k) ok = exchange(k_x++);
+        while (ok && k_s < k) ok = exchange_slice(k_s++);
+        while (ok && k_x < k) ok = exchange_operand(k_x++);
         if (!ok && lane == 0) report_wait_expired(status);
     } else {
         // ---------------- consumer warpgroups ----------------
