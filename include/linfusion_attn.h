@@ -330,6 +330,33 @@ linfusion_status_t linfusion_attn_noalloc_layout(const linfusion_attn_desc_t* de
                                                  int32_t* chunks, size_t* state_offset,
                                                  size_t* bytes_used, size_t* capacity);
 
+/*
+ * The attention fed from the layer input X instead of from Q, K, V (Sec. 3.1, implementation details;
+ * Eq. 2).  In the module, Q = f'(X), K = g'(X) and V = X W_V, with
+ *
+ *     f'(X) = X W_Q + LeakyReLU(LayerNorm(X W_1q + b_1q)),     g'(X) likewise with its own weights:
+ *
+ * a linear branch plus one Linear-LayerNorm-LeakyReLU block, summed.  The entry points below run the
+ * projections on the tensor cores inside the kernels that consume them, so that K, V and Q are never
+ * written to or read from device memory.
+ *
+ * They need a handle with head dim 64 (d_qk = 0), LINFUSION_VARIANT_STREAM and
+ * LINFUSION_LAYOUT_TOKEN_MAJOR (else UNSUPPORTED).  x: device, 16-bit, [B, N, C] with C = H * 64 (the
+ * heads of a token side by side, which is what [B, N, H, d] is).  Every weight matrix: device, 16-bit
+ * (the handle's storage type), [C][C] row-major with row = input channel, column = output channel
+ * (out = x W), 16-byte aligned.
+ *
+ * state_x: S | z of the slabs from X — per 128-token tile and head, [K | V] = X [W_K,h | W_V,h] into
+ * tensor memory, K (+ t_k) through phi, both rounded to 16 bits into shared memory, then the split-N
+ * state accumulation and the fixed-order reduction exactly as in linfusion_attn_state().  t_k (may be
+ * NULL) is the output of g's non-linear branch, LeakyReLU(LayerNorm(X W_1k + b_1k)), 16-bit [B, N, C];
+ * NULL means the branch contributes nothing (the paper's initialization).  Afterwards state_buffer(),
+ * read_state(), apply() and apply_peers() work as after linfusion_attn_state().
+ * Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+linfusion_status_t linfusion_attn_state_x(linfusion_attn_t* h, const void* x, const void* w_k,
+                                          const void* w_v, const void* t_k, void* cuda_stream);
+
 /* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);
 

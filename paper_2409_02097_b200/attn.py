@@ -29,6 +29,7 @@ EXPORTED = [
     "linfusion_attn_forward_noalloc", "linfusion_attn_noalloc_layout",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
     "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait", "linfusion_attn_selftest_counter_wait",
+    "linfusion_attn_state_x",
 ]
 
 
@@ -107,6 +108,8 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_apply_peers.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_void_p), ctypes.c_int32, vp]
     lib.linfusion_attn_state_buffer.restype = st
     lib.linfusion_attn_state_buffer.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
+    lib.linfusion_attn_state_x.restype = st
+    lib.linfusion_attn_state_x.argtypes = [vp, vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -292,6 +295,28 @@ class LinFusionAttention:
         rc = self._lib.linfusion_attn_state(self._h, k.data_ptr(), v.data_ptr(), stream)
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_state")
+
+    # -- fed from the layer input X [B, N, C] and the projection weights [C, C] (x @ w) ------------
+    def _check_x(self, x, weights, extras=()):
+        import torch
+        want = torch.float16 if self.dtype == "fp16" else torch.bfloat16
+        B, H, N, d = self.desc.B, self.desc.H, self.desc.N, self.desc.d
+        C = H * d
+        for t, n, shape in [(x, "x", (B, N, C))] + [(w, "weight", (C, C)) for w in weights] + \
+                           [(t, "branch output", (B, N, C)) for t in extras if t is not None]:
+            if tuple(t.shape) != shape or t.dtype != want or not t.is_contiguous() or not t.is_cuda:
+                raise ValueError(f"{n}: expected contiguous CUDA {self.dtype} tensor of shape {shape}")
+
+    def state_x(self, x, w_k, w_v, t_k=None, stream: Optional[int] = None) -> None:
+        """S | z from the layer input: K = x @ w_k (+ t_k), V = x @ w_v computed inside the kernel."""
+        import torch
+        self._check_x(x, (w_k, w_v), (t_k,))
+        if stream is None:
+            stream = torch.cuda.current_stream(x.device).cuda_stream
+        rc = self._lib.linfusion_attn_state_x(self._h, x.data_ptr(), w_k.data_ptr(), w_v.data_ptr(),
+                                              t_k.data_ptr() if t_k is not None else None, stream)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_state_x")
 
     def apply(self, q, y=None, stream: Optional[int] = None):
         import torch

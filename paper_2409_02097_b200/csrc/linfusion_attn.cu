@@ -12,6 +12,7 @@
 #include "split_kernels.cuh"
 #include "stream_kernels.cuh"
 #include "fused_kernels.cuh"
+#include "producer_kernels.cuh"
 
 using namespace lf;
 
@@ -444,6 +445,9 @@ cudaError_t set_stream_attrs()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(stream_fused_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              FusedCfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(producer_state_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             ProdStateCfg::SMEM_BYTES);
     return e;
 }
 
@@ -1509,5 +1513,98 @@ extern "C" linfusion_status_t linfusion_attn_state_buffer(linfusion_attn_t* h, f
     if (h == nullptr || dev_ptr == nullptr || floats == nullptr) return LINFUSION_ERR_INVALID_ARG;
     *dev_ptr = h->state;
     *floats = static_cast<size_t>(h->plan.slabs) * h->plan.state_floats;
+    return LINFUSION_OK;
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// The attention fed from the layer input X (Sec. 3.1, implementation details; Eq. 2): the
+// projections run inside the kernels that consume their results (producer_kernels.cuh).
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+// X [B, N, C] (16-bit, C = H * 64) -> boxes of 128 tokens x 64 channels, 128-byte swizzle, zero fill past N.
+bool encode_x_map(CUtensorMap* map, const void* x, const linfusion_attn_desc_t& d)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    const cuuint64_t C = static_cast<cuuint64_t>(d.H) * kStreamD;
+    cuuint64_t dims[3] = {C, static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.B)};
+    cuuint64_t strides[2] = {C * 2, static_cast<cuuint64_t>(d.N) * C * 2};
+    cuuint32_t box[3] = {64u, static_cast<cuuint32_t>(ProdStateCfg::TILE), 1u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// W [C_in][C_out] (16-bit, row = input channel) -> boxes of 64 input rows x 64 output columns.
+bool encode_w_map(CUtensorMap* map, const void* w, int C)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(C)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(C) * 2};
+    cuuint32_t box[2] = {64u, 64u};
+    cuuint32_t estr[2] = {1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Handles that can take X: head dim 64 on both sides, the three-launch TMA + tcgen05 plan, and the
+// token-major layout (X and Y are [B, N, C]: the heads of a token side by side).
+bool takes_x(const linfusion_attn* h)
+{
+    return h->plan.variant == kStream && (h->desc.flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u;
+}
+
+template <int KIND>
+cudaError_t launch_state_x(const linfusion_attn* h, const void* x, const void* w_k, const void* w_v, const void* t_k,
+                           cudaStream_t s)
+{
+    const Plan& p = h->plan;
+    const int C = h->desc.H * kStreamD;
+    CUtensorMap mx, mwk, mwv, mt;
+    if (!encode_x_map(&mx, x, h->desc) || !encode_w_map(&mwk, w_k, C) || !encode_w_map(&mwv, w_v, C)) return cudaErrorInvalidValue;
+    if (!encode_slab_map(&mt, t_k != nullptr ? t_k : x, h->desc, ProdStateCfg::TILE)) return cudaErrorInvalidValue;
+    ProducerArgs pa;
+    pa.N = h->desc.N;
+    pa.H = h->desc.H;
+    pa.chunks = C / ProdStateCfg::KC;
+    pa.has_t = t_k != nullptr ? 1 : 0;
+    cudaError_t e = launch_chained(producer_state_kernel<KIND>, dim3(p.G_state), dim3(ProdStateCfg::THREADS),
+                                   ProdStateCfg::SMEM_BYTES, s, mx, mwk, mwv, mt, h->partials, h->status, pa,
+                                   p.tiles_state, p.W_state, p.spans);
+    if (e != cudaSuccess) return e;
+    e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
+                       h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
+                       p.spans, dtype_of(h->desc), operand_scale(h->desc));
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+extern "C" linfusion_status_t linfusion_attn_state_x(linfusion_attn_t* h, const void* x, const void* w_k,
+                                                     const void* w_v, const void* t_k, void* cuda_stream)
+{
+    if (h == nullptr || x == nullptr || w_k == nullptr || w_v == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w_k) || !aligned16(w_v) || !aligned16(t_k)) return LINFUSION_ERR_INVALID_ARG;
+    if (!takes_x(h)) return LINFUSION_ERR_UNSUPPORTED;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV) e = launch_state_x<KV>(h, x, w_k, w_v, t_k, s)
+    LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
+    h->last_stream = s;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
     return LINFUSION_OK;
 }

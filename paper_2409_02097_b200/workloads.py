@@ -117,3 +117,35 @@ def make_small(B: int, H: int, N: int, d: int, seed: int = BASE_SEED, device: st
         q, k, v = (q.float() * scale).bfloat16(), (k.float() * scale).bfloat16(), \
                   (v.float() * scale).bfloat16()
     return q, k, v
+
+
+def make_producer_inputs(B: int, H: int, N: int, d: int, seed: int = BASE_SEED, names=("q", "k", "v"),
+                         device: str = "cpu", dtype=torch.bfloat16, x_mean: float = 0.0):
+    """Layer input and module parameters for the attention fed from X (Sec. 3.1 implementation
+    details; the trained weights the paper uses are not available, these are their stand-ins).
+
+    Returns ``(x, w)``: ``x`` [B, N, C] ~ N(x_mean, 1) with C = H * d, and ``w[name]`` for every name asked
+    for.  A name that starts with "t" gives a [B, N, C] tensor ~ N(0, 0.25) (a stand-in for the output
+    of a non-linear branch); "b..." a bias [C] ~ N(0, 0.25); "g..." a LayerNorm scale [C] ~ N(1, 0.04);
+    "e..." a LayerNorm shift [C] ~ N(0, 0.04); any other name a weight matrix [C, C] (row = input
+    channel) ~ N(0, 1/C), so that x @ w is ~ N(0, 1) per element like the Q, K, V of the other
+    workloads.  Everything is drawn in fp32 from one seeded generator and rounded to ``dtype``."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev)
+    g.manual_seed(int(seed))
+    C = H * d
+    x = (torch.randn((B, N, C), generator=g, device=dev, dtype=torch.float32) + x_mean).to(dtype)
+    w = {}
+    for name in names:
+        if name.startswith("t"):
+            t = 0.5 * torch.randn((B, N, C), generator=g, device=dev, dtype=torch.float32)
+        elif name.startswith("b"):
+            t = 0.5 * torch.randn((C,), generator=g, device=dev, dtype=torch.float32)
+        elif name.startswith("g"):
+            t = 1.0 + 0.2 * torch.randn((C,), generator=g, device=dev, dtype=torch.float32)
+        elif name.startswith("e"):
+            t = 0.2 * torch.randn((C,), generator=g, device=dev, dtype=torch.float32)
+        else:
+            t = torch.randn((C, C), generator=g, device=dev, dtype=torch.float32) / (C ** 0.5)
+        w[name] = t.to(dtype)
+    return x, w
