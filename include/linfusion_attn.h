@@ -356,6 +356,17 @@ linfusion_status_t linfusion_attn_noalloc_layout(const linfusion_attn_desc_t* de
  */
 linfusion_status_t linfusion_attn_state_x(linfusion_attn_t* h, const void* x, const void* w_k,
                                           const void* w_v, const void* t_k, void* cuda_stream);
+/*
+ * apply_x: Y of the local tokens from X and the handle's current state (Prop. 2's output with Eq. 5's
+ * division) — per 128-token tile and head, Q = X W_Q,h into tensor memory, Q (+ t_q) through phi and back
+ * into tensor memory as the A operand of phi(Q) [S | z], rows divided by their denominator, Y tile
+ * stored with TMA.  t_q (may be NULL): output of f's non-linear branch, as t_k above.  y: device, 16-bit,
+ * [B, N, C], written in full; must not overlap x.  The fp32 state is re-read (it may have been summed
+ * over devices since state_x(), Sec. 4.3), so state_x() / all-reduce / apply_x() is the token-sharded
+ * forward from X.  Errors: INVALID_ARG, UNSUPPORTED, CUDA.
+ */
+linfusion_status_t linfusion_attn_apply_x(linfusion_attn_t* h, const void* x, const void* w_q,
+                                          const void* t_q, void* y, void* cuda_stream);
 
 /* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);

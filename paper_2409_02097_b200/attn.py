@@ -29,7 +29,7 @@ EXPORTED = [
     "linfusion_attn_forward_noalloc", "linfusion_attn_noalloc_layout",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
     "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait", "linfusion_attn_selftest_counter_wait",
-    "linfusion_attn_state_x",
+    "linfusion_attn_state_x", "linfusion_attn_apply_x",
 ]
 
 
@@ -110,6 +110,8 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_state_buffer.argtypes = [vp, ctypes.POINTER(vp), ctypes.POINTER(ctypes.c_size_t)]
     lib.linfusion_attn_state_x.restype = st
     lib.linfusion_attn_state_x.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.linfusion_attn_apply_x.restype = st
+    lib.linfusion_attn_apply_x.argtypes = [vp, vp, vp, vp, vp, vp]
     _lib = lib
     return lib
 
@@ -317,6 +319,20 @@ class LinFusionAttention:
                                               t_k.data_ptr() if t_k is not None else None, stream)
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_state_x")
+
+    def apply_x(self, x, w_q, t_q=None, y=None, stream: Optional[int] = None):
+        """Y [B, N, C] from the layer input and the current state: Q = x @ w_q (+ t_q) inside the kernel."""
+        import torch
+        self._check_x(x, (w_q,), (t_q, y))
+        if y is None:
+            y = torch.empty_like(x)
+        if stream is None:
+            stream = torch.cuda.current_stream(x.device).cuda_stream
+        rc = self._lib.linfusion_attn_apply_x(self._h, x.data_ptr(), w_q.data_ptr(),
+                                              t_q.data_ptr() if t_q is not None else None, y.data_ptr(), stream)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_apply_x")
+        return y
 
     def apply(self, q, y=None, stream: Optional[int] = None):
         import torch

@@ -448,6 +448,9 @@ cudaError_t set_stream_attrs()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(producer_state_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              ProdStateCfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(producer_apply_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             ProdApplyCfg::SMEM_BYTES);
     return e;
 }
 
@@ -1584,9 +1587,63 @@ cudaError_t launch_state_x(const linfusion_attn* h, const void* x, const void* w
     return cudaGetLastError();
 }
 
+template <int KIND>
+cudaError_t launch_apply_x(const linfusion_attn* h, const void* x, const void* w_q, const void* t_q, void* y,
+                           cudaStream_t s)
+{
+    const Plan& p = h->plan;
+    const int C = h->desc.H * kStreamD;
+    CUtensorMap mx, mwq, mt, my;
+    if (!encode_x_map(&mx, x, h->desc) || !encode_w_map(&mwq, w_q, C) ||
+        !encode_slab_map(&mt, t_q != nullptr ? t_q : x, h->desc, ProdApplyCfg::TILE) ||
+        !encode_slab_map(&my, y, h->desc, ProdApplyCfg::TILE))
+        return cudaErrorInvalidValue;
+    ProducerArgs pa;
+    pa.N = h->desc.N;
+    pa.H = h->desc.H;
+    pa.chunks = C / ProdApplyCfg::KC;
+    pa.has_t = t_q != nullptr ? 1 : 0;
+    // The fp32 state may have been summed over devices since it was reduced: rebuild its 16-bit image.
+    PeerStates own;
+    own.p[0] = h->state;
+    own.n = 1;
+    cudaError_t e = launch_chained(stream_pack_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
+                                   own, h->operand, h->tile_counters, dtype_of(h->desc), operand_scale(h->desc));
+    if (e != cudaSuccess) return e;
+    e = launch_chained(producer_apply_kernel<KIND>, dim3(p.G_apply), dim3(ProdApplyCfg::THREADS),
+                       ProdApplyCfg::SMEM_BYTES, s, mx, mwq, mt, my, h->operand, h->status, pa, p.tiles_apply,
+                       p.W_apply, apply_scales(h->desc));
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 }  // namespace
+
+extern "C" linfusion_status_t linfusion_attn_apply_x(linfusion_attn_t* h, const void* x, const void* w_q,
+                                                     const void* t_q, void* y, void* cuda_stream)
+{
+    if (h == nullptr || x == nullptr || w_q == nullptr || y == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w_q) || !aligned16(t_q) || !aligned16(y)) return LINFUSION_ERR_INVALID_ARG;
+    if (!takes_x(h)) return LINFUSION_ERR_UNSUPPORTED;
+    const uintptr_t px = reinterpret_cast<uintptr_t>(x), py = reinterpret_cast<uintptr_t>(y);
+    const size_t bytes = bytes_vy(h->desc);
+    if (px < py + bytes && py < px + bytes) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV) e = launch_apply_x<KV>(h, x, w_q, t_q, y, s)
+    LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
+    h->last_stream = s;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
 
 extern "C" linfusion_status_t linfusion_attn_state_x(linfusion_attn_t* h, const void* x, const void* w_k,
                                                      const void* w_v, const void* t_k, void* cuda_stream)

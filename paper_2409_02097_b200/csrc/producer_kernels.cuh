@@ -383,4 +383,316 @@ producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
 }
 
+struct ProdApplyCfg {
+    static constexpr int TILE = 128;
+    static constexpr int KC = 64;
+    static constexpr int STAGES = 4;
+    static constexpr int X_BYTES = TILE * 128;     // 16 KB
+    static constexpr int W_BYTES = KC * 128;       // 8 KB: 64 input rows x 64 Q columns
+    static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
+    static constexpr int Y_BYTES = TILE * 128;     // per epilogue group: T tile in, Y tile out
+    static constexpr int B_ROWS = StreamApplyCfg::B_ROWS;
+    static constexpr int B_BYTES = StreamApplyCfg::B_BYTES;  // S^T | z operand image, two buffers
+    static constexpr int EPI_GROUPS = 2;
+    static constexpr int EPI_WARPS = 4 * EPI_GROUPS;
+    static constexpr int PRODUCER_WARP = EPI_WARPS;
+    static constexpr int MMA_WARP = EPI_WARPS + 1;
+    static constexpr int STORE_WARP = EPI_WARPS + 2;
+    static constexpr int THREADS = 32 * (EPI_WARPS + 3);
+    static constexpr int TMEM_COLS = 512;
+    static constexpr int TMEM_PER_GROUP = 256;  // projection accumulator 64 | phi(Q) operand 32 | output accumulator 80
+    static constexpr int TMEM_A = 64, TMEM_D2 = 96;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_GROUPS * Y_BYTES + 2 * B_BYTES + 1024 + 1024;
+};
+static_assert((ProdApplyCfg::STAGES * ProdApplyCfg::STAGE_BYTES + ProdApplyCfg::EPI_GROUPS * ProdApplyCfg::Y_BYTES) % 1024 == 0 &&
+                  ProdApplyCfg::B_BYTES % 1024 == 0 && ProdApplyCfg::STAGE_BYTES % 1024 == 0,
+              "operands on 1024-byte boundaries");
+static_assert(ProdApplyCfg::SMEM_BYTES > 116 * 1024 && ProdApplyCfg::SMEM_BYTES <= 227 * 1024, "one CTA per SM");
+
+// Y of the slabs from X and the reduced state: CTA g of G owns the contiguous run of (slab, tile)
+// units [g*W/G, (g+1)*W/G).  A run is a sequence of slab VISITS; visit k's operand image S^T | z
+// goes to shared-memory buffer k & 1.
+template <int KIND>
+__global__ void __launch_bounds__(ProdApplyCfg::THREADS, 1)
+producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_wq,
+                      const __grid_constant__ CUtensorMap tmap_t, const __grid_constant__ CUtensorMap tmap_y,
+                      const unsigned char* __restrict__ operand, uint32_t* __restrict__ status, ProducerArgs pa,
+                      int tiles_per_slab, long long W, ApplyScales sc)
+{
+    using C = ProdApplyCfg;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    unsigned char* ybuf = smem + C::STAGES * C::STAGE_BYTES;
+    unsigned char* bsm = ybuf + C::EPI_GROUPS * C::Y_BYTES;
+    uint64_t* full = reinterpret_cast<uint64_t*>(bsm + 2 * C::B_BYTES);
+    uint64_t* empty = full + C::STAGES;
+    uint64_t* d1_done = empty + C::STAGES;  // [2] projection accumulator complete
+    uint64_t* d1_free = d1_done + 2;        // [2] read by its epilogue
+    uint64_t* t_full = d1_free + 2;         // [2] T tile landed in the group's tile buffer
+    uint64_t* a_ready = t_full + 2;         // [2] phi(Q) rows in tensor memory
+    uint64_t* d2_done = a_ready + 2;        // [2] output accumulator complete
+    uint64_t* y_ready = d2_done + 2;        // [2] Y tile in the group's tile buffer
+    uint64_t* y_free = y_ready + 2;         // [2] the store has read it
+    uint64_t* b_ready = y_free + 2;         // [2] operand image of the visit in shared memory
+    uint64_t* b_free = b_ready + 2;         // [2] the MMAs that read it are complete
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b_free + 2);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long G = gridDim.x, g = blockIdx.x;
+    const long long u0 = unit_begin(g, W, G), u1 = unit_begin(g + 1, W, G);
+    const int n_units = static_cast<int>(u1 - u0);
+    const int KCH = pa.chunks;
+
+    if (tid == 0) {
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&d1_done[b], 1);
+            mbar_init(&d1_free[b], 4);
+            mbar_init(&t_full[b], 1);
+            mbar_init(&a_ready[b], 4);
+            mbar_init(&d2_done[b], 1);
+            mbar_init(&y_ready[b], 4);
+            mbar_init(&y_free[b], 1);
+            mbar_init(&b_ready[b], 1);
+            mbar_init(&b_free[b], 1);
+        }
+        mbar_fence_init();
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    if (warp == C::PRODUCER_WARP && lane == 0) {
+        prefetch_tmap(&tmap_x);
+        prefetch_tmap(&tmap_wq);
+        if (pa.has_t != 0) prefetch_tmap(&tmap_t);
+    }
+    if (warp == C::STORE_WARP && lane == 0) prefetch_tmap(&tmap_y);
+    pdl_launch_dependents();
+    pdl_wait();
+
+    if (warp == C::PRODUCER_WARP) {
+        // ---------------- producer warp (lane 0 issues TMA; all lanes copy the operand image) ----------------
+        uint64_t pol_x = 0, pol_w = 0;
+        if (lane == 0) {
+            pol_x = policy_evict_first();
+            pol_w = policy_evict_last();
+        }
+        bool ok = true;
+        int issued = 0, visit = -1, cur_slab = -1;
+        for (int it = 0; it < n_units && ok; ++it) {
+            const long long u = u0 + it;
+            const int slab = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
+            const int b = slab / pa.H, h = slab % pa.H, e = it & 1, n = it >> 1;
+            if (lane == 0) {
+                for (int kc = 0; kc < KCH; ++kc) {
+                    const int c = it * KCH + kc, s = c % C::STAGES;
+                    ok = mbar_wait(&empty[s], ((c / C::STAGES) & 1) ^ 1);
+                    if (!ok) break;
+                    unsigned char* dst = smem + s * C::STAGE_BYTES;
+                    mbar_expect_tx(&full[s], C::STAGE_BYTES);
+                    tma_load_3d(dst, &tmap_x, kc * C::KC, tile * C::TILE, b, &full[s], pol_x);
+                    tma_load_2d(dst + C::X_BYTES, &tmap_wq, h * 64, kc * C::KC, &full[s], pol_w);
+                    ++issued;
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+            if (!ok) break;
+            if (slab != cur_slab) {
+                // A new visit: its operand image, after the unit's own loads are on their way (the MMA
+                // thread frees the buffer of two visits back only once it reaches the visit before this one).
+                cur_slab = slab;
+                ++visit;
+                if (visit >= 2) {
+                    if (lane == 0) ok = mbar_wait(&b_free[visit & 1], ((visit >> 1) - 1) & 1);
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                    if (!ok) break;
+                }
+                const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
+                uint4* dst = reinterpret_cast<uint4*>(bsm + (visit & 1) * C::B_BYTES);
+                for (int i = lane; i < C::B_BYTES / 16; i += 32) dst[i] = __ldg(src + i);
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&b_ready[visit & 1]);
+            }
+            if (pa.has_t != 0 && lane == 0) {
+                // T tile into the group's tile buffer, once the store of two units back has read it
+                if (n >= 1) ok = mbar_wait(&y_free[e], (n - 1) & 1);
+                if (ok) {
+                    mbar_expect_tx(&t_full[e], C::Y_BYTES);
+                    tma_load_4d(ybuf + e * C::Y_BYTES, &tmap_t, 0, tile * C::TILE, h, b, &t_full[e], pol_x);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        }
+        if (lane == 0) {
+            if (!ok) report_wait_expired(status);
+            drain_loads<C::STAGES>(full, 0, issued, status);
+        }
+    } else if (warp == C::MMA_WARP) {
+        // ---------------- MMA warp ----------------
+        if (lane == 0) {
+            const uint32_t idesc1 = umma_idesc_f32acc(kind_dtype(KIND), 128, 64, kUmmaBMnMajor);
+            const uint32_t idesc2 = umma_idesc_f32acc(kind_dtype(KIND), C::TILE, C::B_ROWS);
+            bool ok = true;
+            int visit = -1, cur_slab = -1;
+            uint64_t b_desc = 0;
+            // Output MMAs of unit j: D2 = phi(Q) [S | z].
+            auto apply_mma = [&](int j) {
+                const int e = j & 1;
+                const int slab = static_cast<int>((u0 + j) / tiles_per_slab);
+                if (slab != cur_slab) {
+                    if (visit >= 0) umma_commit(&b_free[visit & 1]);  // the visit before: all its MMAs are issued
+                    ++visit;
+                    cur_slab = slab;
+                    if (!mbar_wait(&b_ready[visit & 1], (visit >> 1) & 1)) return false;
+                    b_desc = umma_desc_kmajor_sw128(smem_u32(bsm + (visit & 1) * C::B_BYTES));
+                }
+                if (!mbar_wait(&a_ready[e], (j >> 1) & 1)) return false;
+                tc_fence_after_sync();
+                const uint32_t a_tmem = tmem_base + e * C::TMEM_PER_GROUP + C::TMEM_A;
+                const uint32_t d_tmem = tmem_base + e * C::TMEM_PER_GROUP + C::TMEM_D2;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) umma_ts(d_tmem, a_tmem + 8 * k, b_desc + 2 * k, idesc2, k > 0 ? 1u : 0u);
+                umma_commit(&d2_done[e]);
+                return true;
+            };
+            for (int it = 0; it < n_units && ok; ++it) {
+                const int e = it & 1;
+                if (it >= 2) ok = mbar_wait(&d1_free[e], ((it >> 1) - 1) & 1);
+                if (!ok) break;
+                const uint32_t d1 = tmem_base + e * C::TMEM_PER_GROUP;
+                for (int kc = 0; kc < KCH; ++kc) {
+                    const int c = it * KCH + kc, s = c % C::STAGES;
+                    ok = mbar_wait(&full[s], (c / C::STAGES) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t x_addr = smem_u32(smem + s * C::STAGE_BYTES), w_addr = x_addr + C::X_BYTES;
+                    const uint64_t a_desc = umma_desc_kmajor_sw128(x_addr);
+#pragma unroll
+                    for (int k = 0; k < C::KC / 16; ++k) {
+                        const uint64_t w_desc = umma_desc_mnmajor_sw128(w_addr + k * 2048, 0, 1024);
+                        umma_ss(d1, a_desc + 2 * k, w_desc, idesc1, (kc == 0 && k == 0) ? 0u : 1u);
+                    }
+                    umma_commit(&empty[s]);
+                }
+                if (!ok) break;
+                umma_commit(&d1_done[e]);
+                if (it >= 1) ok = apply_mma(it - 1);
+            }
+            if (ok && n_units > 0) ok = apply_mma(n_units - 1);
+            if (!ok) report_wait_expired(status);
+        }
+    } else if (warp == C::STORE_WARP) {
+        // ---------------- store warp ----------------
+        if (lane == 0) {
+            const uint64_t policy = policy_evict_first();
+            for (int it = 0; it < n_units; ++it) {
+                const int e = it & 1;
+                if (!mbar_wait(&y_ready[e], (it >> 1) & 1)) {
+                    report_wait_expired(status);
+                    break;
+                }
+                const long long u = u0 + it;
+                const int slab = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
+                tma_store_4d(&tmap_y, ybuf + e * C::Y_BYTES, 0, tile * C::TILE, slab % pa.H, slab / pa.H, policy);
+                tma_store_wait_read();
+                mbar_arrive(&y_free[e]);
+            }
+            tma_store_wait_all();
+        }
+    } else {
+        // ---------------- epilogue warpgroups: group e takes units e, e + 2, ... ----------------
+        const int e = warp >> 2, wq = warp & 3;
+        const int row = wq * 32 + lane;
+        const uint32_t sw = row & 7;
+        const uint32_t t_base = tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + e * C::TMEM_PER_GROUP;
+        const uint32_t y_row = smem_u32(ybuf + e * C::Y_BYTES) + row * 128;
+        bool ok = true;
+        for (int it = e; it < n_units; it += 2) {
+            const int n = it >> 1;
+            ok = mbar_wait(&d1_done[e], n & 1);
+            if (ok && pa.has_t != 0) ok = mbar_wait(&t_full[e], n & 1);
+            __syncwarp();
+            if (!ok) break;
+            tc_fence_after_sync();
+            {
+                // Q row (+ T row), phi in fp32, rounded: the row of the output MMA's A operand
+                uint32_t a[32];
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t d[32];
+                    tmem_load_32cols(t_base + 32 * half, d);
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float f[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(d[8 * c + i]);
+                        if (pa.has_t != 0) {
+                            uint32_t t0, t1, t2, t3;
+                            asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];"
+                                         : "=r"(t0), "=r"(t1), "=r"(t2), "=r"(t3)
+                                         : "r"(y_row + (((4 * half + c) ^ sw) << 4)));
+                            f[0] += pair_lo<KIND>(t0); f[1] += pair_hi<KIND>(t0);
+                            f[2] += pair_lo<KIND>(t1); f[3] += pair_hi<KIND>(t1);
+                            f[4] += pair_lo<KIND>(t2); f[5] += pair_hi<KIND>(t2);
+                            f[6] += pair_lo<KIND>(t3); f[7] += pair_hi<KIND>(t3);
+                        }
+#pragma unroll
+                        for (int i = 0; i < 4; ++i)
+                            a[16 * half + 4 * c + i] = pack_pair<KIND>(phi<KIND>(f[2 * i]), phi<KIND>(f[2 * i + 1]));
+                    }
+                }
+                tmem_store_32cols(t_base + C::TMEM_A, a);
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&d1_free[e]);
+                mbar_arrive(&a_ready[e]);
+            }
+            ok = mbar_wait(&d2_done[e], n & 1);
+            // without a T tile nobody has waited yet for the store of two units back to let go of the buffer
+            if (ok && pa.has_t == 0 && n >= 1) ok = mbar_wait(&y_free[e], (n - 1) & 1);
+            __syncwarp();
+            if (!ok) break;
+            tc_fence_after_sync();
+            const float den = __uint_as_float(tmem_load_1col(t_base + C::TMEM_D2 + 64));  // phi(Q_i) . z
+            const float inv = row_scale(den, sc);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t d[32];
+                tmem_load_32cols(t_base + C::TMEM_D2 + 32 * half, d);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t v0 = pack_pair<KIND>(__uint_as_float(d[8 * c + 0]) * inv, __uint_as_float(d[8 * c + 1]) * inv);
+                    const uint32_t v1 = pack_pair<KIND>(__uint_as_float(d[8 * c + 2]) * inv, __uint_as_float(d[8 * c + 3]) * inv);
+                    const uint32_t v2 = pack_pair<KIND>(__uint_as_float(d[8 * c + 4]) * inv, __uint_as_float(d[8 * c + 5]) * inv);
+                    const uint32_t v3 = pack_pair<KIND>(__uint_as_float(d[8 * c + 6]) * inv, __uint_as_float(d[8 * c + 7]) * inv);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(y_row + (((4 * half + c) ^ sw) << 4)),
+                                 "r"(v0), "r"(v1), "r"(v2), "r"(v3)
+                                 : "memory");
+                }
+            }
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&y_ready[e]);
+        }
+        if (!ok && lane == 0) report_wait_expired(status);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+
 }  // namespace lf

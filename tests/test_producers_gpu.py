@@ -50,3 +50,34 @@ def test_state_from_x_matches_the_oracle(shape):
         S, z = op.read_state()
         assert np.array_equal(S, S2) and np.array_equal(z, z2), "not bit-reproducible"
     op.close()
+
+
+def _module_oracle(x, w, H, t_q=None, t_k=None):
+    """Q = X W_q (+ T_q), K = X W_k (+ T_k), V = X W_v, heads split, attention, heads merged: [B, N, C]."""
+    xf = to_f64(x)
+    q = oracle.linear_map(xf, to_f64(w["q"])) + (to_f64(t_q) if t_q is not None else 0.0)
+    k = oracle.linear_map(xf, to_f64(w["k"])) + (to_f64(t_k) if t_k is not None else 0.0)
+    v = oracle.linear_map(xf, to_f64(w["v"]))
+    y = oracle.linear(oracle.split_heads(q, H), oracle.split_heads(k, H), oracle.split_heads(v, H), EPS)
+    return y  # [B, H, N, d]
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=lambda s: "x".join(map(str, s)))
+def test_state_then_apply_from_x_matches_the_oracle(shape):
+    B, H, N = shape
+    for x_mean in (0.0, 0.5):
+        x, w = wl.make_producer_inputs(B, H, N, 64, seed=93, names=("q", "k", "v", "tq", "tk"), device="cuda",
+                                       x_mean=x_mean)
+        op = attn.LinFusionAttention(B, H, N, 64, eps=EPS, variant="stream", layout="token_major")
+        for t_q, t_k in ((None, None), (w["tq"], w["tk"])):
+            ref = _module_oracle(x, w, H, t_q, t_k)
+            op.state_x(x, w["k"], w["v"], t_k)
+            y = op.apply_x(x, w["q"], t_q)
+            torch.cuda.synchronize()
+            assert op.status() == attn.OK
+            y_bhnd = y.view(B, N, H, 64).permute(0, 2, 1, 3)
+            assert_parity(y_bhnd, ref, f"{shape} x_mean={x_mean} branches={t_q is not None}")
+            y2 = op.apply_x(x, w["q"], t_q)
+            torch.cuda.synchronize()
+            assert torch.equal(y, y2), "not bit-reproducible"
+        op.close()
