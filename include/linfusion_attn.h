@@ -368,6 +368,49 @@ linfusion_status_t linfusion_attn_state_x(linfusion_attn_t* h, const void* x, co
 linfusion_status_t linfusion_attn_apply_x(linfusion_attn_t* h, const void* x, const void* w_q,
                                           const void* t_q, void* y, void* cuda_stream);
 
+/*
+ * branch_x: the output of one non-linear branch, T = LeakyReLU(LayerNorm(X W_1 + b_1; gamma, beta)), into
+ * t_out [B, N, C] (device, 16-bit, must not overlap x).  w_1: [C][C] as the other weights; b_1 (may be
+ * NULL: no bias), gamma, beta: [C], 16-bit.  LayerNorm runs over a token's whole feature vector (all
+ * heads), biased variance, ln_eps inside the root; leaky_slope is LeakyReLU's negative slope.  Two
+ * launches: the projection on the tensor cores, which also leaves every row's mean and
+ * 1 / sqrt(variance + ln_eps) (sums taken in fp32 before U is rounded to 16 bits), and the
+ * element-wise normalization in place.  The first call on a handle allocates the row-statistics
+ * buffer (8 bytes per token; freed by destroy()).  C <= 2048.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALLOC, CUDA.
+ */
+linfusion_status_t linfusion_attn_branch_x(linfusion_attn_t* h, const void* x, const void* w_1,
+                                           const void* b_1, const void* gamma, const void* beta,
+                                           float ln_eps, float leaky_slope, void* t_out,
+                                           void* cuda_stream);
+
+/* The parameters of f' or g': out = x w_lin + LeakyReLU(LayerNorm(x w_1 + b_1; gamma, beta)). */
+typedef struct {
+    const void* w_lin; /* [C][C] linear branch (initialized from W_Q / W_K in the paper)     */
+    const void* w_1;   /* [C][C] the block's Linear; NULL: the non-linear branch is absent   */
+    const void* b_1;   /* [C] its bias; may be NULL                                          */
+    const void* gamma; /* [C] LayerNorm scale                                                */
+    const void* beta;  /* [C] LayerNorm shift                                                */
+} linfusion_mlp_weights_t;
+
+typedef struct {
+    linfusion_mlp_weights_t q; /* f' */
+    linfusion_mlp_weights_t k; /* g' */
+    const void* w_v;           /* [C][C], Eq. 2 */
+    float ln_eps;              /* LayerNorm's epsilon          */
+    float leaky_slope;         /* LeakyReLU's negative slope   */
+} linfusion_module_weights_t;
+
+/*
+ * forward_x: the whole module from the layer input, Y = attention(f'(X), g'(X), X W_V): the non-linear
+ * branches that are present (branch_x into buffers of B*N*C*2 bytes each that the handle allocates on
+ * first use and frees in destroy()), then state_x and apply_x.  x, y: [B, N, C] as above.
+ * Errors: INVALID_ARG, UNSUPPORTED, ALLOC, CUDA.
+ */
+linfusion_status_t linfusion_attn_forward_x(linfusion_attn_t* h, const void* x,
+                                            const linfusion_module_weights_t* w, void* y,
+                                            void* cuda_stream);
+
 /* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);
 

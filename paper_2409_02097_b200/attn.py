@@ -29,7 +29,7 @@ EXPORTED = [
     "linfusion_attn_forward_noalloc", "linfusion_attn_noalloc_layout",
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
     "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait", "linfusion_attn_selftest_counter_wait",
-    "linfusion_attn_state_x", "linfusion_attn_apply_x",
+    "linfusion_attn_state_x", "linfusion_attn_apply_x", "linfusion_attn_branch_x", "linfusion_attn_forward_x",
 ]
 
 
@@ -38,6 +38,18 @@ class Desc(ctypes.Structure):
     _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("N", ctypes.c_int32),
                 ("d", ctypes.c_int32), ("phi", ctypes.c_int32), ("eps", ctypes.c_float),
                 ("device", ctypes.c_int32), ("flags", ctypes.c_uint32), ("d_qk", ctypes.c_int32)]
+
+
+class MlpWeights(ctypes.Structure):
+    """Mirror of ``linfusion_mlp_weights_t``."""
+    _fields_ = [("w_lin", ctypes.c_void_p), ("w_1", ctypes.c_void_p), ("b_1", ctypes.c_void_p),
+                ("gamma", ctypes.c_void_p), ("beta", ctypes.c_void_p)]
+
+
+class ModuleWeights(ctypes.Structure):
+    """Mirror of ``linfusion_module_weights_t``."""
+    _fields_ = [("q", MlpWeights), ("k", MlpWeights), ("w_v", ctypes.c_void_p),
+                ("ln_eps", ctypes.c_float), ("leaky_slope", ctypes.c_float)]
 
 
 class LinFusionError(RuntimeError):
@@ -112,6 +124,10 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_state_x.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.linfusion_attn_apply_x.restype = st
     lib.linfusion_attn_apply_x.argtypes = [vp, vp, vp, vp, vp, vp]
+    lib.linfusion_attn_branch_x.restype = st
+    lib.linfusion_attn_branch_x.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, vp]
+    lib.linfusion_attn_forward_x.restype = st
+    lib.linfusion_attn_forward_x.argtypes = [vp, vp, ctypes.POINTER(ModuleWeights), vp, vp]
     _lib = lib
     return lib
 
@@ -319,6 +335,42 @@ class LinFusionAttention:
                                               t_k.data_ptr() if t_k is not None else None, stream)
         if rc != OK:
             raise LinFusionError(rc, "linfusion_attn_state_x")
+
+    def branch_x(self, x, w_1, b_1, gamma, beta, ln_eps=1e-5, slope=0.01, t_out=None, stream: Optional[int] = None):
+        """T = LeakyReLU(LayerNorm(x @ w_1 + b_1; gamma, beta)) [B, N, C]: one non-linear branch of f' / g'."""
+        import torch
+        self._check_x(x, (w_1,), (t_out,))
+        if t_out is None:
+            t_out = torch.empty_like(x)
+        if stream is None:
+            stream = torch.cuda.current_stream(x.device).cuda_stream
+        rc = self._lib.linfusion_attn_branch_x(self._h, x.data_ptr(), w_1.data_ptr(),
+                                               b_1.data_ptr() if b_1 is not None else None, gamma.data_ptr(),
+                                               beta.data_ptr(), float(ln_eps), float(slope), t_out.data_ptr(), stream)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_branch_x")
+        return t_out
+
+    def forward_x(self, x, weights: dict, ln_eps=1e-5, slope=0.01, y=None, stream: Optional[int] = None):
+        """The module from the layer input.  ``weights``: q_lin, k_lin, v ([C, C]) and, for each
+        non-linear branch that is present, q_w1 / q_b1 / q_gamma / q_beta (and k_...)."""
+        import torch
+        self._check_x(x, (weights["q_lin"], weights["k_lin"], weights["v"]), (y,))
+        if y is None:
+            y = torch.empty_like(x)
+        if stream is None:
+            stream = torch.cuda.current_stream(x.device).cuda_stream
+        ptr = lambda name: weights[name].data_ptr() if weights.get(name) is not None else None
+        mw = ModuleWeights()
+        for side, name in ((mw.q, "q"), (mw.k, "k")):
+            side.w_lin, side.w_1, side.b_1 = ptr(name + "_lin"), ptr(name + "_w1"), ptr(name + "_b1")
+            side.gamma, side.beta = ptr(name + "_gamma"), ptr(name + "_beta")
+        mw.w_v, mw.ln_eps, mw.leaky_slope = ptr("v"), float(ln_eps), float(slope)
+        self._weights_alive = weights
+        rc = self._lib.linfusion_attn_forward_x(self._h, x.data_ptr(), ctypes.byref(mw), y.data_ptr(), stream)
+        if rc != OK:
+            raise LinFusionError(rc, "linfusion_attn_forward_x")
+        return y
 
     def apply_x(self, x, w_q, t_q=None, y=None, stream: Optional[int] = None):
         """Y [B, N, C] from the layer input and the current state: Q = x @ w_q (+ t_q) inside the kernel."""

@@ -354,6 +354,10 @@ struct linfusion_attn {
     long long forward_calls;  // forwards since timing was enabled
     bool sample_now;          // the forward being enqueued is one of them
     struct HostPipe* pipe;  // copy/compute pipeline of the host-buffer entry point (first use)
+    // forward_x(): row statistics of the non-linear branches' LayerNorm and the branches' outputs
+    // T_q, T_k (allocated on first use)
+    float* x_stats;
+    void* x_t[2];
 };
 
 // forward_host() cuts the slabs into groups and overlaps the upload of group i+1, the kernels of
@@ -451,6 +455,9 @@ cudaError_t set_stream_attrs()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(producer_apply_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              ProdApplyCfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(producer_hidden_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             ProdHiddenCfg::SMEM_BYTES);
     return e;
 }
 
@@ -707,6 +714,8 @@ linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linf
     h->forward_calls = 0;
     h->sample_now = false;
     h->pipe = nullptr;
+    h->x_stats = nullptr;
+    h->x_t[0] = h->x_t[1] = nullptr;
     st = make_plan(desc, h->sm_count, &h->plan);
     if (st != LINFUSION_OK) {
         delete h;
@@ -1118,6 +1127,9 @@ linfusion_status_t linfusion_attn_destroy(linfusion_attn_t* h)
         if (h->owns_ws && h->ws != nullptr && cudaFree(h->ws) != cudaSuccess) st = LINFUSION_ERR_CUDA;
         for (int i = 0; i < 4; ++i)
             if (h->stage[i] != nullptr && cudaFree(h->stage[i]) != cudaSuccess) st = LINFUSION_ERR_CUDA;
+        if (h->x_stats != nullptr && cudaFree(h->x_stats) != cudaSuccess) st = LINFUSION_ERR_CUDA;
+        for (int i = 0; i < 2; ++i)
+            if (h->x_t[i] != nullptr && cudaFree(h->x_t[i]) != cudaSuccess) st = LINFUSION_ERR_CUDA;
         if (h->events != nullptr) {
             for (int i = 0; i < h->timing_slots * 4; ++i) cudaEventDestroy(h->events[i]);
             delete[] h->events;
@@ -1347,6 +1359,8 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     view.forward_calls = 0;
     view.sample_now = false;
     view.pipe = nullptr;
+    view.x_stats = nullptr;
+    view.x_t[0] = view.x_t[1] = nullptr;
 
     cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
     const __nv_bfloat16* Q = static_cast<const __nv_bfloat16*>(q);
@@ -1617,9 +1631,110 @@ cudaError_t launch_apply_x(const linfusion_attn* h, const void* x, const void* w
     return cudaGetLastError();
 }
 
+// T = LeakyReLU(LayerNorm(X W_1 + b_1; gamma, beta)) into `t` [B, N, C].
+template <int KIND>
+cudaError_t launch_branch_x(const linfusion_attn* h, const void* x, const void* w_1, const void* b_1, const void* gamma,
+                            const void* beta, float ln_eps, float slope, void* t, cudaStream_t s)
+{
+    const int C = h->desc.H * kStreamD, N = h->desc.N, B = h->desc.B;
+    CUtensorMap mx, mw, mu;
+    if (!encode_x_map(&mx, x, h->desc) || !encode_w_map(&mw, w_1, C) || !encode_x_map(&mu, t, h->desc)) return cudaErrorInvalidValue;
+    const int tiles = (N + ProdHiddenCfg::TILE - 1) / ProdHiddenCfg::TILE;
+    const long long W = static_cast<long long>(B) * tiles;
+    const int G = static_cast<int>(W < h->sm_count ? W : h->sm_count);
+    cudaError_t e = launch_chained(producer_hidden_kernel<KIND>, dim3(G), dim3(ProdHiddenCfg::THREADS),
+                                   ProdHiddenCfg::SMEM_BYTES, s, mx, mw, mu, static_cast<const __nv_bfloat16*>(b_1),
+                                   h->x_stats, h->status, N, C, tiles, W, ln_eps);
+    if (e != cudaSuccess) return e;
+    const long long rows = static_cast<long long>(B) * N, total = rows * (C / 8);
+    long long blocks = (total + 255) / 256;
+    if (blocks > 8ll * 148 * 8) blocks = 8ll * 148 * 8;
+    e = launch_chained(producer_norm_kernel<KIND>, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, s,
+                       static_cast<__nv_bfloat16*>(t), static_cast<const float*>(h->x_stats),
+                       static_cast<const __nv_bfloat16*>(gamma), static_cast<const __nv_bfloat16*>(beta), rows, C, slope);
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Row statistics buffer of the branches' LayerNorm, on first use.
+linfusion_status_t ensure_x_stats(linfusion_attn* h)
+{
+    if (h->x_stats != nullptr) return LINFUSION_OK;
+    void* p = nullptr;
+    if (cudaMalloc(&p, static_cast<size_t>(h->desc.B) * h->desc.N * 2 * sizeof(float)) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_ALLOC;
+    }
+    h->x_stats = static_cast<float*>(p);
+    return LINFUSION_OK;
+}
+
 }  // namespace
+
+extern "C" linfusion_status_t linfusion_attn_branch_x(linfusion_attn_t* h, const void* x, const void* w_1,
+                                                      const void* b_1, const void* gamma, const void* beta,
+                                                      float ln_eps, float leaky_slope, void* t_out,
+                                                      void* cuda_stream)
+{
+    if (h == nullptr || x == nullptr || w_1 == nullptr || gamma == nullptr || beta == nullptr || t_out == nullptr)
+        return LINFUSION_ERR_INVALID_ARG;
+    if (!aligned16(x) || !aligned16(w_1) || !aligned16(gamma) || !aligned16(beta) || !aligned16(t_out) ||
+        (reinterpret_cast<uintptr_t>(b_1) & 1u) != 0)
+        return LINFUSION_ERR_INVALID_ARG;
+    if (!std::isfinite(ln_eps) || ln_eps < 0.0f || !std::isfinite(leaky_slope)) return LINFUSION_ERR_INVALID_ARG;
+    if (!takes_x(h)) return LINFUSION_ERR_UNSUPPORTED;
+    if (h->desc.H * kStreamD > ProdHiddenCfg::MAX_C) return LINFUSION_ERR_UNSUPPORTED;
+    const uintptr_t px = reinterpret_cast<uintptr_t>(x), pt = reinterpret_cast<uintptr_t>(t_out);
+    const size_t bytes = bytes_vy(h->desc);
+    if (px < pt + bytes && pt < px + bytes) return LINFUSION_ERR_INVALID_ARG;
+    DeviceGuard guard(h->desc.device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    linfusion_status_t st = ensure_x_stats(h);
+    if (st != LINFUSION_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV) e = launch_branch_x<KV>(h, x, w_1, b_1, gamma, beta, ln_eps, leaky_slope, t_out, s)
+    LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
+    h->last_stream = s;
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    return LINFUSION_OK;
+}
+
+extern "C" linfusion_status_t linfusion_attn_forward_x(linfusion_attn_t* h, const void* x,
+                                                       const linfusion_module_weights_t* w, void* y,
+                                                       void* cuda_stream)
+{
+    if (h == nullptr || x == nullptr || w == nullptr || y == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    if (w->q.w_lin == nullptr || w->k.w_lin == nullptr || w->w_v == nullptr) return LINFUSION_ERR_INVALID_ARG;
+    if (!takes_x(h)) return LINFUSION_ERR_UNSUPPORTED;
+    const linfusion_mlp_weights_t* br[2] = {&w->q, &w->k};
+    const void* t[2] = {nullptr, nullptr};
+    for (int i = 0; i < 2; ++i) {
+        if (br[i]->w_1 == nullptr) continue;  // the branch is absent: it contributes nothing
+        if (h->x_t[i] == nullptr) {
+            DeviceGuard guard(h->desc.device);
+            if (!guard.ok) return LINFUSION_ERR_CUDA;
+            if (cudaMalloc(&h->x_t[i], bytes_vy(h->desc)) != cudaSuccess) {
+                cudaGetLastError();
+                h->x_t[i] = nullptr;
+                return LINFUSION_ERR_ALLOC;
+            }
+        }
+        linfusion_status_t st = linfusion_attn_branch_x(h, x, br[i]->w_1, br[i]->b_1, br[i]->gamma, br[i]->beta,
+                                                        w->ln_eps, w->leaky_slope, h->x_t[i], cuda_stream);
+        if (st != LINFUSION_OK) return st;
+        t[i] = h->x_t[i];
+    }
+    linfusion_status_t st = linfusion_attn_state_x(h, x, w->k.w_lin, w->w_v, t[1], cuda_stream);
+    if (st != LINFUSION_OK) return st;
+    return linfusion_attn_apply_x(h, x, w->q.w_lin, t[0], y, cuda_stream);
+}
 
 extern "C" linfusion_status_t linfusion_attn_apply_x(linfusion_attn_t* h, const void* x, const void* w_q,
                                                      const void* t_q, void* y, void* cuda_stream)

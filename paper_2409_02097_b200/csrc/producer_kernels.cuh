@@ -28,6 +28,8 @@
 // Every wait is bounded.
 #pragma once
 
+#include <cuda_fp16.h>
+
 #include "stream_kernels.cuh"
 
 namespace lf {
@@ -691,6 +693,291 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     if (warp == 0) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+
+// 3-D tiled TMA store (x = channel, y = token, z = batch), clipped at the tensor's extents.
+__device__ __forceinline__ void tma_store_3d(const void* tmap, const void* smem_src, int x, int y, int z,
+                                             uint64_t cache_policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group.L2::cache_hint [%0, {%1, %2, %3}], [%4], %5;"
+        ::"l"(tmap), "r"(x), "r"(y), "r"(z), "r"(smem_u32(smem_src)), "l"(cache_policy)
+        : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+// ---------------------------------------------------------------------------------------------
+// The non-linear branch of f' / g' (Sec. 3.1, implementation details): T = LeakyReLU(LayerNorm(X W_1 + b_1)).
+// LayerNorm runs over a token's whole feature vector, so it is taken in two steps:
+//   producer_hidden_kernel — U = X W_1 + b_1 on tcgen05, 128 tokens x 128 output columns at a time,
+//                            rounded to 16 bits and stored by TMA; the thread that owns a token row
+//                            sums u and u^2 (fp32, before rounding) over all its column blocks and
+//                            leaves the row's mean and 1 / sqrt(variance + ln_eps);
+//   producer_norm_kernel   — T = LeakyReLU((U - mean) * rstd * gamma + beta), elementwise, in place.
+// ---------------------------------------------------------------------------------------------
+struct ProdHiddenCfg {
+    static constexpr int TILE = 128;
+    static constexpr int KC = 64;
+    static constexpr int NB_COLS = 128;              // output columns per block
+    static constexpr int STAGES = 4;
+    static constexpr int X_BYTES = TILE * 128;
+    static constexpr int W_BYTES = 2 * KC * 128;     // two 64-column boxes
+    static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
+    static constexpr int OUT_BYTES = 2 * TILE * 128;  // 128 rows x (64 | 64) columns
+    static constexpr int MAX_C = 2048;
+    static constexpr int EPI_WARPS = 4;
+    static constexpr int PRODUCER_WARP = EPI_WARPS;
+    static constexpr int MMA_WARP = EPI_WARPS + 1;
+    static constexpr int STORE_WARP = EPI_WARPS + 2;
+    static constexpr int THREADS = 32 * (EPI_WARPS + 3);
+    static constexpr int TMEM_COLS = 256;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_BYTES + MAX_C * 4 + 1024 + 1024;
+};
+static_assert(ProdHiddenCfg::SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+// grid: CTA g of G owns token tiles [g*W/G, (g+1)*W/G) of the W = B * tiles tiles.  stats: [B*N][2] fp32.
+template <int KIND>
+__global__ void __launch_bounds__(ProdHiddenCfg::THREADS, 1)
+producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w1,
+                       const __grid_constant__ CUtensorMap tmap_u, const __nv_bfloat16* __restrict__ bias,
+                       float* __restrict__ stats, uint32_t* __restrict__ status, int N, int Cdim, int tiles_per_batch,
+                       long long W, float ln_eps)
+{
+    using C = ProdHiddenCfg;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    unsigned char* outb = smem + C::STAGES * C::STAGE_BYTES;
+    float* bias_s = reinterpret_cast<float*>(outb + 2 * C::OUT_BYTES);
+    uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(bias_s) + C::MAX_C * 4);
+    uint64_t* empty = full + C::STAGES;
+    uint64_t* d1_done = empty + C::STAGES;  // [2]
+    uint64_t* d1_free = d1_done + 2;        // [2]
+    uint64_t* out_ready = d1_free + 2;      // [2]
+    uint64_t* out_free = out_ready + 2;     // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_free + 2);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long G = gridDim.x, g = blockIdx.x;
+    const long long u0 = unit_begin(g, W, G), u1 = unit_begin(g + 1, W, G);
+    const int n_units = static_cast<int>(u1 - u0);
+    const int KCH = Cdim / C::KC;
+    const int NB = (Cdim + C::NB_COLS - 1) / C::NB_COLS;
+    const int n_blocks = n_units * NB;  // (tile, column block) pairs of this CTA, in order
+
+    if (tid == 0) {
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&d1_done[b], 1);
+            mbar_init(&d1_free[b], 4);
+            mbar_init(&out_ready[b], 4);
+            mbar_init(&out_free[b], 1);
+        }
+        mbar_fence_init();
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    if (warp == C::PRODUCER_WARP && lane == 0) {
+        prefetch_tmap(&tmap_x);
+        prefetch_tmap(&tmap_w1);
+    }
+    if (warp == C::STORE_WARP && lane == 0) prefetch_tmap(&tmap_u);
+    pdl_launch_dependents();
+    pdl_wait();
+    // the bias as fp32, for every role that wants it (zero when there is none)
+    for (int i = tid; i < Cdim; i += C::THREADS)
+        bias_s[i] = bias != nullptr ? (kind_dtype(KIND) == kDtypeFp16 ? __half2float(reinterpret_cast<const __half*>(bias)[i])
+                                                                    : __bfloat162float(bias[i]))
+                                    : 0.0f;
+    __syncthreads();
+
+    if (warp == C::PRODUCER_WARP) {
+        if (lane == 0) {
+            const uint64_t pol_x = policy_evict_first(), pol_w = policy_evict_last();
+            bool ok = true;
+            int issued = 0;
+            for (int j = 0; j < n_blocks && ok; ++j) {
+                const long long u = u0 + j / NB;
+                const int nb = j % NB;
+                const int b = static_cast<int>(u / tiles_per_batch), tile = static_cast<int>(u % tiles_per_batch);
+                for (int kc = 0; kc < KCH; ++kc) {
+                    const int c = j * KCH + kc, s = c % C::STAGES;
+                    ok = mbar_wait(&empty[s], ((c / C::STAGES) & 1) ^ 1);
+                    if (!ok) break;
+                    unsigned char* dst = smem + s * C::STAGE_BYTES;
+                    mbar_expect_tx(&full[s], C::STAGE_BYTES);
+                    tma_load_3d(dst, &tmap_x, kc * C::KC, tile * C::TILE, b, &full[s], pol_x);
+                    // (the second box of an odd last block lies past the last column: zero fill)
+                    tma_load_2d(dst + C::X_BYTES, &tmap_w1, nb * C::NB_COLS, kc * C::KC, &full[s], pol_w);
+                    tma_load_2d(dst + C::X_BYTES + C::KC * 128, &tmap_w1, nb * C::NB_COLS + 64, kc * C::KC, &full[s], pol_w);
+                    ++issued;
+                }
+            }
+            if (!ok) report_wait_expired(status);
+            drain_loads<C::STAGES>(full, 0, issued, status);
+        }
+    } else if (warp == C::MMA_WARP) {
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), 128, 128, kUmmaBMnMajor);
+            bool ok = true;
+            for (int j = 0; j < n_blocks && ok; ++j) {
+                const int e = j & 1;
+                if (j >= 2) ok = mbar_wait(&d1_free[e], ((j >> 1) - 1) & 1);
+                if (!ok) break;
+                const uint32_t d1 = tmem_base + e * 128;
+                for (int kc = 0; kc < KCH; ++kc) {
+                    const int c = j * KCH + kc, s = c % C::STAGES;
+                    ok = mbar_wait(&full[s], (c / C::STAGES) & 1);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint32_t x_addr = smem_u32(smem + s * C::STAGE_BYTES), w_addr = x_addr + C::X_BYTES;
+                    const uint64_t a_desc = umma_desc_kmajor_sw128(x_addr);
+#pragma unroll
+                    for (int k = 0; k < C::KC / 16; ++k) {
+                        const uint64_t b_desc = umma_desc_mnmajor_sw128(w_addr + k * 2048, C::KC * 128, 1024);
+                        umma_ss(d1, a_desc + 2 * k, b_desc, idesc, (kc == 0 && k == 0) ? 0u : 1u);
+                    }
+                    umma_commit(&empty[s]);
+                }
+                if (!ok) break;
+                umma_commit(&d1_done[e]);
+            }
+            if (!ok) report_wait_expired(status);
+        }
+    } else if (warp == C::STORE_WARP) {
+        if (lane == 0) {
+            const uint64_t policy = policy_evict_last();  // read again soon by the normalization
+            for (int j = 0; j < n_blocks; ++j) {
+                const int e = j & 1;
+                if (!mbar_wait(&out_ready[e], (j >> 1) & 1)) {
+                    report_wait_expired(status);
+                    break;
+                }
+                const long long u = u0 + j / NB;
+                const int nb = j % NB;
+                const int b = static_cast<int>(u / tiles_per_batch), tile = static_cast<int>(u % tiles_per_batch);
+                tma_store_3d(&tmap_u, outb + e * C::OUT_BYTES, nb * C::NB_COLS, tile * C::TILE, b, policy);
+                if (nb * C::NB_COLS + 64 < Cdim)
+                    tma_store_3d(&tmap_u, outb + e * C::OUT_BYTES + C::TILE * 128, nb * C::NB_COLS + 64, tile * C::TILE, b, policy);
+                tma_store_wait_read();
+                mbar_arrive(&out_free[e]);
+            }
+            tma_store_wait_all();
+        }
+    } else {
+        // ---------------- epilogue warpgroup: thread r owns token row r of every tile ----------------
+        const int wq = warp & 3;
+        const int row = wq * 32 + lane;
+        const uint32_t sw = row & 7;
+        float sum = 0.0f, sq = 0.0f;
+        bool ok = true;
+        for (int j = 0; j < n_blocks; ++j) {
+            const int e = j & 1, nb = j % NB;
+            ok = mbar_wait(&d1_done[e], (j >> 1) & 1);
+            if (ok && j >= 2) ok = mbar_wait(&out_free[e], ((j >> 1) - 1) & 1);
+            __syncwarp();
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + e * 128;
+            const uint32_t o_row = smem_u32(outb + e * C::OUT_BYTES) + row * 128;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                // columns 32 q .. + 31 of the block: half q / 2 of the staging tile, chunks 4 (q % 2) ..
+                uint32_t d[32];
+                tmem_load_32cols(t_row + 32 * q, d);
+                const int col0 = nb * C::NB_COLS + 32 * q;
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    float f[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int col = col0 + 8 * c + i;
+                        f[i] = 0.0f;
+                        if (col < Cdim) {
+                            f[i] = __uint_as_float(d[8 * c + i]) + bias_s[col];
+                            sum += f[i];
+                            sq += f[i] * f[i];
+                        }
+                    }
+                    const uint32_t addr = o_row + (q >> 1) * (C::TILE * 128) + (((4 * (q & 1) + c) ^ sw) << 4);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(pack_pair<KIND>(f[0], f[1])),
+                                 "r"(pack_pair<KIND>(f[2], f[3])), "r"(pack_pair<KIND>(f[4], f[5])),
+                                 "r"(pack_pair<KIND>(f[6], f[7]))
+                                 : "memory");
+                }
+            }
+            tc_fence_before_sync();
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(&d1_free[e]);
+                mbar_arrive(&out_ready[e]);
+            }
+            if (nb == NB - 1) {
+                // the row is complete: mean and 1 / sqrt(biased variance + ln_eps) over its Cdim features
+                const long long u = u0 + j / NB;
+                const int b = static_cast<int>(u / tiles_per_batch), tile = static_cast<int>(u % tiles_per_batch);
+                const int tok = tile * C::TILE + row;
+                if (tok < N) {
+                    const float mean = sum / static_cast<float>(Cdim);
+                    const float var = fmaxf(sq / static_cast<float>(Cdim) - mean * mean, 0.0f);
+                    float2* dst = reinterpret_cast<float2*>(stats) + static_cast<size_t>(b) * N + tok;
+                    *dst = make_float2(mean, rsqrtf(var + ln_eps));
+                }
+                sum = 0.0f;
+                sq = 0.0f;
+            }
+        }
+        if (!ok && lane == 0) report_wait_expired(status);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// T = LeakyReLU((U - mean) * rstd * gamma + beta), in place over t [rows][Cdim] (16-bit), eight
+// channels per thread; stats [rows][2] = (mean, rstd) per row.
+template <int KIND>
+__global__ void __launch_bounds__(256)
+producer_norm_kernel(__nv_bfloat16* __restrict__ t, const float* __restrict__ stats,
+                     const __nv_bfloat16* __restrict__ gamma, const __nv_bfloat16* __restrict__ beta, long long rows,
+                     int Cdim, float slope)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int vecs = Cdim / 8;
+    const long long total = rows * vecs;
+    for (long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x; i < total;
+         i += static_cast<long long>(gridDim.x) * blockDim.x) {
+        const long long row = i / vecs;
+        const int c8 = static_cast<int>(i - row * vecs);
+        const float2 st = __ldg(reinterpret_cast<const float2*>(stats) + row);
+        uint4* p = reinterpret_cast<uint4*>(t + row * Cdim) + c8;
+        const uint4 u = *p;
+        const uint4 gm = __ldg(reinterpret_cast<const uint4*>(gamma) + c8);
+        const uint4 bt = __ldg(reinterpret_cast<const uint4*>(beta) + c8);
+        const uint32_t uu[4] = {u.x, u.y, u.z, u.w}, gg[4] = {gm.x, gm.y, gm.z, gm.w}, bb[4] = {bt.x, bt.y, bt.z, bt.w};
+        uint32_t out[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            float lo = (pair_lo<KIND>(uu[k]) - st.x) * st.y * pair_lo<KIND>(gg[k]) + pair_lo<KIND>(bb[k]);
+            float hi = (pair_hi<KIND>(uu[k]) - st.x) * st.y * pair_hi<KIND>(gg[k]) + pair_hi<KIND>(bb[k]);
+            lo = lo >= 0.0f ? lo : slope * lo;
+            hi = hi >= 0.0f ? hi : slope * hi;
+            out[k] = pack_pair<KIND>(lo, hi);
+        }
+        *p = make_uint4(out[0], out[1], out[2], out[3]);
     }
 }
 

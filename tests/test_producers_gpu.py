@@ -81,3 +81,69 @@ def test_state_then_apply_from_x_matches_the_oracle(shape):
             torch.cuda.synchronize()
             assert torch.equal(y, y2), "not bit-reproducible"
         op.close()
+
+
+MODULE_NAMES = ("q_lin", "q_w1", "b_q", "g_q", "e_q", "k_lin", "k_w1", "b_k", "g_k", "e_k", "v")
+
+
+def _module_weights(B, H, N, seed, x_mean=0.0):
+    x, w = wl.make_producer_inputs(B, H, N, 64, seed=seed, names=MODULE_NAMES, device="cuda", x_mean=x_mean)
+    w = dict(w)
+    for side in ("q", "k"):
+        w[f"{side}_b1"], w[f"{side}_gamma"], w[f"{side}_beta"] = w.pop(f"b_{side}"), w.pop(f"g_{side}"), w.pop(f"e_{side}")
+    return x, w
+
+
+@pytest.mark.parametrize("shape", [(1, 2, 1), (2, 3, 129), (1, 5, 300), (2, 10, 520)], ids=lambda s: "x".join(map(str, s)))
+def test_non_linear_branch_matches_the_oracle(shape):
+    """T = LeakyReLU(LayerNorm(X W_1 + b_1)): C = 128 (one column block), 192 (an odd half block), 320, 640."""
+    B, H, N = shape
+    x, w = _module_weights(B, H, N, seed=95, x_mean=0.25)
+    op = attn.LinFusionAttention(B, H, N, 64, eps=EPS, variant="stream", layout="token_major")
+    f = to_f64
+    for slope in (0.01, 0.5):
+        pre = oracle.linear_map(f(x), f(w["k_w1"]), f(w["k_b1"]))
+        nrm = oracle.layernorm(pre, f(w["k_gamma"]), f(w["k_beta"]), oracle.LN_EPS)
+        ref = np.where(nrm >= 0.0, nrm, slope * nrm)
+        t = op.branch_x(x, w["k_w1"], w["k_b1"], w["k_gamma"], w["k_beta"], oracle.LN_EPS, slope)
+        torch.cuda.synchronize()
+        assert op.status() == attn.OK
+        diff = np.abs(f(t) - ref)
+        # U is rounded to 16 bits before it is normalized and T after: two unit roundoffs of 2^-8 on values of
+        # order 1 (|T| <= ~4), plus the fp32 statistics
+        assert diff.max() <= 3e-2 and diff.mean() <= 3e-3, (shape, slope, diff.max(), diff.mean())
+        assert np.linalg.norm(diff) <= 6e-3 * np.linalg.norm(ref), (shape, slope)
+    # no bias
+    ref0 = oracle.layernorm(oracle.linear_map(f(x), f(w["k_w1"])), f(w["k_gamma"]), f(w["k_beta"]), oracle.LN_EPS)
+    ref0 = np.where(ref0 >= 0.0, ref0, 0.01 * ref0)
+    t0 = op.branch_x(x, w["k_w1"], None, w["k_gamma"], w["k_beta"], oracle.LN_EPS, 0.01)
+    torch.cuda.synchronize()
+    assert np.linalg.norm(f(t0) - ref0) <= 6e-3 * np.linalg.norm(ref0)
+    op.close()
+
+
+@pytest.mark.parametrize("shape", [(2, 2, 129), (1, 5, 300), (2, 10, 1000)], ids=lambda s: "x".join(map(str, s)))
+def test_whole_module_from_x_matches_the_oracle(shape):
+    B, H, N = shape
+    x, w = _module_weights(B, H, N, seed=97, x_mean=0.25)
+    ref = oracle.linfusion_from_x(to_f64(x), {k: to_f64(v) for k, v in w.items()}, H, EPS)   # [B, N, C]
+    ref = oracle.split_heads(ref, H)
+    op = attn.LinFusionAttention(B, H, N, 64, eps=EPS, variant="stream", layout="token_major")
+    y = op.forward_x(x, w, oracle.LN_EPS, oracle.LEAKY_SLOPE)
+    torch.cuda.synchronize()
+    assert op.status() == attn.OK
+    assert_parity(y.view(B, N, H, 64).permute(0, 2, 1, 3), ref, f"module {shape}")
+    y2 = op.forward_x(x, w, oracle.LN_EPS, oracle.LEAKY_SLOPE)
+    torch.cuda.synchronize()
+    assert torch.equal(y, y2)
+    # the paper's initialization: zero scale and shift => the module is the plain projections
+    w0 = dict(w)
+    for side in ("q", "k"):
+        w0[f"{side}_gamma"] = torch.zeros_like(w[f"{side}_gamma"])
+        w0[f"{side}_beta"] = torch.zeros_like(w[f"{side}_beta"])
+    y0 = op.forward_x(x, w0, oracle.LN_EPS, oracle.LEAKY_SLOPE)
+    w_lin_only = {"q_lin": w["q_lin"], "k_lin": w["k_lin"], "v": w["v"]}
+    y_lin = op.forward_x(x, w_lin_only)
+    torch.cuda.synchronize()
+    assert torch.equal(y0, y_lin)
+    op.close()
