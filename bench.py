@@ -592,6 +592,103 @@ def run_sweep(args):
             torch.cuda.empty_cache()
 
 
+def measured_tensor_peaks():
+    """(burst, sustained) dense bf16 TFLOP/s from MEASURED_PEAKS.json, else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["bf16_tflops"]), float(d["bf16_tflops_sustained"]), "measured"
+    except Exception:
+        return 1590.0, 1400.0, "fallback"
+
+
+def run_from_x(args):
+    """The module fed from the layer input X (projections fused into the state and apply kernels),
+    one JSON line per shape: each kernel's time and tensor-core rate, the whole forward with and
+    without the non-linear branches, and beside it the un-fused route — Q, K, V from a library GEMM
+    (torch.matmul), written to and read back from device memory, then the attention kernels."""
+    import torch
+    from paper_2409_02097_b200 import attn, build, workloads as wl
+
+    build.build_library()
+    torch.cuda.set_device(0)
+    burst, sustained, kind = measured_tensor_peaks()
+    names = ("q_lin", "q_w1", "b_q", "g_q", "e_q", "k_lin", "k_w1", "b_k", "g_k", "e_k", "v")
+    shapes = [wl.find_shape(n) for n in (args.only.split(",") if args.only else
+                                         ["sdxl_2048_L1", "sdxl_2048_L2", "sdxl_16k_L2", "sdxl_16k_L1"])]
+    for s in shapes:
+        assert s.d == 64
+        B, H, N, C = s.B, s.H, s.N, s.C
+        x, w = wl.make_producer_inputs(B, H, N, 64, seed=wl.BASE_SEED, names=names, device="cuda:0")
+        w = dict(w)
+        for side in ("q", "k"):
+            w[f"{side}_b1"], w[f"{side}_gamma"], w[f"{side}_beta"] = w.pop(f"b_{side}"), w.pop(f"g_{side}"), w.pop(f"e_{side}")
+        w_lin = {"q_lin": w["q_lin"], "k_lin": w["k_lin"], "v": w["v"]}
+        op = attn.LinFusionAttention(B, H, N, 64, device=0, variant="stream", layout="token_major")
+        y = torch.empty_like(x)
+        t = torch.empty_like(x)
+        tokens = B * N
+        steps = max(5, min(args.steps, int(4e13 // (tokens * 10 * C * C))))
+
+        def timed(fn):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(steps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / steps
+
+        ms_state = timed(lambda: op.state_x(x, w["k_lin"], w["v"]))
+        ms_apply = timed(lambda: op.apply_x(x, w["q_lin"], None, y))
+        ms_branch = timed(lambda: op.branch_x(x, w["k_w1"], w["k_b1"], w["k_gamma"], w["k_beta"], 1e-5, 0.01, t))
+        ms_lin = timed(lambda: op.forward_x(x, w_lin, y=y))
+        ms_full = timed(lambda: op.forward_x(x, w, y=y))
+        assert op.status() == attn.OK
+        # un-fused: library GEMMs produce Q, K, V in device memory, then the three attention kernels
+        q = torch.empty_like(x)
+        k = torch.empty_like(x)
+        v = torch.empty_like(x)
+        x2 = x.view(B * N, C)
+
+        def unfused():
+            torch.matmul(x2, w["q_lin"], out=q.view(B * N, C))
+            torch.matmul(x2, w["k_lin"], out=k.view(B * N, C))
+            torch.matmul(x2, w["v"], out=v.view(B * N, C))
+            op.forward(q.view(B, N, H, 64), k.view(B, N, H, 64), v.view(B, N, H, 64), y.view(B, N, H, 64))
+        ms_unfused = timed(unfused)
+        ms_gemm = timed(lambda: torch.matmul(x2, w["v"], out=v.view(B * N, C)))
+        proj = 2.0 * tokens * C * C             # flops of one C x C projection
+        attn_half = 2.0 * tokens * C * 64       # flops of the state (or the apply) contraction
+        tf = lambda flops, ms: flops / (ms * 1e-3) / 1e12
+        line = {
+            "mode": "from_x", "shape": s.name, "B": B, "H": H, "N": N, "C": C, "dtype": "bf16", "steps": steps,
+            "peak_tflops": {"burst": burst, "sustained": sustained, "kind": "of " + kind},
+            "kernels": {
+                "producer_state_kernel+reduce": {"ms": ms_state, "tflops": tf(2 * proj + attn_half, ms_state)},
+                "pack+producer_apply_kernel": {"ms": ms_apply, "tflops": tf(proj + attn_half, ms_apply)},
+                "producer_hidden_kernel+norm (one branch)": {"ms": ms_branch, "tflops": tf(proj, ms_branch)},
+            },
+            "forward_x_linear_branches": {"ms": ms_lin, "tflops": tf(3 * proj + 2 * attn_half, ms_lin),
+                                          "tokens_per_s": tokens / (ms_lin * 1e-3)},
+            "forward_x_with_non_linear_branches": {"ms": ms_full, "tflops": tf(5 * proj + 2 * attn_half, ms_full),
+                                                   "tokens_per_s": tokens / (ms_full * 1e-3)},
+            "unfused_library_gemm_then_attention": {"ms": ms_unfused, "tokens_per_s": tokens / (ms_unfused * 1e-3),
+                                                    "one_library_gemm_ms": ms_gemm, "one_library_gemm_tflops": tf(proj, ms_gemm)},
+            "roofline": {"bound": "tensor", "kernel": "producer_state_kernel", "achieved": tf(2 * proj + attn_half, ms_state),
+                         "peak": sustained, "peak_kind": "of " + kind + " (sustained bf16)", "unit": "TFLOP/s",
+                         "frac": tf(2 * proj + attn_half, ms_state) / sustained, "traffic": None},
+        }
+        print(json.dumps(line), flush=True)
+        op.close()
+        del x, w, y, t, q, k, v
+        torch.cuda.empty_cache()
+
+
 def main(argv=None):
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -613,9 +710,13 @@ def main(argv=None):
                     help="storage type of Q, K, V, Y (the headline number is bf16)")
     ap.add_argument("--sweep", action="store_true",
                     help="time every shape of the five workload families with every variant")
-    ap.add_argument("--only", default="", help="with --sweep: restrict to one shape, e.g. sd15_512_L1")
+    ap.add_argument("--only", default="", help="with --sweep / --from-x: restrict to one shape, e.g. sd15_512_L1")
+    ap.add_argument("--from-x", action="store_true",
+                    help="time the module fed from the layer input X (fused projections) beside the un-fused route")
     argv = sys.argv[1:] if argv is None else argv
     args = ap.parse_args(argv)
+    if args.from_x:
+        return run_from_x(args)
     if args.sweep:
         run_sweep(args)
     elif maybe_relaunch(args, argv):
