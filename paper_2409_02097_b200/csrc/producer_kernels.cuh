@@ -53,6 +53,56 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, in
         "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(cache_policy)
         : "memory");
 }
+// Position in a ring of STAGES stages: stage index and the parity of its current use.  The K loops
+// below run on one thread each (the TMA issuer, the MMA issuer); at four MMAs per chunk the thread's
+// own instruction stream sets the pace, so the loops carry running positions and descriptors instead
+// of recomputing them (no divisions, no descriptor assembly per chunk).
+template <int STAGES>
+struct RingPos {
+    int s = 0;
+    uint32_t phase = 0;
+    __device__ __forceinline__ void next()
+    {
+        if (++s == STAGES) {
+            s = 0;
+            phase ^= 1u;
+        }
+    }
+};
+// mbar_wait on a shared-memory address that is already 32-bit.
+__device__ __forceinline__ bool mbar_wait_addr(uint32_t addr, uint32_t parity)
+{
+    if (mbar_try_wait(addr, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    do {
+        if (mbar_try_wait(addr, parity)) return true;
+    } while (global_timer_ns() - t0 < kMaxBarrierWaitNs);
+    return false;
+}
+__device__ __forceinline__ void mbar_expect_tx_addr(uint32_t addr, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(addr), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void umma_commit_addr(uint32_t addr)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(addr) : "memory");
+}
+// TMA loads with shared-memory addresses already 32-bit.
+__device__ __forceinline__ void tma_load_3d_addr(uint32_t dst, const void* tmap, int x, int y, int z, uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(z), "r"(bar), "l"(policy)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_addr(uint32_t dst, const void* tmap, int x, int y, uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;" ::"r"(dst), "l"(tmap), "r"(x), "r"(y), "r"(bar), "l"(policy)
+        : "memory");
+}
+
 __device__ __forceinline__ uint64_t policy_evict_last()
 {
     uint64_t p;
@@ -72,9 +122,10 @@ struct ProdStateCfg {
     static constexpr int EPI_GROUPS = 2;
     static constexpr int EPI_WARPS = 4 * EPI_GROUPS;  // warps 0..7: warp % 4 = the TMEM lane quarter
     static constexpr int FLUSH_WARP0 = EPI_WARPS;      // warps 8, 9, 10 = lane quarters 0, 1, 2
-    static constexpr int PRODUCER_WARP = EPI_WARPS + 3;
+    static constexpr int PRODUCER_WARP = EPI_WARPS + 3;   // X chunks (and T tiles)
     static constexpr int MMA_WARP = EPI_WARPS + 4;
-    static constexpr int THREADS = 32 * (EPI_WARPS + 5);
+    static constexpr int WPRODUCER_WARP = EPI_WARPS + 5;  // W chunks: two issuing threads halve the issue time per chunk
+    static constexpr int THREADS = 32 * (EPI_WARPS + 6);
     static constexpr int SEGMENT_TILES = 32;
     static constexpr int TMEM_COLS = 512;   // [0,256): two projection accumulators; [256,384): two state accumulators
     static constexpr int TMEM_STATE0 = 256;
@@ -125,7 +176,7 @@ producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
-            mbar_init(&full[s], 1);
+            mbar_init(&full[s], 2);  // the X and the W issuer each announce their bytes
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -151,32 +202,54 @@ producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const uint32_t tmem_base = *tmem_slot;
     if (warp == C::PRODUCER_WARP && lane == 0) {
         prefetch_tmap(&tmap_x);
+        if (pa.has_t != 0) prefetch_tmap(&tmap_t);
+    }
+    if (warp == C::WPRODUCER_WARP && lane == 0) {
         prefetch_tmap(&tmap_wk);
         prefetch_tmap(&tmap_wv);
-        if (pa.has_t != 0) prefetch_tmap(&tmap_t);
     }
     pdl_launch_dependents();
     pdl_wait();
 
-    if (warp == C::PRODUCER_WARP) {
-        // ---------------- producer ----------------
+    if (warp == C::WPRODUCER_WARP) {
+        // ---------------- W producer: the weight chunks of every unit ----------------
         if (lane == 0) {
-            const uint64_t pol_x = policy_evict_first(), pol_w = policy_evict_last();
+            const uint64_t pol_w = policy_evict_last();
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), w0 = smem_u32(smem) + C::X_BYTES;
+            RingPos<C::STAGES> r;
+            bool ok = true;
+            for (int it = 0; it < n_units && ok; ++it) {
+                const int h64 = static_cast<int>(((u0 + it) / tiles_per_slab) % pa.H) * 64;
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
+                    if (!ok) break;
+                    const uint32_t dst = w0 + r.s * C::STAGE_BYTES, bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::W_BYTES);
+                    tma_load_2d_addr(dst, &tmap_wk, h64, kc * C::KC, bar, pol_w);
+                    tma_load_2d_addr(dst + C::KC * 128, &tmap_wv, h64, kc * C::KC, bar, pol_w);
+                }
+            }
+            if (!ok) report_wait_expired(status);
+        }
+    } else if (warp == C::PRODUCER_WARP) {
+        // ---------------- X producer (its drain at the end covers the W loads too: a stage's
+        // `full` phase completes only when both issuers' bytes have landed) ----------------
+        if (lane == 0) {
+            const uint64_t pol_x = policy_evict_first();
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), x0 = smem_u32(smem);
+            RingPos<C::STAGES> r;
             bool ok = true;
             int issued = 0;
             for (int it = 0; it < n_units && ok; ++it) {
                 const long long u = u0 + it;
                 const int slab = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
                 const int b = slab / pa.H, h = slab % pa.H;
-                for (int kc = 0; kc < KCH; ++kc) {
-                    const int c = it * KCH + kc, s = c % C::STAGES;
-                    ok = mbar_wait(&empty[s], ((c / C::STAGES) & 1) ^ 1);
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
                     if (!ok) break;
-                    unsigned char* dst = smem + s * C::STAGE_BYTES;
-                    mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                    tma_load_3d(dst, &tmap_x, kc * C::KC, tile * C::TILE, b, &full[s], pol_x);
-                    tma_load_2d(dst + C::X_BYTES, &tmap_wk, h * 64, kc * C::KC, &full[s], pol_w);
-                    tma_load_2d(dst + C::X_BYTES + C::KC * 128, &tmap_wv, h * 64, kc * C::KC, &full[s], pol_w);
+                    const uint32_t bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::X_BYTES);
+                    tma_load_3d_addr(x0 + r.s * C::STAGE_BYTES, &tmap_x, kc * C::KC, tile * C::TILE, b, bar, pol_x);
                     ++issued;
                 }
                 if (ok && pa.has_t != 0) {
@@ -227,26 +300,29 @@ producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 umma_commit(&kv_free[e]);
                 return true;
             };
+            // Descriptors of stage 0; a stage further on adds STAGE_BYTES / 16 to the address field.  A: the X
+            // chunk, K-major, one K step = 32 bytes.  B: the W chunk, 16 input rows per K step (2048
+            // bytes), its two 64-column blocks (K, V) 8 KB apart.
+            const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
+            const uint64_t b_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, C::KC * 128, 1024);
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty);
+            RingPos<C::STAGES> r;
             for (int it = 0; it < n_units && ok; ++it) {
                 const int e = it & 1;
                 // the accumulator's previous epilogue (two units back) must have read it
                 if (it >= 2) ok = mbar_wait(&d1_free[e], ((it >> 1) - 1) & 1);
                 if (!ok) break;
                 const uint32_t d1 = tmem_base + e * 128;
-                for (int kc = 0; kc < KCH; ++kc) {
-                    const int c = it * KCH + kc, s = c % C::STAGES;
-                    ok = mbar_wait(&full[s], (c / C::STAGES) & 1);
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(full0 + 8 * r.s, r.phase);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t x_addr = smem_u32(smem + s * C::STAGE_BYTES), w_addr = x_addr + C::X_BYTES;
-                    const uint64_t a_desc = umma_desc_kmajor_sw128(x_addr);
+                    const uint64_t step = static_cast<uint64_t>(r.s * (C::STAGE_BYTES >> 4));
+                    const uint64_t a_desc = a_desc0 + step, b_desc = b_desc0 + step;
+                    umma_ss(d1, a_desc, b_desc, idesc1, kc > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 0; k < C::KC / 16; ++k) {
-                        // B: 16 input rows from k*2048; its two 64-column blocks (K, V) are 8 KB apart
-                        const uint64_t b_desc = umma_desc_mnmajor_sw128(w_addr + k * 2048, C::KC * 128, 1024);
-                        umma_ss(d1, a_desc + 2 * k, b_desc, idesc1, (kc == 0 && k == 0) ? 0u : 1u);
-                    }
-                    umma_commit(&empty[s]);
+                    for (int k = 1; k < C::KC / 16; ++k) umma_ss(d1, a_desc + 2 * k, b_desc + 128 * k, idesc1, 1u);
+                    umma_commit_addr(empty0 + 8 * r.s);
                 }
                 if (!ok) break;
                 umma_commit(&d1_done[e]);
@@ -388,7 +464,9 @@ producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 struct ProdApplyCfg {
     static constexpr int TILE = 128;
     static constexpr int KC = 64;
-    static constexpr int STAGES = 4;
+    // The K loop is bound by the bytes in flight per SM (ring size / load round trip of ~1.4 us), not
+    // by L2 bandwidth or the tensor pipe: as many stages as shared memory holds.
+    static constexpr int STAGES = 7;
     static constexpr int X_BYTES = TILE * 128;     // 16 KB
     static constexpr int W_BYTES = KC * 128;       // 8 KB: 64 input rows x 64 Q columns
     static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
@@ -400,7 +478,8 @@ struct ProdApplyCfg {
     static constexpr int PRODUCER_WARP = EPI_WARPS;
     static constexpr int MMA_WARP = EPI_WARPS + 1;
     static constexpr int STORE_WARP = EPI_WARPS + 2;
-    static constexpr int THREADS = 32 * (EPI_WARPS + 3);
+    static constexpr int WPRODUCER_WARP = EPI_WARPS + 3;  // W chunks (the producer warp issues the X chunks)
+    static constexpr int THREADS = 32 * (EPI_WARPS + 4);
     static constexpr int TMEM_COLS = 512;
     static constexpr int TMEM_PER_GROUP = 256;  // projection accumulator 64 | phi(Q) operand 32 | output accumulator 80
     static constexpr int TMEM_A = 64, TMEM_D2 = 96;
@@ -448,7 +527,7 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
-            mbar_init(&full[s], 1);
+            mbar_init(&full[s], 2);  // the X and the W issuer each announce their bytes
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -471,20 +550,39 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const uint32_t tmem_base = *tmem_slot;
     if (warp == C::PRODUCER_WARP && lane == 0) {
         prefetch_tmap(&tmap_x);
-        prefetch_tmap(&tmap_wq);
         if (pa.has_t != 0) prefetch_tmap(&tmap_t);
     }
+    if (warp == C::WPRODUCER_WARP && lane == 0) prefetch_tmap(&tmap_wq);
     if (warp == C::STORE_WARP && lane == 0) prefetch_tmap(&tmap_y);
     pdl_launch_dependents();
     pdl_wait();
 
-    if (warp == C::PRODUCER_WARP) {
-        // ---------------- producer warp (lane 0 issues TMA; all lanes copy the operand image) ----------------
-        uint64_t pol_x = 0, pol_w = 0;
+    if (warp == C::WPRODUCER_WARP) {
+        // ---------------- W producer: the weight chunks of every unit ----------------
         if (lane == 0) {
-            pol_x = policy_evict_first();
-            pol_w = policy_evict_last();
+            const uint64_t pol_w = policy_evict_last();
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), w0 = smem_u32(smem) + C::X_BYTES;
+            RingPos<C::STAGES> r;
+            bool ok = true;
+            for (int it = 0; it < n_units && ok; ++it) {
+                const int h64 = static_cast<int>(((u0 + it) / tiles_per_slab) % pa.H) * 64;
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
+                    if (!ok) break;
+                    const uint32_t bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::W_BYTES);
+                    tma_load_2d_addr(w0 + r.s * C::STAGE_BYTES, &tmap_wq, h64, kc * C::KC, bar, pol_w);
+                }
+            }
+            if (!ok) report_wait_expired(status);
         }
+    } else if (warp == C::PRODUCER_WARP) {
+        // ---------------- producer warp (lane 0 issues the X chunks and T tiles; all lanes copy the
+        // operand image; its drain at the end covers the W loads too) ----------------
+        uint64_t pol_x = 0;
+        if (lane == 0) pol_x = policy_evict_first();
+        const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), x0 = smem_u32(smem);
+        RingPos<C::STAGES> r;
         bool ok = true;
         int issued = 0, visit = -1, cur_slab = -1;
         for (int it = 0; it < n_units && ok; ++it) {
@@ -492,14 +590,12 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             const int slab = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
             const int b = slab / pa.H, h = slab % pa.H, e = it & 1, n = it >> 1;
             if (lane == 0) {
-                for (int kc = 0; kc < KCH; ++kc) {
-                    const int c = it * KCH + kc, s = c % C::STAGES;
-                    ok = mbar_wait(&empty[s], ((c / C::STAGES) & 1) ^ 1);
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
                     if (!ok) break;
-                    unsigned char* dst = smem + s * C::STAGE_BYTES;
-                    mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                    tma_load_3d(dst, &tmap_x, kc * C::KC, tile * C::TILE, b, &full[s], pol_x);
-                    tma_load_2d(dst + C::X_BYTES, &tmap_wq, h * 64, kc * C::KC, &full[s], pol_w);
+                    const uint32_t bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::X_BYTES);
+                    tma_load_3d_addr(x0 + r.s * C::STAGE_BYTES, &tmap_x, kc * C::KC, tile * C::TILE, b, bar, pol_x);
                     ++issued;
                 }
             }
@@ -564,24 +660,26 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                 umma_commit(&d2_done[e]);
                 return true;
             };
+            // Descriptors of stage 0 (a stage further on adds STAGE_BYTES / 16 to the address field).
+            const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
+            const uint64_t w_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, 0, 1024);
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty);
+            RingPos<C::STAGES> r;
             for (int it = 0; it < n_units && ok; ++it) {
                 const int e = it & 1;
                 if (it >= 2) ok = mbar_wait(&d1_free[e], ((it >> 1) - 1) & 1);
                 if (!ok) break;
                 const uint32_t d1 = tmem_base + e * C::TMEM_PER_GROUP;
-                for (int kc = 0; kc < KCH; ++kc) {
-                    const int c = it * KCH + kc, s = c % C::STAGES;
-                    ok = mbar_wait(&full[s], (c / C::STAGES) & 1);
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(full0 + 8 * r.s, r.phase);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t x_addr = smem_u32(smem + s * C::STAGE_BYTES), w_addr = x_addr + C::X_BYTES;
-                    const uint64_t a_desc = umma_desc_kmajor_sw128(x_addr);
+                    const uint64_t step = static_cast<uint64_t>(r.s * (C::STAGE_BYTES >> 4));
+                    const uint64_t a_desc = a_desc0 + step, w_desc = w_desc0 + step;
+                    umma_ss(d1, a_desc, w_desc, idesc1, kc > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 0; k < C::KC / 16; ++k) {
-                        const uint64_t w_desc = umma_desc_mnmajor_sw128(w_addr + k * 2048, 0, 1024);
-                        umma_ss(d1, a_desc + 2 * k, w_desc, idesc1, (kc == 0 && k == 0) ? 0u : 1u);
-                    }
-                    umma_commit(&empty[s]);
+                    for (int k = 1; k < C::KC / 16; ++k) umma_ss(d1, a_desc + 2 * k, w_desc + 128 * k, idesc1, 1u);
+                    umma_commit_addr(empty0 + 8 * r.s);
                 }
                 if (!ok) break;
                 umma_commit(&d1_done[e]);
@@ -731,7 +829,8 @@ struct ProdHiddenCfg {
     static constexpr int PRODUCER_WARP = EPI_WARPS;
     static constexpr int MMA_WARP = EPI_WARPS + 1;
     static constexpr int STORE_WARP = EPI_WARPS + 2;
-    static constexpr int THREADS = 32 * (EPI_WARPS + 3);
+    static constexpr int WPRODUCER_WARP = EPI_WARPS + 3;  // W chunks (the producer warp issues the X chunks)
+    static constexpr int THREADS = 32 * (EPI_WARPS + 4);
     static constexpr int TMEM_COLS = 256;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_BYTES + MAX_C * 4 + 1024 + 1024;
 };
@@ -769,7 +868,7 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
-            mbar_init(&full[s], 1);
+            mbar_init(&full[s], 2);  // the X and the W issuer each announce their bytes
             mbar_init(&empty[s], 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -785,10 +884,8 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    if (warp == C::PRODUCER_WARP && lane == 0) {
-        prefetch_tmap(&tmap_x);
-        prefetch_tmap(&tmap_w1);
-    }
+    if (warp == C::PRODUCER_WARP && lane == 0) prefetch_tmap(&tmap_x);
+    if (warp == C::WPRODUCER_WARP && lane == 0) prefetch_tmap(&tmap_w1);
     if (warp == C::STORE_WARP && lane == 0) prefetch_tmap(&tmap_u);
     pdl_launch_dependents();
     pdl_wait();
@@ -799,53 +896,71 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                                     : 0.0f;
     __syncthreads();
 
-    if (warp == C::PRODUCER_WARP) {
+    if (warp == C::WPRODUCER_WARP) {
         if (lane == 0) {
-            const uint64_t pol_x = policy_evict_first(), pol_w = policy_evict_last();
+            const uint64_t pol_w = policy_evict_last();
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), w0 = smem_u32(smem) + C::X_BYTES;
+            RingPos<C::STAGES> r;
+            bool ok = true;
+            for (int j = 0; j < n_blocks && ok; ++j) {
+                const int col = (j % NB) * C::NB_COLS;
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
+                    if (!ok) break;
+                    const uint32_t dst = w0 + r.s * C::STAGE_BYTES, bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::W_BYTES);
+                    // (the second box of an odd last block lies past the last column: zero fill)
+                    tma_load_2d_addr(dst, &tmap_w1, col, kc * C::KC, bar, pol_w);
+                    tma_load_2d_addr(dst + C::KC * 128, &tmap_w1, col + 64, kc * C::KC, bar, pol_w);
+                }
+            }
+            if (!ok) report_wait_expired(status);
+        }
+    } else if (warp == C::PRODUCER_WARP) {
+        if (lane == 0) {
+            const uint64_t pol_x = policy_evict_first();
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), x0 = smem_u32(smem);
+            RingPos<C::STAGES> r;
             bool ok = true;
             int issued = 0;
             for (int j = 0; j < n_blocks && ok; ++j) {
                 const long long u = u0 + j / NB;
-                const int nb = j % NB;
                 const int b = static_cast<int>(u / tiles_per_batch), tile = static_cast<int>(u % tiles_per_batch);
-                for (int kc = 0; kc < KCH; ++kc) {
-                    const int c = j * KCH + kc, s = c % C::STAGES;
-                    ok = mbar_wait(&empty[s], ((c / C::STAGES) & 1) ^ 1);
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
                     if (!ok) break;
-                    unsigned char* dst = smem + s * C::STAGE_BYTES;
-                    mbar_expect_tx(&full[s], C::STAGE_BYTES);
-                    tma_load_3d(dst, &tmap_x, kc * C::KC, tile * C::TILE, b, &full[s], pol_x);
-                    // (the second box of an odd last block lies past the last column: zero fill)
-                    tma_load_2d(dst + C::X_BYTES, &tmap_w1, nb * C::NB_COLS, kc * C::KC, &full[s], pol_w);
-                    tma_load_2d(dst + C::X_BYTES + C::KC * 128, &tmap_w1, nb * C::NB_COLS + 64, kc * C::KC, &full[s], pol_w);
+                    const uint32_t bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::X_BYTES);
+                    tma_load_3d_addr(x0 + r.s * C::STAGE_BYTES, &tmap_x, kc * C::KC, tile * C::TILE, b, bar, pol_x);
                     ++issued;
                 }
             }
             if (!ok) report_wait_expired(status);
-            drain_loads<C::STAGES>(full, 0, issued, status);
+            drain_loads<C::STAGES>(full, 0, issued, status);  // covers the W loads too (same barriers)
         }
     } else if (warp == C::MMA_WARP) {
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), 128, 128, kUmmaBMnMajor);
             bool ok = true;
+            const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
+            const uint64_t b_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, C::KC * 128, 1024);
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty);
+            RingPos<C::STAGES> r;
             for (int j = 0; j < n_blocks && ok; ++j) {
                 const int e = j & 1;
                 if (j >= 2) ok = mbar_wait(&d1_free[e], ((j >> 1) - 1) & 1);
                 if (!ok) break;
                 const uint32_t d1 = tmem_base + e * 128;
-                for (int kc = 0; kc < KCH; ++kc) {
-                    const int c = j * KCH + kc, s = c % C::STAGES;
-                    ok = mbar_wait(&full[s], (c / C::STAGES) & 1);
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(full0 + 8 * r.s, r.phase);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    const uint32_t x_addr = smem_u32(smem + s * C::STAGE_BYTES), w_addr = x_addr + C::X_BYTES;
-                    const uint64_t a_desc = umma_desc_kmajor_sw128(x_addr);
+                    const uint64_t step = static_cast<uint64_t>(r.s * (C::STAGE_BYTES >> 4));
+                    const uint64_t a_desc = a_desc0 + step, b_desc = b_desc0 + step;
+                    umma_ss(d1, a_desc, b_desc, idesc, kc > 0 ? 1u : 0u);
 #pragma unroll
-                    for (int k = 0; k < C::KC / 16; ++k) {
-                        const uint64_t b_desc = umma_desc_mnmajor_sw128(w_addr + k * 2048, C::KC * 128, 1024);
-                        umma_ss(d1, a_desc + 2 * k, b_desc, idesc, (kc == 0 && k == 0) ? 0u : 1u);
-                    }
-                    umma_commit(&empty[s]);
+                    for (int k = 1; k < C::KC / 16; ++k) umma_ss(d1, a_desc + 2 * k, b_desc + 128 * k, idesc, 1u);
+                    umma_commit_addr(empty0 + 8 * r.s);
                 }
                 if (!ok) break;
                 umma_commit(&d1_done[e]);
