@@ -1624,9 +1624,18 @@ cudaError_t launch_apply_x(const linfusion_attn* h, const void* x, const void* w
     cudaError_t e = launch_chained(stream_pack_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
                                    own, h->operand, h->tile_counters, dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
-    e = launch_chained(producer_apply_kernel<KIND>, dim3(p.G_apply), dim3(ProdApplyCfg::THREADS),
+    // Units are (batch, head pair, tile); the same number of CTAs on every (batch, head pair) where that
+    // keeps at least four fifths of the SMs busy, so that the CTAs of a token's head pairs walk through
+    // X in step and share its tiles in L2.
+    const long long groups = static_cast<long long>(h->desc.B) * head_pairs(h->desc.H);
+    const long long W = groups * p.tiles_apply;
+    long long G = h->sm_count;
+    const long long aligned = (G / groups) * groups;
+    if (aligned * 5 >= G * 4) G = aligned;
+    if (G > W) G = W;
+    e = launch_chained(producer_apply_kernel<KIND>, dim3(static_cast<unsigned>(G)), dim3(ProdApplyCfg::THREADS),
                        ProdApplyCfg::SMEM_BYTES, s, mx, mwq, mt, my, h->operand, h->status, pa, p.tiles_apply,
-                       p.W_apply, apply_scales(h->desc));
+                       W, apply_scales(h->desc));
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

@@ -464,16 +464,17 @@ producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
 struct ProdApplyCfg {
     static constexpr int TILE = 128;
     static constexpr int KC = 64;
-    // The K loop is bound by the bytes in flight per SM (ring size / load round trip of ~1.4 us), not
-    // by L2 bandwidth or the tensor pipe: as many stages as shared memory holds.
-    static constexpr int STAGES = 7;
+    // One tcgen05.mma of this thread costs about 125 cycles to issue whatever its N (measured: the
+    // K loop took the same time per chunk with N = 64 as with N = 128), so a unit takes TWO heads:
+    // D1[128 x 128] = X_tile [W_Q,h0 | W_Q,h1], twice the work per instruction.
+    static constexpr int STAGES = 4;
     static constexpr int X_BYTES = TILE * 128;     // 16 KB
-    static constexpr int W_BYTES = KC * 128;       // 8 KB: 64 input rows x 64 Q columns
+    static constexpr int W_BYTES = 2 * KC * 128;   // 16 KB: 64 input rows x (64 | 64) Q columns of the two heads
     static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
-    static constexpr int Y_BYTES = TILE * 128;     // per epilogue group: T tile in, Y tile out
+    static constexpr int Y_BYTES = TILE * 128;     // per head of the pair: T tile in, Y tile out
     static constexpr int B_ROWS = StreamApplyCfg::B_ROWS;
-    static constexpr int B_BYTES = StreamApplyCfg::B_BYTES;  // S^T | z operand image, two buffers
-    static constexpr int EPI_GROUPS = 2;
+    static constexpr int B_BYTES = StreamApplyCfg::B_BYTES;  // S^T | z operand image of one head
+    static constexpr int EPI_GROUPS = 2;           // group e works on head e of every pair
     static constexpr int EPI_WARPS = 4 * EPI_GROUPS;
     static constexpr int PRODUCER_WARP = EPI_WARPS;
     static constexpr int MMA_WARP = EPI_WARPS + 1;
@@ -481,18 +482,24 @@ struct ProdApplyCfg {
     static constexpr int WPRODUCER_WARP = EPI_WARPS + 3;  // W chunks (the producer warp issues the X chunks)
     static constexpr int THREADS = 32 * (EPI_WARPS + 4);
     static constexpr int TMEM_COLS = 512;
-    static constexpr int TMEM_PER_GROUP = 256;  // projection accumulator 64 | phi(Q) operand 32 | output accumulator 80
-    static constexpr int TMEM_A = 64, TMEM_D2 = 96;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_GROUPS * Y_BYTES + 2 * B_BYTES + 1024 + 1024;
+    // [0,256): two projection accumulators of 128 columns; per head e: phi(Q) operand (32) and output accumulator (80)
+    static constexpr int TMEM_A0 = 256, TMEM_A_STEP = 32, TMEM_D2_0 = 320, TMEM_D2_STEP = 80;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_GROUPS * Y_BYTES + 4 * B_BYTES + 1024 + 1024;
 };
 static_assert((ProdApplyCfg::STAGES * ProdApplyCfg::STAGE_BYTES + ProdApplyCfg::EPI_GROUPS * ProdApplyCfg::Y_BYTES) % 1024 == 0 &&
                   ProdApplyCfg::B_BYTES % 1024 == 0 && ProdApplyCfg::STAGE_BYTES % 1024 == 0,
               "operands on 1024-byte boundaries");
+static_assert(ProdApplyCfg::TMEM_D2_0 + 2 * ProdApplyCfg::TMEM_D2_STEP <= ProdApplyCfg::TMEM_COLS, "TMEM budget");
 static_assert(ProdApplyCfg::SMEM_BYTES > 116 * 1024 && ProdApplyCfg::SMEM_BYTES <= 227 * 1024, "one CTA per SM");
 
-// Y of the slabs from X and the reduced state: CTA g of G owns the contiguous run of (slab, tile)
-// units [g*W/G, (g+1)*W/G).  A run is a sequence of slab VISITS; visit k's operand image S^T | z
-// goes to shared-memory buffer k & 1.
+// Heads are taken in pairs (2p, 2p + 1); with an odd head count the last pair's second head does
+// not exist: its weight box and T tile lie past the tensors' extents (TMA fills zeros) and its Y
+// tile is not stored.
+__host__ __device__ __forceinline__ int head_pairs(int H) { return (H + 1) / 2; }
+
+// Y from X and the reduced state.  Units are (batch, head pair, 128-token tile), numbered
+// pair-major; CTA g of G owns the contiguous run [g*W/G, (g+1)*W/G).  A run is a sequence of VISITS
+// to (batch, head pair)s; visit k's two operand images S^T | z go to shared-memory buffers 2 (k & 1) + e.
 template <int KIND>
 __global__ void __launch_bounds__(ProdApplyCfg::THREADS, 1)
 producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_wq,
@@ -506,17 +513,17 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     unsigned char* ybuf = smem + C::STAGES * C::STAGE_BYTES;
     unsigned char* bsm = ybuf + C::EPI_GROUPS * C::Y_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(bsm + 2 * C::B_BYTES);
+    uint64_t* full = reinterpret_cast<uint64_t*>(bsm + 4 * C::B_BYTES);
     uint64_t* empty = full + C::STAGES;
-    uint64_t* d1_done = empty + C::STAGES;  // [2] projection accumulator complete
-    uint64_t* d1_free = d1_done + 2;        // [2] read by its epilogue
-    uint64_t* t_full = d1_free + 2;         // [2] T tile landed in the group's tile buffer
-    uint64_t* a_ready = t_full + 2;         // [2] phi(Q) rows in tensor memory
-    uint64_t* d2_done = a_ready + 2;        // [2] output accumulator complete
-    uint64_t* y_ready = d2_done + 2;        // [2] Y tile in the group's tile buffer
-    uint64_t* y_free = y_ready + 2;         // [2] the store has read it
-    uint64_t* b_ready = y_free + 2;         // [2] operand image of the visit in shared memory
-    uint64_t* b_free = b_ready + 2;         // [2] the MMAs that read it are complete
+    uint64_t* d1_done = empty + C::STAGES;  // [2] projection accumulator (unit parity) complete
+    uint64_t* d1_free = d1_done + 2;        // [2] read by both heads' epilogues
+    uint64_t* t_full = d1_free + 2;         // [2] per head: T tile landed in the head's tile buffer
+    uint64_t* a_ready = t_full + 2;         // [2] per head: phi(Q) rows in tensor memory
+    uint64_t* d2_done = a_ready + 2;        // [2] per head: output accumulator complete
+    uint64_t* y_ready = d2_done + 2;        // [2] per head: Y tile in the tile buffer
+    uint64_t* y_free = y_ready + 2;         // [2] per head: the store has read it
+    uint64_t* b_ready = y_free + 2;         // [2] per visit parity: operand images in shared memory
+    uint64_t* b_free = b_ready + 2;         // [2] the MMAs that read them are complete
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b_free + 2);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -524,6 +531,7 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     const long long u0 = unit_begin(g, W, G), u1 = unit_begin(g + 1, W, G);
     const int n_units = static_cast<int>(u1 - u0);
     const int KCH = pa.chunks;
+    const int HP = head_pairs(pa.H);
 
     if (tid == 0) {
         for (int s = 0; s < C::STAGES; ++s) {
@@ -532,7 +540,7 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(&d1_done[b], 1);
-            mbar_init(&d1_free[b], 4);
+            mbar_init(&d1_free[b], 8);
             mbar_init(&t_full[b], 1);
             mbar_init(&a_ready[b], 4);
             mbar_init(&d2_done[b], 1);
@@ -565,30 +573,31 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             RingPos<C::STAGES> r;
             bool ok = true;
             for (int it = 0; it < n_units && ok; ++it) {
-                const int h64 = static_cast<int>(((u0 + it) / tiles_per_slab) % pa.H) * 64;
+                const int col = static_cast<int>(((u0 + it) / tiles_per_slab) % HP) * 128;  // first column of head 2p
                 for (int kc = 0; kc < KCH; ++kc, r.next()) {
                     ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
                     if (!ok) break;
-                    const uint32_t bar = full0 + 8 * r.s;
+                    const uint32_t dst = w0 + r.s * C::STAGE_BYTES, bar = full0 + 8 * r.s;
                     mbar_expect_tx_addr(bar, C::W_BYTES);
-                    tma_load_2d_addr(w0 + r.s * C::STAGE_BYTES, &tmap_wq, h64, kc * C::KC, bar, pol_w);
+                    tma_load_2d_addr(dst, &tmap_wq, col, kc * C::KC, bar, pol_w);
+                    tma_load_2d_addr(dst + C::KC * 128, &tmap_wq, col + 64, kc * C::KC, bar, pol_w);
                 }
             }
             if (!ok) report_wait_expired(status);
         }
     } else if (warp == C::PRODUCER_WARP) {
         // ---------------- producer warp (lane 0 issues the X chunks and T tiles; all lanes copy the
-        // operand image; its drain at the end covers the W loads too) ----------------
+        // operand images; its drain at the end covers the W loads too) ----------------
         uint64_t pol_x = 0;
         if (lane == 0) pol_x = policy_evict_first();
         const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), x0 = smem_u32(smem);
         RingPos<C::STAGES> r;
         bool ok = true;
-        int issued = 0, visit = -1, cur_slab = -1;
+        int issued = 0, visit = -1, cur_ps = -1;
         for (int it = 0; it < n_units && ok; ++it) {
             const long long u = u0 + it;
-            const int slab = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
-            const int b = slab / pa.H, h = slab % pa.H, e = it & 1, n = it >> 1;
+            const int ps = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
+            const int b = ps / HP, h0 = 2 * (ps % HP);
             if (lane == 0) {
                 for (int kc = 0; kc < KCH; ++kc, r.next()) {
                     ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
@@ -601,29 +610,36 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
             if (!ok) break;
-            if (slab != cur_slab) {
-                // A new visit: its operand image, after the unit's own loads are on their way (the MMA
-                // thread frees the buffer of two visits back only once it reaches the visit before this one).
-                cur_slab = slab;
+            if (ps != cur_ps) {
+                // A new visit: its operand images, after the unit's own loads are on their way (the MMA
+                // thread frees the buffers of two visits back only once it reaches the visit before this one).
+                cur_ps = ps;
                 ++visit;
                 if (visit >= 2) {
                     if (lane == 0) ok = mbar_wait(&b_free[visit & 1], ((visit >> 1) - 1) & 1);
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                     if (!ok) break;
                 }
-                const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
-                uint4* dst = reinterpret_cast<uint4*>(bsm + (visit & 1) * C::B_BYTES);
-                for (int i = lane; i < C::B_BYTES / 16; i += 32) dst[i] = __ldg(src + i);
+                for (int e = 0; e < 2; ++e) {
+                    if (h0 + e >= pa.H) break;
+                    const int slab = b * pa.H + h0 + e;
+                    const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
+                    uint4* dst = reinterpret_cast<uint4*>(bsm + (2 * (visit & 1) + e) * C::B_BYTES);
+                    for (int i = lane; i < C::B_BYTES / 16; i += 32) dst[i] = __ldg(src + i);
+                }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(&b_ready[visit & 1]);
             }
             if (pa.has_t != 0 && lane == 0) {
-                // T tile into the group's tile buffer, once the store of two units back has read it
-                if (n >= 1) ok = mbar_wait(&y_free[e], (n - 1) & 1);
-                if (ok) {
-                    mbar_expect_tx(&t_full[e], C::Y_BYTES);
-                    tma_load_4d(ybuf + e * C::Y_BYTES, &tmap_t, 0, tile * C::TILE, h, b, &t_full[e], pol_x);
+                // T tiles of the two heads into their tile buffers, once the stores of the unit before
+                // have read them (a head past the last one: the box lies outside the tensor, zeros)
+                for (int e = 0; e < 2 && ok; ++e) {
+                    if (it >= 1) ok = mbar_wait(&y_free[e], (it - 1) & 1);
+                    if (ok) {
+                        mbar_expect_tx(&t_full[e], C::Y_BYTES);
+                        tma_load_4d(ybuf + e * C::Y_BYTES, &tmap_t, 0, tile * C::TILE, h0 + e, b, &t_full[e], pol_x);
+                    }
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -635,41 +651,45 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     } else if (warp == C::MMA_WARP) {
         // ---------------- MMA warp ----------------
         if (lane == 0) {
-            const uint32_t idesc1 = umma_idesc_f32acc(kind_dtype(KIND), 128, 64, kUmmaBMnMajor);
+            const uint32_t idesc1 = umma_idesc_f32acc(kind_dtype(KIND), 128, 128, kUmmaBMnMajor);
             const uint32_t idesc2 = umma_idesc_f32acc(kind_dtype(KIND), C::TILE, C::B_ROWS);
             bool ok = true;
-            int visit = -1, cur_slab = -1;
-            uint64_t b_desc = 0;
-            // Output MMAs of unit j: D2 = phi(Q) [S | z].
+            int visit = -1, cur_ps = -1;
+            uint64_t b_desc[2] = {0, 0};
+            // Output MMAs of unit j, head by head: D2_e = phi(Q_e) [S_e | z_e].
             auto apply_mma = [&](int j) {
-                const int e = j & 1;
-                const int slab = static_cast<int>((u0 + j) / tiles_per_slab);
-                if (slab != cur_slab) {
+                const int ps = static_cast<int>((u0 + j) / tiles_per_slab);
+                if (ps != cur_ps) {
                     if (visit >= 0) umma_commit(&b_free[visit & 1]);  // the visit before: all its MMAs are issued
                     ++visit;
-                    cur_slab = slab;
+                    cur_ps = ps;
                     if (!mbar_wait(&b_ready[visit & 1], (visit >> 1) & 1)) return false;
-                    b_desc = umma_desc_kmajor_sw128(smem_u32(bsm + (visit & 1) * C::B_BYTES));
+                    b_desc[0] = umma_desc_kmajor_sw128(smem_u32(bsm + (2 * (visit & 1)) * C::B_BYTES));
+                    b_desc[1] = umma_desc_kmajor_sw128(smem_u32(bsm + (2 * (visit & 1) + 1) * C::B_BYTES));
                 }
-                if (!mbar_wait(&a_ready[e], (j >> 1) & 1)) return false;
-                tc_fence_after_sync();
-                const uint32_t a_tmem = tmem_base + e * C::TMEM_PER_GROUP + C::TMEM_A;
-                const uint32_t d_tmem = tmem_base + e * C::TMEM_PER_GROUP + C::TMEM_D2;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) umma_ts(d_tmem, a_tmem + 8 * k, b_desc + 2 * k, idesc2, k > 0 ? 1u : 0u);
-                umma_commit(&d2_done[e]);
+                for (int e = 0; e < 2; ++e) {
+                    if (!mbar_wait(&a_ready[e], j & 1)) return false;
+                    tc_fence_after_sync();
+                    const uint32_t a_tmem = tmem_base + C::TMEM_A0 + e * C::TMEM_A_STEP;
+                    const uint32_t d_tmem = tmem_base + C::TMEM_D2_0 + e * C::TMEM_D2_STEP;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) umma_ts(d_tmem, a_tmem + 8 * k, b_desc[e] + 2 * k, idesc2, k > 0 ? 1u : 0u);
+                    umma_commit(&d2_done[e]);
+                }
                 return true;
             };
-            // Descriptors of stage 0 (a stage further on adds STAGE_BYTES / 16 to the address field).
+            // Descriptors of stage 0 (a stage further on adds STAGE_BYTES / 16 to the address field); the W
+            // chunk's two 64-column blocks (the two heads) are 8 KB apart.
             const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
-            const uint64_t w_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, 0, 1024);
+            const uint64_t w_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, C::KC * 128, 1024);
             const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty);
             RingPos<C::STAGES> r;
             for (int it = 0; it < n_units && ok; ++it) {
-                const int e = it & 1;
-                if (it >= 2) ok = mbar_wait(&d1_free[e], ((it >> 1) - 1) & 1);
+                const int buf = it & 1;
+                if (it >= 2) ok = mbar_wait(&d1_free[buf], ((it >> 1) - 1) & 1);
                 if (!ok) break;
-                const uint32_t d1 = tmem_base + e * C::TMEM_PER_GROUP;
+                const uint32_t d1 = tmem_base + buf * 128;
                 for (int kc = 0; kc < KCH; ++kc, r.next()) {
                     ok = mbar_wait_addr(full0 + 8 * r.s, r.phase);
                     if (!ok) break;
@@ -682,7 +702,7 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                     umma_commit_addr(empty0 + 8 * r.s);
                 }
                 if (!ok) break;
-                umma_commit(&d1_done[e]);
+                umma_commit(&d1_done[buf]);
                 if (it >= 1) ok = apply_mma(it - 1);
             }
             if (ok && n_units > 0) ok = apply_mma(n_units - 1);
@@ -692,42 +712,50 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         // ---------------- store warp ----------------
         if (lane == 0) {
             const uint64_t policy = policy_evict_first();
-            for (int it = 0; it < n_units; ++it) {
-                const int e = it & 1;
-                if (!mbar_wait(&y_ready[e], (it >> 1) & 1)) {
-                    report_wait_expired(status);
-                    break;
-                }
+            bool ok = true;
+            for (int it = 0; it < n_units && ok; ++it) {
                 const long long u = u0 + it;
-                const int slab = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
-                tma_store_4d(&tmap_y, ybuf + e * C::Y_BYTES, 0, tile * C::TILE, slab % pa.H, slab / pa.H, policy);
-                tma_store_wait_read();
-                mbar_arrive(&y_free[e]);
+                const int ps = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
+                const int b = ps / HP, h0 = 2 * (ps % HP);
+                for (int e = 0; e < 2; ++e) {
+                    if (!mbar_wait(&y_ready[e], it & 1)) {
+                        report_wait_expired(status);
+                        ok = false;
+                        break;
+                    }
+                    if (h0 + e < pa.H) {
+                        tma_store_4d(&tmap_y, ybuf + e * C::Y_BYTES, 0, tile * C::TILE, h0 + e, b, policy);
+                        tma_store_wait_read();
+                    }
+                    mbar_arrive(&y_free[e]);
+                }
             }
             tma_store_wait_all();
         }
     } else {
-        // ---------------- epilogue warpgroups: group e takes units e, e + 2, ... ----------------
+        // ---------------- epilogue warpgroups: group e works on head e of every unit's pair ----------------
         const int e = warp >> 2, wq = warp & 3;
         const int row = wq * 32 + lane;
         const uint32_t sw = row & 7;
-        const uint32_t t_base = tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + e * C::TMEM_PER_GROUP;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(wq * 32) << 16);
+        const uint32_t a_tmem = t_lane + C::TMEM_A0 + e * C::TMEM_A_STEP;
+        const uint32_t d2_tmem = t_lane + C::TMEM_D2_0 + e * C::TMEM_D2_STEP;
         const uint32_t y_row = smem_u32(ybuf + e * C::Y_BYTES) + row * 128;
         bool ok = true;
-        for (int it = e; it < n_units; it += 2) {
-            const int n = it >> 1;
-            ok = mbar_wait(&d1_done[e], n & 1);
-            if (ok && pa.has_t != 0) ok = mbar_wait(&t_full[e], n & 1);
+        for (int it = 0; it < n_units; ++it) {
+            const int buf = it & 1;
+            ok = mbar_wait(&d1_done[buf], (it >> 1) & 1);
+            if (ok && pa.has_t != 0) ok = mbar_wait(&t_full[e], it & 1);
             __syncwarp();
             if (!ok) break;
             tc_fence_after_sync();
             {
-                // Q row (+ T row), phi in fp32, rounded: the row of the output MMA's A operand
+                // Q row of this head (+ T row), phi in fp32, rounded: the row of the output MMA's A operand
                 uint32_t a[32];
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     uint32_t d[32];
-                    tmem_load_32cols(t_base + 32 * half, d);
+                    tmem_load_32cols(t_lane + buf * 128 + e * 64 + 32 * half, d);
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
                         float f[8];
@@ -748,26 +776,26 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
                             a[16 * half + 4 * c + i] = pack_pair<KIND>(phi<KIND>(f[2 * i]), phi<KIND>(f[2 * i + 1]));
                     }
                 }
-                tmem_store_32cols(t_base + C::TMEM_A, a);
+                tmem_store_32cols(a_tmem, a);
             }
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) {
-                mbar_arrive(&d1_free[e]);
+                mbar_arrive(&d1_free[buf]);
                 mbar_arrive(&a_ready[e]);
             }
-            ok = mbar_wait(&d2_done[e], n & 1);
-            // without a T tile nobody has waited yet for the store of two units back to let go of the buffer
-            if (ok && pa.has_t == 0 && n >= 1) ok = mbar_wait(&y_free[e], (n - 1) & 1);
+            ok = mbar_wait(&d2_done[e], it & 1);
+            // without a T tile nobody has waited yet for the store of the unit before to let go of the buffer
+            if (ok && pa.has_t == 0 && it >= 1) ok = mbar_wait(&y_free[e], (it - 1) & 1);
             __syncwarp();
             if (!ok) break;
             tc_fence_after_sync();
-            const float den = __uint_as_float(tmem_load_1col(t_base + C::TMEM_D2 + 64));  // phi(Q_i) . z
+            const float den = __uint_as_float(tmem_load_1col(d2_tmem + 64));  // phi(Q_i) . z
             const float inv = row_scale(den, sc);
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t d[32];
-                tmem_load_32cols(t_base + C::TMEM_D2 + 32 * half, d);
+                tmem_load_32cols(d2_tmem + 32 * half, d);
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
                     const uint32_t v0 = pack_pair<KIND>(__uint_as_float(d[8 * c + 0]) * inv, __uint_as_float(d[8 * c + 1]) * inv);
@@ -793,7 +821,6 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         tmem_dealloc(tmem_base, C::TMEM_COLS);
     }
 }
-
 
 // 3-D tiled TMA store (x = channel, y = token, z = batch), clipped at the tensor's extents.
 __device__ __forceinline__ void tma_store_3d(const void* tmap, const void* smem_src, int x, int y, int z,
