@@ -54,7 +54,7 @@ typedef enum {
 #define LINFUSION_VARIANT_AUTO 0u
 #define LINFUSION_VARIANT_SPLIT 1u   /* three launches: split-N state, reduction, apply (any supported d) */
 #define LINFUSION_VARIANT_STREAM 2u  /* three launches, TMA-pipelined persistent kernels (d = 64 only)    */
-#define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N)               */
+#define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N); one CTA per slab for N <= 192 */
 #define LINFUSION_VARIANT_FUSED 4u   /* one launch, persistent TMA + tcgen05 kernel with per-slab counters (d = 64) */
 #define LINFUSION_VARIANT_MASK 0xFu
 /*
@@ -223,7 +223,7 @@ linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host,
  * state_buffer: *dev_ptr is the device address of [B*H][d*d S (row = feature c of K, column =
  * channel e of V), then d z] fp32, *floats its length; it stays valid until the handle is
  * destroyed or its workspace is replaced.  Handles that resolved to a single-launch variant
- * (CLUSTER, FUSED; AUTO picks FUSED for many small slabs of head dim 64) cannot be split in two:
+ * (CLUSTER, FUSED; AUTO picks CLUSTER for N <= 192 and FUSED for many small slabs of head dim 64) cannot be split in two:
  * state() and apply() return UNSUPPORTED for them (create the handle with LINFUSION_VARIANT_SPLIT
  * or _STREAM).  Other errors as for forward().
  */
@@ -411,7 +411,7 @@ linfusion_status_t linfusion_attn_forward_x(linfusion_attn_t* h, const void* x,
                                             const linfusion_module_weights_t* w, void* y,
                                             void* cuda_stream);
 
-/* Name of the kernel variant the handle resolved to ("split", "stream", "cluster"). */
+/* Name of the kernel variant the handle resolved to ("split", "stream", "cluster", "fused"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);
 
 /* Number of kernel launches one forward() enqueues for this handle. */

@@ -1,6 +1,6 @@
-// Device helpers shared by the attention kernels: the activation phi, bf16 packing,
+// Device helpers shared by the attention kernels: the activation phi, 16-bit packing,
 // warp-level tensor-core fragments (ldmatrix / mma.sync), bounded mbarrier + TMA wrappers, and the
-// tcgen05 (tensor memory) wrappers of the apply kernel.
+// tcgen05 (tensor memory, 5th-generation MMA) wrappers of the stream, fused and producer kernels.
 #pragma once
 
 #include <cuda.h>

@@ -84,8 +84,16 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
     return LINFUSION_OK;
 }
 
+// Up to this many 64-token K/V tiles one CTA takes a slab alone: one launch, no partial states, the
+// state goes from the MMA fragments straight into the apply operand.  Measured: 15.8 vs 22.4 us (three
+// chained launches) at N = 64, d = 160 x 16 slabs and 9.8 vs 12.3 us (the persistent tcgen05 launch) at
+// N = 144, d = 64 x 40 slabs; at four tiles (N = 256, d = 160) one CTA per slab is already the slower
+// (35 vs 24.5 us: 16 CTAs working through their tiles one after the other).
+constexpr int kLocalMaxTilesKv = 3;
+
 int largest_cluster(int tiles_kv)
 {
+    if (tiles_kv <= kLocalMaxTilesKv) return 1;
     int c = kMaxClusterSize;
     while (c > 1 && c > tiles_kv) c >>= 1;
     return c;
@@ -123,7 +131,9 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // boundaries (32 vs 22 us at N = 2304 x 20, 106 vs 47 us at N = 16384 x 20), so it is not
         // chosen there.
         const int fused_tiles = (d->N + FusedCfg::TILE - 1) / FusedCfg::TILE;
-        if (square64 && stream_tiles >= 8ll * sm_count)
+        if (tiles_kv <= kLocalMaxTilesKv)
+            v = LINFUSION_VARIANT_CLUSTER;  // resolves to one CTA per slab (largest_cluster())
+        else if (square64 && stream_tiles >= 8ll * sm_count)
             v = LINFUSION_VARIANT_STREAM;
         else if (square64 && fused_tiles <= 8 && 4 * slabs >= sm_count && stream_tiles < 4ll * sm_count)
             v = LINFUSION_VARIANT_FUSED;
@@ -533,8 +543,13 @@ cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, cons
     cudaLaunchAttribute attr[1];
     cluster_config<DK, DV>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
     mark(h, 0, s);
-    cudaError_t e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<DK, DV, KIND>, q, k, v, y, h->state,
-                                       h->desc.N, apply_scales(h->desc), layout_qk(h->desc), layout_vy(h->desc));
+    cudaError_t e;
+    if (h->plan.cluster_size == 1)  // one CTA per slab: a plain launch, chained to its neighbours in the stream
+        e = launch_chained(cluster_fused_kernel<DK, DV, KIND>, cfg.gridDim, cfg.blockDim, cfg.dynamicSmemBytes, s, q, k,
+                           v, y, h->state, h->desc.N, apply_scales(h->desc), layout_qk(h->desc), layout_vy(h->desc));
+    else
+        e = cudaLaunchKernelEx(&cfg, cluster_fused_kernel<DK, DV, KIND>, q, k, v, y, h->state, h->desc.N,
+                               apply_scales(h->desc), layout_qk(h->desc), layout_vy(h->desc));
     mark(h, 1, s);
     return e;
 }

@@ -413,6 +413,43 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
                              chunk_begin(p, tiles, chunks), chunk_begin(p + 1, tiles, chunks), St, Qsm, sc);
 }
 
+// The state fragments of accumulate_state() -> the 16-bit S^T | z operand in shared memory (which must
+// have been cleared: pad rows and columns stay zero).  For a CTA that holds a slab's whole state.
+template <int DK, int DV, int KIND>
+__device__ __forceinline__ void state_fragments_to_operand(unsigned char* St, const float (&acc)[SplitCfg<DK, DV>::NBT][4],
+                                                           float scale)
+{
+    using C = SplitCfg<DK, DV>;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int c0 = warp * 16 + g, c1 = c0 + 8;
+    auto put = [&](int row, int c, float v) {
+        *reinterpret_cast<uint16_t*>(St + row * C::PITCHK + c * 2) = to_storage16(v * scale, kind_dtype(KIND));
+    };
+#pragma unroll
+    for (int nb = 0; nb < C::NBV; ++nb) {
+        const int e = nb * 8 + 2 * t;  // S[c][e] goes to row e, column c
+        if (c0 < DK) {
+            put(e, c0, acc[nb][0]);
+            put(e + 1, c0, acc[nb][1]);
+        }
+        if (c1 < DK) {
+            put(e, c1, acc[nb][2]);
+            put(e + 1, c1, acc[nb][3]);
+        }
+    }
+    // z[c] to column c of rows DV .. DV+7: lane t of a quad writes rows DV + 2t, DV + 2t + 1 (every
+    // column of the z block holds the same sum)
+    if (c0 < DK) {
+        put(DV + 2 * t, c0, acc[C::NBV][0]);
+        put(DV + 2 * t + 1, c0, acc[C::NBV][0]);
+    }
+    if (c1 < DK) {
+        put(DV + 2 * t, c1, acc[C::NBV][2]);
+        put(DV + 2 * t + 1, c1, acc[C::NBV][2]);
+    }
+}
+
 // One cluster of `cluster_size` CTAs per slab (grid.x = cluster_size, grid.y = slabs).  CTA r
 // accumulates the partial state of its run of K/V tiles into its own shared memory; after a
 // cluster barrier CTA r sums slice r of the partials over ranks 0, 1, ... in that order and pushes
@@ -436,6 +473,25 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
     const int csize = static_cast<int>(cluster.num_blocks());
     const int slab = blockIdx.y;
     const size_t off_k = slab_base(LK, slab), off_v = slab_base(LV, slab);
+
+    if (csize == 1) {
+        // One CTA holds the slab's whole state: nothing to exchange.  The state goes from the MMA
+        // fragments straight into the apply operand (and, in fp32, to state_out).
+        pdl_launch_dependents();
+        pdl_wait();
+        for (int i = threadIdx.x; i < C::SMEM_ST / 16; i += blockDim.x)
+            reinterpret_cast<uint4*>(St)[i] = make_uint4(0u, 0u, 0u, 0u);
+        const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;
+        float acc[C::NBT][4];
+        accumulate_state<DK, DV, KIND>(K + off_k, V + off_v, N, LK.row_stride, LV.row_stride, 0, tiles, stage, acc);
+        // (accumulate_state ends with a barrier: the clear above is complete)
+        state_fragments_to_operand<DK, DV, KIND>(St, acc, sc.operand);
+        if (state_out != nullptr) store_state<DK, DV>(state_out + static_cast<size_t>(slab) * C::STATE_FLOATS, acc);
+        __syncthreads();
+        const int qtiles = (N + C::TILE_Q - 1) / C::TILE_Q;
+        apply_tiles<DK, DV, KIND>(Q + off_k, Y + off_v, N, LK.row_stride, LV.row_stride, 0, qtiles, St, stage, sc);
+        return;
+    }
 
     {
         const int tiles = (N + C::TILE_KV - 1) / C::TILE_KV;

@@ -147,8 +147,9 @@ def test_stream_variant_tail_and_slab_crossing():
 
 def test_auto_policy_follows_the_measured_crossovers():
     for dims, want in [((2, 10, 16384, 64), "stream"), ((2, 20, 4096, 64), "stream"),
-                       ((2, 20, 2304, 64), "split"), ((2, 20, 144, 64), "fused"), ((2, 20, 576, 64), "fused"),
-                       ((2, 2, 144, 64), "split"), ((2, 8, 4096, 40), "split")]:
+                       ((2, 20, 2304, 64), "split"), ((2, 20, 144, 64), "cluster"), ((2, 20, 576, 64), "fused"),
+                       ((2, 2, 144, 64), "cluster"), ((2, 8, 4096, 40), "split"), ((2, 8, 64, 160), "cluster"),
+                       ((2, 8, 256, 160), "split")]:
         op = attn.LinFusionAttention(*dims)
         assert op.variant == want, (dims, op.variant)
         op.close()
