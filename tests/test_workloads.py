@@ -50,3 +50,21 @@ def test_outlier_rows_hit_all_three_tensors_and_all_heads():
     assert torch.equal(hot, rms(k) > 4.0) and torch.equal(hot, rms(v) > 4.0)
     per_head = q.float().pow(2).mean(dim=3).sqrt()               # [B, H, N]
     assert ((per_head > 4.0) == hot[:, None, :]).all()
+
+
+def test_generated_inputs_match_the_committed_checksums():
+    """The recipe is pinned: the CPU generator must reproduce, bit for bit, the inputs whose checksums are
+    committed (a change of the generator's stream, of the draw order or of the rounding shows up here)."""
+    import importlib.util
+    import json
+    import os
+    here = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+    spec = importlib.util.spec_from_file_location("make_workload_checksums", os.path.join(here, "make_workload_checksums.py"))
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    with open(os.path.join(here, "workload_checksums.json")) as f:
+        want = json.load(f)["cases"]
+    got = mod.cases()
+    assert got.keys() == want.keys()
+    for name in want:
+        assert got[name] == want[name], name
