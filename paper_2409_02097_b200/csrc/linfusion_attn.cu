@@ -54,6 +54,9 @@ struct Plan {
     int G_state = 0, G_apply = 0, spans = 0;
     // cluster
     int cluster_size = 0;
+    // stream, fed from X (token-major handles): units are (batch, head pair, tile)
+    long long W_x = 0;
+    int G_x = 0, spans_x = 0;
     // fused
     int fused_split = 0, fused_whole = 0;
     // workspace (bytes, offsets)
@@ -178,6 +181,29 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         }
         p->spans = spans;
         partial_floats = static_cast<size_t>(p->G_state) * spans * kStreamStateFloats;
+        if ((d->flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u) {
+            // The state from X (state_x): two heads per unit, the same number of CTAs on every (batch, head
+            // pair) where that keeps at least four fifths of the SMs busy (the CTAs of a token's head pairs
+            // then walk through X in step and share its tiles in L2); two partials per visit.
+            const long long groups = static_cast<long long>(d->B) * head_pairs(d->H);
+            p->W_x = groups * p->tiles_state;
+            long long gx = sm_count;
+            const long long aligned_x = (gx / groups) * groups;
+            if (aligned_x * 5 >= gx * 4) gx = aligned_x;
+            if (gx > p->W_x) gx = p->W_x;
+            p->G_x = static_cast<int>(gx);
+            int sx = 1;
+            for (int g = 0; g < p->G_x; ++g) {
+                long long b = unit_begin(g, p->W_x, p->G_x), e = unit_begin(g + 1, p->W_x, p->G_x);
+                if (e > b) {
+                    int n = static_cast<int>((e - 1) / p->tiles_state - b / p->tiles_state) + 1;
+                    if (n > sx) sx = n;
+                }
+            }
+            p->spans_x = sx;
+            const size_t need = static_cast<size_t>(p->G_x) * sx * 2 * kStreamStateFloats;
+            if (need > partial_floats) partial_floats = need;
+        }
         p->launches = 3;
     } else if (v == LINFUSION_VARIANT_FUSED) {
         // One persistent launch.  Two waves of slabs once every CTA has a couple of tiles in each
@@ -465,6 +491,9 @@ cudaError_t set_stream_attrs()
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(producer_apply_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              ProdApplyCfg::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(producer_state2_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             ProdState2Cfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(producer_hidden_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              ProdHiddenCfg::SMEM_BYTES);
@@ -1584,6 +1613,22 @@ bool encode_w_map(CUtensorMap* map, const void* w, int C)
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same matrix seen as (column within head 64, input row C, head H) -> boxes of 64 input rows x the
+// 64-column blocks of TWO heads, which land in shared memory as two consecutive 8 KB blocks (head, row,
+// column): one copy per weight matrix and K chunk.  A head index past the last head reads as zeros.
+bool encode_w_pair_map(CUtensorMap* map, const void* w, int C, int H)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    cuuint64_t dims[3] = {64u, static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(H)};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(C) * 2, 128u};
+    cuuint32_t box[3] = {64u, 64u, 2u};
+    cuuint32_t estr[3] = {1u, 1u, 1u};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(w), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Handles that can take X: head dim 64 on both sides, the three-launch TMA + tcgen05 plan, and the
 // token-major layout (X and Y are [B, N, C]: the heads of a token side by side).
 bool takes_x(const linfusion_attn* h)
@@ -1597,21 +1642,22 @@ cudaError_t launch_state_x(const linfusion_attn* h, const void* x, const void* w
 {
     const Plan& p = h->plan;
     const int C = h->desc.H * kStreamD;
-    CUtensorMap mx, mwk, mwv, mt;
-    if (!encode_x_map(&mx, x, h->desc) || !encode_w_map(&mwk, w_k, C) || !encode_w_map(&mwv, w_v, C)) return cudaErrorInvalidValue;
-    if (!encode_slab_map(&mt, t_k != nullptr ? t_k : x, h->desc, ProdStateCfg::TILE)) return cudaErrorInvalidValue;
+    CUtensorMap mx, mwk, mwv;
+    if (!encode_x_map(&mx, x, h->desc) || !encode_w_pair_map(&mwk, w_k, C, h->desc.H) ||
+        !encode_w_pair_map(&mwv, w_v, C, h->desc.H))
+        return cudaErrorInvalidValue;
     ProducerArgs pa;
     pa.N = h->desc.N;
     pa.H = h->desc.H;
-    pa.chunks = C / ProdStateCfg::KC;
+    pa.chunks = C / ProdState2Cfg::KC;
     pa.has_t = t_k != nullptr ? 1 : 0;
-    cudaError_t e = launch_chained(producer_state_kernel<KIND>, dim3(p.G_state), dim3(ProdStateCfg::THREADS),
-                                   ProdStateCfg::SMEM_BYTES, s, mx, mwk, mwv, mt, h->partials, h->status, pa,
-                                   p.tiles_state, p.W_state, p.spans);
+    cudaError_t e = launch_chained(producer_state2_kernel<KIND>, dim3(p.G_x), dim3(ProdState2Cfg::THREADS),
+                                   ProdState2Cfg::SMEM_BYTES, s, mx, mwk, mwv, static_cast<const __nv_bfloat16*>(t_k),
+                                   h->partials, h->status, pa, p.tiles_state, p.W_x, p.spans_x);
     if (e != cudaSuccess) return e;
-    e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
-                       h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
-                       p.spans, dtype_of(h->desc), operand_scale(h->desc));
+    e = launch_chained(producer_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
+                       h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_x, p.G_x, p.spans_x,
+                       h->desc.H, dtype_of(h->desc), operand_scale(h->desc));
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
@@ -1623,7 +1669,7 @@ cudaError_t launch_apply_x(const linfusion_attn* h, const void* x, const void* w
     const Plan& p = h->plan;
     const int C = h->desc.H * kStreamD;
     CUtensorMap mx, mwq, mt, my;
-    if (!encode_x_map(&mx, x, h->desc) || !encode_w_map(&mwq, w_q, C) ||
+    if (!encode_x_map(&mx, x, h->desc) || !encode_w_pair_map(&mwq, w_q, C, h->desc.H) ||
         !encode_slab_map(&mt, t_q != nullptr ? t_q : x, h->desc, ProdApplyCfg::TILE) ||
         !encode_slab_map(&my, y, h->desc, ProdApplyCfg::TILE))
         return cudaErrorInvalidValue;

@@ -103,6 +103,11 @@ __device__ __forceinline__ void tma_load_2d_addr(uint32_t dst, const void* tmap,
         : "memory");
 }
 
+// Heads are taken in pairs (2p, 2p + 1); with an odd head count the last pair's second head does
+// not exist: its weight boxes and T tile lie past the tensors' extents (TMA fills zeros), and nothing
+// of it is stored.
+__host__ __device__ __forceinline__ int head_pairs(int H) { return (H + 1) / 2; }
+
 __device__ __forceinline__ uint64_t policy_evict_last()
 {
     uint64_t p;
@@ -461,6 +466,357 @@ producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// State from X, two heads per unit.  One tcgen05.mma costs its issuing thread about 125 cycles
+// whatever its N, so the projection runs at N = 256: D1[128 x 256] = X_tile [W_K,h0 | W_K,h1 | W_V,h0 | W_V,h1].
+// A double-buffered accumulator of that width is all of tensor memory, so the state contraction
+// itself moves to the epilogue warps: group e (four warps) writes phi(K_e) | V_e of the tile into
+// padded shared memory and accumulates S_e^T-by-rows with warp-level MMAs, fp32 in registers, exactly
+// as the split path does (warp w of the group owns features 16 w .. 16 w + 15 of S and z).
+// Units are (batch, head pair, 128-token tile), pair-major; CTA g of G owns a contiguous run; a run is
+// a sequence of visits to (batch, head pair)s; partials[((g * spans + visit) * 2 + e)][S 64x64 | z 64].
+// ---------------------------------------------------------------------------------------------
+struct ProdState2Cfg {
+    static constexpr int TILE = 128;
+    static constexpr int KC = 64;
+    static constexpr int STAGES = 3;
+    static constexpr int X_BYTES = TILE * 128;       // 16 KB
+    static constexpr int W_BYTES = 4 * KC * 128;     // 32 KB: 64 input rows x four 64-column blocks
+    static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
+    static constexpr int PITCH = 144;                // bytes per token row of a staged tile: odd in 16-byte units
+    static constexpr int KV_BYTES = 2 * TILE * PITCH;  // phi(K) tile then V tile of one head
+    static constexpr int EPI_GROUPS = 2;
+    static constexpr int EPI_WARPS = 4 * EPI_GROUPS;
+    static constexpr int PRODUCER_WARP = EPI_WARPS;
+    static constexpr int MMA_WARP = EPI_WARPS + 1;
+    static constexpr int WPRODUCER_WARP = EPI_WARPS + 2;
+    static constexpr int THREADS = 32 * (EPI_WARPS + 3);
+    static constexpr int TMEM_COLS = 512;            // two projection accumulators of 256 columns
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_GROUPS * KV_BYTES + 1024 + 1024;
+};
+static_assert(ProdState2Cfg::SMEM_BYTES > 116 * 1024 && ProdState2Cfg::SMEM_BYTES <= 227 * 1024, "one CTA per SM");
+static_assert(ProdState2Cfg::STAGE_BYTES % 1024 == 0, "operands on 1024-byte boundaries");
+
+__device__ __forceinline__ void named_barrier_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+// Barrier over `threads` threads that also tells everybody whether `ok` held for all of them, so
+// that a group leaves a loop that contains barriers together or not at all.
+__device__ __forceinline__ bool named_barrier_all(int id, int threads, bool ok)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(ok ? 1u : 0u), "r"(id), "r"(threads)
+        : "memory");
+    return r != 0u;
+}
+
+template <int KIND>
+__global__ void __launch_bounds__(ProdState2Cfg::THREADS, 1)
+producer_state2_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_wk,
+                       const __grid_constant__ CUtensorMap tmap_wv, const __nv_bfloat16* __restrict__ t_k,
+                       float* __restrict__ partials, uint32_t* __restrict__ status, ProducerArgs pa,
+                       int tiles_per_slab, long long W, int spans)
+{
+    using C = ProdState2Cfg;
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* smem = reinterpret_cast<unsigned char*>(
+        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    unsigned char* kv = smem + C::STAGES * C::STAGE_BYTES;  // per head of the pair: phi(K) tile | V tile, padded rows
+    uint64_t* full = reinterpret_cast<uint64_t*>(kv + C::EPI_GROUPS * C::KV_BYTES);
+    uint64_t* empty = full + C::STAGES;
+    uint64_t* d1_done = empty + C::STAGES;  // [2]
+    uint64_t* d1_free = d1_done + 2;        // [2]
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(d1_free + 2);
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const long long G = gridDim.x, g = blockIdx.x;
+    const long long u0 = unit_begin(g, W, G), u1 = unit_begin(g + 1, W, G);
+    const int n_units = static_cast<int>(u1 - u0);
+    const int KCH = pa.chunks;
+    const int HP = head_pairs(pa.H);
+
+    if (tid == 0) {
+        for (int s = 0; s < C::STAGES; ++s) {
+            mbar_init(&full[s], 2);
+            mbar_init(&empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&d1_done[b], 1);
+            mbar_init(&d1_free[b], 8);
+        }
+        mbar_fence_init();
+    }
+    if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+    if (warp == C::PRODUCER_WARP && lane == 0) prefetch_tmap(&tmap_x);
+    if (warp == C::WPRODUCER_WARP && lane == 0) {
+        prefetch_tmap(&tmap_wk);
+        prefetch_tmap(&tmap_wv);
+    }
+    pdl_launch_dependents();
+    pdl_wait();
+
+    if (warp == C::WPRODUCER_WARP) {
+        // ---------------- W producer: [W_K | W_V] chunks of both heads (a head past the last: zero fill) ----------------
+        if (lane == 0) {
+            const uint64_t pol_w = policy_evict_last();
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), w0 = smem_u32(smem) + C::X_BYTES;
+            RingPos<C::STAGES> r;
+            bool ok = true;
+            for (int it = 0; it < n_units && ok; ++it) {
+                const int h0 = static_cast<int>(((u0 + it) / tiles_per_slab) % HP) * 2;
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
+                    if (!ok) break;
+                    const uint32_t dst = w0 + r.s * C::STAGE_BYTES, bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::W_BYTES);
+                    // one box per weight matrix: 64 input rows x the 64-column blocks of both heads
+                    tma_load_3d_addr(dst, &tmap_wk, 0, kc * C::KC, h0, bar, pol_w);
+                    tma_load_3d_addr(dst + 16384, &tmap_wv, 0, kc * C::KC, h0, bar, pol_w);
+                }
+            }
+            if (!ok) report_wait_expired(status);
+        }
+    } else if (warp == C::PRODUCER_WARP) {
+        // ---------------- X producer (its drain covers the W loads too) ----------------
+        if (lane == 0) {
+            const uint64_t pol_x = policy_evict_first();
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), x0 = smem_u32(smem);
+            RingPos<C::STAGES> r;
+            bool ok = true;
+            int issued = 0;
+            for (int it = 0; it < n_units && ok; ++it) {
+                const long long u = u0 + it;
+                const int ps = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
+                const int b = ps / HP;
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
+                    if (!ok) break;
+                    const uint32_t bar = full0 + 8 * r.s;
+                    mbar_expect_tx_addr(bar, C::X_BYTES);
+                    tma_load_3d_addr(x0 + r.s * C::STAGE_BYTES, &tmap_x, kc * C::KC, tile * C::TILE, b, bar, pol_x);
+                    ++issued;
+                }
+            }
+            if (!ok) report_wait_expired(status);
+            drain_loads<C::STAGES>(full, 0, issued, status);
+        }
+    } else if (warp == C::MMA_WARP) {
+        // ---------------- MMA warp: the projections only ----------------
+        if (lane == 0) {
+            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), 128, 256, kUmmaBMnMajor);
+            const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
+            const uint64_t b_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, C::KC * 128, 1024);
+            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty);
+            RingPos<C::STAGES> r;
+            bool ok = true;
+            for (int it = 0; it < n_units && ok; ++it) {
+                const int buf = it & 1;
+                if (it >= 2) ok = mbar_wait(&d1_free[buf], ((it >> 1) - 1) & 1);
+                if (!ok) break;
+                const uint32_t d1 = tmem_base + buf * 256;
+                for (int kc = 0; kc < KCH; ++kc, r.next()) {
+                    ok = mbar_wait_addr(full0 + 8 * r.s, r.phase);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const uint64_t step = static_cast<uint64_t>(r.s * (C::STAGE_BYTES >> 4));
+                    const uint64_t a_desc = a_desc0 + step, b_desc = b_desc0 + step;
+                    umma_ss(d1, a_desc, b_desc, idesc, kc > 0 ? 1u : 0u);
+#pragma unroll
+                    for (int k = 1; k < C::KC / 16; ++k) umma_ss(d1, a_desc + 2 * k, b_desc + 128 * k, idesc, 1u);
+                    umma_commit_addr(empty0 + 8 * r.s);
+                }
+                if (!ok) break;
+                umma_commit(&d1_done[buf]);
+            }
+            if (!ok) report_wait_expired(status);
+        }
+    } else {
+        // ---------------- epilogue warpgroups: group e owns head e of every pair ----------------
+        const int e = warp >> 2, wg = warp & 3;
+        const int row = wg * 32 + lane;
+        const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(wg * 32) << 16) + e * 64;  // K_e at +0, V_e at +128
+        unsigned char* Ksm = kv + e * C::KV_BYTES;
+        unsigned char* Vsm = Ksm + C::TILE * C::PITCH;
+        const uint32_t k_row = smem_u32(Ksm) + row * C::PITCH, v_row = smem_u32(Vsm) + row * C::PITCH;
+        // ldmatrix.trans lane addressing of the state MMA (A = phi(K)^T from the tile stored [token][feature],
+        // B = V from the tile stored [token][channel]); warp wg owns features 16 wg .. 16 wg + 15
+        const uint32_t a_off = smem_u32(Ksm) + ((lane & 7) + ((lane >> 4) << 3)) * C::PITCH + (wg * 16 + ((lane >> 3) & 1) * 8) * 2;
+        const uint32_t b_off = smem_u32(Vsm) + ((lane & 7) + (((lane >> 3) & 1) << 3)) * C::PITCH + ((lane >> 4) * 8) * 2;
+        const uint32_t ones = ones_pair<KIND>();
+        const int gq = lane >> 2, tq = lane & 3;
+        const int Cdim = pa.H * 64;
+        float acc[9][4];
+#pragma unroll
+        for (int nb = 0; nb < 9; ++nb)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[nb][i] = 0.0f;
+        bool ok = true;
+        int visit = -1, cur_ps = -1;
+        for (int it = 0; it < n_units; ++it) {
+            const long long u = u0 + it;
+            const int ps = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
+            const int b = ps / HP, h = 2 * (ps % HP) + e;
+            const bool head = h < pa.H;
+            const int tok = tile * C::TILE + row;
+            const bool live = tok < pa.N && head;  // rows past N (and a head that does not exist) count for nothing
+            if (ps != cur_ps) {
+                cur_ps = ps;
+                ++visit;
+            }
+            // the T row of this token and head, if any, on its way while the projection completes
+            uint4 tr[8];
+            if (pa.has_t != 0 && live) {
+                const uint4* src = reinterpret_cast<const uint4*>(t_k + (static_cast<size_t>(b) * pa.N + tok) * Cdim + h * 64);
+#pragma unroll
+                for (int c = 0; c < 8; ++c) tr[c] = ld_stream_16B(src + c);
+            }
+            const int buf = it & 1;
+            ok = named_barrier_all(3 + e, 128, mbar_wait(&d1_done[buf], (it >> 1) & 1));
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t d[32];
+                tmem_load_32cols(t_lane + buf * 256 + 32 * half, d);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    float f[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(d[8 * c + i]);
+                    if (pa.has_t != 0 && live) {
+                        const uint4 t4 = tr[4 * half + c];
+                        f[0] += pair_lo<KIND>(t4.x); f[1] += pair_hi<KIND>(t4.x);
+                        f[2] += pair_lo<KIND>(t4.y); f[3] += pair_hi<KIND>(t4.y);
+                        f[4] += pair_lo<KIND>(t4.z); f[5] += pair_hi<KIND>(t4.z);
+                        f[6] += pair_lo<KIND>(t4.w); f[7] += pair_hi<KIND>(t4.w);
+                    }
+                    uint32_t p0 = 0u, p1 = 0u, p2 = 0u, p3 = 0u;
+                    if (live) {
+                        p0 = pack_pair<KIND>(phi<KIND>(f[0]), phi<KIND>(f[1]));
+                        p1 = pack_pair<KIND>(phi<KIND>(f[2]), phi<KIND>(f[3]));
+                        p2 = pack_pair<KIND>(phi<KIND>(f[4]), phi<KIND>(f[5]));
+                        p3 = pack_pair<KIND>(phi<KIND>(f[6]), phi<KIND>(f[7]));
+                    }
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(k_row + (4 * half + c) * 16), "r"(p0), "r"(p1),
+                                 "r"(p2), "r"(p3)
+                                 : "memory");
+                }
+            }
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t d[32];
+                tmem_load_32cols(t_lane + buf * 256 + 128 + 32 * half, d);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint32_t p0 = pack_pair<KIND>(__uint_as_float(d[8 * c + 0]), __uint_as_float(d[8 * c + 1]));
+                    const uint32_t p1 = pack_pair<KIND>(__uint_as_float(d[8 * c + 2]), __uint_as_float(d[8 * c + 3]));
+                    const uint32_t p2 = pack_pair<KIND>(__uint_as_float(d[8 * c + 4]), __uint_as_float(d[8 * c + 5]));
+                    const uint32_t p3 = pack_pair<KIND>(__uint_as_float(d[8 * c + 6]), __uint_as_float(d[8 * c + 7]));
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(v_row + (4 * half + c) * 16), "r"(p0), "r"(p1),
+                                 "r"(p2), "r"(p3)
+                                 : "memory");
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&d1_free[buf]);
+            named_barrier_sync(1 + e, 128);  // the group's tiles are complete
+            // S^T rows 16 wg .. += phi(K)^T V over the tile's 128 tokens, z from a block of ones
+#pragma unroll
+            for (int ks = 0; ks < C::TILE / 16; ++ks) {
+                uint32_t a0, a1, a2, a3;
+                ldmatrix_x4_trans(a_off + ks * 16 * C::PITCH, a0, a1, a2, a3);
+#pragma unroll
+                for (int nbp = 0; nbp < 4; ++nbp) {
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(b_off + ks * 16 * C::PITCH + nbp * 32, b0, b1, b2, b3);
+                    mma_16816<KIND>(acc[2 * nbp], a0, a1, a2, a3, b0, b1);
+                    mma_16816<KIND>(acc[2 * nbp + 1], a0, a1, a2, a3, b2, b3);
+                }
+                mma_16816<KIND>(acc[8], a0, a1, a2, a3, ones, ones);
+            }
+            named_barrier_sync(1 + e, 128);  // everybody has read the tiles: the next unit may overwrite them
+            const bool visit_ends = it + 1 == n_units || static_cast<int>((u + 1) / tiles_per_slab) != ps;
+            if (visit_ends) {
+                // this CTA's share of slab (b, h): S [64][64] (row = feature c) then z [64]
+                if (head) {
+                    float* dst = partials + ((static_cast<size_t>(g) * spans + visit) * 2 + e) * kStreamStateFloats;
+                    const int c0 = wg * 16 + gq, c1 = c0 + 8;
+#pragma unroll
+                    for (int nb = 0; nb < 8; ++nb) {
+                        const int ee = nb * 8 + 2 * tq;
+                        *reinterpret_cast<float2*>(dst + c0 * 64 + ee) = make_float2(acc[nb][0], acc[nb][1]);
+                        *reinterpret_cast<float2*>(dst + c1 * 64 + ee) = make_float2(acc[nb][2], acc[nb][3]);
+                    }
+                    if (tq == 0) {
+                        dst[64 * 64 + c0] = acc[8][0];
+                        dst[64 * 64 + c1] = acc[8][2];
+                    }
+                }
+#pragma unroll
+                for (int nb = 0; nb < 9; ++nb)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) acc[nb][i] = 0.0f;
+            }
+        }
+        if (!ok && lane == 0) report_wait_expired(status);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, C::TMEM_COLS);
+    }
+}
+
+// The second stage for producer_state2_kernel's partials: grid (17, slabs), 256 threads; slab (b, h) is
+// head h % 2 of pair-slab (b, h / 2); its partials come from the CTAs whose run meets that pair-slab,
+// summed in CTA order.  Output as stream_reduce_kernel's: fp32 S | z, the 16-bit operand image, the tile counter.
+__global__ void __launch_bounds__(256)
+producer_reduce_kernel(const float* __restrict__ partials, float* __restrict__ state,
+                       unsigned char* __restrict__ operand, int* __restrict__ tile_counters, int tiles_per_slab,
+                       long long W, int G, int spans, int H, int dtype, float operand_scale)
+{
+    __shared__ float sums[256];
+    const int tid = threadIdx.x;
+    const int idx = blockIdx.x * 256 + tid;
+    const int slab = blockIdx.y;
+    pdl_launch_dependents();
+    pdl_wait();
+    if (blockIdx.x == 0 && tid == 0) tile_counters[slab] = 0;
+    float sum = 0.0f;
+    if (idx < kStreamStateFloats) {
+        const int HP = head_pairs(H);
+        const int ps = (slab / H) * HP + (slab % H) / 2, e = (slab % H) & 1;
+        const long long lo = static_cast<long long>(ps) * tiles_per_slab, hi = lo + tiles_per_slab;
+        long long g0 = (lo * G) / W;
+        while (g0 + 1 < G && unit_begin(g0 + 1, W, G) <= lo) ++g0;
+        while (g0 > 0 && unit_begin(g0, W, G) > lo) --g0;
+        long long g1 = (hi * G) / W;
+        while (g1 < G && unit_begin(g1, W, G) < hi) ++g1;
+        while (g1 > 0 && unit_begin(g1 - 1, W, G) >= hi) --g1;
+        // visit index of pair-slab ps in CTA g0's run; every later CTA starts inside it (its visit 0)
+        const int slot0 = ps - static_cast<int>(unit_begin(g0, W, G) / tiles_per_slab);
+        const size_t F = kStreamStateFloats;
+        const float* src = partials + idx;
+        sum += src[((static_cast<size_t>(g0) * spans + slot0) * 2 + e) * F];
+#pragma unroll 4
+        for (long long g = g0 + 1; g < g1; ++g) sum += src[((static_cast<size_t>(g) * spans) * 2 + e) * F];
+        state[static_cast<size_t>(slab) * F + idx] = sum;
+    }
+    sums[tid] = sum;
+    __syncthreads();
+    emit_state_operand(sums, operand + static_cast<size_t>(slab) * kStreamOperandBytes, dtype, operand_scale);
+}
+
 struct ProdApplyCfg {
     static constexpr int TILE = 128;
     static constexpr int KC = 64;
@@ -491,11 +847,6 @@ static_assert((ProdApplyCfg::STAGES * ProdApplyCfg::STAGE_BYTES + ProdApplyCfg::
               "operands on 1024-byte boundaries");
 static_assert(ProdApplyCfg::TMEM_D2_0 + 2 * ProdApplyCfg::TMEM_D2_STEP <= ProdApplyCfg::TMEM_COLS, "TMEM budget");
 static_assert(ProdApplyCfg::SMEM_BYTES > 116 * 1024 && ProdApplyCfg::SMEM_BYTES <= 227 * 1024, "one CTA per SM");
-
-// Heads are taken in pairs (2p, 2p + 1); with an odd head count the last pair's second head does
-// not exist: its weight box and T tile lie past the tensors' extents (TMA fills zeros) and its Y
-// tile is not stored.
-__host__ __device__ __forceinline__ int head_pairs(int H) { return (H + 1) / 2; }
 
 // Y from X and the reduced state.  Units are (batch, head pair, 128-token tile), numbered
 // pair-major; CTA g of G owns the contiguous run [g*W/G, (g+1)*W/G).  A run is a sequence of VISITS
@@ -573,14 +924,14 @@ producer_apply_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
             RingPos<C::STAGES> r;
             bool ok = true;
             for (int it = 0; it < n_units && ok; ++it) {
-                const int col = static_cast<int>(((u0 + it) / tiles_per_slab) % HP) * 128;  // first column of head 2p
+                const int h0 = static_cast<int>(((u0 + it) / tiles_per_slab) % HP) * 2;
                 for (int kc = 0; kc < KCH; ++kc, r.next()) {
                     ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
                     if (!ok) break;
-                    const uint32_t dst = w0 + r.s * C::STAGE_BYTES, bar = full0 + 8 * r.s;
+                    const uint32_t bar = full0 + 8 * r.s;
                     mbar_expect_tx_addr(bar, C::W_BYTES);
-                    tma_load_2d_addr(dst, &tmap_wq, col, kc * C::KC, bar, pol_w);
-                    tma_load_2d_addr(dst + C::KC * 128, &tmap_wq, col + 64, kc * C::KC, bar, pol_w);
+                    // one box: 64 input rows x the 64-column blocks of both heads
+                    tma_load_3d_addr(w0 + r.s * C::STAGE_BYTES, &tmap_wq, 0, kc * C::KC, h0, bar, pol_w);
                 }
             }
             if (!ok) report_wait_expired(status);
