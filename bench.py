@@ -669,7 +669,7 @@ def run_from_x(args):
             "mode": "from_x", "shape": s.name, "B": B, "H": H, "N": N, "C": C, "dtype": "bf16", "steps": steps,
             "peak_tflops": {"burst": burst, "sustained": sustained, "kind": "of " + kind},
             "kernels": {
-                "producer_state_kernel+reduce": {"ms": ms_state, "tflops": tf(2 * proj + attn_half, ms_state)},
+                "producer_state2_kernel+reduce": {"ms": ms_state, "tflops": tf(2 * proj + attn_half, ms_state)},
                 "pack+producer_apply_kernel": {"ms": ms_apply, "tflops": tf(proj + attn_half, ms_apply)},
                 "producer_hidden_kernel+norm (one branch)": {"ms": ms_branch, "tflops": tf(proj, ms_branch)},
             },
@@ -679,7 +679,7 @@ def run_from_x(args):
                                                    "tokens_per_s": tokens / (ms_full * 1e-3)},
             "unfused_library_gemm_then_attention": {"ms": ms_unfused, "tokens_per_s": tokens / (ms_unfused * 1e-3),
                                                     "one_library_gemm_ms": ms_gemm, "one_library_gemm_tflops": tf(proj, ms_gemm)},
-            "roofline": {"bound": "tensor", "kernel": "producer_state_kernel", "achieved": tf(2 * proj + attn_half, ms_state),
+            "roofline": {"bound": "tensor", "kernel": "producer_state2_kernel", "achieved": tf(2 * proj + attn_half, ms_state),
                          "peak": sustained, "peak_kind": "of " + kind + " (sustained bf16)", "unit": "TFLOP/s",
                          "frac": tf(2 * proj + attn_half, ms_state) / sustained, "traffic": None},
         }

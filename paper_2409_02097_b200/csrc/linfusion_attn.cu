@@ -486,9 +486,6 @@ cudaError_t set_stream_attrs()
     e = cudaFuncSetAttribute(stream_fused_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              FusedCfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(producer_state_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             ProdStateCfg::SMEM_BYTES);
-    if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(producer_apply_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              ProdApplyCfg::SMEM_BYTES);
     if (e != cudaSuccess) return e;
@@ -1592,7 +1589,7 @@ bool encode_x_map(CUtensorMap* map, const void* x, const linfusion_attn_desc_t& 
     const cuuint64_t C = static_cast<cuuint64_t>(d.H) * kStreamD;
     cuuint64_t dims[3] = {C, static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.B)};
     cuuint64_t strides[2] = {C * 2, static_cast<cuuint64_t>(d.N) * C * 2};
-    cuuint32_t box[3] = {64u, static_cast<cuuint32_t>(ProdStateCfg::TILE), 1u};
+    cuuint32_t box[3] = {64u, static_cast<cuuint32_t>(ProdState2Cfg::TILE), 1u};
     cuuint32_t estr[3] = {1u, 1u, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,

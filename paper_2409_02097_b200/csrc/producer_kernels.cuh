@@ -10,22 +10,20 @@
 // feature vector, all heads, so it cannot be taken tile by tile per head) and added tile by tile
 // here; without that branch (its output is zero at the paper's initialization) T is absent.
 //
-// producer_state_kernel — per (batch, head) slab and 128-token tile:
-//     D1[128 x 128] = X_tile[128 x C] [W_K,h | W_V,h]      K loop over C in chunks of 64, operands by
-//                                                           TMA (X: K-major; W: [c_in][c_out] rows =
-//                                                           MN-major), accumulator in tensor memory
-//     epilogue: K = D1[:, 0:64] (+ T tile), phi(K) and V = D1[:, 64:128] rounded to 16 bits and laid
-//               out in shared memory exactly as TMA would have delivered a K and a V tile
-//     state MMA: the stream kernel's  D[128 x 64] += [V^T ; 1 ; 0] phi(K)^T   (Prop. 2, Eq. 5)
-//   The units, their split over CTAs and the partial-state format are stream_state_kernel's, so
-//   stream_reduce_kernel follows unchanged.
-// producer_apply_kernel — per slab and 128-token tile:
-//     D1[128 x 64] = X_tile W_Q,h ; epilogue: Q (+ T tile), phi(Q) -> tensor memory as the A operand
-//     D2[128 x 80] = phi(Q) [S | z] ; Y = D2[:, 0:64] / (D2[:, 64] + eps) -> shared -> TMA store
+// producer_state2_kernel — per (batch, head pair) and 128-token tile:
+//     D1[128 x 256] = X_tile[128 x C] [W_K,h0 | W_K,h1 | W_V,h0 | W_V,h1]   K loop over C in chunks of 64,
+//                                                           operands by TMA (X: K-major; W: [c_in][c_out]
+//                                                           rows = MN-major), accumulator in tensor memory
+//     epilogue (one warpgroup per head): K = D1 columns (+ T row), phi(K) and V rounded to 16 bits into
+//               padded shared-memory tiles; S^T rows += phi(K)^T V and z on warp-level MMAs (Prop. 2, Eq. 5)
+//   producer_reduce_kernel sums the CTAs' partial states in CTA order (fixed order).
+// producer_apply_kernel — per (batch, head pair) and 128-token tile:
+//     D1[128 x 128] = X_tile [W_Q,h0 | W_Q,h1] ; epilogue per head: Q (+ T tile), phi(Q) -> tensor memory as
+//     the A operand; D2[128 x 80] = phi(Q) [S | z] ; Y = D2[:, 0:64] / (D2[:, 64] + eps) -> shared -> TMA store
 //
-// Roles per CTA (one per SM): producer warp (TMA), MMA warp (one thread issues every tcgen05.mma),
-// two epilogue warpgroups that alternate units, and for the state kernel three flush warps.
-// Every wait is bounded.
+// Roles per CTA (one per SM): two producer warps (TMA: X chunks; W chunks), MMA warp (one thread issues
+// every tcgen05.mma), two epilogue warpgroups (one per head of the pair), a store warp where Y or U is
+// written.  Every wait is bounded.
 #pragma once
 
 #include <cuda_fp16.h>
@@ -115,30 +113,6 @@ __device__ __forceinline__ uint64_t policy_evict_last()
     return p;
 }
 
-struct ProdStateCfg {
-    static constexpr int TILE = 128;                 // tokens per unit = rows of the projection MMA
-    static constexpr int KC = 64;                    // input channels per K-loop chunk (one swizzle span)
-    static constexpr int STAGES = 4;                 // ring of (X chunk, W chunk) pairs
-    static constexpr int X_BYTES = TILE * 128;       // 16 KB: 128 tokens x 64 channels
-    static constexpr int W_BYTES = 2 * KC * 128;     // 16 KB: 64 input rows x (64 K columns | 64 V columns)
-    static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
-    static constexpr int KV_BYTES = 2 * TILE * 128;  // phi(K) tile then V tile, as the state MMA reads them
-    static constexpr int ONES_BYTES = 16 * 128;
-    static constexpr int EPI_GROUPS = 2;
-    static constexpr int EPI_WARPS = 4 * EPI_GROUPS;  // warps 0..7: warp % 4 = the TMEM lane quarter
-    static constexpr int FLUSH_WARP0 = EPI_WARPS;      // warps 8, 9, 10 = lane quarters 0, 1, 2
-    static constexpr int PRODUCER_WARP = EPI_WARPS + 3;   // X chunks (and T tiles)
-    static constexpr int MMA_WARP = EPI_WARPS + 4;
-    static constexpr int WPRODUCER_WARP = EPI_WARPS + 5;  // W chunks: two issuing threads halve the issue time per chunk
-    static constexpr int THREADS = 32 * (EPI_WARPS + 6);
-    static constexpr int SEGMENT_TILES = 32;
-    static constexpr int TMEM_COLS = 512;   // [0,256): two projection accumulators; [256,384): two state accumulators
-    static constexpr int TMEM_STATE0 = 256;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + EPI_GROUPS * KV_BYTES + ONES_BYTES + 1024 + 1024;
-};
-static_assert(ProdStateCfg::FLUSH_WARP0 % 4 == 0, "flush warps must cover TMEM lane quarters 0, 1, 2");
-static_assert(ProdStateCfg::SMEM_BYTES > 116 * 1024 && ProdStateCfg::SMEM_BYTES <= 227 * 1024, "one CTA per SM");
-
 // What the epilogues need besides the accumulator: whether a tile of the non-linear branch's
 // output is added, and the token count (rows past it must count for nothing).
 struct ProducerArgs {
@@ -147,324 +121,6 @@ struct ProducerArgs {
     int chunks;   // C / 64: K-loop length
     int has_t;    // nonzero: T tiles are loaded and added
 };
-
-template <int KIND>
-__global__ void __launch_bounds__(ProdStateCfg::THREADS, 1)
-producer_state_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_wk,
-                      const __grid_constant__ CUtensorMap tmap_wv, const __grid_constant__ CUtensorMap tmap_t,
-                      float* __restrict__ partials, uint32_t* __restrict__ status, ProducerArgs pa,
-                      int tiles_per_slab, long long W, int spans)
-{
-    using C = ProdStateCfg;
-    extern __shared__ unsigned char smem_raw[];
-    unsigned char* smem = reinterpret_cast<unsigned char*>(
-        (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    unsigned char* kv = smem + C::STAGES * C::STAGE_BYTES;       // two (phi(K) | V) operand tiles
-    unsigned char* ones = kv + C::EPI_GROUPS * C::KV_BYTES;
-    uint64_t* full = reinterpret_cast<uint64_t*>(ones + C::ONES_BYTES);
-    uint64_t* empty = full + C::STAGES;
-    uint64_t* d1_done = empty + C::STAGES;   // [2] projection accumulator complete
-    uint64_t* d1_free = d1_done + 2;         // [2] its epilogue has read it
-    uint64_t* t_full = d1_free + 2;          // [2] T tile landed in the operand buffer
-    uint64_t* kv_ready = t_full + 2;         // [2] phi(K) | V written
-    uint64_t* kv_free = kv_ready + 2;        // [2] the state MMAs that read them are complete
-    uint64_t* acc_done = kv_free + 2;        // [2]
-    uint64_t* acc_free = acc_done + 2;       // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(acc_free + 2);
-
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const long long G = gridDim.x, g = blockIdx.x;
-    const long long u0 = unit_begin(g, W, G), u1 = unit_begin(g + 1, W, G);
-    const int n_units = static_cast<int>(u1 - u0);
-    const int slab_first = static_cast<int>(u0 / tiles_per_slab);
-    const int KCH = pa.chunks;
-
-    if (tid == 0) {
-        for (int s = 0; s < C::STAGES; ++s) {
-            mbar_init(&full[s], 2);  // the X and the W issuer each announce their bytes
-            mbar_init(&empty[s], 1);
-        }
-        for (int b = 0; b < 2; ++b) {
-            mbar_init(&d1_done[b], 1);
-            mbar_init(&d1_free[b], 4);
-            mbar_init(&t_full[b], 1);
-            mbar_init(&kv_ready[b], 4);
-            mbar_init(&kv_free[b], 1);
-            mbar_init(&acc_done[b], 1);
-            mbar_init(&acc_free[b], 3);
-        }
-        mbar_fence_init();
-    }
-    for (int i = tid; i < C::ONES_BYTES / 4; i += C::THREADS) reinterpret_cast<uint32_t*>(ones)[i] = 0u;
-    __syncthreads();
-    if (tid < 16)
-        *reinterpret_cast<uint16_t*>(ones + tid * 128 + ((tid & 7) << 4)) = static_cast<uint16_t>(ones_pair<KIND>() & 0xffffu);
-    fence_proxy_async_smem();
-    if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
-    tc_fence_before_sync();
-    __syncthreads();
-    tc_fence_after_sync();
-    const uint32_t tmem_base = *tmem_slot;
-    if (warp == C::PRODUCER_WARP && lane == 0) {
-        prefetch_tmap(&tmap_x);
-        if (pa.has_t != 0) prefetch_tmap(&tmap_t);
-    }
-    if (warp == C::WPRODUCER_WARP && lane == 0) {
-        prefetch_tmap(&tmap_wk);
-        prefetch_tmap(&tmap_wv);
-    }
-    pdl_launch_dependents();
-    pdl_wait();
-
-    if (warp == C::WPRODUCER_WARP) {
-        // ---------------- W producer: the weight chunks of every unit ----------------
-        if (lane == 0) {
-            const uint64_t pol_w = policy_evict_last();
-            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), w0 = smem_u32(smem) + C::X_BYTES;
-            RingPos<C::STAGES> r;
-            bool ok = true;
-            for (int it = 0; it < n_units && ok; ++it) {
-                const int h64 = static_cast<int>(((u0 + it) / tiles_per_slab) % pa.H) * 64;
-                for (int kc = 0; kc < KCH; ++kc, r.next()) {
-                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
-                    if (!ok) break;
-                    const uint32_t dst = w0 + r.s * C::STAGE_BYTES, bar = full0 + 8 * r.s;
-                    mbar_expect_tx_addr(bar, C::W_BYTES);
-                    tma_load_2d_addr(dst, &tmap_wk, h64, kc * C::KC, bar, pol_w);
-                    tma_load_2d_addr(dst + C::KC * 128, &tmap_wv, h64, kc * C::KC, bar, pol_w);
-                }
-            }
-            if (!ok) report_wait_expired(status);
-        }
-    } else if (warp == C::PRODUCER_WARP) {
-        // ---------------- X producer (its drain at the end covers the W loads too: a stage's
-        // `full` phase completes only when both issuers' bytes have landed) ----------------
-        if (lane == 0) {
-            const uint64_t pol_x = policy_evict_first();
-            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty), x0 = smem_u32(smem);
-            RingPos<C::STAGES> r;
-            bool ok = true;
-            int issued = 0;
-            for (int it = 0; it < n_units && ok; ++it) {
-                const long long u = u0 + it;
-                const int slab = static_cast<int>(u / tiles_per_slab), tile = static_cast<int>(u % tiles_per_slab);
-                const int b = slab / pa.H, h = slab % pa.H;
-                for (int kc = 0; kc < KCH; ++kc, r.next()) {
-                    ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
-                    if (!ok) break;
-                    const uint32_t bar = full0 + 8 * r.s;
-                    mbar_expect_tx_addr(bar, C::X_BYTES);
-                    tma_load_3d_addr(x0 + r.s * C::STAGE_BYTES, &tmap_x, kc * C::KC, tile * C::TILE, b, bar, pol_x);
-                    ++issued;
-                }
-                if (ok && pa.has_t != 0) {
-                    // The non-linear branch's tile lands where phi(K) will be written; the buffer's
-                    // previous user (two units back) must be through with it.
-                    const int e = it & 1;
-                    if (it >= 2) ok = mbar_wait(&kv_free[e], ((it >> 1) - 1) & 1);
-                    if (!ok) break;
-                    mbar_expect_tx(&t_full[e], C::TILE * 128);
-                    tma_load_4d(kv + e * C::KV_BYTES, &tmap_t, 0, tile * C::TILE, h, b, &t_full[e], pol_x);
-                }
-            }
-            if (!ok) report_wait_expired(status);
-            drain_loads<C::STAGES>(full, 0, issued, status);
-        }
-    } else if (warp == C::MMA_WARP) {
-        // ---------------- MMA warp ----------------
-        if (lane == 0) {
-            const uint32_t idesc1 = umma_idesc_f32acc(kind_dtype(KIND), 128, 128, kUmmaBMnMajor);
-            const uint32_t idesc2 = umma_idesc_f32acc(kind_dtype(KIND), 128, 64, kUmmaAMnMajor | kUmmaBMnMajor);
-            const uint32_t ones_addr = smem_u32(ones);
-            bool ok = true;
-            int cur_slab = -1, in_segment = 0, segments = 0, abuf = 1;
-            // State MMAs of unit j (its phi(K) | V tile is in operand buffer j & 1).
-            auto state_mma = [&](int j) {
-                const int e = j & 1;
-                const int slab = static_cast<int>((u0 + j) / tiles_per_slab);
-                if (slab != cur_slab || in_segment == C::SEGMENT_TILES) {
-                    if (cur_slab >= 0) umma_commit(&acc_done[abuf]);
-                    abuf ^= 1;
-                    if (segments >= 2 && !mbar_wait(&acc_free[abuf], ((segments - 2) >> 1) & 1)) return false;
-                    ++segments;
-                    cur_slab = slab;
-                    in_segment = 0;
-                }
-                if (!mbar_wait(&kv_ready[e], (j >> 1) & 1)) return false;
-                tc_fence_after_sync();
-                const uint32_t k_addr = smem_u32(kv + e * C::KV_BYTES), v_addr = k_addr + C::TILE * 128;
-                const uint32_t d_tmem = tmem_base + C::TMEM_STATE0 + abuf * 64;
-#pragma unroll
-                for (int k = 0; k < C::TILE / 16; ++k) {
-                    const uint32_t va = v_addr + k * 2048;
-                    const uint64_t a_desc = umma_desc_mnmajor_sw128(va, ones_addr - va, 1024);
-                    const uint64_t b_desc = umma_desc_mnmajor_sw128(k_addr + k * 2048, 0, 1024);
-                    umma_ss(d_tmem, a_desc, b_desc, idesc2, (in_segment == 0 && k == 0) ? 0u : 1u);
-                }
-                ++in_segment;
-                umma_commit(&kv_free[e]);
-                return true;
-            };
-            // Descriptors of stage 0; a stage further on adds STAGE_BYTES / 16 to the address field.  A: the X
-            // chunk, K-major, one K step = 32 bytes.  B: the W chunk, 16 input rows per K step (2048
-            // bytes), its two 64-column blocks (K, V) 8 KB apart.
-            const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
-            const uint64_t b_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, C::KC * 128, 1024);
-            const uint32_t full0 = smem_u32(full), empty0 = smem_u32(empty);
-            RingPos<C::STAGES> r;
-            for (int it = 0; it < n_units && ok; ++it) {
-                const int e = it & 1;
-                // the accumulator's previous epilogue (two units back) must have read it
-                if (it >= 2) ok = mbar_wait(&d1_free[e], ((it >> 1) - 1) & 1);
-                if (!ok) break;
-                const uint32_t d1 = tmem_base + e * 128;
-                for (int kc = 0; kc < KCH; ++kc, r.next()) {
-                    ok = mbar_wait_addr(full0 + 8 * r.s, r.phase);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const uint64_t step = static_cast<uint64_t>(r.s * (C::STAGE_BYTES >> 4));
-                    const uint64_t a_desc = a_desc0 + step, b_desc = b_desc0 + step;
-                    umma_ss(d1, a_desc, b_desc, idesc1, kc > 0 ? 1u : 0u);
-#pragma unroll
-                    for (int k = 1; k < C::KC / 16; ++k) umma_ss(d1, a_desc + 2 * k, b_desc + 128 * k, idesc1, 1u);
-                    umma_commit_addr(empty0 + 8 * r.s);
-                }
-                if (!ok) break;
-                umma_commit(&d1_done[e]);
-                if (it >= 1) ok = state_mma(it - 1);
-            }
-            if (ok && n_units > 0) ok = state_mma(n_units - 1);
-            if (ok && cur_slab >= 0) umma_commit(&acc_done[abuf]);
-            if (!ok) report_wait_expired(status);
-        }
-    } else if (warp >= C::FLUSH_WARP0 && warp < C::FLUSH_WARP0 + 3) {
-        // ---------------- flush warps: the stream state kernel's, on the state accumulators ----------------
-        const int wq = warp & 3;
-        const uint32_t t_lane = tmem_base + C::TMEM_STATE0 + (static_cast<uint32_t>(wq * 32) << 16);
-        float acc[64];
-#pragma unroll
-        for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
-        int seg = 0;
-        bool ok = true;
-        for (int it = 0; it < n_units && ok;) {
-            const int slab = static_cast<int>((u0 + it) / tiles_per_slab);
-            const long long slab_end = static_cast<long long>(slab + 1) * tiles_per_slab - u0;
-            int len = static_cast<int>(slab_end < n_units ? slab_end : n_units) - it;
-            if (len > C::SEGMENT_TILES) len = C::SEGMENT_TILES;
-            it += len;
-            const int buf = seg & 1;
-            ok = mbar_wait(&acc_done[buf], (seg >> 1) & 1);
-            ++seg;
-            __syncwarp();
-            if (!ok) {
-                if (lane == 0) report_wait_expired(status);
-                break;
-            }
-            tc_fence_after_sync();
-#pragma unroll
-            for (int q4 = 0; q4 < 4; ++q4) {
-                uint32_t d[16];
-                tmem_load_16cols(t_lane + buf * 64 + 16 * q4, d);
-#pragma unroll
-                for (int c = 0; c < 16; ++c) acc[16 * q4 + c] += __uint_as_float(d[c]);
-            }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&acc_free[buf]);
-            if (it == n_units || it == slab_end) {
-                float* dst = partials + (static_cast<size_t>(g) * spans + (slab - slab_first)) * kStreamStateFloats;
-                if (wq < 2) {
-                    const int e = wq * 32 + lane;
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) dst[c * 64 + e] = acc[c];
-                } else if (lane == 0) {
-#pragma unroll
-                    for (int c = 0; c < 64; ++c) dst[64 * 64 + c] = acc[c];
-                }
-#pragma unroll
-                for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
-            }
-        }
-    } else if (warp < C::EPI_WARPS) {
-        // ---------------- epilogue warpgroups: group e takes units e, e + 2, ... ----------------
-        const int e = warp >> 2, wq = warp & 3;
-        const int row = wq * 32 + lane;
-        const uint32_t sw = row & 7;
-        const uint32_t t_row = tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + e * 128;
-        const uint32_t k_row = smem_u32(kv + e * C::KV_BYTES) + row * 128, v_row = k_row + C::TILE * 128;
-        bool ok = true;
-        for (int it = e; it < n_units; it += 2) {
-            const int n = it >> 1;
-            const int tile = static_cast<int>((u0 + it) % tiles_per_slab);
-            const bool live = tile * C::TILE + row < pa.N;  // rows past N must count for nothing
-            ok = mbar_wait(&d1_done[e], n & 1);
-            // the operand buffer's previous user (two units back): its state MMAs must be complete
-            if (ok && n >= 1) ok = mbar_wait(&kv_free[e], (n - 1) & 1);
-            if (ok && pa.has_t != 0) ok = mbar_wait(&t_full[e], n & 1);
-            __syncwarp();
-            if (!ok) break;
-            tc_fence_after_sync();
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                // K columns 32*half .. +31: (+ T), phi in fp32, round, store as the tile's row
-                uint32_t d[32];
-                tmem_load_32cols(t_row + 32 * half, d);
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t addr = k_row + (((4 * half + c) ^ sw) << 4);
-                    float f[8];
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(d[8 * c + i]);
-                    if (pa.has_t != 0) {
-                        uint32_t t0, t1, t2, t3;
-                        asm volatile("ld.shared.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(t0), "=r"(t1), "=r"(t2), "=r"(t3) : "r"(addr));
-                        f[0] += pair_lo<KIND>(t0); f[1] += pair_hi<KIND>(t0);
-                        f[2] += pair_lo<KIND>(t1); f[3] += pair_hi<KIND>(t1);
-                        f[4] += pair_lo<KIND>(t2); f[5] += pair_hi<KIND>(t2);
-                        f[6] += pair_lo<KIND>(t3); f[7] += pair_hi<KIND>(t3);
-                    }
-                    uint32_t p0 = 0u, p1 = 0u, p2 = 0u, p3 = 0u;
-                    if (live) {
-                        p0 = pack_pair<KIND>(phi<KIND>(f[0]), phi<KIND>(f[1]));
-                        p1 = pack_pair<KIND>(phi<KIND>(f[2]), phi<KIND>(f[3]));
-                        p2 = pack_pair<KIND>(phi<KIND>(f[4]), phi<KIND>(f[5]));
-                        p3 = pack_pair<KIND>(phi<KIND>(f[6]), phi<KIND>(f[7]));
-                    }
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(p0), "r"(p1), "r"(p2), "r"(p3) : "memory");
-                }
-            }
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                // V columns (rows past N are zero already: X was zero-filled there)
-                uint32_t d[32];
-                tmem_load_32cols(t_row + 64 + 32 * half, d);
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint32_t addr = v_row + (((4 * half + c) ^ sw) << 4);
-                    const uint32_t p0 = pack_pair<KIND>(__uint_as_float(d[8 * c + 0]), __uint_as_float(d[8 * c + 1]));
-                    const uint32_t p1 = pack_pair<KIND>(__uint_as_float(d[8 * c + 2]), __uint_as_float(d[8 * c + 3]));
-                    const uint32_t p2 = pack_pair<KIND>(__uint_as_float(d[8 * c + 4]), __uint_as_float(d[8 * c + 5]));
-                    const uint32_t p3 = pack_pair<KIND>(__uint_as_float(d[8 * c + 6]), __uint_as_float(d[8 * c + 7]));
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(p0), "r"(p1), "r"(p2), "r"(p3) : "memory");
-                }
-            }
-            tc_fence_before_sync();
-            fence_proxy_async_smem();
-            __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(&d1_free[e]);
-                mbar_arrive(&kv_ready[e]);
-            }
-        }
-        if (!ok && lane == 0) report_wait_expired(status);
-    }
-    tc_fence_before_sync();
-    __syncthreads();
-    if (warp == 0) {
-        tc_fence_after_sync();
-        tmem_dealloc(tmem_base, C::TMEM_COLS);
-    }
-}
 
 // ---------------------------------------------------------------------------------------------
 // State from X, two heads per unit.  One tcgen05.mma costs its issuing thread about 125 cycles
