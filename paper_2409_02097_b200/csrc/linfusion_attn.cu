@@ -1611,15 +1611,15 @@ bool encode_w_map(CUtensorMap* map, const void* w, int C)
 }
 
 // The same matrix seen as (column within head 64, input row C, head H) -> boxes of 64 input rows x the
-// 64-column blocks of TWO heads, which land in shared memory as two consecutive 8 KB blocks (head, row,
-// column): one copy per weight matrix and K chunk.  A head index past the last head reads as zeros.
-bool encode_w_pair_map(CUtensorMap* map, const void* w, int C, int H)
+// 64-column blocks of `heads` consecutive heads, which land in shared memory as consecutive 8 KB blocks
+// (head, row, column): one copy per weight matrix and K chunk.  A head index past the last head reads as zeros.
+bool encode_w_pair_map(CUtensorMap* map, const void* w, int C, int H, int heads = 2)
 {
     EncodeTiledFn fn = get_encode_fn();
     if (fn == nullptr) return false;
     cuuint64_t dims[3] = {64u, static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(H)};
     cuuint64_t strides[2] = {static_cast<cuuint64_t>(C) * 2, 128u};
-    cuuint32_t box[3] = {64u, 64u, 2u};
+    cuuint32_t box[3] = {64u, 64u, static_cast<cuuint32_t>(heads)};
     cuuint32_t estr[3] = {1u, 1u, 1u};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(w), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -1705,7 +1705,9 @@ cudaError_t launch_branch_x(const linfusion_attn* h, const void* x, const void* 
 {
     const int C = h->desc.H * kStreamD, N = h->desc.N, B = h->desc.B;
     CUtensorMap mx, mw, mu;
-    if (!encode_x_map(&mx, x, h->desc) || !encode_w_map(&mw, w_1, C) || !encode_x_map(&mu, t, h->desc)) return cudaErrorInvalidValue;
+    if (!encode_x_map(&mx, x, h->desc) || !encode_w_pair_map(&mw, w_1, C, h->desc.H, ProdHiddenCfg::NB_COLS / 64) ||
+        !encode_x_map(&mu, t, h->desc))
+        return cudaErrorInvalidValue;
     const int tiles = (N + ProdHiddenCfg::TILE - 1) / ProdHiddenCfg::TILE;
     const long long W = static_cast<long long>(B) * tiles;
     const int G = static_cast<int>(W < h->sm_count ? W : h->sm_count);

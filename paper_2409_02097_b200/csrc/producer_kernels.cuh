@@ -843,7 +843,7 @@ __device__ __forceinline__ void tma_store_3d(const void* tmap, const void* smem_
 // ---------------------------------------------------------------------------------------------
 // The non-linear branch of f' / g' (Sec. 3.1, implementation details): T = LeakyReLU(LayerNorm(X W_1 + b_1)).
 // LayerNorm runs over a token's whole feature vector, so it is taken in two steps:
-//   producer_hidden_kernel — U = X W_1 + b_1 on tcgen05, 128 tokens x 128 output columns at a time,
+//   producer_hidden_kernel — U = X W_1 + b_1 on tcgen05, 128 tokens x 256 output columns at a time,
 //                            rounded to 16 bits and stored by TMA; the thread that owns a token row
 //                            sums u and u^2 (fp32, before rounding) over all its column blocks and
 //                            leaves the row's mean and 1 / sqrt(variance + ln_eps);
@@ -852,12 +852,12 @@ __device__ __forceinline__ void tma_store_3d(const void* tmap, const void* smem_
 struct ProdHiddenCfg {
     static constexpr int TILE = 128;
     static constexpr int KC = 64;
-    static constexpr int NB_COLS = 128;              // output columns per block
-    static constexpr int STAGES = 4;
+    static constexpr int NB_COLS = 256;              // output columns per block: the widest MMA one CTA can issue
+    static constexpr int STAGES = 3;
     static constexpr int X_BYTES = TILE * 128;
-    static constexpr int W_BYTES = 2 * KC * 128;     // two 64-column boxes
+    static constexpr int W_BYTES = 4 * KC * 128;     // 64 input rows x four 64-column blocks (one TMA box)
     static constexpr int STAGE_BYTES = X_BYTES + W_BYTES;
-    static constexpr int OUT_BYTES = 2 * TILE * 128;  // 128 rows x (64 | 64) columns
+    static constexpr int OUT_BYTES = 4 * TILE * 128;  // 128 rows x four 64-column blocks
     static constexpr int MAX_C = 2048;
     static constexpr int EPI_WARPS = 4;
     static constexpr int PRODUCER_WARP = EPI_WARPS;
@@ -865,8 +865,8 @@ struct ProdHiddenCfg {
     static constexpr int STORE_WARP = EPI_WARPS + 2;
     static constexpr int WPRODUCER_WARP = EPI_WARPS + 3;  // W chunks (the producer warp issues the X chunks)
     static constexpr int THREADS = 32 * (EPI_WARPS + 4);
-    static constexpr int TMEM_COLS = 256;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 2 * OUT_BYTES + MAX_C * 4 + 1024 + 1024;
+    static constexpr int TMEM_COLS = 512;            // two accumulators of 256 columns
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + OUT_BYTES + MAX_C * 4 + 1024 + 1024;
 };
 static_assert(ProdHiddenCfg::SMEM_BYTES <= 227 * 1024, "shared memory budget");
 
@@ -883,14 +883,14 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     unsigned char* outb = smem + C::STAGES * C::STAGE_BYTES;
-    float* bias_s = reinterpret_cast<float*>(outb + 2 * C::OUT_BYTES);
+    float* bias_s = reinterpret_cast<float*>(outb + C::OUT_BYTES);
     uint64_t* full = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(bias_s) + C::MAX_C * 4);
     uint64_t* empty = full + C::STAGES;
     uint64_t* d1_done = empty + C::STAGES;  // [2]
     uint64_t* d1_free = d1_done + 2;        // [2]
-    uint64_t* out_ready = d1_free + 2;      // [2]
-    uint64_t* out_free = out_ready + 2;     // [2]
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_free + 2);
+    uint64_t* out_ready = d1_free + 2;      // the staged block is complete
+    uint64_t* out_free = out_ready + 1;     // the stores have read it
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(out_free + 1);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const long long G = gridDim.x, g = blockIdx.x;
@@ -908,9 +908,9 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int b = 0; b < 2; ++b) {
             mbar_init(&d1_done[b], 1);
             mbar_init(&d1_free[b], 4);
-            mbar_init(&out_ready[b], 4);
-            mbar_init(&out_free[b], 1);
         }
+        mbar_init(out_ready, 4);
+        mbar_init(out_free, 1);
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
@@ -937,15 +937,14 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             RingPos<C::STAGES> r;
             bool ok = true;
             for (int j = 0; j < n_blocks && ok; ++j) {
-                const int col = (j % NB) * C::NB_COLS;
+                const int blk64 = (j % NB) * (C::NB_COLS / 64);  // first 64-column block of this column block
                 for (int kc = 0; kc < KCH; ++kc, r.next()) {
                     ok = mbar_wait_addr(empty0 + 8 * r.s, r.phase ^ 1u);
                     if (!ok) break;
-                    const uint32_t dst = w0 + r.s * C::STAGE_BYTES, bar = full0 + 8 * r.s;
+                    const uint32_t bar = full0 + 8 * r.s;
                     mbar_expect_tx_addr(bar, C::W_BYTES);
-                    // (the second box of an odd last block lies past the last column: zero fill)
-                    tma_load_2d_addr(dst, &tmap_w1, col, kc * C::KC, bar, pol_w);
-                    tma_load_2d_addr(dst + C::KC * 128, &tmap_w1, col + 64, kc * C::KC, bar, pol_w);
+                    // one box of four 64-column blocks (those past the last column: zero fill)
+                    tma_load_3d_addr(w0 + r.s * C::STAGE_BYTES, &tmap_w1, 0, kc * C::KC, blk64, bar, pol_w);
                 }
             }
             if (!ok) report_wait_expired(status);
@@ -974,7 +973,7 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         }
     } else if (warp == C::MMA_WARP) {
         if (lane == 0) {
-            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), 128, 128, kUmmaBMnMajor);
+            const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), 128, 256, kUmmaBMnMajor);
             bool ok = true;
             const uint64_t a_desc0 = umma_desc_kmajor_sw128(smem_u32(smem));
             const uint64_t b_desc0 = umma_desc_mnmajor_sw128(smem_u32(smem) + C::X_BYTES, C::KC * 128, 1024);
@@ -984,7 +983,7 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
                 const int e = j & 1;
                 if (j >= 2) ok = mbar_wait(&d1_free[e], ((j >> 1) - 1) & 1);
                 if (!ok) break;
-                const uint32_t d1 = tmem_base + e * 128;
+                const uint32_t d1 = tmem_base + e * 256;
                 for (int kc = 0; kc < KCH; ++kc, r.next()) {
                     ok = mbar_wait_addr(full0 + 8 * r.s, r.phase);
                     if (!ok) break;
@@ -1005,19 +1004,18 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         if (lane == 0) {
             const uint64_t policy = policy_evict_last();  // read again soon by the normalization
             for (int j = 0; j < n_blocks; ++j) {
-                const int e = j & 1;
-                if (!mbar_wait(&out_ready[e], (j >> 1) & 1)) {
+                if (!mbar_wait(out_ready, j & 1)) {
                     report_wait_expired(status);
                     break;
                 }
                 const long long u = u0 + j / NB;
                 const int nb = j % NB;
                 const int b = static_cast<int>(u / tiles_per_batch), tile = static_cast<int>(u % tiles_per_batch);
-                tma_store_3d(&tmap_u, outb + e * C::OUT_BYTES, nb * C::NB_COLS, tile * C::TILE, b, policy);
-                if (nb * C::NB_COLS + 64 < Cdim)
-                    tma_store_3d(&tmap_u, outb + e * C::OUT_BYTES + C::TILE * 128, nb * C::NB_COLS + 64, tile * C::TILE, b, policy);
+                for (int q = 0; q < C::NB_COLS / 64; ++q)
+                    if (nb * C::NB_COLS + 64 * q < Cdim)
+                        tma_store_3d(&tmap_u, outb + q * (C::TILE * 128), nb * C::NB_COLS + 64 * q, tile * C::TILE, b, policy);
                 tma_store_wait_read();
-                mbar_arrive(&out_free[e]);
+                mbar_arrive(out_free);
             }
             tma_store_wait_all();
         }
@@ -1031,14 +1029,14 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         for (int j = 0; j < n_blocks; ++j) {
             const int e = j & 1, nb = j % NB;
             ok = mbar_wait(&d1_done[e], (j >> 1) & 1);
-            if (ok && j >= 2) ok = mbar_wait(&out_free[e], ((j >> 1) - 1) & 1);
+            if (ok && j >= 1) ok = mbar_wait(out_free, (j - 1) & 1);
             __syncwarp();
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + e * 128;
-            const uint32_t o_row = smem_u32(outb + e * C::OUT_BYTES) + row * 128;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(wq * 32) << 16) + e * 256;
+            const uint32_t o_row = smem_u32(outb) + row * 128;
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
+            for (int q = 0; q < C::NB_COLS / 32; ++q) {
                 // columns 32 q .. + 31 of the block: half q / 2 of the staging tile, chunks 4 (q % 2) ..
                 uint32_t d[32];
                 tmem_load_32cols(t_row + 32 * q, d);
@@ -1068,7 +1066,7 @@ producer_hidden_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
             __syncwarp();
             if (lane == 0) {
                 mbar_arrive(&d1_free[e]);
-                mbar_arrive(&out_ready[e]);
+                mbar_arrive(out_ready);
             }
             if (nb == NB - 1) {
                 // the row is complete: mean and 1 / sqrt(biased variance + ln_eps) over its Cdim features
