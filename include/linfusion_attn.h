@@ -411,6 +411,28 @@ linfusion_status_t linfusion_attn_forward_x(linfusion_attn_t* h, const void* x,
                                             const linfusion_module_weights_t* w, void* y,
                                             void* cuda_stream);
 
+/*
+ * The bounds-checked debugging build (the paper has no counterpart; it stands in for a memory checker).
+ * The same sources compiled with -DLF_CHECKED give a second library in which forward(), forward_noalloc(),
+ * state(), apply() and apply_peers() of the SPLIT and CLUSTER variants first tell the device which byte
+ * ranges the call may touch (Q, K, V, Y, the workspace, peers' states), and every global-memory address
+ * these kernels compute is compared with them: an access that does not lie wholly inside one range is
+ * counted and skipped (loads return zero) — nothing traps or faults, the call completes.  One range table
+ * per device: checked calls on different streams must not overlap in time.
+ *   checked_build():       1 in that library, 0 in the normal one.
+ *   checked_violations():  synchronizes `device` and returns the number of skipped accesses since the
+ *                          last reset in *count (reset != 0 clears it).  UNSUPPORTED in the normal build
+ *                          (*count = 0).  Errors: INVALID_ARG, CUDA.
+ *   checked_shrink_y():    self-test of the check itself: from now on the registered range of Y is cut
+ *                          short by `bytes` at its end, so that the (valid) stores to the last rows of Y
+ *                          are reported and skipped and those rows keep what they held; 0 restores the
+ *                          full range.  No access leaves its buffer either way.  UNSUPPORTED in the
+ *                          normal build.
+ */
+int32_t linfusion_attn_checked_build(void);
+linfusion_status_t linfusion_attn_checked_violations(int32_t device, uint32_t* count, int32_t reset);
+linfusion_status_t linfusion_attn_checked_shrink_y(size_t bytes);
+
 /* Name of the kernel variant the handle resolved to ("split", "stream", "cluster", "fused"). */
 const char* linfusion_attn_variant_name(const linfusion_attn_t* h);
 

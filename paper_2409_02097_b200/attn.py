@@ -11,7 +11,8 @@ import os
 from typing import Optional
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "liblinfusion_attn.so")
+# LINFUSION_ATTN_LIB selects another build of the same library (the bounds-checked debugging build)
+LIB_PATH = os.environ.get("LINFUSION_ATTN_LIB") or os.path.join(_PKG, "liblinfusion_attn.so")
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT = range(6)
 PHI_ELU_PLUS_ONE, PHI_IDENTITY = 0, 1
@@ -30,6 +31,7 @@ EXPORTED = [
     "linfusion_attn_state", "linfusion_attn_apply", "linfusion_attn_state_buffer",
     "linfusion_attn_apply_peers", "linfusion_attn_selftest_wait", "linfusion_attn_selftest_counter_wait",
     "linfusion_attn_state_x", "linfusion_attn_apply_x", "linfusion_attn_branch_x", "linfusion_attn_forward_x",
+    "linfusion_attn_checked_build", "linfusion_attn_checked_violations", "linfusion_attn_checked_shrink_y",
 ]
 
 
@@ -128,8 +130,35 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_branch_x.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, vp]
     lib.linfusion_attn_forward_x.restype = st
     lib.linfusion_attn_forward_x.argtypes = [vp, vp, ctypes.POINTER(ModuleWeights), vp, vp]
+    lib.linfusion_attn_checked_build.restype = ctypes.c_int32
+    lib.linfusion_attn_checked_build.argtypes = []
+    lib.linfusion_attn_checked_violations.restype = st
+    lib.linfusion_attn_checked_violations.argtypes = [ctypes.c_int32, ctypes.POINTER(ctypes.c_uint32), ctypes.c_int32]
+    lib.linfusion_attn_checked_shrink_y.restype = st
+    lib.linfusion_attn_checked_shrink_y.argtypes = [ctypes.c_size_t]
     _lib = lib
     return lib
+
+
+def checked_build() -> bool:
+    """True when the loaded library is the bounds-checked debugging build."""
+    return bool(load_library().linfusion_attn_checked_build())
+
+
+def checked_shrink_y(nbytes: int) -> None:
+    """Self-test of the checked build: register Y ``nbytes`` short, so that its last rows count as out of range."""
+    rc = load_library().linfusion_attn_checked_shrink_y(int(nbytes))
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_checked_shrink_y")
+
+
+def checked_violations(device: int = 0, reset: bool = True) -> int:
+    """Global-memory accesses the checked build found outside the buffers of their call (and skipped)."""
+    n = ctypes.c_uint32(0)
+    rc = load_library().linfusion_attn_checked_violations(int(device), ctypes.byref(n), 1 if reset else 0)
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_checked_violations")
+    return int(n.value)
 
 
 def status_string(code: int) -> str:

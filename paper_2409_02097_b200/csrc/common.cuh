@@ -90,12 +90,6 @@ struct PeerStates {
     const float* p[kMaxPeers];
     int n;
 };
-__device__ __forceinline__ float peer_sum(const PeerStates& ps, size_t i)
-{
-    float sum = 0.0f;
-    for (int r = 0; r < ps.n; ++r) sum += ps.p[r][i];
-    return sum;
-}
 
 __device__ __forceinline__ float bf16_lo(uint32_t p) { return __uint_as_float(p << 16); }
 __device__ __forceinline__ float bf16_hi(uint32_t p) { return __uint_as_float(p & 0xffff0000u); }
@@ -238,11 +232,70 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
 }
 
 // ---------------------------------------------------------------------------------------------
+// Checked build (-DLF_CHECKED; a second library, for debugging, never the one that is benchmarked).
+// The host registers the byte ranges a forward may touch (Q, K, V, Y, the workspace, peers' states);
+// every global-memory access the split / cluster kernels compute an address for goes through
+// lf_in_bounds(): an access that does not lie wholly inside one registered range is counted and
+// SKIPPED (a load returns zeros) — no trap, no fault, the kernel runs to its end and the host reads
+// the count.  Addresses in shared memory (the cluster kernel keeps partial states there) pass.
+// In the normal build lf_in_bounds() is the constant true and costs nothing.
+// ---------------------------------------------------------------------------------------------
+#ifdef LF_CHECKED
+constexpr int kCheckedMaxRanges = 24;
+struct CheckedRanges {
+    unsigned long long lo[kCheckedMaxRanges];
+    unsigned long long hi[kCheckedMaxRanges];
+    int n;
+};
+__device__ CheckedRanges g_checked_ranges;
+__device__ unsigned int g_checked_violations;
+__device__ __forceinline__ bool lf_in_bounds(const void* p, unsigned int bytes)
+{
+    if (!__isGlobal(p)) return true;
+    const unsigned long long a = reinterpret_cast<unsigned long long>(p);
+    for (int i = 0; i < g_checked_ranges.n; ++i)
+        if (a >= g_checked_ranges.lo[i] && a + bytes <= g_checked_ranges.hi[i]) return true;
+    atomicAdd(&g_checked_violations, 1u);
+    return false;
+}
+#else
+__device__ __forceinline__ constexpr bool lf_in_bounds(const void*, unsigned int) { return true; }
+#endif
+
+// Plain global loads and stores of the split / cluster kernels, through the check above.
+template <typename T>
+__device__ __forceinline__ T g_load(const T* p)
+{
+    if (!lf_in_bounds(p, sizeof(T))) return T{};
+    return *p;
+}
+template <typename T>
+__device__ __forceinline__ T g_load_ro(const T* p)  // read-only data path
+{
+    if (!lf_in_bounds(p, sizeof(T))) return T{};
+    return __ldg(p);
+}
+template <typename T>
+__device__ __forceinline__ void g_store(T* p, T v)
+{
+    if (lf_in_bounds(p, sizeof(T))) *p = v;
+}
+
+// Element i of the sum of the devices' states, in list order (see PeerStates).
+__device__ __forceinline__ float peer_sum(const PeerStates& ps, size_t i)
+{
+    float sum = 0.0f;
+    for (int r = 0; r < ps.n; ++r) sum += g_load(ps.p[r] + i);
+    return sum;
+}
+
+// ---------------------------------------------------------------------------------------------
 // Global memory access with streaming hints (each byte of Q, K, V, Y is touched once)
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint4 ld_stream_16B(const void* p)
 {
     uint4 v;
+    if (!lf_in_bounds(p, 16)) return make_uint4(0u, 0u, 0u, 0u);
     asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                  : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
                  : "l"(p));
@@ -251,6 +304,7 @@ __device__ __forceinline__ uint4 ld_stream_16B(const void* p)
 
 __device__ __forceinline__ void st_stream_16B(void* p, uint4 v)
 {
+    if (!lf_in_bounds(p, 16)) return;
     asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
                  "r"(v.w)
                  : "memory");
@@ -258,6 +312,7 @@ __device__ __forceinline__ void st_stream_16B(void* p, uint4 v)
 
 __device__ __forceinline__ void st_stream_4B(void* p, uint32_t v)
 {
+    if (!lf_in_bounds(p, 4)) return;
     asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 

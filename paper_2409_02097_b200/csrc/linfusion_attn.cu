@@ -374,6 +374,7 @@ struct linfusion_attn {
     Plan plan;
     int sm_count;
     void* ws;  // device workspace in use
+    size_t ws_bytes;
     bool owns_ws;
     float* partials;
     float* state;
@@ -412,6 +413,7 @@ namespace {
 void bind_workspace(linfusion_attn* h, void* ws)
 {
     h->ws = ws;
+    h->ws_bytes = h->plan.total_bytes;
     unsigned char* base = static_cast<unsigned char*>(ws);
     h->partials = reinterpret_cast<float*>(base);
     h->state = reinterpret_cast<float*>(base + h->plan.state_off);
@@ -516,10 +518,46 @@ cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
+// Checked build: tell the kernels, in stream order, which byte ranges this call may touch (Q and K,
+// V and Y, the workspace, and for the peer-summed apply the devices' state buffers).  One table per
+// device: checked calls on different streams must not overlap.  Nothing in the normal build.
+#ifdef LF_CHECKED
+// Self-test of the check: the registered Y range is cut short by this many bytes, so that the (valid)
+// stores to the end of Y are reported and skipped.
+std::atomic<size_t> g_checked_shrink_y{0};
+#endif
+
+void register_checked_ranges(const linfusion_attn* h, const void* q, const void* k, const void* v, const void* y,
+                             cudaStream_t s, const PeerStates* peers = nullptr)
+{
+#ifdef LF_CHECKED
+    CheckedRanges r;
+    r.n = 0;
+    auto add = [&](const void* p, size_t bytes) {
+        if (p == nullptr || r.n >= kCheckedMaxRanges) return;
+        r.lo[r.n] = reinterpret_cast<unsigned long long>(p);
+        r.hi[r.n] = r.lo[r.n] + bytes;
+        ++r.n;
+    };
+    add(q, bytes_qk(h->desc));
+    add(k, bytes_qk(h->desc));
+    add(v, bytes_vy(h->desc));
+    const size_t shrink = g_checked_shrink_y.load();
+    add(y, bytes_vy(h->desc) > shrink ? bytes_vy(h->desc) - shrink : 0);
+    add(h->ws, h->ws_bytes);
+    if (peers != nullptr)
+        for (int i = 0; i < peers->n; ++i) add(peers->p[i], static_cast<size_t>(h->plan.slabs) * h->plan.state_floats * 4);
+    cudaMemcpyToSymbolAsync(g_checked_ranges, &r, sizeof(r), 0, cudaMemcpyHostToDevice, s);
+#else
+    (void)h; (void)q; (void)k; (void)v; (void)y; (void)s; (void)peers;
+#endif
+}
+
 template <int DK, int DV, int KIND>
 cudaError_t launch_split(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                          const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
+    register_checked_ranges(h, q, k, v, y, s);
     using C = SplitCfg<DK, DV>;
     const Plan& p = h->plan;
     const int N = h->desc.N;
@@ -565,6 +603,7 @@ template <int DK, int DV, int KIND>
 cudaError_t launch_cluster(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
                            const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
 {
+    register_checked_ranges(h, q, k, v, y, s);
     cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[1];
     cluster_config<DK, DV>(&cfg, attr, h->plan.cluster_size, h->plan.slabs, s);
@@ -1385,6 +1424,7 @@ extern "C" linfusion_status_t linfusion_attn_forward_noalloc(const linfusion_att
     if (bytes_used > kNoAllocScratchBytes) return LINFUSION_ERR_ALLOC;  // cannot happen; the array is never overrun
     view.sm_count = dev.sm_count;
     view.ws = dev.scratch;
+    view.ws_bytes = bytes_used;
     view.owns_ws = false;
     view.partials = reinterpret_cast<float*>(dev.scratch);
     view.state = reinterpret_cast<float*>(dev.scratch + state_off);
@@ -1434,6 +1474,10 @@ cudaError_t launch_split_half(const linfusion_attn* h, bool state_half, const __
 {
     using C = SplitCfg<DK, DV>;
     const SlabLayout LK = layout_qk(h->desc), LV = layout_vy(h->desc);
+    if (state_half)
+        register_checked_ranges(h, nullptr, a, b, nullptr, s);
+    else
+        register_checked_ranges(h, a, nullptr, nullptr, y, s, peers);
     const Plan& p = h->plan;
     const int N = h->desc.N;
     if (state_half) {
@@ -1596,21 +1640,7 @@ bool encode_x_map(CUtensorMap* map, const void* x, const linfusion_attn_desc_t& 
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// W [C_in][C_out] (16-bit, row = input channel) -> boxes of 64 input rows x 64 output columns.
-bool encode_w_map(CUtensorMap* map, const void* w, int C)
-{
-    EncodeTiledFn fn = get_encode_fn();
-    if (fn == nullptr) return false;
-    cuuint64_t dims[2] = {static_cast<cuuint64_t>(C), static_cast<cuuint64_t>(C)};
-    cuuint64_t strides[1] = {static_cast<cuuint64_t>(C) * 2};
-    cuuint32_t box[2] = {64u, 64u};
-    cuuint32_t estr[2] = {1u, 1u};
-    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(w), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
-// The same matrix seen as (column within head 64, input row C, head H) -> boxes of 64 input rows x the
+// A weight matrix W [C_in][C_out] (16-bit, row = input channel) seen as (column within head 64, input row C, head H) -> boxes of 64 input rows x the
 // 64-column blocks of `heads` consecutive heads, which land in shared memory as consecutive 8 KB blocks
 // (head, row, column): one copy per weight matrix and K chunk.  A head index past the last head reads as zeros.
 bool encode_w_pair_map(CUtensorMap* map, const void* w, int C, int H, int heads = 2)
@@ -1848,4 +1878,56 @@ extern "C" linfusion_status_t linfusion_attn_state_x(linfusion_attn_t* h, const 
         return LINFUSION_ERR_CUDA;
     }
     return LINFUSION_OK;
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// The bounds-checked debugging build (see lf_in_bounds() in common.cuh).
+// ---------------------------------------------------------------------------------------------
+extern "C" int32_t linfusion_attn_checked_build(void)
+{
+#ifdef LF_CHECKED
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+extern "C" linfusion_status_t linfusion_attn_checked_shrink_y(size_t bytes)
+{
+#ifdef LF_CHECKED
+    g_checked_shrink_y.store(bytes);
+    return LINFUSION_OK;
+#else
+    (void)bytes;
+    return LINFUSION_ERR_UNSUPPORTED;
+#endif
+}
+
+extern "C" linfusion_status_t linfusion_attn_checked_violations(int32_t device, uint32_t* count, int32_t reset)
+{
+    if (count == nullptr || device < 0) return LINFUSION_ERR_INVALID_ARG;
+#ifdef LF_CHECKED
+    DeviceGuard guard(device);
+    if (!guard.ok) return LINFUSION_ERR_CUDA;
+    unsigned int c = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess ||
+        cudaMemcpyFromSymbol(&c, g_checked_violations, sizeof(c)) != cudaSuccess) {
+        cudaGetLastError();
+        return LINFUSION_ERR_CUDA;
+    }
+    *count = c;
+    if (reset != 0) {
+        c = 0;
+        if (cudaMemcpyToSymbol(g_checked_violations, &c, sizeof(c)) != cudaSuccess) {
+            cudaGetLastError();
+            return LINFUSION_ERR_CUDA;
+        }
+    }
+    return LINFUSION_OK;
+#else
+    (void)reset;
+    *count = 0;
+    return LINFUSION_ERR_UNSUPPORTED;
+#endif
 }

@@ -171,12 +171,12 @@ __device__ __forceinline__ void store_state(float* dst, const float (&acc)[Split
 #pragma unroll
     for (int nb = 0; nb < C::NBV; ++nb) {
         int e = nb * 8 + 2 * t;
-        if (c0 < DK) *reinterpret_cast<float2*>(dst + c0 * DV + e) = make_float2(acc[nb][0], acc[nb][1]);
-        if (c1 < DK) *reinterpret_cast<float2*>(dst + c1 * DV + e) = make_float2(acc[nb][2], acc[nb][3]);
+        if (c0 < DK) g_store(reinterpret_cast<float2*>(dst + c0 * DV + e), make_float2(acc[nb][0], acc[nb][1]));
+        if (c1 < DK) g_store(reinterpret_cast<float2*>(dst + c1 * DV + e), make_float2(acc[nb][2], acc[nb][3]));
     }
     if (t == 0) {
-        if (c0 < DK) dst[DK * DV + c0] = acc[C::NBV][0];
-        if (c1 < DK) dst[DK * DV + c1] = acc[C::NBV][2];
+        if (c0 < DK) g_store(dst + DK * DV + c0, acc[C::NBV][0]);
+        if (c1 < DK) g_store(dst + DK * DV + c1, acc[C::NBV][2]);
     }
 }
 
@@ -331,10 +331,10 @@ __device__ __forceinline__ void put_state_operand(unsigned char* img, int idx, u
 {
     if (idx < dk * dv) {
         const int c = idx / dv, e = idx - c * dv;
-        *reinterpret_cast<uint16_t*>(img + e * pitch + c * 2) = b;
+        g_store(reinterpret_cast<uint16_t*>(img + e * pitch + c * 2), b);
     } else {
         const int c = idx - dk * dv;
-        for (int j = 0; j < 8; ++j) *reinterpret_cast<uint16_t*>(img + (dv + j) * pitch + c * 2) = b;
+        for (int j = 0; j < 8; ++j) g_store(reinterpret_cast<uint16_t*>(img + (dv + j) * pitch + c * 2), b);
     }
 }
 
@@ -357,8 +357,8 @@ state_reduce_kernel(const float* __restrict__ partials, float* __restrict__ stat
     const int slab = blockIdx.y;
     const float* src = partials + static_cast<size_t>(slab) * chunks * state_floats + idx;
     float sum = 0.0f;
-    for (int p = 0; p < chunks; ++p) sum += src[static_cast<size_t>(p) * state_floats];
-    state[static_cast<size_t>(slab) * state_floats + idx] = sum;
+    for (int p = 0; p < chunks; ++p) sum += g_load(src + static_cast<size_t>(p) * state_floats);
+    g_store(state + static_cast<size_t>(slab) * state_floats + idx, sum);
     if (st_image != nullptr)
         put_state_operand(st_image + static_cast<size_t>(slab) * image_bytes, idx,
                           to_storage16(sum * operand_scale, dtype), dk, dv, pitch);
@@ -403,10 +403,10 @@ apply_kernel(const __nv_bfloat16* __restrict__ Q, const float* __restrict__ stat
         // The reduction kernel left the operand in its shared-memory layout: plain 16-byte copy.
         const uint4* img = reinterpret_cast<const uint4*>(st_image + static_cast<size_t>(slab) * C::SMEM_ST);
         for (int i = threadIdx.x; i < C::SMEM_ST / 16; i += blockDim.x)
-            reinterpret_cast<uint4*>(St)[i] = __ldg(img + i);
+            reinterpret_cast<uint4*>(St)[i] = g_load_ro(img + i);
     } else {
         const float* st = state + static_cast<size_t>(slab) * C::STATE_FLOATS;
-        fill_state_operand<DK, DV>(St, [&](int i) { return __ldg(st + i); }, kind_dtype(KIND), sc.operand);
+        fill_state_operand<DK, DV>(St, [&](int i) { return g_load_ro(st + i); }, kind_dtype(KIND), sc.operand);
     }
     __syncthreads();
     apply_tiles<DK, DV, KIND>(Q + slab_base(LK, slab), Y + slab_base(LV, slab), N, LK.row_stride, LV.row_stride,
@@ -535,7 +535,7 @@ cluster_fused_kernel(const __nv_bfloat16* __restrict__ Q, const __nv_bfloat16* _
             for (int u = 0; u < kBatch; ++u) {
                 const int i = base + u * blockDim.x;
                 if (i >= end) continue;
-                if (gout != nullptr) gout[i] = sum[u];
+                if (gout != nullptr) g_store(gout + i, sum[u]);
                 const uint16_t b = to_storage16(sum[u] * sc.operand, kind_dtype(KIND));
                 // S[c][e] goes to row e, column c of the operand; z[c] to column c of rows DV .. DV+7.
                 const bool is_z = i >= DK * DV;
