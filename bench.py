@@ -424,7 +424,9 @@ def run_cuda(args):
         if sharded or kernel_times_taken.get(s.name) is None:
             continue
         sums, calls = kernel_times_taken[s.name]
-        for name, total in zip(names, sums):
+        # three launches: state, reduction, apply; two when the apply kernel takes over the reduction
+        op_names = names if op.launches_per_forward == 3 else [names[0], names[2]]
+        for name, total in zip(op_names, sums):
             if calls == 0:
                 continue
             avg_ms = total / calls

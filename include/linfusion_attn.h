@@ -53,7 +53,8 @@ typedef enum {
 /* flags: kernel-variant selection.  0 lets the library choose from (N, d, B*H). */
 #define LINFUSION_VARIANT_AUTO 0u
 #define LINFUSION_VARIANT_SPLIT 1u   /* three launches: split-N state, reduction, apply (any supported d) */
-#define LINFUSION_VARIANT_STREAM 2u  /* three launches, TMA-pipelined persistent kernels (d = 64 only)    */
+#define LINFUSION_VARIANT_STREAM 2u  /* TMA-pipelined persistent tcgen05 kernels (d = 64 only): two launches, the
+                                        apply kernel sums the partial states itself (three when slabs > SMs) */
 #define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N); one CTA per slab for N <= 192 */
 #define LINFUSION_VARIANT_FUSED 4u   /* one launch, persistent TMA + tcgen05 kernel with per-slab counters (d = 64) */
 #define LINFUSION_VARIANT_MASK 0xFu

@@ -136,30 +136,6 @@ __device__ __forceinline__ FusedWalk fused_walk(const FusedPlan& p, long long g,
     return w;
 }
 
-__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p)
-{
-    uint32_t v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void red_release_gpu_add(uint32_t* p, uint32_t v)
-{
-    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-
-// Spin (bounded by the global timer, like the mbarrier waits) until the counter has advanced by at
-// least `need` from `base`.  Counters only grow; the difference is taken modulo 2^32.
-__device__ __forceinline__ bool counter_wait(const uint32_t* ctr, uint32_t base, uint32_t need)
-{
-    if (ld_acquire_gpu(ctr) - base >= need) return true;
-    const unsigned long long t0 = global_timer_ns();
-    do {
-        __nanosleep(40);
-        if (ld_acquire_gpu(ctr) - base >= need) return true;
-    } while (global_timer_ns() - t0 < kMaxBarrierWaitNs);
-    return false;
-}
-
 // One warp waits for a counter nobody advances: the bounded wait must give up and leave the error
 // word behind.  Run by the library's self-test only.
 __global__ void __launch_bounds__(32)

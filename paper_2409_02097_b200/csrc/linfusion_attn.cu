@@ -52,6 +52,7 @@ struct Plan {
     int tiles_state = 0, tiles_apply = 0;  // per slab
     long long W_state = 0, W_apply = 0;
     int G_state = 0, G_apply = 0, spans = 0;
+    int merged_reduce = 0;  // stream: the apply kernel sums the partials itself (two launches)
     // cluster
     int cluster_size = 0;
     // stream, fed from X (token-major handles): units are (batch, head pair, tile)
@@ -119,13 +120,12 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v == LINFUSION_VARIANT_AUTO) {
         // Measured on B200 over the SD-v1.5 / v2.1 / XL layer shapes, forwards back to back.  The
-        // persistent TMA + tcgen05 kernels (d = 64) pay a few microseconds of set-up (tensor-memory
-        // allocation, one CTA per SM working through its tiles in turn) and win once every SM has
-        // about eight 128-token tiles (35 vs 41 us at N = 4096 x 40 slabs, 47 vs 70 us at
-        // N = 16384 x 20; 29 vs 29 us at N = 9216 x 10, 24 vs 22 us at N = 2304 x 10).  Below that the three chained launches of
-        // the split path are the fastest at every shape measured, the smallest levels included
-        // (12.9 us at N = 144, d = 64, against 14.4 us for the single clustered launch; 21.9 vs 27 us
-        // at N = 64, d = 160), so the cluster kernel is only run on request.
+        // persistent TMA + tcgen05 kernels (d = 64; two launches, the apply kernel sums the partial states
+        // itself) pay a few microseconds of set-up (tensor-memory allocation, one CTA per SM working through
+        // its tiles in turn) and win from about two 128-token tiles per SM on (18.8 vs 22.8 us at
+        // N = 2304 x 20 slabs, 24.8 vs 30.1 us at N = 9216 x 10, 36 vs 43 us at N = 4096 x 40, 46 vs 73 us at
+        // N = 16384 x 20).  Below that the three chained launches of the split path, the single persistent
+        // launch (many small slabs) or one CTA per slab (N <= 192) are faster.
         const long long stream_tiles = static_cast<long long>(slabs) * ((d->N + StreamStateCfg::TILE - 1) / StreamStateCfg::TILE);
         // The single persistent launch wins where no state has to cross CTAs: slabs of at most eight
         // 128-token tiles, enough of them to occupy a quarter of the SMs, each handled whole by one
@@ -136,7 +136,7 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         const int fused_tiles = (d->N + FusedCfg::TILE - 1) / FusedCfg::TILE;
         if (tiles_kv <= kLocalMaxTilesKv)
             v = LINFUSION_VARIANT_CLUSTER;  // resolves to one CTA per slab (largest_cluster())
-        else if (square64 && stream_tiles >= 8ll * sm_count)
+        else if (square64 && stream_tiles >= 2ll * sm_count)
             v = LINFUSION_VARIANT_STREAM;
         else if (square64 && fused_tiles <= 8 && 4 * slabs >= sm_count && stream_tiles < 4ll * sm_count)
             v = LINFUSION_VARIANT_FUSED;
@@ -160,11 +160,14 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         p->W_apply = static_cast<long long>(slabs) * p->tiles_apply;
         long long gs = static_cast<long long>(sm_count) * StreamStateCfg::CTAS_PER_SM;
         long long ga = sm_count;
-        if ((d->flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u) {
-            // Token-major: the 128-byte rows of all heads of a token are adjacent in memory.  With
-            // the same number of CTAs on every slab, the CTAs of different heads walk through the
-            // same tokens at the same time and DRAM pages are used while they are open: 140 CTAs
-            // (7 per slab) beat 148 by 7-8 % at 20 slabs, and 120 (3 per slab) equal 148 at 40.
+        // The same number of CTAs on every slab, where that keeps at least four fifths of the SMs busy:
+        // (1) token-major: the 128-byte rows of all heads of a token are adjacent in memory, and with equal
+        // counts the CTAs of different heads walk through the same tokens at the same time, so DRAM pages
+        // are used while they are open: 140 CTAs (7 per slab) beat 148 by 7-8 % at 20 slabs, and 120 (3 per
+        // slab) equal 148 at 40; (2) either layout when a CTA's share is only a few dozen tiles: with 7 CTAs
+        // on some slabs and 8 on others the kernels end with a tail that the tile hand-out cannot level
+        // (41.8 vs 46.3 us at N = 16384 x 20 slabs, 31.0 vs 36.3 us at N = 4096 x 40).
+        if ((d->flags & LINFUSION_LAYOUT_TOKEN_MAJOR) != 0u || p->W_state < 64ll * sm_count) {
             const long long aligned = (static_cast<long long>(sm_count) / slabs) * slabs;
             if (aligned * 5 >= static_cast<long long>(sm_count) * 4) gs = ga = aligned;
         }
@@ -204,7 +207,10 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
             const size_t need = static_cast<size_t>(p->G_x) * sx * 2 * kStreamStateFloats;
             if (need > partial_floats) partial_floats = need;
         }
-        p->launches = 3;
+        // Every slab needs an apply CTA that starts on it for the apply kernel to take over the second
+        // stage of the reduction (see MergedReduce); otherwise the reduction keeps its own kernel.
+        p->merged_reduce = slabs <= p->G_apply ? 1 : 0;
+        p->launches = p->merged_reduce != 0 ? 2 : 3;
     } else if (v == LINFUSION_VARIANT_FUSED) {
         // One persistent launch.  Two waves of slabs once every CTA has a couple of tiles in each
         // (the exchange of one wave's states then hides behind the other wave's streaming); at
@@ -254,8 +260,8 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamOperandBytes
                               : v == LINFUSION_VARIANT_SPLIT ? static_cast<size_t>(slabs) * split_image
                                                              : 0;
-    // Stream: one tile counter per slab.  Fused: two arrival counters per slab, then the control words.
-    const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM  ? align_up(static_cast<size_t>(slabs) * 4, 256)
+    // Stream: one tile counter and one ready flag per slab.  Fused: two arrival counters per slab, then the control words.
+    const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM  ? align_up(static_cast<size_t>(slabs) * 8, 256)
                                  : v == LINFUSION_VARIANT_FUSED ? align_up(static_cast<size_t>(slabs) * 8, 256) + 256
                                                                 : 0;
     p->counters_off = p->operand_off + align_up(frag_bytes, 256);
@@ -631,22 +637,40 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
         !encode_slab_map(&mq, q, h->desc, ApplyCfg::TILE) || !encode_slab_map(&my, y, h->desc, ApplyCfg::TILE))
         return cudaErrorInvalidValue;
     cudaError_t e;
+    MergedReduce mr = {};
+    uint32_t* per_slab_words = reinterpret_cast<uint32_t*>(h->tile_counters);  // tile counters, then ready flags
+    if (p.merged_reduce != 0) {
+        mr.partials = h->partials;
+        mr.state = h->state;
+        mr.operand = h->operand;
+        mr.ready = per_slab_words + p.slabs;
+        mr.W = p.W_state;
+        mr.G = p.G_state;
+        mr.spans = p.spans;
+        mr.tiles_per_slab = p.tiles_state;
+        mr.dtype = dtype_of(h->desc);
+        mr.scale = operand_scale(h->desc);
+        mr.enabled = 1;
+    }
     mark(h, 0, s);
     e = launch_chained(stream_state_kernel<KIND>, dim3(p.G_state), dim3(StreamStateCfg::THREADS),
                        StreamStateCfg::SMEM_BYTES, s, mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state,
-                       p.spans, h->desc.H);
+                       p.spans, h->desc.H, p.merged_reduce != 0 ? per_slab_words : nullptr,
+                       p.merged_reduce != 0 ? 2 * p.slabs : 0);
     if (e != cudaSuccess) return e;
     mark(h, 1, s);
-    e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
-                       h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
-                       p.spans, dtype_of(h->desc), operand_scale(h->desc));
-    if (e != cudaSuccess) return e;
-    mark(h, 2, s);
+    if (p.merged_reduce == 0) {
+        e = launch_chained(stream_reduce_kernel, dim3((kStreamStateFloats + 255) / 256, p.slabs), dim3(256), 0, s,
+                           h->partials, h->state, h->operand, h->tile_counters, p.tiles_state, p.W_state, p.G_state,
+                           p.spans, dtype_of(h->desc), operand_scale(h->desc));
+        if (e != cudaSuccess) return e;
+        mark(h, 2, s);
+    }
     e = launch_chained(stream_apply_kernel<KIND>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
                        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs,
-                       apply_scales(h->desc), h->desc.H);
+                       apply_scales(h->desc), h->desc.H, mr);
     if (e != cudaSuccess) return e;
-    mark(h, 3, s);
+    mark(h, p.merged_reduce != 0 ? 2 : 3, s);
     return cudaGetLastError();
 }
 
@@ -1513,7 +1537,7 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
             !encode_slab_map(&mv, b, h->desc, StreamStateCfg::TILE))
             return cudaErrorInvalidValue;
         stream_state_kernel<KIND><<<p.G_state, StreamStateCfg::THREADS, StreamStateCfg::SMEM_BYTES, s>>>(
-            mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H);
+            mk, mv, h->partials, h->status, N, p.tiles_state, p.W_state, p.spans, h->desc.H, nullptr, 0);
         stream_reduce_kernel<<<rgrid, 256, 0, s>>>(h->partials, h->state, h->operand, h->tile_counters,
                                                   p.tiles_state, p.W_state, p.G_state, p.spans,
                                                   dtype_of(h->desc), operand_scale(h->desc));
@@ -1529,7 +1553,8 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
         stream_pack_kernel<<<rgrid, 256, 0, s>>>(peers != nullptr ? *peers : own, h->operand, h->tile_counters,
                                                 dtype_of(h->desc), operand_scale(h->desc));
         stream_apply_kernel<KIND><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
-            mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, apply_scales(h->desc), h->desc.H);
+            mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, apply_scales(h->desc), h->desc.H,
+            MergedReduce{});
     }
     return cudaGetLastError();
 }

@@ -153,10 +153,6 @@ struct ProdState2Cfg {
 static_assert(ProdState2Cfg::SMEM_BYTES > 116 * 1024 && ProdState2Cfg::SMEM_BYTES <= 227 * 1024, "one CTA per SM");
 static_assert(ProdState2Cfg::STAGE_BYTES % 1024 == 0, "operands on 1024-byte boundaries");
 
-__device__ __forceinline__ void named_barrier_sync(int id, int threads)
-{
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
-}
 // Barrier over `threads` threads that also tells everybody whether `ok` held for all of them, so
 // that a group leaves a loop that contains barriers together or not at all.
 __device__ __forceinline__ bool named_barrier_all(int id, int threads, bool ok)

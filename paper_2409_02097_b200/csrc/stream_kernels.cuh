@@ -53,6 +53,7 @@ struct StreamStateCfg {
     static constexpr int PHI_WARPS = 4 * GROUPS;
     static constexpr int PRODUCER_WARP = PHI_WARPS;
     static constexpr int MMA_WARP = PHI_WARPS + 1;
+    static constexpr int CLEAR_WARP = PHI_WARPS + 2;   // zeroes the apply kernel's per-slab words
     static constexpr int FLUSH_WARP0 = PHI_WARPS + 4;  // three warps whose index is 0, 1, 2 mod 4
     static constexpr int THREADS = 32 * (PHI_WARPS + 7);
     static constexpr int STAGES = 6;
@@ -97,6 +98,36 @@ __host__ __device__ __forceinline__ long long unit_begin(long long g, long long 
 __device__ __forceinline__ void report_wait_expired(uint32_t* status)
 {
     atomicExch(status, kStatusWaitExpired);
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void red_release_gpu_add(uint32_t* p, uint32_t v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Spin (bounded by the global timer, like the mbarrier waits) until the counter has advanced by at
+// least `need` from `base`.  Counters only grow; the difference is taken modulo 2^32.
+__device__ __forceinline__ bool counter_wait(const uint32_t* ctr, uint32_t base, uint32_t need)
+{
+    if (ld_acquire_gpu(ctr) - base >= need) return true;
+    const unsigned long long t0 = global_timer_ns();
+    do {
+        __nanosleep(40);
+        if (ld_acquire_gpu(ctr) - base >= need) return true;
+    } while (global_timer_ns() - t0 < kMaxBarrierWaitNs);
+    return false;
+}
+
+// Barrier among `threads` threads of the CTA (ids 1..15; 0 is __syncthreads).
+__device__ __forceinline__ void named_barrier_sync(int id, int threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
 }
 
 // One warp waits on an mbarrier that nothing ever arrives on: the bounded wait must give up after
@@ -147,7 +178,8 @@ template <int KIND>
 __global__ void __launch_bounds__(StreamStateCfg::THREADS, StreamStateCfg::CTAS_PER_SM)
 stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                     const __grid_constant__ CUtensorMap tmap_v, float* __restrict__ partials,
-                    uint32_t* __restrict__ status, int N, int tiles_per_slab, long long W, int spans, int H)
+                    uint32_t* __restrict__ status, int N, int tiles_per_slab, long long W, int spans, int H,
+                    uint32_t* __restrict__ clear_words, int n_clear)
 {
     using C = StreamStateCfg;
     extern __shared__ unsigned char smem_raw[];
@@ -315,6 +347,10 @@ stream_state_kernel(const __grid_constant__ CUtensorMap tmap_k,
                 for (int c = 0; c < 64; ++c) acc[c] = 0.0f;
             }
         }
+    } else if (warp == C::CLEAR_WARP) {
+        // ---------------- the apply kernel's per-slab words (tile counters, ready flags) start every forward
+        // at zero; the forward before has completed (dependency wait above) ----------------
+        for (int i = static_cast<int>(g) * 32 + lane; i < n_clear; i += static_cast<int>(G) * 32) clear_words[i] = 0u;
     } else if (warp < C::PHI_WARPS) {
         // ---------------- phi warpgroups ----------------
         const int group = warp >> 2;
@@ -469,11 +505,29 @@ stream_pack_kernel(PeerStates states, unsigned char* __restrict__ operand,
 // Per stage s: full[s] (TMA bytes landed) -> a_ready[g] (4 warps: phi(Q) rows in TMEM) ->
 // mma_done[g] (tcgen05.commit) -> y_ready[s] (4 warps: Y rows in the stage) -> empty[s].
 // ---------------------------------------------------------------------------------------------
+// The second stage of the state reduction done by the apply kernel itself (no kernel of its own between
+// the state kernel and the apply kernel): every apply CTA sums, in CTA order, the partials of its HOME slab
+// (the slab it starts on) straight into its shared-memory operand; the lowest-numbered CTA of a slab's
+// home CTAs also leaves the fp32 state and the 16-bit operand image in global memory and then raises the
+// slab's ready flag, which a CTA that later helps out on that slab waits for (bounded) before it copies
+// the image.  Every slab needs a home CTA: the host enables this only when slabs <= grid size.
+struct MergedReduce {
+    const float* partials;   // of stream_state_kernel
+    float* state;            // [slab][S 64x64 | z 64] fp32
+    unsigned char* operand;  // [slab] 16-bit images
+    uint32_t* ready;         // [slab] flags, zero at kernel start
+    long long W;             // the state kernel's units, grid and partial slots per CTA
+    int G, spans, tiles_per_slab;
+    int dtype;
+    float scale;
+    int enabled;
+};
+
 template <int KIND>
 __global__ void __launch_bounds__(StreamApplyCfg::THREADS, 1)
 stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_y,
                     const unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
-                    uint32_t* __restrict__ status, int tiles_per_slab, int slabs, ApplyScales sc, int H)
+                    uint32_t* __restrict__ status, int tiles_per_slab, int slabs, ApplyScales sc, int H, MergedReduce mr)
 {
     using C = StreamApplyCfg;
     extern __shared__ unsigned char smem_raw[];
@@ -486,7 +540,8 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     uint64_t* a_ready = y_ready + C::STAGES;  // per group
     uint64_t* mma_done = a_ready + C::GROUPS;  // per group
     uint64_t* b_ready = mma_done + C::GROUPS;  // the operand of the slab now being posted is in shared memory
-    int2* meta = reinterpret_cast<int2*>(b_ready + 1);  // (slab, tile) of each stage; slab < 0 ends
+    uint64_t* home_done = b_ready + 1;         // the home slab's operand has been summed into shared memory
+    int2* meta = reinterpret_cast<int2*>(home_done + 1);  // (slab, tile) of each stage; slab < 0 ends
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(meta + C::STAGES);
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -502,6 +557,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             mbar_init(&mma_done[g], 1);
         }
         mbar_init(b_ready, 1);
+        mbar_init(home_done, 1);
         mbar_fence_init();
     }
     if (warp == 0) tmem_alloc(tmem_slot, C::TMEM_COLS);
@@ -514,14 +570,102 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     // tensor maps are kernel parameters: fetching them does not depend on earlier work.)
     if (warp == C::PRODUCER_WARP && lane == 0) prefetch_tmap(&tmap_q);
     if (warp == C::STORE_WARP && lane == 0) prefetch_tmap(&tmap_y);
+    const int home = static_cast<int>((static_cast<long long>(blockIdx.x) * slabs) / gridDim.x);
+    constexpr int TEAM = C::THREADS - 32;  // every warp but the producer
+    const int ttid = tid < 32 * C::PRODUCER_WARP ? tid : tid - 32;
+    int* ctrb = reinterpret_cast<int*>(tmem_slot + 1);  // g0, g1, first contributor's slot
+    if (mr.enabled != 0 && warp != C::PRODUCER_WARP) {
+        // (pure index arithmetic and shared memory: done while the kernel ahead is still running)
+        if (ttid == 0) {
+            const long long lo = static_cast<long long>(home) * mr.tiles_per_slab, hi = lo + mr.tiles_per_slab;
+            const long long Gs = mr.G, Ws = mr.W;
+            long long g0 = (lo * Gs) / Ws;
+            while (g0 + 1 < Gs && unit_begin(g0 + 1, Ws, Gs) <= lo) ++g0;
+            while (g0 > 0 && unit_begin(g0, Ws, Gs) > lo) --g0;
+            long long g1 = (hi * Gs) / Ws;
+            while (g1 < Gs && unit_begin(g1, Ws, Gs) < hi) ++g1;
+            while (g1 > 0 && unit_begin(g1 - 1, Ws, Gs) >= hi) --g1;
+            ctrb[0] = static_cast<int>(g0);
+            ctrb[1] = static_cast<int>(g1);
+            ctrb[2] = home - static_cast<int>(unit_begin(g0, Ws, Gs) / mr.tiles_per_slab);
+        }
+        for (int i = ttid; i < 15 * 128 / 16; i += TEAM) reinterpret_cast<uint4*>(bsm + 65 * 128)[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
     pdl_launch_dependents();
     pdl_wait();
+
+    if (mr.enabled != 0 && warp != C::PRODUCER_WARP) {
+        // ---------------- every warp but the producer (which is already fetching Q tiles): the home
+        // slab's state, summed over the state kernel's CTAs ----------------
+        named_barrier_sync(1, TEAM);
+        const int g0 = ctrb[0], g1 = ctrb[1], slot0 = ctrb[2];
+        const bool writer = blockIdx.x == 0 ||
+                            static_cast<int>((static_cast<long long>(blockIdx.x - 1) * slabs) / gridDim.x) != home;
+        const float4* part4 = reinterpret_cast<const float4*>(mr.partials);
+        constexpr int V4 = kStreamStateFloats / 4;  // 1040: S rows as 16 float4 each, then z as 16
+        float4* st4 = reinterpret_cast<float4*>(mr.state + static_cast<size_t>(home) * kStreamStateFloats);
+        for (int idx = ttid; idx < V4; idx += TEAM) {
+            // contributor g0's partial of this slab sits in its slot `slot0`; every later contributor's run
+            // starts inside the slab (its slot 0).  Eight loads in flight, summed in CTA order.
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int gb = g0; gb < g1; gb += 8) {
+                float4 v[8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    v[j] = gb + j < g1 ? __ldcg(part4 + (static_cast<size_t>(gb + j) * mr.spans + (gb + j == g0 ? slot0 : 0)) * V4 + idx)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    if (gb + j == g0) {
+                        sum = v[j];  // the first term as it is: the same bits as a sum that starts from it
+                    } else if (gb + j < g1) {
+                        sum.x += v[j].x;
+                        sum.y += v[j].y;
+                        sum.z += v[j].z;
+                        sum.w += v[j].w;
+                    }
+                }
+            }
+            if (writer) st4[idx] = sum;
+            const float f[4] = {sum.x * mr.scale, sum.y * mr.scale, sum.z * mr.scale, sum.w * mr.scale};
+            if (idx < 1024) {
+                const int c = idx >> 4, e0 = (idx & 15) * 4;  // S[c][e0 .. e0+3] -> B rows e0 .., column c
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = e0 + i;
+                    *reinterpret_cast<uint16_t*>(bsm + row * 128 + (((c >> 3) ^ (row & 7)) << 4) + (c & 7) * 2) =
+                        to_storage16(f[i], mr.dtype);
+                }
+            } else {
+                // z[4 t .. 4 t + 3] -> row 64 (64 & 7 = 0: chunks in place)
+                const int t4 = idx - 1024;
+                uint2 wv;
+                wv.x = to_storage16(f[0], mr.dtype) | (static_cast<uint32_t>(to_storage16(f[1], mr.dtype)) << 16);
+                wv.y = to_storage16(f[2], mr.dtype) | (static_cast<uint32_t>(to_storage16(f[3], mr.dtype)) << 16);
+                *reinterpret_cast<uint2*>(bsm + 64 * 128 + t4 * 8) = wv;
+            }
+        }
+        fence_proxy_async_smem();
+        named_barrier_sync(1, TEAM);
+        if (ttid == 0) mbar_arrive(home_done);
+        if (writer) {
+            uint4* img = reinterpret_cast<uint4*>(mr.operand + static_cast<size_t>(home) * C::B_BYTES);
+            for (int i = ttid; i < C::B_BYTES / 16; i += TEAM) img[i] = reinterpret_cast<const uint4*>(bsm)[i];
+            named_barrier_sync(1, TEAM);
+            if (ttid == 0) {
+                __threadfence();
+                red_release_gpu_add(&mr.ready[home], 1u);
+            }
+        }
+    }
 
     if (warp == C::PRODUCER_WARP) {
         // ---------------- producer warp (lane 0 issues; all lanes help to find work and copy B) ----------------
         uint64_t policy = 0;
         if (lane == 0) policy = policy_evict_first();
-        int slab = static_cast<int>((static_cast<long long>(blockIdx.x) * slabs) / gridDim.x);
+        int slab = home;
+        int smem_slab = mr.enabled != 0 ? home : -1;  // whose operand the shared-memory buffer holds (or will, once home_done)
+        bool home_pending = mr.enabled != 0;          // the other warps may still be writing it
         int it = 0, issued = 0, loaded_slab = -1;
         bool ok = true;
         int next = 0;
@@ -548,7 +692,8 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             // tile takes) overlaps the wait for a free stage and the copy below.
             if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
             const bool new_slab = slab != loaded_slab;
-            if (new_slab) {
+            const bool copy_b = new_slab && slab != smem_slab;
+            if (copy_b) {
                 // Every tile posted so far must have left (its MMAs, which read B, are then
                 // complete as well) before B is overwritten.
                 if (lane == 0) {
@@ -575,10 +720,26 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             if (!ok) break;
             ++it;
             if (new_slab) {
-                // The slab's operand, copied while the tile above is on its way; the MMA thread
-                // waits for b_ready before the first MMA of a slab.
-                const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
-                for (int i = lane; i < C::B_BYTES / 16; i += 32) reinterpret_cast<uint4*>(bsm)[i] = __ldg(src + i);
+                // The slab's operand, copied while the tile above is on its way (unless the buffer holds
+                // it already: the home slab's, summed above); the MMA thread waits for b_ready before
+                // the first MMA of a slab.
+                if (copy_b) {
+                    if (mr.enabled != 0) {
+                        // the buffer must not be overwritten while the home slab's sum is still being written
+                        // into it; the image is written during this kernel by the slab's first home CTA
+                        if (lane == 0 && home_pending) ok = mbar_wait(home_done, 0);
+                        home_pending = false;
+                        if (lane == 0 && ok) ok = counter_wait(&mr.ready[slab], 0u, 1u);
+                        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                        if (!ok) {
+                            if (lane == 0) report_wait_expired(status);
+                            break;
+                        }
+                    }
+                    const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
+                    for (int i = lane; i < C::B_BYTES / 16; i += 32) reinterpret_cast<uint4*>(bsm)[i] = __ldcg(src + i);
+                    smem_slab = slab;
+                }
                 fence_proxy_async_smem();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(b_ready);
@@ -632,6 +793,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             const uint64_t b_desc = umma_desc_kmajor_sw128(smem_u32(bsm));
             int cur_slab = -1;
             uint32_t operands_seen = 0;
+            if (mr.enabled != 0 && !mbar_wait(home_done, 0)) report_wait_expired(status);
             for (int it = 0;; ++it) {
                 const int s = it % C::STAGES, g = it % C::GROUPS;
                 if (!mbar_wait(&full[s], (it / C::STAGES) & 1)) {

@@ -147,7 +147,7 @@ def test_stream_variant_tail_and_slab_crossing():
 
 def test_auto_policy_follows_the_measured_crossovers():
     for dims, want in [((2, 10, 16384, 64), "stream"), ((2, 20, 4096, 64), "stream"),
-                       ((2, 20, 2304, 64), "split"), ((2, 20, 144, 64), "cluster"), ((2, 20, 576, 64), "fused"),
+                       ((2, 20, 2304, 64), "stream"), ((2, 10, 9216, 64), "stream"), ((1, 10, 2304, 64), "split"), ((2, 20, 144, 64), "cluster"), ((2, 20, 576, 64), "fused"),
                        ((2, 2, 144, 64), "cluster"), ((2, 8, 4096, 40), "split"), ((2, 8, 64, 160), "cluster"),
                        ((2, 8, 256, 160), "split")]:
         op = attn.LinFusionAttention(*dims)
@@ -343,7 +343,7 @@ def test_kernel_timing_stride_samples_every_nth_forward():
     outs = [op.forward(q, k, v).clone() for _ in range(10)]
     sums, calls = op.kernel_times()
     assert calls == 3                      # forwards 0, 4 and 8
-    assert all(t > 0 for t in sums)
+    assert all(t > 0 for t in sums[:op.launches_per_forward])
     op.enable_kernel_timing(0)
     for o in outs:                         # timed or not, chained or not: the same bits
         assert torch.equal(o.view(torch.int16), y.view(torch.int16))
