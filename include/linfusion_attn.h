@@ -56,7 +56,8 @@ typedef enum {
 #define LINFUSION_VARIANT_STREAM 2u  /* TMA-pipelined persistent tcgen05 kernels (d = 64 only): two launches, the
                                         apply kernel sums the partial states itself (three when slabs > SMs) */
 #define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N); one CTA per slab for N <= 192 */
-#define LINFUSION_VARIANT_FUSED 4u   /* one launch, persistent TMA + tcgen05 kernel with per-slab counters (d = 64) */
+#define LINFUSION_VARIANT_FUSED 4u   /* one launch, persistent TMA + tcgen05 kernel with per-slab counters: d = 64, and
+                                        d = 40 / 80 / 160 (d' = d) when B*H <= SM count and N <= 4096 * (SMs / (B*H)) */
 #define LINFUSION_VARIANT_MASK 0xFu
 /*
  * flags: memory layout of Q, K, V and Y.  Default (bit clear): head-major [B, H, N, d].  Bit set:
@@ -109,7 +110,7 @@ typedef struct {
  *
  * desc.d is the value width d, desc.d_qk the feature width d' (0: the same as d, the released
  * model's case).  The three-launch split path and the cluster kernel serve d' != d; the TMA +
- * tcgen05 variants (STREAM, FUSED) are for d' = d = 64.  Everywhere this header says [.., d] for Q
+ * tcgen05 variants are for d' = d: STREAM at 64, FUSED at 40, 64, 80 and 160.  Everywhere this header says [.., d] for Q
  * or K, or d x d for S, or d for z, read d' for the feature side.
  */
 
@@ -224,7 +225,8 @@ linfusion_status_t linfusion_attn_read_state(linfusion_attn_t* h, float* S_host,
  * state_buffer: *dev_ptr is the device address of [B*H][d*d S (row = feature c of K, column =
  * channel e of V), then d z] fp32, *floats its length; it stays valid until the handle is
  * destroyed or its workspace is replaced.  Handles that resolved to a single-launch variant
- * (CLUSTER, FUSED; AUTO picks CLUSTER for N <= 192 and FUSED for many small slabs of head dim 64) cannot be split in two:
+ * (CLUSTER, FUSED; AUTO picks CLUSTER for N <= 192, FUSED for many small slabs of head dim 64 and for
+ * head dims 40 / 80 / 160 wherever that kernel applies) cannot be split in two:
  * state() and apply() return UNSUPPORTED for them (create the handle with LINFUSION_VARIANT_SPLIT
  * or _STREAM).  Other errors as for forward().
  */

@@ -8,7 +8,8 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_PKG, "csrc")
 LIB_PATH = os.path.join(_PKG, "liblinfusion_attn.so")
 _SOURCES = ["linfusion_attn.cu"]
-_HEADERS = ["common.cuh", "split_kernels.cuh", "stream_kernels.cuh", "fused_kernels.cuh", "producer_kernels.cuh"]
+_HEADERS = ["common.cuh", "split_kernels.cuh", "stream_kernels.cuh", "fused_kernels.cuh", "producer_kernels.cuh",
+            "padded_kernels.cuh"]
 CHECKED_LIB_PATH = os.path.join(_PKG, "liblinfusion_attn_checked.so")
 
 

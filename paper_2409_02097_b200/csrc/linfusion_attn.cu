@@ -13,6 +13,7 @@
 #include "stream_kernels.cuh"
 #include "fused_kernels.cuh"
 #include "producer_kernels.cuh"
+#include "padded_kernels.cuh"
 
 using namespace lf;
 
@@ -41,6 +42,31 @@ bool supported_widths(int dk, int dv)
     return (dk == 128 && dv == 64) || (dk == 80 && dv == 40) || (dk == 32 && dv == 64);
 }
 
+// Head widths of the single-launch tcgen05 kernel for widths that are not a multiple of 64
+// (padded_kernels.cuh), d' = d.
+bool padded_width(int dk, int dv) { return dk == dv && (dv == 40 || dv == 80 || dv == 160); }
+int padded_partial_floats(int d) { return ((d + 15) / 16 * 16) * ((d + 1 + 15) / 16 * 16); }
+
+// CTAs per slab of that kernel, or 0 where it does not apply: every slab needs a CTA of its own (all
+// of them resident together), and a CTA's run of tiles must fit one accumulation in tensor memory.
+// Every CTA of a slab reads all of the slab's partials (9 KB each at d = 40, 30 KB at 80, 110 KB at 160),
+// so their number is kept to what makes that a couple of hundred KB at most (more only where the runs
+// would otherwise be too long); then the smallest count that gives the CTAs the same longest run is taken.
+int padded_per_slab(int N, int slabs, int sm_count, int d)
+{
+    if (slabs > sm_count) return 0;
+    const int tiles = (N + 127) / 128;
+    int k = sm_count / slabs;
+    if (k > tiles) k = tiles;
+    int cap = static_cast<int>((192u * 1024u) / (static_cast<unsigned>(padded_partial_floats(d)) * 4u));
+    const int need = (tiles + 31) / 32;  // CTAs that the longest run allows
+    if (cap < need) cap = need;
+    if (k > cap) k = cap;
+    const int longest = (tiles + k - 1) / k;
+    if (longest > 32) return 0;
+    return (tiles + longest - 1) / longest;
+}
+
 // Everything that follows from (descriptor, SM count) alone.
 struct Plan {
     int variant = 0;
@@ -60,6 +86,7 @@ struct Plan {
     int G_x = 0, spans_x = 0;
     // fused
     int fused_split = 0, fused_whole = 0;
+    int padded_per_slab = 0;  // fused, widths 40 / 80 / 160: CTAs per slab
     // workspace (bytes, offsets)
     size_t partial_bytes = 0, state_off = 0, operand_off = 0, counters_off = 0, status_off = 0, total_bytes = 0;
     int launches = 0;
@@ -83,8 +110,9 @@ linfusion_status_t validate(const linfusion_attn_desc_t* d)
         return LINFUSION_ERR_UNSUPPORTED;
     uint32_t v = d->flags & LINFUSION_VARIANT_MASK;
     if (v > LINFUSION_VARIANT_FUSED) return LINFUSION_ERR_UNSUPPORTED;
-    if ((v == LINFUSION_VARIANT_STREAM || v == LINFUSION_VARIANT_FUSED) && (d->d != kStreamD || dk_of(*d) != kStreamD))
-        return LINFUSION_ERR_UNSUPPORTED;
+    const bool square64 = d->d == kStreamD && dk_of(*d) == kStreamD;
+    if (v == LINFUSION_VARIANT_STREAM && !square64) return LINFUSION_ERR_UNSUPPORTED;
+    if (v == LINFUSION_VARIANT_FUSED && !square64 && !padded_width(dk_of(*d), d->d)) return LINFUSION_ERR_UNSUPPORTED;
     return LINFUSION_OK;
 }
 
@@ -134,7 +162,13 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // boundaries (32 vs 22 us at N = 2304 x 20, 106 vs 47 us at N = 16384 x 20), so it is not
         // chosen there.
         const int fused_tiles = (d->N + FusedCfg::TILE - 1) / FusedCfg::TILE;
-        if (tiles_kv <= kLocalMaxTilesKv)
+        // Widths 40 / 80 / 160 (the SD-v1.5 levels): the single TMA + tcgen05 launch wherever its limits allow
+        // (19.4 vs 20.8 us for three chained launches at N = 4096, d = 40 x 16 slabs; 16.6 vs 17.4 us at
+        // N = 1024, d = 80; 19.4 vs 24.6 us at N = 256, d = 160; 13.5 vs 14.7 us for one CTA per slab of the
+        // warp-level kernel at N = 64, d = 160).
+        if (padded_width(dk, dv) && padded_per_slab(d->N, slabs, sm_count, dv) > 0)
+            v = LINFUSION_VARIANT_FUSED;
+        else if (tiles_kv <= kLocalMaxTilesKv)
             v = LINFUSION_VARIANT_CLUSTER;  // resolves to one CTA per slab (largest_cluster())
         else if (square64 && stream_tiles >= 2ll * sm_count)
             v = LINFUSION_VARIANT_STREAM;
@@ -211,6 +245,14 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // stage of the reduction (see MergedReduce); otherwise the reduction keeps its own kernel.
         p->merged_reduce = slabs <= p->G_apply ? 1 : 0;
         p->launches = p->merged_reduce != 0 ? 2 : 3;
+    } else if (v == LINFUSION_VARIANT_FUSED && !square64) {
+        // One persistent launch, widths 40 / 80 / 160: per_slab CTAs on every slab, one partial each.
+        p->padded_per_slab = padded_per_slab(d->N, slabs, sm_count, dv);
+        if (p->padded_per_slab == 0) return LINFUSION_ERR_UNSUPPORTED;
+        p->tiles_state = p->tiles_apply = (d->N + 127) / 128;
+        p->G_state = p->G_apply = slabs * p->padded_per_slab;
+        partial_floats = static_cast<size_t>(p->G_state) * padded_partial_floats(dv);
+        p->launches = 1;
     } else if (v == LINFUSION_VARIANT_FUSED) {
         // One persistent launch.  Two waves of slabs once every CTA has a couple of tiles in each
         // (the exchange of one wave's states then hides behind the other wave's streaming); at
@@ -370,6 +412,25 @@ bool encode_slab_map(CUtensorMap* map, const void* base, const linfusion_attn_de
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box,
                     estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// The same view for the widths 40 / 80 / 160: the channel extent is d, the box is 64 channels wide, so
+// the part of a box past channel d lies outside the tensor (zeros on loads, not written by stores).
+bool encode_padded_map(CUtensorMap* map, const void* base, const linfusion_attn_desc_t& d)
+{
+    EncodeTiledFn fn = get_encode_fn();
+    if (fn == nullptr) return false;
+    const SlabLayout L = layout_vy(d);  // d' = d
+    cuuint64_t dims[4] = {static_cast<cuuint64_t>(d.d), static_cast<cuuint64_t>(d.N), static_cast<cuuint64_t>(d.H),
+                          static_cast<cuuint64_t>(d.B)};
+    cuuint64_t strides[3] = {static_cast<cuuint64_t>(L.row_stride) * 2, static_cast<cuuint64_t>(L.head_stride) * 2,
+                             static_cast<cuuint64_t>(L.batch_stride) * 2};
+    cuuint32_t box[4] = {64u, 128u, 1u, 1u};
+    cuuint32_t estr[4] = {1u, 1u, 1u, 1u};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
@@ -695,6 +756,38 @@ cudaError_t launch_fused(const linfusion_attn* h, const __nv_bfloat16* q, const 
     return cudaGetLastError();
 }
 
+template <int D, int KIND>
+cudaError_t launch_padded(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                          const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
+{
+    using C = PaddedCfg<D>;
+    const Plan& p = h->plan;
+    CUtensorMap mq, mk, mv, my;
+    if (!encode_padded_map(&mk, k, h->desc) || !encode_padded_map(&mv, v, h->desc) ||
+        !encode_padded_map(&mq, q, h->desc) || !encode_padded_map(&my, y, h->desc))
+        return cudaErrorInvalidValue;
+    uint32_t* counters = reinterpret_cast<uint32_t*>(h->tile_counters);
+    uint32_t* ctrl = counters + align_up(static_cast<size_t>(p.slabs) * 8, 256) / 4;
+    mark(h, 0, s);
+    cudaError_t e = launch_chained(padded_fused_kernel<D, KIND>, dim3(p.G_state), dim3(C::THREADS), C::SMEM_BYTES, s, mk,
+                                   mv, mq, my, h->partials, h->state, counters, ctrl, h->status, h->desc.N,
+                                   p.tiles_state, p.padded_per_slab, p.slabs, h->desc.H, apply_scales(h->desc));
+    if (e != cudaSuccess) return e;
+    mark(h, 1, s);
+    return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_padded_d(const linfusion_attn* h, const __nv_bfloat16* q, const __nv_bfloat16* k,
+                            const __nv_bfloat16* v, __nv_bfloat16* y, cudaStream_t s)
+{
+    cudaError_t e = cudaErrorInvalidValue;
+#define LF_K(KV) e = launch_padded<D, KV>(h, q, k, v, y, s)
+    LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
+#undef LF_K
+    return e;
+}
+
 template <int DK, int DV>
 cudaError_t set_attrs_d(int kind)
 {
@@ -702,6 +795,13 @@ cudaError_t set_attrs_d(int kind)
 #define LF_K(KV) e = set_split_attrs<DK, DV, KV>()
     LF_DISPATCH_KIND(kind, LF_K)
 #undef LF_K
+    if constexpr (DK == DV && (DV == 40 || DV == 80 || DV == 160)) {
+        if (e != cudaSuccess) return e;
+#define LF_K(KV) \
+    e = cudaFuncSetAttribute(padded_fused_kernel<DV, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, PaddedCfg<DV>::SMEM_BYTES)
+        LF_DISPATCH_KIND(kind, LF_K)
+#undef LF_K
+    }
     return e;
 }
 
@@ -921,6 +1021,13 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
 #define LF_K(KV) e = launch_stream<KV>(h, Q, K, V, Y, s)
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)
 #undef LF_K
+    } else if (h->plan.variant == kFused && h->plan.padded_per_slab > 0) {
+        switch (h->desc.d) {
+            case 40: e = launch_padded_d<40>(h, Q, K, V, Y, s); break;
+            case 80: e = launch_padded_d<80>(h, Q, K, V, Y, s); break;
+            case 160: e = launch_padded_d<160>(h, Q, K, V, Y, s); break;
+            default: break;
+        }
     } else if (h->plan.variant == kFused) {
 #define LF_K(KV) e = launch_fused<KV>(h, Q, K, V, Y, s)
         LF_DISPATCH_KIND(kind_of(h->desc), LF_K)

@@ -59,6 +59,12 @@ def test_workspace_bytes_is_pure_host_and_monotone():
     # cluster: no partials in global memory
     c = _ws(attn.make_desc(2, 8, 256, 160, variant="cluster"))
     assert c == (16 * 160 * 161 * 4 + 255) // 256 * 256 + 256
+    # the single tcgen05 launch at widths 40 / 80 / 160: per_slab partials of [roundup16(d)][roundup16(d + 1)] floats
+    # per slab (8 CTAs per slab at N = 4096 x 16 slabs, d = 40), state, two words per slab + control, status
+    f = _ws(attn.make_desc(2, 8, 4096, 40, variant="fused"))
+    assert f == (16 * 8 * 48 * 48 * 4 + 255) // 256 * 256 + (16 * 40 * 41 * 4 + 255) // 256 * 256 + 256 + 256 + 256
+    assert _ws(attn.make_desc(2, 8, 256, 160, variant="fused")) == \
+        (16 * 160 * 176 * 4 + 255) // 256 * 256 + (16 * 160 * 161 * 4 + 255) // 256 * 256 + 256 + 256 + 256
     # the plan depends on the SM count it is given
     assert _ws(attn.make_desc(2, 10, 524288, 64, variant="stream"), 74) < s
 
@@ -80,8 +86,22 @@ def test_invalid_descriptors(kw):
 
 
 @pytest.mark.parametrize("kw", [
+    dict(d=40, variant="fused", H=80),                    # more slabs than SMs: no CTA per slab
+    dict(d=160, variant="fused", B=74, H=2, N=128 * 33),  # one CTA per slab, more than 32 tiles each
+])
+def test_shapes_the_single_launch_at_padded_widths_cannot_take(kw):
+    args = dict(B=2, H=8, N=4096, d=64, eps=1e-6, device=0)
+    args.update(kw)
+    with pytest.raises(attn.LinFusionError) as e:
+        _ws(attn.make_desc(**args))
+    assert e.value.code == attn.ERR_UNSUPPORTED
+    args["variant"] = "auto"                              # AUTO plans something else
+    assert _ws(attn.make_desc(**args)) > 0
+
+
+@pytest.mark.parametrize("kw", [
     dict(d=48), dict(d=7), dict(d=256), dict(phi=7), dict(variant=9), dict(variant=0x80),
-    dict(d=40, variant="stream"), dict(d=40, variant="fused"),
+    dict(d=40, variant="stream"), dict(d=128, variant="fused"), dict(d=32, variant="fused"),
 ])
 def test_unsupported_descriptors(kw):
     args = dict(B=2, H=8, N=4096, d=64, eps=1e-6, device=0)

@@ -47,8 +47,8 @@ def _variants(N, d):
     out = ["split", "cluster"]
     if d == 64:
         out += ["stream"]
-        if hasattr(attn, "VARIANT_FUSED"):
-            out += ["fused"]
+    if d in (40, 64, 80, 160):
+        out += ["fused"]
     return out
 
 

@@ -30,6 +30,7 @@ def variants_for(shape):
     out = ["auto", "split"]
     if shape.d == 64:
         out.append("stream")
+    if shape.d in (40, 64, 80, 160):
         out.append("fused")
     if shape.N <= 16384:
         out.append("cluster")
@@ -148,8 +149,9 @@ def test_stream_variant_tail_and_slab_crossing():
 def test_auto_policy_follows_the_measured_crossovers():
     for dims, want in [((2, 10, 16384, 64), "stream"), ((2, 20, 4096, 64), "stream"),
                        ((2, 20, 2304, 64), "stream"), ((2, 10, 9216, 64), "stream"), ((1, 10, 2304, 64), "split"), ((2, 20, 144, 64), "cluster"), ((2, 20, 576, 64), "fused"),
-                       ((2, 2, 144, 64), "cluster"), ((2, 8, 4096, 40), "split"), ((2, 8, 64, 160), "cluster"),
-                       ((2, 8, 256, 160), "split")]:
+                       ((2, 2, 144, 64), "cluster"), ((2, 8, 4096, 40), "fused"), ((2, 8, 1024, 80), "fused"),
+                       ((2, 8, 64, 160), "fused"), ((2, 8, 256, 160), "fused"), ((2, 100, 256, 160), "split"),
+                       ((2, 100, 64, 160), "cluster"), ((2, 8, 4096, 128), "split")]:
         op = attn.LinFusionAttention(*dims)
         assert op.variant == want, (dims, op.variant)
         op.close()
@@ -160,6 +162,8 @@ def test_bit_reproducible_run_to_run():
                            (wl.find_shape("sdxl_2048_L2"), "fused"),
                            (wl.find_shape("sd21_768_L4"), "fused"),
                            (wl.find_shape("sd15_512_L1"), "split"),
+                           (wl.find_shape("sd15_512_L1"), "fused"),
+                           (wl.find_shape("sd15_512_L3"), "fused"),
                            (wl.find_shape("sd15_512_L2"), "cluster")]:
         q, k, v = wl.make_qkv(shape, seed=3, device="cuda")
         y1, op = run_gpu(q, k, v, variant)
