@@ -560,8 +560,8 @@ def run_sweep(args):
                 if args.dtype == "fp16":
                     q, k, v = (t.half() for t in (q, k, v))
                 bufs.append((q, k, v, torch.empty_like(q)))
-            variants = ["auto", "split"] + (["stream", "fused"] if s.d == 64 else []) + \
-                       (["cluster"] if s.N <= 16384 else [])
+            variants = ["auto", "split"] + (["stream"] if s.d == 64 else []) + \
+                       (["fused"] if s.d in (40, 64, 80, 160) else []) + (["cluster"] if s.N <= 16384 else [])
             for variant in variants:
                 op = attn.LinFusionAttention(s.B, s.H, s.N, s.d, device=0, variant=variant, layout=args.layout,
                                              dtype=args.dtype)

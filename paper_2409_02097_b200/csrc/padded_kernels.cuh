@@ -79,6 +79,19 @@ __host__ __device__ __forceinline__ int padded_run_begin(int r, int tiles, int r
 // Control words behind the per-slab counters: ctrl[0] = CTAs of the running forward that have finished.
 constexpr int kPaddedCtrlWords = 1;
 
+// 16 columns of the lane's TMEM row into registers, without waiting: r[] may be read only after a
+// tmem_wait_loads() that follows.  Lets the next block's load run while the previous one is consumed.
+__device__ __forceinline__ void tmem_load_16cols_async(uint32_t taddr, uint32_t (&r)[16])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_loads() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // phi on the D real channels of one 128-token row held as atoms of 128-byte rows (`row_addr` = the
 // row inside atom 0, `sw` = row & 7: 16-byte chunk c of a row sits at chunk position c ^ sw).
 template <int D, int KIND>
@@ -323,10 +336,13 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             if (warp_has_rows) {
                 float* dst = partials + (static_cast<size_t>(slab) * per_slab + run) * C::PARTIAL_FLOATS + e;
                 const uint32_t b_row = smem_u32(bsm) + (e >> 6) * C::B_ATOM_BYTES + (e & 7) * 2;
+                uint32_t dd[2][16];
+                tmem_load_16cols_async(lane_base + group * C::DKN, dd[0]);
 #pragma unroll
                 for (int c0 = 0; c0 < C::DKN; c0 += 16) {
-                    uint32_t d[16];
-                    tmem_load_16cols(lane_base + group * C::DKN + c0, d);
+                    uint32_t (&d)[16] = dd[(c0 >> 4) & 1];
+                    tmem_wait_loads();
+                    if (c0 + 16 < C::DKN) tmem_load_16cols_async(lane_base + group * C::DKN + c0 + 16, dd[((c0 >> 4) + 1) & 1]);
                     if (e < C::DVN) {
                         if (per_slab == 1) {
                             // alone on the slab: S[c][e] | z[c] -> operand row c, channel e (eight lanes fill one
@@ -457,12 +473,15 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 break;
             }
             tc_fence_after_sync();
-            const float den = __uint_as_float(tmem_load_1col(d_tmem + D));  // phi(Q_i) . z
+            uint32_t dd[2][16];
+            tmem_load_16cols_async(d_tmem, dd[0]);
+            const float den = __uint_as_float(tmem_load_1col(d_tmem + D));  // phi(Q_i) . z (waits for both loads)
             const float inv = row_scale(den, sc);
 #pragma unroll
             for (int cb = 0; cb < C::DKN / 16; ++cb) {
-                uint32_t d[16];
-                tmem_load_16cols(d_tmem + 16 * cb, d);
+                uint32_t (&d)[16] = dd[cb & 1];
+                if (cb > 0) tmem_wait_loads();
+                if (cb + 1 < C::DKN / 16) tmem_load_16cols_async(d_tmem + 16 * (cb + 1), dd[(cb + 1) & 1]);
 #pragma unroll
                 for (int h2 = 0; h2 < 2; ++h2) {
                     const int cc = 2 * cb + h2;  // 16-byte chunk of the output row
