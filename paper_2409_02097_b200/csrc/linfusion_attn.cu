@@ -79,6 +79,7 @@ struct Plan {
     long long W_state = 0, W_apply = 0;
     int G_state = 0, G_apply = 0, spans = 0;
     int merged_reduce = 0;  // stream: the apply kernel sums the partials itself (two launches)
+    int apply_static_runs = 0;  // stream: CTAs per slab when the apply kernel's CTAs take fixed runs of tiles
     // cluster
     int cluster_size = 0;
     // stream, fed from X (token-major handles): units are (batch, head pair, tile)
@@ -244,6 +245,13 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // Every slab needs an apply CTA that starts on it for the apply kernel to take over the second
         // stage of the reduction (see MergedReduce); otherwise the reduction keeps its own kernel.
         p->merged_reduce = slabs <= p->G_apply ? 1 : 0;
+        // Fixed runs of tiles in the apply kernel where every slab has the same number of CTAs and a CTA's
+        // share is a few dozen tiles (measured: the hand-out through counters ends such kernels with a tail
+        // of 7 us at N = 4096 x 40 slabs and N = 16384 x 20 slabs — CTAs that got fewer tiles than their
+        // neighbours move to other slabs for a tile or two and drain their ring for each new operand).
+        if (p->G_apply % slabs == 0 && p->G_apply / slabs <= p->tiles_apply &&
+            p->tiles_apply <= 64ll * (p->G_apply / slabs))
+            p->apply_static_runs = p->G_apply / slabs;
         p->launches = p->merged_reduce != 0 ? 2 : 3;
     } else if (v == LINFUSION_VARIANT_FUSED && !square64) {
         // One persistent launch, widths 40 / 80 / 160: per_slab CTAs on every slab, one partial each.
@@ -729,7 +737,7 @@ cudaError_t launch_stream(const linfusion_attn* h, const __nv_bfloat16* q, const
     }
     e = launch_chained(stream_apply_kernel<KIND>, dim3(p.G_apply), dim3(ApplyCfg::THREADS), ApplyCfg::SMEM_BYTES, s,
                        mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs,
-                       apply_scales(h->desc), h->desc.H, mr);
+                       apply_scales(h->desc), h->desc.H, mr, p.apply_static_runs);
     if (e != cudaSuccess) return e;
     mark(h, p.merged_reduce != 0 ? 2 : 3, s);
     return cudaGetLastError();
@@ -1661,7 +1669,7 @@ cudaError_t launch_stream_half(const linfusion_attn* h, bool state_half, const _
                                                 dtype_of(h->desc), operand_scale(h->desc));
         stream_apply_kernel<KIND><<<p.G_apply, ApplyCfg::THREADS, ApplyCfg::SMEM_BYTES, s>>>(
             mq, my, h->operand, h->tile_counters, h->status, p.tiles_apply, p.slabs, apply_scales(h->desc), h->desc.H,
-            MergedReduce{});
+            MergedReduce{}, p.apply_static_runs);
     }
     return cudaGetLastError();
 }

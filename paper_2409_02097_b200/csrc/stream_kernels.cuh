@@ -491,7 +491,8 @@ stream_pack_kernel(PeerStates states, unsigned char* __restrict__ operand,
 // Apply.  Tiles are handed out per slab through an atomic counter: CTA g starts on its home slab
 // g*slabs/G and moves to the next slab that still has tiles when one runs dry, so the CTAs of a
 // slab share its tail and early finishers help elsewhere.  Each output tile depends only on its
-// own Q rows and the slab's S | z, so the result does not depend on who computes it.
+// own Q rows and the slab's S | z, so the result does not depend on who computes it.  For short
+// runs with the same number of CTAs on every slab the host asks for fixed runs instead (static_runs).
 //
 // Roles in a CTA (one CTA per SM; it owns all 512 TMEM columns):
 //   producer warp — claims tiles, copies the slab's B operand into shared memory when the slab
@@ -527,7 +528,8 @@ template <int KIND>
 __global__ void __launch_bounds__(StreamApplyCfg::THREADS, 1)
 stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_y,
                     const unsigned char* __restrict__ operand, int* __restrict__ tile_counters,
-                    uint32_t* __restrict__ status, int tiles_per_slab, int slabs, ApplyScales sc, int H, MergedReduce mr)
+                    uint32_t* __restrict__ status, int tiles_per_slab, int slabs, ApplyScales sc, int H, MergedReduce mr,
+                    int static_runs)
 {
     using C = StreamApplyCfg;
     extern __shared__ unsigned char smem_raw[];
@@ -604,28 +606,10 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         const float4* part4 = reinterpret_cast<const float4*>(mr.partials);
         constexpr int V4 = kStreamStateFloats / 4;  // 1040: S rows as 16 float4 each, then z as 16
         float4* st4 = reinterpret_cast<float4*>(mr.state + static_cast<size_t>(home) * kStreamStateFloats);
-        for (int idx = ttid; idx < V4; idx += TEAM) {
-            // contributor g0's partial of this slab sits in its slot `slot0`; every later contributor's run
-            // starts inside the slab (its slot 0).  Eight loads in flight, summed in CTA order.
-            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int gb = g0; gb < g1; gb += 8) {
-                float4 v[8];
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    v[j] = gb + j < g1 ? __ldcg(part4 + (static_cast<size_t>(gb + j) * mr.spans + (gb + j == g0 ? slot0 : 0)) * V4 + idx)
-                                       : make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    if (gb + j == g0) {
-                        sum = v[j];  // the first term as it is: the same bits as a sum that starts from it
-                    } else if (gb + j < g1) {
-                        sum.x += v[j].x;
-                        sum.y += v[j].y;
-                        sum.z += v[j].z;
-                        sum.w += v[j].w;
-                    }
-                }
-            }
+        // contributor g0's partial of this slab sits in its slot `slot0`; every later contributor's run starts
+        // inside the slab (its slot 0).  A thread walks through the (element, contributor) pairs of its
+        // elements with twelve 16-byte loads in flight and adds them in CTA order.
+        auto emit = [&](int idx, const float4& sum) {
             if (writer) st4[idx] = sum;
             const float f[4] = {sum.x * mr.scale, sum.y * mr.scale, sum.z * mr.scale, sum.w * mr.scale};
             if (idx < 1024) {
@@ -643,6 +627,43 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 wv.x = to_storage16(f[0], mr.dtype) | (static_cast<uint32_t>(to_storage16(f[1], mr.dtype)) << 16);
                 wv.y = to_storage16(f[2], mr.dtype) | (static_cast<uint32_t>(to_storage16(f[3], mr.dtype)) << 16);
                 *reinterpret_cast<uint2*>(bsm + 64 * 128 + t4 * 8) = wv;
+            }
+        };
+        {
+            constexpr int kInFlight = 12;
+            int idx = ttid, gc = g0;
+            float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+            while (idx < V4) {
+                float4 v[kInFlight];
+                int idx2 = idx, gc2 = gc;
+#pragma unroll
+                for (int u = 0; u < kInFlight; ++u) {
+                    if (idx2 < V4) {
+                        v[u] = __ldcg(part4 + (static_cast<size_t>(gc2) * mr.spans + (gc2 == g0 ? slot0 : 0)) * V4 + idx2);
+                        if (++gc2 == g1) {
+                            gc2 = g0;
+                            idx2 += TEAM;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kInFlight; ++u) {
+                    if (idx < V4) {
+                        if (gc == g0) {
+                            sum = v[u];  // the first term as it is: the same bits as a sum that starts from it
+                        } else {
+                            sum.x += v[u].x;
+                            sum.y += v[u].y;
+                            sum.z += v[u].z;
+                            sum.w += v[u].w;
+                        }
+                        if (++gc == g1) {
+                            emit(idx, sum);
+                            gc = g0;
+                            idx += TEAM;
+                        }
+                    }
+                }
             }
         }
         fence_proxy_async_smem();
@@ -668,11 +689,23 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         bool home_pending = mr.enabled != 0;          // the other warps may still be writing it
         int it = 0, issued = 0, loaded_slab = -1;
         bool ok = true;
+        // static_runs > 0 (the grid is static_runs CTAs per slab): this CTA takes a fixed run of its home
+        // slab's tiles and nothing else.  A CTA's share is then shorter than the ring is deep, and tiles
+        // claimed through the counters would go to whichever CTA asks first, leave the others short, and
+        // send them to other slabs for a tile or two at the price of draining the ring for the new operand.
+        const int run = static_runs > 0 ? static_cast<int>(blockIdx.x) % static_runs : 0;
+        int s_next = static_runs > 0 ? static_cast<int>((static_cast<long long>(run) * tiles_per_slab) / static_runs) : 0;
+        const int s_end = static_runs > 0 ? static_cast<int>((static_cast<long long>(run + 1) * tiles_per_slab) / static_runs) : 0;
+        auto claim = [&]() {
+            if (static_runs > 0) return s_next < s_end ? s_next++ : tiles_per_slab;
+            return atomicAdd(&tile_counters[slab], 1);
+        };
         int next = 0;
-        if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
+        if (lane == 0) next = claim();
         while (true) {
             const int tile = __shfl_sync(0xffffffffu, next, 0);
             if (tile >= tiles_per_slab) {
+                if (static_runs > 0) break;
                 // Next slab, in cyclic order, whose counter has not run past its tiles.
                 int found = -1;
                 for (int base = 0; base < slabs && found < 0; base += 32) {
@@ -685,12 +718,12 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 }
                 if (found < 0) break;
                 slab = found;
-                if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
+                if (lane == 0) next = claim();
                 continue;
             }
             // Claim the tile after this one now: the atomic's round trip (comparable to the time a
             // tile takes) overlaps the wait for a free stage and the copy below.
-            if (lane == 0) next = atomicAdd(&tile_counters[slab], 1);
+            if (lane == 0) next = claim();
             const bool new_slab = slab != loaded_slab;
             const bool copy_b = new_slab && slab != smem_slab;
             if (copy_b) {
