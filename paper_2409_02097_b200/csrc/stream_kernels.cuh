@@ -669,7 +669,8 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         fence_proxy_async_smem();
         named_barrier_sync(1, TEAM);
         if (ttid == 0) mbar_arrive(home_done);
-        if (writer) {
+        if (writer && static_runs == 0) {
+            // (with fixed runs nobody works on another CTA's slab: no image, no flag)
             uint4* img = reinterpret_cast<uint4*>(mr.operand + static_cast<size_t>(home) * C::B_BYTES);
             for (int i = ttid; i < C::B_BYTES / 16; i += TEAM) img[i] = reinterpret_cast<const uint4*>(bsm)[i];
             named_barrier_sync(1, TEAM);
