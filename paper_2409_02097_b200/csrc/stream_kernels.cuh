@@ -80,9 +80,10 @@ struct StreamApplyCfg {
     static constexpr int STAGES = 12;
     static constexpr int B_ROWS = 80;  // N of the MMA: 64 channels of S^T, z, padding to a multiple of 16
     static constexpr int B_BYTES = B_ROWS * kStreamRowBytes;    // 10 KB
+    static constexpr int B_BUFFERS = 2;                         // the next slab's operand is copied while the last one is in use
     static constexpr int TMEM_COLS_PER_GROUP = 128;             // A: 32 columns, D: 80
     static constexpr int TMEM_COLS = 512;                       // a power of two >= GROUPS * 128
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + B_BYTES + 1024 /*align*/ + 1024 /*barriers, meta*/;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + B_BUFFERS * B_BYTES + 1024 /*align*/ + 1024 /*barriers, meta*/;
 };
 static_assert(StreamApplyCfg::GROUPS * StreamApplyCfg::TMEM_COLS_PER_GROUP <= StreamApplyCfg::TMEM_COLS, "TMEM budget");
 static_assert(StreamApplyCfg::STAGES >= 2 * StreamApplyCfg::GROUPS + 2, "end markers need released stages");
@@ -535,14 +536,14 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = reinterpret_cast<unsigned char*>(
         (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    unsigned char* bsm = smem + C::STAGES * C::STAGE_BYTES;  // B operand, on a 1024-byte boundary
-    uint64_t* full = reinterpret_cast<uint64_t*>(bsm + C::B_BYTES);
+    unsigned char* bsm = smem + C::STAGES * C::STAGE_BYTES;  // B operands (two buffers), on 1024-byte boundaries
+    uint64_t* full = reinterpret_cast<uint64_t*>(bsm + C::B_BUFFERS * C::B_BYTES);
     uint64_t* empty = full + C::STAGES;
     uint64_t* y_ready = empty + C::STAGES;
     uint64_t* a_ready = y_ready + C::STAGES;  // per group
     uint64_t* mma_done = a_ready + C::GROUPS;  // per group
-    uint64_t* b_ready = mma_done + C::GROUPS;  // the operand of the slab now being posted is in shared memory
-    uint64_t* home_done = b_ready + 1;         // the home slab's operand has been summed into shared memory
+    uint64_t* b_ready = mma_done + C::GROUPS;  // [B_BUFFERS]: a slab's operand has been put into that buffer
+    uint64_t* home_done = b_ready + C::B_BUFFERS;  // the home slab's operand has been summed into buffer 0
     int2* meta = reinterpret_cast<int2*>(home_done + 1);  // (slab, tile) of each stage; slab < 0 ends
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(meta + C::STAGES);
 
@@ -558,7 +559,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             mbar_init(&a_ready[g], 4);
             mbar_init(&mma_done[g], 1);
         }
-        mbar_init(b_ready, 1);
+        for (int b = 0; b < C::B_BUFFERS; ++b) mbar_init(&b_ready[b], 1);
         mbar_init(home_done, 1);
         mbar_fence_init();
     }
@@ -686,9 +687,14 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         uint64_t policy = 0;
         if (lane == 0) policy = policy_evict_first();
         int slab = home;
-        int smem_slab = mr.enabled != 0 ? home : -1;  // whose operand the shared-memory buffer holds (or will, once home_done)
-        bool home_pending = mr.enabled != 0;          // the other warps may still be writing it
-        int it = 0, issued = 0, loaded_slab = -1;
+        // Two operand buffers: the operand of the slab being posted sits in buffer cur_buf; when the slab
+        // changes the new operand goes to the other buffer, which was last read by the tiles posted before
+        // the previous change (long gone, as a rule), so the ring is not drained for it.  Buffer 0 starts
+        // as the home slab's, summed in place by the other warps (complete once home_done).
+        int cur_buf = 0;
+        const bool home_in_place = mr.enabled != 0;
+        bool home_pending = mr.enabled != 0;          // the other warps may still be writing buffer 0
+        int it = 0, issued = 0, loaded_slab = -1, last_switch_it = 0;
         bool ok = true;
         // static_runs > 0 (the grid is static_runs CTAs per slab): this CTA takes a fixed run of its home
         // slab's tiles and nothing else.  A CTA's share is then shorter than the ring is deep, and tiles
@@ -726,12 +732,14 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             // tile takes) overlaps the wait for a free stage and the copy below.
             if (lane == 0) next = claim();
             const bool new_slab = slab != loaded_slab;
-            const bool copy_b = new_slab && slab != smem_slab;
-            if (copy_b) {
-                // Every tile posted so far must have left (its MMAs, which read B, are then
-                // complete as well) before B is overwritten.
+            const bool first_slab = loaded_slab < 0;
+            const bool copy_b = new_slab && !(first_slab && home_in_place);
+            const int use_buf = new_slab ? (first_slab ? 0 : cur_buf ^ 1) : cur_buf;
+            if (copy_b && !first_slab) {
+                // The tiles that read buffer use_buf are those posted before the previous change of slab:
+                // they must have left (their MMAs are then complete as well) before it is overwritten.
                 if (lane == 0) {
-                    for (int j = it > C::STAGES ? it - C::STAGES : 0; j < it && ok; ++j)
+                    for (int j = it > C::STAGES ? it - C::STAGES : 0; j < last_switch_it && ok; ++j)
                         ok = mbar_wait(&empty[j % C::STAGES], (j / C::STAGES) & 1);
                     if (!ok) report_wait_expired(status);
                 }
@@ -742,7 +750,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
             if (lane == 0) {
                 ok = mbar_wait(&empty[s], ((it / C::STAGES) & 1) ^ 1);
                 if (ok) {
-                    meta[s] = make_int2(slab, tile);
+                    meta[s] = make_int2(slab, tile | (use_buf << 30));
                     mbar_expect_tx(&full[s], C::STAGE_BYTES);
                     tma_load_4d(smem + s * C::STAGE_BYTES, &tmap_q, 0, tile * C::TILE, slab % H, slab / H, &full[s], policy);
                     ++issued;
@@ -759,10 +767,10 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 // the first MMA of a slab.
                 if (copy_b) {
                     if (mr.enabled != 0) {
-                        // the buffer must not be overwritten while the home slab's sum is still being written
+                        // buffer 0 must not be overwritten while the home slab's sum is still being written
                         // into it; the image is written during this kernel by the slab's first home CTA
-                        if (lane == 0 && home_pending) ok = mbar_wait(home_done, 0);
-                        home_pending = false;
+                        if (lane == 0 && home_pending && use_buf == 0) ok = mbar_wait(home_done, 0);
+                        if (use_buf == 0) home_pending = false;
                         if (lane == 0 && ok) ok = counter_wait(&mr.ready[slab], 0u, 1u);
                         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
                         if (!ok) {
@@ -771,13 +779,15 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                         }
                     }
                     const uint4* src = reinterpret_cast<const uint4*>(operand + static_cast<size_t>(slab) * C::B_BYTES);
-                    for (int i = lane; i < C::B_BYTES / 16; i += 32) reinterpret_cast<uint4*>(bsm)[i] = __ldcg(src + i);
-                    smem_slab = slab;
+                    uint4* dst = reinterpret_cast<uint4*>(bsm + use_buf * C::B_BYTES);
+                    for (int i = lane; i < C::B_BYTES / 16; i += 32) dst[i] = __ldcg(src + i);
                 }
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(b_ready);
+                if (lane == 0) mbar_arrive(&b_ready[use_buf]);
                 loaded_slab = slab;
+                cur_buf = use_buf;
+                last_switch_it = it - 1;  // the tile just posted is the first of this slab
             }
         }
         if (lane == 0) {
@@ -812,7 +822,7 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                 }
                 const int2 m = meta[s];
                 if (m.x < 0) break;  // the first end marker: every tile posted before it has left
-                tma_store_4d(&tmap_y, smem + s * C::STAGE_BYTES, 0, m.y * C::TILE, m.x % H, m.x / H, policy);
+                tma_store_4d(&tmap_y, smem + s * C::STAGE_BYTES, 0, (m.y & 0x3fffffff) * C::TILE, m.x % H, m.x / H, policy);
                 tma_store_wait_read();
                 mbar_arrive(&empty[s]);
             }
@@ -824,9 +834,10 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
         // then; with a single issuing thread it has not.)
         if (lane == 0) {
             const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), C::TILE, C::B_ROWS);
-            const uint64_t b_desc = umma_desc_kmajor_sw128(smem_u32(bsm));
+            const uint64_t b_desc0 = umma_desc_kmajor_sw128(smem_u32(bsm));
+            uint64_t b_desc = b_desc0;
             int cur_slab = -1;
-            uint32_t operands_seen = 0;
+            uint32_t operands_seen[C::B_BUFFERS] = {0u, 0u};
             if (mr.enabled != 0 && !mbar_wait(home_done, 0)) report_wait_expired(status);
             for (int it = 0;; ++it) {
                 const int s = it % C::STAGES, g = it % C::GROUPS;
@@ -834,15 +845,18 @@ stream_apply_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_con
                     report_wait_expired(status);
                     break;
                 }
-                const int slab = meta[s].x;
+                const int2 m = meta[s];
+                const int slab = m.x;
                 if (slab < 0) break;
                 if (slab != cur_slab) {
-                    if (!mbar_wait(b_ready, operands_seen & 1)) {
+                    const int buf = (m.y >> 30) & 1;
+                    if (!mbar_wait(&b_ready[buf], operands_seen[buf] & 1u)) {
                         report_wait_expired(status);
                         break;
                     }
-                    ++operands_seen;
+                    ++operands_seen[buf];
                     cur_slab = slab;
+                    b_desc = b_desc0 + static_cast<uint64_t>(buf * (C::B_BYTES >> 4));  // start address field, 16-byte units
                 }
                 if (!mbar_wait(&a_ready[g], (it / C::GROUPS) & 1)) {
                     report_wait_expired(status);
