@@ -142,7 +142,7 @@ linfusion_status_t linfusion_attn_forward(linfusion_attn_t* h, const void* q, co
  * The same operation for callers whose tensors live in HOST memory (pinned memory makes the
  * copies asynchronous): copies K, V, Q to device staging buffers owned by the handle, runs
  * forward() on them and copies Y back, ordered after the earlier work and before the later work
- * of `cuda_stream`.  Large problems are cut into up to 8 groups of (b, h) slabs so that the upload
+ * of `cuda_stream`.  Large problems are cut into up to 20 groups of (b, h) slabs so that the upload
  * of one group, the kernels of the previous one and the download of the one before overlap (two
  * internal copy streams); each group then has its own fixed split of N, so Y may differ from
  * forward()'s in the last bits while staying bit-identical from call to call.  The staging

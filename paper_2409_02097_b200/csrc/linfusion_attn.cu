@@ -474,7 +474,7 @@ struct linfusion_attn {
 
 // forward_host() cuts the slabs into groups and overlaps the upload of group i+1, the kernels of
 // group i and the download of group i-1 on three streams.
-constexpr int kMaxHostGroups = 8;
+constexpr int kMaxHostGroups = 20;
 struct HostPipe {
     int groups = 1;
     linfusion_attn* sub = nullptr;  // handle for one group of slabs (null when groups == 1)
