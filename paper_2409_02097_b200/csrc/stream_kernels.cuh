@@ -70,7 +70,7 @@ static_assert(StreamStateCfg::SMEM_BYTES > 116 * 1024, "one state CTA per SM");
 
 struct StreamApplyCfg {
     static constexpr int TILE = 128;   // tokens per stage = rows of one MMA tile = TMEM lanes
-    static constexpr int GROUPS = 3;   // warpgroups, each working on its own tile
+    static constexpr int GROUPS = 4;   // warpgroups, each working on its own tile
     static constexpr int CONSUMER_WARPS = 4 * GROUPS;
     static constexpr int PRODUCER_WARP = CONSUMER_WARPS;
     static constexpr int STORE_WARP = CONSUMER_WARPS + 1;
@@ -498,7 +498,7 @@ stream_pack_kernel(PeerStates states, unsigned char* __restrict__ operand,
 // Roles in a CTA (one CTA per SM; it owns all 512 TMEM columns):
 //   producer warp — claims tiles, copies the slab's B operand into shared memory when the slab
 //                   changes (after every posted tile has left), loads Q tiles with TMA;
-//   3 warpgroups  — group g takes the tiles posted g-th, (g+3)-th, ...; thread r of a group owns
+//   4 warpgroups  — group g takes the tiles posted g-th, (g+4)-th, ...; thread r of a group owns
 //                   row r of the tile = TMEM lane r (a warp may only touch the 32 lanes of its
 //                   quarter, so warp w of the CTA works on rows 32*(w%4) ..);
 //   MMA warp      — one thread issues every tcgen05.mma of the CTA, in posting order;
