@@ -136,6 +136,11 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint64_t* acc_done = mma_done + C::APPLY_GROUPS;
     uint64_t* b_ready = acc_done + 1;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b_ready + 1);
+    // Ring positions the producer has issued so far.  A consumer looks at a slot's `full` barrier only once
+    // the position it wants has been issued: the parity of an mbarrier wait tells phase n from phase n + 1,
+    // not from phase n - 1, and a warpgroup whose first tile already sits in a reused slot would otherwise
+    // take the completion of the slot's earlier use for its own.
+    uint32_t* issued_pos = tmem_slot + 1;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int slab = blockIdx.x / per_slab, run = blockIdx.x % per_slab;
@@ -156,6 +161,7 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         }
         mbar_init(acc_done, 1);
         mbar_init(b_ready, C::CONSUMER_WARPS);
+        *issued_pos = 0u;
         mbar_fence_init();
     }
     // The apply operand's padding (rows c >= D everywhere; channels e > D where a CTA builds the operand
@@ -202,6 +208,7 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 for (int a = 0; a < C::NA; ++a)
                     tma_load_4d(dst + a * C::ATOM_BYTES, map, 64 * a, tile * C::TILE, head, batch, &full[s], policy);
                 ++issued;
+                asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_u32(issued_pos)), "r"(static_cast<uint32_t>(issued)) : "memory");
             }
             drain_loads<C::SLOTS>(full, 0, issued, status);
         }
@@ -297,11 +304,25 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         const uint32_t sw = row & 7;
         const uint32_t lane_base = tmem_base + (static_cast<uint32_t>(wq * 32) << 16);
         bool ok = true;
+        // Until the producer has issued ring position `pos` (bounded like every other wait).
+        auto wait_issued = [&](int pos) {
+            const uint32_t addr = smem_u32(issued_pos);
+            uint32_t v;
+            asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+            if (v > static_cast<uint32_t>(pos)) return true;
+            const unsigned long long t0 = global_timer_ns();
+            do {
+                __nanosleep(20);
+                asm volatile("ld.acquire.cta.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+                if (v > static_cast<uint32_t>(pos)) return true;
+            } while (global_timer_ns() - t0 < kMaxBarrierWaitNs);
+            return false;
+        };
 
         // 1. phi(K) in place, a one into channel D of V
         for (int i = group; i < n && ok; i += C::APPLY_GROUPS) {
             const int sk = slot_of(2 * i), sv = slot_of(2 * i + 1);
-            ok = mbar_wait(&full[sk], phase_of(2 * i)) && mbar_wait(&full[sv], phase_of(2 * i + 1));
+            ok = wait_issued(2 * i + 1) && mbar_wait(&full[sk], phase_of(2 * i)) && mbar_wait(&full[sv], phase_of(2 * i + 1));
             __syncwarp();
             if (!ok) {
                 if (lane == 0) report_wait_expired(status);
@@ -454,7 +475,7 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         const uint32_t d_tmem = lane_base + group * C::DVN;
         for (int j = group; j < n && ok; j += C::APPLY_GROUPS) {
             const int pos = 2 * n + j, s = slot_of(pos);
-            ok = mbar_wait(&full[s], phase_of(pos));
+            ok = wait_issued(pos) && mbar_wait(&full[s], phase_of(pos));
             __syncwarp();
             if (!ok) {
                 if (lane == 0) report_wait_expired(status);
