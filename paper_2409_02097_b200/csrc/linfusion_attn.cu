@@ -19,6 +19,14 @@ using namespace lf;
 
 namespace {
 
+// In the stream and fused kernels a ring stage is always served by the same warpgroup (stage = it % STAGES,
+// group = it % GROUPS), so a group has consumed a stage's previous use before it waits for the next one and
+// the parity of its mbarrier wait is unambiguous.  That needs the ring depth to be a multiple of the group
+// count.  (The padded-width kernel's ring can be odd; it guards its waits with the producer's issue count.)
+static_assert(StreamStateCfg::STAGES % StreamStateCfg::GROUPS == 0 && StreamApplyCfg::STAGES % StreamApplyCfg::GROUPS == 0 &&
+                  FusedCfg::SLOTS % FusedCfg::GROUPS == 0 && FusedCfg::KV_STAGES % FusedCfg::GROUPS == 0,
+              "a ring stage must stay with one warpgroup");
+
 constexpr int kDefaultSmCount = 148;
 using ApplyCfg = StreamApplyCfg;
 
