@@ -136,7 +136,9 @@ def test_stream_variant_tail_and_slab_crossing():
     """Many slabs, ragged N: every CTA's run crosses slab boundaries and tail tiles are masked."""
     # the last case gives every CTA a run of 60 tiles: more than one tensor-memory segment per slab
     # and, for the CTAs at the seams, a change of slab in mid-run
-    for (B, H, N) in [(2, 37, 1000), (1, 100, 130), (2, 20, 2500), (1, 3, 378917)]:
+    # (1, 7, 200000): long enough for the apply kernel to hand its tiles out through the per-slab counters
+    # (the shorter cases get fixed runs), with CTAs moving on to other slabs at the end
+    for (B, H, N) in [(2, 37, 1000), (1, 100, 130), (2, 20, 2500), (1, 3, 378917), (1, 7, 200000)]:
         q, k, v = wl.make_small(B, H, N, 64, seed=5, device="cuda")
         ref = oracle_y(q, k, v)
         for variant in ("stream", "fused"):
