@@ -55,15 +55,15 @@ bool supported_widths(int dk, int dv)
 bool padded_width(int dk, int dv) { return dk == dv && (dv == 40 || dv == 80 || dv == 160); }
 int padded_partial_floats(int d) { return ((d + 15) / 16 * 16) * ((d + 1 + 15) / 16 * 16); }
 
-// CTAs per slab of that kernel, or 0 where it does not apply: every slab needs a CTA of its own (all
-// of them resident together), and a CTA's run of tiles must fit one accumulation in tensor memory.
+// CTAs per slab of that kernel, or 0 where it does not apply: a CTA's run of tiles must fit one
+// accumulation in tensor memory (with more slabs than SMs a CTA takes whole slabs, several in turn).
 // Every CTA of a slab reads all of the slab's partials (9 KB each at d = 40, 30 KB at 80, 110 KB at 160),
 // so their number is kept to what makes that a couple of hundred KB at most (more only where the runs
 // would otherwise be too long); then the smallest count that gives the CTAs the same longest run is taken.
 int padded_per_slab(int N, int slabs, int sm_count, int d)
 {
-    if (slabs > sm_count) return 0;
     const int tiles = (N + 127) / 128;
+    if (slabs > sm_count) return tiles <= 32 ? 1 : 0;
     int k = sm_count / slabs;
     if (k > tiles) k = tiles;
     int cap = static_cast<int>((192u * 1024u) / (static_cast<unsigned>(padded_partial_floats(d)) * 4u));
@@ -266,8 +266,8 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         p->padded_per_slab = padded_per_slab(d->N, slabs, sm_count, dv);
         if (p->padded_per_slab == 0) return LINFUSION_ERR_UNSUPPORTED;
         p->tiles_state = p->tiles_apply = (d->N + 127) / 128;
-        p->G_state = p->G_apply = slabs * p->padded_per_slab;
-        partial_floats = static_cast<size_t>(p->G_state) * padded_partial_floats(dv);
+        p->G_state = p->G_apply = slabs > sm_count ? sm_count : slabs * p->padded_per_slab;
+        partial_floats = p->padded_per_slab > 1 ? static_cast<size_t>(p->G_state) * padded_partial_floats(dv) : 0;
         p->launches = 1;
     } else if (v == LINFUSION_VARIANT_FUSED) {
         // One persistent launch.  Two waves of slabs once every CTA has a couple of tiles in each

@@ -11,7 +11,8 @@
 // is z = sum phi(K_j) (Eq. 5) and no separate operand block of ones is needed.
 //
 // Work split.  Every slab is cut into `per_slab` runs of whole tiles, one CTA per run (grid =
-// slabs * per_slab <= SM count; all CTAs resident together).  A CTA
+// slabs * per_slab <= SM count; all CTAs resident together; per_slab = 1 and grid = SM count when
+// there are more slabs than SMs).  A CTA
 //   1. streams the K and V tiles of its run through a ring of tile slots, applies phi to the K
 //      rows in place, and accumulates  D[e][c] += sum_j [V | 1]_je phi(K)_jc  in tensor memory
 //      (A = [V | 1]^T and B = phi(K)^T, both MN-major as TMA delivers them);
@@ -29,8 +30,10 @@
 //      over the Q row, and a TMA store (clipped at D channels and N tokens) sends the tile to Y.
 // Every CTA of a slab reads all of its partials, so the host keeps per_slab small enough for that
 // to stay a few hundred KB.  A CTA that has its slab to itself (per_slab = 1) skips 2-3: it builds
-// the operand and the fp32 state straight from the accumulator.  The counters are zeroed again by
-// the CTA that finishes last, so every forward starts from zero.
+// the operand and the fp32 state straight from the accumulator; with more slabs than SMs such a CTA
+// takes several whole slabs one after the other (the K/V tiles of the next slab are fetched while the
+// current one is applied).  The counters are zeroed again by the CTA that finishes last, so every
+// forward starts from zero.
 #pragma once
 
 #include "stream_kernels.cuh"
@@ -111,7 +114,8 @@ __device__ __forceinline__ void phi_row_in_place(uint32_t row_addr, uint32_t sw)
     }
 }
 
-// grid = slabs * per_slab CTAs; CTA g works on slab g / per_slab, run g % per_slab of its tiles.
+// grid = slabs * per_slab CTAs; CTA g works on slab g / per_slab, run g % per_slab of its tiles (per_slab = 1:
+// grid <= slabs, CTA g on slabs g, g + grid, ...).
 // partials: [slab][run][DKN][DVN] fp32; state: [slab][D*D + D] fp32 (S [c][e], then z [c]); counters: one
 // word per slab, zero between forwards; ctrl: kPaddedCtrlWords words, zero between forwards.
 template <int D, int KIND>
@@ -135,7 +139,8 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint64_t* mma_done = q_ready + C::APPLY_GROUPS;  // [APPLY_GROUPS]
     uint64_t* acc_done = mma_done + C::APPLY_GROUPS;
     uint64_t* b_ready = acc_done + 1;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(b_ready + 1);
+    uint64_t* drained = b_ready + 1;  // every consumer warp is through with the apply tiles of a visit
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drained + 1);
     // Ring positions the producer has issued so far.  A consumer looks at a slot's `full` barrier only once
     // the position it wants has been issued: the parity of an mbarrier wait tells phase n from phase n + 1,
     // not from phase n - 1, and a warpgroup whose first tile already sits in a reused slot would otherwise
@@ -143,10 +148,14 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     uint32_t* issued_pos = tmem_slot + 1;
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int slab = blockIdx.x / per_slab, run = blockIdx.x % per_slab;
+    // A CTA visits one run of one slab (per_slab > 1) or, with its slabs to itself, the whole slabs
+    // blockIdx.x, blockIdx.x + gridDim.x, ... one after the other (more slabs than SMs).
+    const int run = per_slab > 1 ? static_cast<int>(blockIdx.x) % per_slab : 0;
+    const int first_slab = per_slab > 1 ? static_cast<int>(blockIdx.x) / per_slab : static_cast<int>(blockIdx.x);
+    const int slab_step = static_cast<int>(gridDim.x);
+    const int visits = per_slab > 1 ? 1 : (slabs - first_slab + slab_step - 1) / slab_step;
     const int t0 = padded_run_begin(run, tiles_per_slab, per_slab);
-    const int n = padded_run_begin(run + 1, tiles_per_slab, per_slab) - t0;  // tiles of this CTA (>= 1)
-    const int head = slab % H, batch = slab / H;
+    const int n = padded_run_begin(run + 1, tiles_per_slab, per_slab) - t0;  // tiles per visit (>= 1)
 
     if (tid == 0) {
         for (int s = 0; s < C::SLOTS; ++s) {
@@ -161,6 +170,7 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         }
         mbar_init(acc_done, 1);
         mbar_init(b_ready, C::CONSUMER_WARPS);
+        mbar_init(drained, C::CONSUMER_WARPS);
         *issued_pos = 0u;
         mbar_fence_init();
     }
@@ -183,7 +193,8 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     pdl_launch_dependents();
     pdl_wait();
 
-    // Ring positions: K of state tile i at 2i, V at 2i + 1; Q (later Y) of apply tile j at 2n + j.
+    // Ring positions of visit v, from base = 3 n v: K of state tile i at base + 2i, V at base + 2i + 1; Q (later Y)
+    // of apply tile j at base + 2n + j.
     auto slot_of = [](int pos) { return pos % C::SLOTS; };
     auto phase_of = [](int pos) { return static_cast<uint32_t>((pos / C::SLOTS) & 1); };
 
@@ -193,22 +204,25 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             const uint64_t policy = policy_evict_first();
             int issued = 0;
             bool ok = true;
-            for (int pos = 0; pos < 3 * n && ok; ++pos) {
-                const int s = slot_of(pos);
-                if (!mbar_wait(&empty[s], phase_of(pos) ^ 1u)) {
-                    report_wait_expired(status);
-                    ok = false;
-                    break;
-                }
-                const void* map = pos >= 2 * n ? &tmap_q : ((pos & 1) != 0 ? &tmap_v : &tmap_k);
-                const int tile = t0 + (pos >= 2 * n ? pos - 2 * n : pos >> 1);
-                unsigned char* dst = smem + s * C::SLOT_BYTES;
-                mbar_expect_tx(&full[s], C::SLOT_BYTES);
+            for (int visit = 0; visit < visits && ok; ++visit) {
+                const int slab = first_slab + visit * slab_step, head = slab % H, batch = slab / H;
+                for (int pos = 0; pos < 3 * n && ok; ++pos) {
+                    const int gp = visit * 3 * n + pos, s = slot_of(gp);
+                    if (!mbar_wait(&empty[s], phase_of(gp) ^ 1u)) {
+                        report_wait_expired(status);
+                        ok = false;
+                        break;
+                    }
+                    const void* map = pos >= 2 * n ? &tmap_q : ((pos & 1) != 0 ? &tmap_v : &tmap_k);
+                    const int tile = t0 + (pos >= 2 * n ? pos - 2 * n : pos >> 1);
+                    unsigned char* dst = smem + s * C::SLOT_BYTES;
+                    mbar_expect_tx(&full[s], C::SLOT_BYTES);
 #pragma unroll
-                for (int a = 0; a < C::NA; ++a)
-                    tma_load_4d(dst + a * C::ATOM_BYTES, map, 64 * a, tile * C::TILE, head, batch, &full[s], policy);
-                ++issued;
-                asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_u32(issued_pos)), "r"(static_cast<uint32_t>(issued)) : "memory");
+                    for (int a = 0; a < C::NA; ++a)
+                        tma_load_4d(dst + a * C::ATOM_BYTES, map, 64 * a, tile * C::TILE, head, batch, &full[s], policy);
+                    ++issued;
+                    asm volatile("st.release.cta.shared.u32 [%0], %1;" ::"r"(smem_u32(issued_pos)), "r"(static_cast<uint32_t>(issued)) : "memory");
+                }
             }
             drain_loads<C::SLOTS>(full, 0, issued, status);
         }
@@ -216,12 +230,23 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         // ---------------- MMA warp: one thread issues every tcgen05.mma ----------------
         if (lane == 0) {
             bool ok = true;
-            // state: D[e][c] += [V | 1]^T phi(K), 16 tokens per step
-            {
-                const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), 128, C::DKN, kUmmaAMnMajor | kUmmaBMnMajor);
-                uint32_t k_phase = 0u;  // bit s = phase of k_ready[s] to wait for next
+            const uint32_t idesc_state = umma_idesc_f32acc(kind_dtype(KIND), 128, C::DKN, kUmmaAMnMajor | kUmmaBMnMajor);
+            const uint32_t idesc_apply = umma_idesc_f32acc(kind_dtype(KIND), C::TILE, C::DVN, kUmmaBMnMajor);
+            const uint32_t b_addr = smem_u32(bsm);
+            uint32_t k_phase = 0u;  // bit s = phase of k_ready[s] to wait for next
+            int jj = 0;             // apply tiles so far, over all visits: tile jj belongs to warpgroup jj % APPLY_GROUPS
+            for (int visit = 0; visit < visits && ok; ++visit) {
+                const int base = visit * 3 * n;
+                // The accumulator shares its columns with the apply tiles of the visit before: those must
+                // have been read out.
+                if (visit > 0 && !mbar_wait(drained, static_cast<uint32_t>((visit - 1) & 1))) {
+                    report_wait_expired(status);
+                    ok = false;
+                    break;
+                }
+                // state: D[e][c] += [V | 1]^T phi(K), 16 tokens per step
                 for (int i = 0; i < n && ok; ++i) {
-                    const int sk = slot_of(2 * i), sv = slot_of(2 * i + 1);
+                    const int sk = slot_of(base + 2 * i), sv = slot_of(base + 2 * i + 1);
                     if (!mbar_wait(&k_ready[sk], (k_phase >> sk) & 1u)) {
                         report_wait_expired(status);
                         ok = false;
@@ -236,30 +261,29 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                         const uint64_t b_desc = umma_desc_mnmajor_sw128(k_addr + ks * 2048, C::ATOM_BYTES, 1024);
                         // rows e 0..127: atoms 0 and 1 of V (one atom: both halves read atom 0, rows 64.. are not used)
                         const uint64_t a_desc = umma_desc_mnmajor_sw128(v_addr + ks * 2048, C::NA >= 2 ? C::ATOM_BYTES : 0, 1024);
-                        umma_ss(tmem_base, a_desc, b_desc, idesc, acc);
+                        umma_ss(tmem_base, a_desc, b_desc, idesc_state, acc);
                         if (C::STATE_MMAS == 2) {
                             // rows e 128..191: atom 2 (read twice; rows 192.. are not used)
                             const uint64_t a2 = umma_desc_mnmajor_sw128(v_addr + 2 * C::ATOM_BYTES + ks * 2048, 0, 1024);
-                            umma_ss(tmem_base + C::DKN, a2, b_desc, idesc, acc);
+                            umma_ss(tmem_base + C::DKN, a2, b_desc, idesc_state, acc);
                         }
                     }
                     umma_commit(&empty[sk]);  // the slots are free once these MMAs have read them
                     umma_commit(&empty[sv]);
                 }
-                if (ok) umma_commit(acc_done);
-            }
-            // apply: D[i][e] = phi(Q) (S | z), 16 features per step
-            if (ok && !mbar_wait(b_ready, 0)) {
-                report_wait_expired(status);
-                ok = false;
-            }
-            if (ok) {
-                const uint32_t idesc = umma_idesc_f32acc(kind_dtype(KIND), C::TILE, C::DVN, kUmmaBMnMajor);
-                const uint32_t b_addr = smem_u32(bsm);
-                for (int j = 0; j < n; ++j) {
-                    const int g = j % C::APPLY_GROUPS, s = slot_of(2 * n + j);
-                    if (!mbar_wait(&q_ready[g], static_cast<uint32_t>((j / C::APPLY_GROUPS) & 1))) {
+                if (!ok) break;
+                umma_commit(acc_done);
+                // apply: D[i][e] = phi(Q) (S | z), 16 features per step
+                if (!mbar_wait(b_ready, static_cast<uint32_t>(visit & 1))) {
+                    report_wait_expired(status);
+                    ok = false;
+                    break;
+                }
+                for (int j = 0; j < n; ++j, ++jj) {
+                    const int g = jj % C::APPLY_GROUPS, s = slot_of(base + 2 * n + j);
+                    if (!mbar_wait(&q_ready[g], static_cast<uint32_t>((jj / C::APPLY_GROUPS) & 1))) {
                         report_wait_expired(status);
+                        ok = false;
                         break;
                     }
                     tc_fence_after_sync();
@@ -269,7 +293,7 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                     for (int ks = 0; ks < C::DKN / 16; ++ks) {
                         const uint64_t a_desc = umma_desc_kmajor_sw128(q_addr + (ks >> 2) * C::ATOM_BYTES + (ks & 3) * 32);
                         const uint64_t b_desc = umma_desc_mnmajor_sw128(b_addr + ks * 2048, C::B_ATOM_BYTES, 1024);
-                        umma_ss(d_tmem, a_desc, b_desc, idesc, ks > 0 ? 1u : 0u);
+                        umma_ss(d_tmem, a_desc, b_desc, idesc_apply, ks > 0 ? 1u : 0u);
                     }
                     umma_commit(&mma_done[g]);
                 }
@@ -280,19 +304,24 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         if (lane == 0) {
             const uint64_t policy = policy_evict_first();
             uint32_t y_phase = 0u;
-            for (int j = 0; j < n; ++j) {
-                const int pos = 2 * n + j, s = slot_of(pos);
-                if (!mbar_wait(&y_ready[s], (y_phase >> s) & 1u)) {
-                    report_wait_expired(status);
-                    break;
-                }
-                y_phase ^= 1u << s;
-                const unsigned char* src = smem + s * C::SLOT_BYTES;
+            bool ok = true;
+            for (int visit = 0; visit < visits && ok; ++visit) {
+                const int slab = first_slab + visit * slab_step, head = slab % H, batch = slab / H;
+                for (int j = 0; j < n; ++j) {
+                    const int s = slot_of(visit * 3 * n + 2 * n + j);
+                    if (!mbar_wait(&y_ready[s], (y_phase >> s) & 1u)) {
+                        report_wait_expired(status);
+                        ok = false;
+                        break;
+                    }
+                    y_phase ^= 1u << s;
+                    const unsigned char* src = smem + s * C::SLOT_BYTES;
 #pragma unroll
-                for (int a = 0; a < C::NA; ++a)
-                    tma_store_4d(&tmap_y, src + a * C::ATOM_BYTES, 64 * a, (t0 + j) * C::TILE, head, batch, policy);
-                tma_store_wait_read();
-                mbar_arrive(&empty[s]);
+                    for (int a = 0; a < C::NA; ++a)
+                        tma_store_4d(&tmap_y, src + a * C::ATOM_BYTES, 64 * a, (t0 + j) * C::TILE, head, batch, policy);
+                    tma_store_wait_read();
+                    mbar_arrive(&empty[s]);
+                }
             }
             tma_store_wait_all();
         }
@@ -319,10 +348,16 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             return false;
         };
 
+        uint32_t tiles_done = 0;  // apply tiles of this warpgroup so far, over all visits
+        const uint32_t d_tmem = lane_base + group * C::DVN;
+        const int dtype = kind_dtype(KIND);
+        for (int visit = 0; visit < visits && ok; ++visit) {
+        const int slab = first_slab + visit * slab_step, base = visit * 3 * n;
         // 1. phi(K) in place, a one into channel D of V
         for (int i = group; i < n && ok; i += C::APPLY_GROUPS) {
-            const int sk = slot_of(2 * i), sv = slot_of(2 * i + 1);
-            ok = wait_issued(2 * i + 1) && mbar_wait(&full[sk], phase_of(2 * i)) && mbar_wait(&full[sv], phase_of(2 * i + 1));
+            const int sk = slot_of(base + 2 * i), sv = slot_of(base + 2 * i + 1);
+            ok = wait_issued(base + 2 * i + 1) && mbar_wait(&full[sk], phase_of(base + 2 * i)) &&
+                 mbar_wait(&full[sv], phase_of(base + 2 * i + 1));
             __syncwarp();
             if (!ok) {
                 if (lane == 0) report_wait_expired(status);
@@ -341,11 +376,10 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         }
 
         float* st = state + static_cast<size_t>(slab) * (D * D + D);
-        const int dtype = kind_dtype(KIND);
 
         // 2. the accumulator (row e = TMEM lane, DKN columns c)
         if (ok) {
-            ok = mbar_wait(acc_done, 0);
+            ok = mbar_wait(acc_done, static_cast<uint32_t>(visit & 1));
             __syncwarp();
             if (!ok && lane == 0) report_wait_expired(status);
         }
@@ -470,11 +504,10 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         __syncwarp();
         if (ok && lane == 0) mbar_arrive(b_ready);
 
-        // 4. apply
-        uint32_t tiles_done = 0;
-        const uint32_t d_tmem = lane_base + group * C::DVN;
-        for (int j = group; j < n && ok; j += C::APPLY_GROUPS) {
-            const int pos = 2 * n + j, s = slot_of(pos);
+        // 4. apply: tile j of this visit is tile visit * n + j overall, and goes to warpgroup (visit * n + j) % APPLY_GROUPS
+        const int j_first = ((group - visit * n) % C::APPLY_GROUPS + C::APPLY_GROUPS) % C::APPLY_GROUPS;
+        for (int j = j_first; j < n && ok; j += C::APPLY_GROUPS) {
+            const int pos = base + 2 * n + j, s = slot_of(pos);
             ok = wait_issued(pos) && mbar_wait(&full[s], phase_of(pos));
             __syncwarp();
             if (!ok) {
@@ -520,6 +553,10 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(&y_ready[s]);
         }
+        // this warp has read its last tile of the visit out of tensor memory
+        __syncwarp();
+        if (ok && lane == 0) mbar_arrive(drained);
+        }  // visits
     }
     tc_fence_before_sync();
     __syncthreads();

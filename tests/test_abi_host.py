@@ -63,8 +63,12 @@ def test_workspace_bytes_is_pure_host_and_monotone():
     # per slab (8 CTAs per slab at N = 4096 x 16 slabs, d = 40), state, two words per slab + control, status
     f = _ws(attn.make_desc(2, 8, 4096, 40, variant="fused"))
     assert f == (16 * 8 * 48 * 48 * 4 + 255) // 256 * 256 + (16 * 40 * 41 * 4 + 255) // 256 * 256 + 256 + 256 + 256
+    # one CTA per slab (d = 160: a partial is 110 KB, so slabs are not shared): no partials at all
     assert _ws(attn.make_desc(2, 8, 256, 160, variant="fused")) == \
-        (16 * 160 * 176 * 4 + 255) // 256 * 256 + (16 * 160 * 161 * 4 + 255) // 256 * 256 + 256 + 256 + 256
+        (16 * 160 * 161 * 4 + 255) // 256 * 256 + 256 + 256 + 256
+    # more slabs than SMs: whole slabs per CTA, no partials either
+    assert _ws(attn.make_desc(2, 100, 256, 40, variant="fused")) == \
+        (200 * 40 * 41 * 4 + 255) // 256 * 256 + (200 * 8 + 255) // 256 * 256 + 256 + 256
     # the plan depends on the SM count it is given
     assert _ws(attn.make_desc(2, 10, 524288, 64, variant="stream"), 74) < s
 
@@ -86,7 +90,7 @@ def test_invalid_descriptors(kw):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(d=40, variant="fused", H=80),                    # more slabs than SMs: no CTA per slab
+    dict(d=40, variant="fused", H=80, N=128 * 33),        # more slabs than SMs and more than 32 tiles per slab
     dict(d=160, variant="fused", B=74, H=2, N=128 * 33),  # one CTA per slab, more than 32 tiles each
 ])
 def test_shapes_the_single_launch_at_padded_widths_cannot_take(kw):
