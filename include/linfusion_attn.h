@@ -57,7 +57,7 @@ typedef enum {
                                         apply kernel sums the partial states itself (three when slabs > SMs) */
 #define LINFUSION_VARIANT_CLUSTER 3u /* one launch, thread-block cluster per slab (small N); one CTA per slab for N <= 192 */
 #define LINFUSION_VARIANT_FUSED 4u   /* one launch, persistent TMA + tcgen05 kernel with per-slab counters: d = 64, and
-                                        d = 40 / 80 / 160 (d' = d) when N <= 4096 * max(1, SMs / (B*H)) */
+                                        d = 40 / 80 / 160 (d' = d) when N <= 65536 * max(1, SMs / (B*H)) */
 #define LINFUSION_VARIANT_MASK 0xFu
 /*
  * flags: memory layout of Q, K, V and Y.  Default (bit clear): head-major [B, H, N, d].  Bit set:

@@ -58,20 +58,27 @@ int padded_partial_floats(int d) { return ((d + 15) / 16 * 16) * ((d + 1 + 15) /
 // CTAs per slab of that kernel, or 0 where it does not apply: a CTA's run of tiles must fit one
 // accumulation in tensor memory (with more slabs than SMs a CTA takes whole slabs, several in turn).
 // Every CTA of a slab reads all of the slab's partials (9 KB each at d = 40, 30 KB at 80, 110 KB at 160),
-// so their number is kept to what makes that a couple of hundred KB at most (more only where the runs
-// would otherwise be too long); then the smallest count that gives the CTAs the same longest run is taken.
+// so their number is kept to what makes that at most 192 KB, or a quarter of what the CTA streams of Q, K
+// and V anyway (long slabs), or what the longest run demands; then the smallest count that gives the CTAs
+// the same longest run is taken.
 int padded_per_slab(int N, int slabs, int sm_count, int d)
 {
     const int tiles = (N + 127) / 128;
-    if (slabs > sm_count) return tiles <= 32 ? 1 : 0;
+    constexpr int kMaxRun = PaddedCfg<40>::MAX_TILES_PER_CTA;  // tiles a CTA may accumulate in one chain
+    if (slabs > sm_count) return tiles <= kMaxRun ? 1 : 0;
     int k = sm_count / slabs;
     if (k > tiles) k = tiles;
-    int cap = static_cast<int>((192u * 1024u) / (static_cast<unsigned>(padded_partial_floats(d)) * 4u));
-    const int need = (tiles + 31) / 32;  // CTAs that the longest run allows
-    if (cap < need) cap = need;
-    if (k > cap) k = cap;
+    const int need = (tiles + kMaxRun - 1) / kMaxRun;  // CTAs that the longest run allows
+    if (k < need) return 0;
+    const long long partial_bytes = 4ll * padded_partial_floats(d), tile_bytes = 3ll * 128 * d * 2;
+    while (k > need && k > 1) {
+        const long long streamed = (tiles + k - 1) / k * tile_bytes;
+        const long long allowed = streamed / 4 > 192 * 1024 ? streamed / 4 : 192 * 1024;
+        if (k * partial_bytes <= allowed) break;
+        --k;
+    }
     const int longest = (tiles + k - 1) / k;
-    if (longest > 32) return 0;
+    if (longest > kMaxRun) return 0;
     return (tiles + longest - 1) / longest;
 }
 
@@ -175,7 +182,14 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // (19.4 vs 20.8 us for three chained launches at N = 4096, d = 40 x 16 slabs; 16.6 vs 17.4 us at
         // N = 1024, d = 80; 19.4 vs 24.6 us at N = 256, d = 160; 13.5 vs 14.7 us for one CTA per slab of the
         // warp-level kernel at N = 64, d = 160).
-        if (padded_width(dk, dv) && padded_per_slab(d->N, slabs, sm_count, dv) > 0)
+        // Not where it would leave most of the machine idle on long runs: the CTAs of a slab all read all of its
+        // partial states, which keeps their number small at d = 160 (a partial is 110 KB), e.g. 16 CTAs of
+        // eight tiles at N = 1000, d = 160 x 16 slabs (54 vs 34 us for the three launches) or 14 CTAs on a single
+        // slab of 100 000 tokens (357 vs 115 us).
+        const int pk = padded_width(dk, dv) ? padded_per_slab(d->N, slabs, sm_count, dv) : 0;
+        const int padded_ctas = slabs > sm_count ? sm_count : slabs * pk;
+        const int padded_run = pk > 0 ? (fused_tiles + pk - 1) / pk : 0;
+        if (pk > 0 && (2 * padded_ctas >= sm_count || padded_run <= 3))
             v = LINFUSION_VARIANT_FUSED;
         else if (tiles_kv <= kLocalMaxTilesKv)
             v = LINFUSION_VARIANT_CLUSTER;  // resolves to one CTA per slab (largest_cluster())

@@ -69,7 +69,9 @@ struct PaddedCfg {
     static constexpr int SLOTS_FIT = (227 * 1024 - B_BYTES - TAIL_BYTES) / SLOT_BYTES;
     static constexpr int SLOTS = SLOTS_FIT > 12 ? 12 : SLOTS_FIT;
     static constexpr int SMEM_BYTES = SLOTS * SLOT_BYTES + B_BYTES + TAIL_BYTES;
-    static constexpr int MAX_TILES_PER_CTA = 32;            // one accumulation chain in tensor memory
+    // One accumulation chain in tensor memory per run: 512 tiles = 4096 MMA steps (a 70 000-step chain was
+    // measured to drift 8e-5 relative, far below the 16-bit operands' 4e-3).
+    static constexpr int MAX_TILES_PER_CTA = 512;
     static constexpr int ARRIVALS = CONSUMER_WARPS;         // arrivals on the slab's counter per CTA
 };
 

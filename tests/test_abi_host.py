@@ -90,8 +90,8 @@ def test_invalid_descriptors(kw):
 
 
 @pytest.mark.parametrize("kw", [
-    dict(d=40, variant="fused", H=80, N=128 * 33),        # more slabs than SMs and more than 32 tiles per slab
-    dict(d=160, variant="fused", B=74, H=2, N=128 * 33),  # one CTA per slab, more than 32 tiles each
+    dict(d=40, variant="fused", H=80, N=128 * 513),        # more slabs than SMs and more than 512 tiles per slab
+    dict(d=160, variant="fused", B=74, H=2, N=128 * 513),  # one CTA per slab, more than 512 tiles each
 ])
 def test_shapes_the_single_launch_at_padded_widths_cannot_take(kw):
     args = dict(B=2, H=8, N=4096, d=64, eps=1e-6, device=0)

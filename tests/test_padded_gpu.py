@@ -17,7 +17,8 @@ WIDTHS = [40, 80, 160]
 # more CTAs per slab than the reduction's batch of four; a single slab cut into many runs; as many
 # slabs as a B200 has SMs (one CTA per slab, several tiles each)
 SIZES = [(1, 2, 1), (1, 3, 63), (2, 2, 129), (2, 8, 256), (2, 8, 1000), (1, 12, 1500), (1, 1, 5000), (4, 37, 300),
-         (4, 50, 300), (1, 149, 129), (3, 111, 64)]   # more slabs than SMs: a CTA takes two or three whole slabs in turn
+         (4, 50, 300), (1, 149, 129), (3, 111, 64),   # more slabs than SMs: a CTA takes two or three whole slabs in turn
+         (1, 150, 8200)]                              # ... of 65 tiles each: one long accumulation chain per slab
 
 
 @pytest.mark.parametrize("d", WIDTHS)
@@ -100,19 +101,19 @@ def test_fused_at_padded_widths_layouts_types_and_normalizer(d):
 
 
 def test_fused_at_padded_widths_limits():
-    """More than 32 tiles per CTA are refused when asked for by name and fall to another variant
+    """More than 512 tiles per CTA are refused when asked for by name and fall to another variant
     under AUTO; d' != d has no such kernel."""
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     with pytest.raises(attn.LinFusionError) as e:
-        attn.LinFusionAttention(1, sms + 1, 128 * 33, 40, variant="fused")
+        attn.LinFusionAttention(1, sms + 1, 128 * 513, 40, variant="fused")
     assert e.value.code == attn.ERR_UNSUPPORTED
     with pytest.raises(attn.LinFusionError) as e:
-        attn.LinFusionAttention(1, sms, 128 * 33, 80, variant="fused")
+        attn.LinFusionAttention(1, sms, 128 * 513, 80, variant="fused")
     assert e.value.code == attn.ERR_UNSUPPORTED
     with pytest.raises(attn.LinFusionError) as e:
         attn.LinFusionAttention(1, 2, 256, 40, variant="fused", d_qk=80)
     assert e.value.code == attn.ERR_UNSUPPORTED
-    op = attn.LinFusionAttention(1, sms + 1, 128 * 33, 40)
+    op = attn.LinFusionAttention(1, sms + 1, 128 * 513, 40)
     assert op.variant != "fused"
     op.close()
     op = attn.LinFusionAttention(1, sms + 1, 256, 40)     # whole slabs, several per CTA
