@@ -546,12 +546,22 @@ def run_sweep(args):
     torch.cuda.set_device(0)
     peak, _ = measured_peak_gbs()
     seen = set()
-    for cfg_idx, cfg in enumerate(wl.CONFIGS):
+    configs = list(wl.CONFIGS)
+    if args.shape:
+        # extra shapes given on the command line (beyond the five workload families): B,H,N,d each
+        extra = []
+        for spec in args.shape:
+            B, H, N, d = (int(x) for x in spec.split(","))
+            extra.append(wl.AttnShape(f"B{B}_H{H}_N{N}_d{d}", B, H, N, d))
+        configs = [extra]
+    for cfg_idx, cfg in enumerate(configs):
         for s in cfg:
             if s.name in seen or (args.only and s.name != args.only):
                 continue
             seen.add(s.name)
             sets = max(1, min(64, -(-400_000_000 // s.min_bytes)))
+            if s.min_bytes > (2 << 30):
+                sets = 1
             bufs = []
             for r in range(sets):
                 q, k, v = wl.make_qkv(s, seed=wl.BASE_SEED + r, device="cuda:0")
@@ -713,6 +723,8 @@ def main(argv=None):
     ap.add_argument("--sweep", action="store_true",
                     help="time every shape of the five workload families with every variant")
     ap.add_argument("--only", default="", help="with --sweep / --from-x: restrict to one shape, e.g. sd15_512_L1")
+    ap.add_argument("--shape", action="append", default=[], metavar="B,H,N,d",
+                    help="with --sweep: time this shape instead of the workload families (may be given several times)")
     ap.add_argument("--from-x", action="store_true",
                     help="time the module fed from the layer input X (fused projections) beside the un-fused route")
     argv = sys.argv[1:] if argv is None else argv
