@@ -170,6 +170,17 @@ linfusion_status_t linfusion_attn_workspace_bytes(const linfusion_attn_desc_t* d
                                                   size_t* bytes);
 
 /*
+ * What a handle for `desc` would run on a device with `sm_count` SMs (<= 0: 148), without creating
+ * one: *variant receives the LINFUSION_VARIANT_* that desc.flags resolves to (AUTO resolved from
+ * (N, d, B*H) as create() does it, before any fall-back create() may take when a cluster cannot be
+ * scheduled), *launches the kernel launches per forward, *ctas the grid size of its largest kernel
+ * (0 for the split and cluster variants, whose grids are two-dimensional).  Pure host computation (no
+ * CUDA call); any of the three pointers may be NULL.  Errors: INVALID_ARG, UNSUPPORTED.
+ */
+linfusion_status_t linfusion_attn_plan(const linfusion_attn_desc_t* desc, int sm_count, int32_t* variant,
+                                       int32_t* launches, int32_t* ctas);
+
+/*
  * Lend a device workspace (256-byte aligned, at least workspace_bytes) to the handle, which
  * stops using — and frees — its own.  The caller keeps ownership and must keep it alive
  * until the handle is destroyed.  Errors: INVALID_ARG, ALLOC (too small).

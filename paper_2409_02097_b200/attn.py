@@ -84,6 +84,9 @@ def load_library() -> ctypes.CDLL:
     lib.linfusion_attn_destroy.argtypes = [vp]
     lib.linfusion_status_string.restype = ctypes.c_char_p
     lib.linfusion_status_string.argtypes = [st]
+    lib.linfusion_attn_plan.restype = st
+    lib.linfusion_attn_plan.argtypes = [ctypes.POINTER(Desc), ctypes.c_int, ctypes.POINTER(ctypes.c_int32),
+                                        ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32)]
     lib.linfusion_attn_workspace_bytes.restype = st
     lib.linfusion_attn_workspace_bytes.argtypes = [ctypes.POINTER(Desc), ctypes.c_int,
                                                    ctypes.POINTER(ctypes.c_size_t)]
@@ -195,6 +198,17 @@ def linfusion_attn_workspace_bytes(desc: Desc, sm_count: int = 0) -> int:
     if rc != OK:
         raise LinFusionError(rc, "linfusion_attn_workspace_bytes")
     return int(out.value)
+
+
+def linfusion_attn_plan(desc: Desc, sm_count: int = 0):
+    """(variant name, launches per forward, CTAs of the largest one-dimensional grid) for ``desc``, no GPU needed."""
+    variant, launches, ctas = ctypes.c_int32(0), ctypes.c_int32(0), ctypes.c_int32(0)
+    rc = load_library().linfusion_attn_plan(ctypes.byref(desc), int(sm_count), ctypes.byref(variant),
+                                            ctypes.byref(launches), ctypes.byref(ctas))
+    if rc != OK:
+        raise LinFusionError(rc, "linfusion_attn_plan")
+    names = {v: k for k, v in VARIANTS.items()}
+    return names[variant.value], int(launches.value), int(ctas.value)
 
 
 def linfusion_attn_create(desc: Desc) -> ctypes.c_void_p:

@@ -913,6 +913,18 @@ linfusion_status_t linfusion_attn_workspace_bytes(const linfusion_attn_desc_t* d
     return LINFUSION_OK;
 }
 
+linfusion_status_t linfusion_attn_plan(const linfusion_attn_desc_t* desc, int sm_count, int32_t* variant,
+                                       int32_t* launches, int32_t* ctas)
+{
+    Plan p;
+    linfusion_status_t st = make_plan(desc, sm_count, &p);
+    if (st != LINFUSION_OK) return st;
+    if (variant != nullptr) *variant = p.variant;
+    if (launches != nullptr) *launches = p.launches;
+    if (ctas != nullptr) *ctas = p.G_state > p.G_apply ? p.G_state : p.G_apply;
+    return LINFUSION_OK;
+}
+
 linfusion_status_t linfusion_attn_create(const linfusion_attn_desc_t* desc, linfusion_attn_t** out)
 {
     if (out == nullptr) return LINFUSION_ERR_INVALID_ARG;

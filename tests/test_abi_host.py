@@ -205,3 +205,41 @@ def test_two_widths_in_the_descriptor():
     # the allocation-free entry point sizes its array use by d' * (d + 1) too
     chunks, off, used, cap = attn.linfusion_attn_noalloc_layout(attn.make_desc(2, 8, 4096, 64, d_qk=128), 148)
     assert used - off == 16 * 128 * 65 * 4 and used <= cap and chunks >= 1
+
+
+# (B, H, N, d) -> what AUTO resolves to on a 148-SM device (the crossovers measured on B200; the GPU tests check
+# the same table against handles created on the device)
+AUTO_POLICY = [
+    ((2, 10, 524288, 64), "stream", 2), ((2, 20, 131072, 64), "stream", 2),
+    ((2, 10, 16384, 64), "stream", 2), ((2, 20, 4096, 64), "stream", 2), ((2, 20, 2304, 64), "stream", 2),
+    ((2, 10, 9216, 64), "stream", 2), ((1, 10, 2304, 64), "split", 3), ((2, 20, 144, 64), "cluster", 1),
+    ((2, 20, 576, 64), "fused", 1), ((2, 2, 144, 64), "cluster", 1),
+    ((2, 8, 4096, 40), "fused", 1), ((2, 8, 1024, 80), "fused", 1), ((2, 8, 256, 160), "fused", 1),
+    ((2, 8, 64, 160), "fused", 1), ((2, 100, 256, 160), "fused", 1), ((2, 100, 8192, 160), "fused", 1),
+    ((2, 100, 131072, 160), "split", 3), ((2, 8, 1000, 160), "split", 3), ((1, 1, 100000, 160), "split", 3),
+    ((2, 8, 16384, 160), "fused", 1), ((32, 8, 4096, 40), "fused", 1), ((2, 8, 4096, 128), "split", 3),
+    ((2, 8, 64, 128), "cluster", 1), ((300, 1, 4096, 64), "stream", 3),
+]
+
+
+def test_auto_policy_without_a_device():
+    for dims, want, launches in AUTO_POLICY:
+        variant, n, ctas = attn.linfusion_attn_plan(attn.make_desc(*dims), 148)
+        assert (variant, n) == (want, launches), (dims, variant, n)
+        assert 0 <= ctas <= 148
+    # the grids of the one-dimensional kernels: equal CTA counts per slab for short runs, every SM for long ones
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 20, 4096, 64), 148)[2] == 120
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 10, 16384, 64), 148)[2] == 140
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 10, 524288, 64), 148)[2] == 148
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 4096, 40), 148)[2] == 128        # 8 CTAs per slab
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 1024, 80), 148)[2] == 64         # 4 per slab
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 256, 160), 148)[2] == 16         # one per slab
+    assert attn.linfusion_attn_plan(attn.make_desc(32, 8, 4096, 40), 148)[2] == 148       # whole slabs in turn
+    # a requested variant is kept; a smaller device changes the split
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 4096, 40, variant="split"), 148)[0] == "split"
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 20, 4096, 64), 74)[2] == 74         # 40 of 74 SMs would be too few
+    lib = attn.load_library()
+    assert lib.linfusion_attn_plan(None, 0, None, None, None) == attn.ERR_INVALID_ARG
+    with pytest.raises(attn.LinFusionError) as e:
+        attn.linfusion_attn_plan(attn.make_desc(2, 8, 4096, 48), 148)
+    assert e.value.code == attn.ERR_UNSUPPORTED
