@@ -440,3 +440,27 @@ def test_fused_variant_many_forwards_in_a_row_and_its_bounded_counter_wait():
         op.state(ka, va)                       # one launch cannot be split in two halves
     assert e.value.code == attn.ERR_UNSUPPORTED
     op.close()
+
+
+def test_many_back_to_back_forwards_give_the_same_bits():
+    """A hundred chained forwards per shape (each starts while the one before drains) into rotating outputs:
+    every one must equal the first bit for bit.  Covers the paths with cross-CTA hand-offs: counters and
+    operand buffers of the stream kernels, fixed runs, the single launches with their slab counters, a CTA
+    taking several slabs in turn."""
+    cases = [(2, 8, 4096, 40, "fused"), (2, 8, 1024, 80, "fused"), (3, 111, 64, 160, "fused"), (4, 50, 300, 80, "fused"),
+             (2, 20, 4096, 64, "stream"), (2, 5, 9216, 64, "stream"), (8, 25, 300, 64, "stream"),
+             (3, 100, 100, 64, "stream"), (1, 7, 200000, 64, "stream"), (2, 20, 576, 64, "fused")]
+    for (B, H, N, d, variant) in cases:
+        q, k, v = wl.make_small(B, H, N, d, seed=17, device="cuda", v_mean=1.0)
+        op = attn.LinFusionAttention(B, H, N, d, variant=variant)
+        y0 = op.forward(q, k, v).clone()
+        ys = [torch.empty_like(y0) for _ in range(4)]
+        reps = 100 if N < 100000 else 24
+        for r in range(reps):
+            op.forward(q, k, v, y=ys[r % 4])
+            if r % 4 == 3:
+                torch.cuda.synchronize()
+                for t in ys:
+                    assert torch.equal(t, y0), (B, H, N, d, variant, r)
+        assert op.status() == attn.OK
+        op.close()
