@@ -54,6 +54,8 @@ bool supported_widths(int dk, int dv)
 // (padded_kernels.cuh), d' = d.
 bool padded_width(int dk, int dv) { return dk == dv && (dv == 40 || dv == 80 || dv == 160); }
 int padded_partial_floats(int d) { return ((d + 15) / 16 * 16) * ((d + 1 + 15) / 16 * 16); }
+// Bytes of its apply operand per slab (64-channel atoms of one 128-byte row per feature).
+size_t padded_image_bytes(int d) { return static_cast<size_t>(((d + 1 + 15) / 16 * 16 + 63) / 64) * ((d + 15) / 16 * 16) * 128; }
 
 // CTAs per slab of that kernel, or 0 where it does not apply: a CTA's run of tiles must fit one
 // accumulation in tensor memory (with more slabs than SMs a CTA takes whole slabs, several in turn).
@@ -61,13 +63,14 @@ int padded_partial_floats(int d) { return ((d + 15) / 16 * 16) * ((d + 1 + 15) /
 // so their number is kept to what makes that at most 192 KB, or a quarter of what the CTA streams of Q, K
 // and V anyway (long slabs), or what the longest run demands; then the smallest count that gives the CTAs
 // the same longest run is taken.
-int padded_per_slab(int N, int slabs, int sm_count, int d)
+int padded_per_slab(int N, int slabs, int sm_count, int d, int* scatter = nullptr)
 {
+    if (scatter != nullptr) *scatter = 0;
     const int tiles = (N + 127) / 128;
     constexpr int kMaxRun = PaddedCfg<40>::MAX_TILES_PER_CTA;  // tiles a CTA may accumulate in one chain
     if (slabs > sm_count) return tiles <= kMaxRun ? 1 : 0;
-    int k = sm_count / slabs;
-    if (k > tiles) k = tiles;
+    const int k_max = sm_count / slabs < tiles ? sm_count / slabs : tiles;
+    int k = k_max;
     const int need = (tiles + kMaxRun - 1) / kMaxRun;  // CTAs that the longest run allows
     if (k < need) return 0;
     const long long partial_bytes = 4ll * padded_partial_floats(d), tile_bytes = 3ll * 128 * d * 2;
@@ -77,8 +80,17 @@ int padded_per_slab(int N, int slabs, int sm_count, int d)
         if (k * partial_bytes <= allowed) break;
         --k;
     }
-    const int longest = (tiles + k - 1) / k;
+    int longest = (tiles + k - 1) / k;
     if (longest > kMaxRun) return 0;
+    // Where that rule leaves runs of four tiles or more and every SM's worth of CTAs would at least halve
+    // them, the CTAs of a slab share the summing instead (two exchange rounds, see the kernel): each reads
+    // one partial's worth and the 16-bit operand, however many they are.  Needs a row of S per CTA.
+    const int k_all = k_max < d ? k_max : d;
+    const int longest_all = (tiles + k_all - 1) / k_all;
+    if (longest >= 4 && 2 * longest_all <= longest) {
+        if (scatter != nullptr) *scatter = 1;
+        longest = longest_all;
+    }
     return (tiles + longest - 1) / longest;
 }
 
@@ -103,6 +115,7 @@ struct Plan {
     // fused
     int fused_split = 0, fused_whole = 0;
     int padded_per_slab = 0;  // fused, widths 40 / 80 / 160: CTAs per slab
+    int padded_scatter = 0;   // ... and whether they share the summing of the partial states (two rounds)
     // workspace (bytes, offsets)
     size_t partial_bytes = 0, state_off = 0, operand_off = 0, counters_off = 0, status_off = 0, total_bytes = 0;
     int launches = 0;
@@ -277,7 +290,7 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         p->launches = p->merged_reduce != 0 ? 2 : 3;
     } else if (v == LINFUSION_VARIANT_FUSED && !square64) {
         // One persistent launch, widths 40 / 80 / 160: per_slab CTAs on every slab, one partial each.
-        p->padded_per_slab = padded_per_slab(d->N, slabs, sm_count, dv);
+        p->padded_per_slab = padded_per_slab(d->N, slabs, sm_count, dv, &p->padded_scatter);
         if (p->padded_per_slab == 0) return LINFUSION_ERR_UNSUPPORTED;
         p->tiles_state = p->tiles_apply = (d->N + 127) / 128;
         p->G_state = p->G_apply = slabs > sm_count ? sm_count : slabs * p->padded_per_slab;
@@ -331,6 +344,7 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
     const size_t split_image = static_cast<size_t>((dv + 8 + 15) / 16 * 16) * (((dkp / 8) | 1) * 16);
     const size_t frag_bytes = v == LINFUSION_VARIANT_STREAM  ? static_cast<size_t>(slabs) * kStreamOperandBytes
                               : v == LINFUSION_VARIANT_SPLIT ? static_cast<size_t>(slabs) * split_image
+                              : p->padded_scatter != 0       ? static_cast<size_t>(slabs) * padded_image_bytes(dv)
                                                              : 0;
     // Stream: one tile counter and one ready flag per slab.  Fused: two arrival counters per slab, then the control words.
     const size_t counter_bytes = v == LINFUSION_VARIANT_STREAM  ? align_up(static_cast<size_t>(slabs) * 8, 256)
@@ -799,9 +813,14 @@ cudaError_t launch_padded(const linfusion_attn* h, const __nv_bfloat16* q, const
     uint32_t* counters = reinterpret_cast<uint32_t*>(h->tile_counters);
     uint32_t* ctrl = counters + align_up(static_cast<size_t>(p.slabs) * 8, 256) / 4;
     mark(h, 0, s);
-    cudaError_t e = launch_chained(padded_fused_kernel<D, KIND>, dim3(p.G_state), dim3(C::THREADS), C::SMEM_BYTES, s, mk,
-                                   mv, mq, my, h->partials, h->state, counters, ctrl, h->status, h->desc.N,
-                                   p.tiles_state, p.padded_per_slab, p.slabs, h->desc.H, apply_scales(h->desc));
+    cudaError_t e =
+        p.padded_scatter != 0
+            ? launch_chained(padded_fused_kernel<D, KIND, 1>, dim3(p.G_state), dim3(C::THREADS), C::SMEM_BYTES, s, mk, mv, mq,
+                             my, h->partials, h->state, h->operand, counters, ctrl, h->status, h->desc.N, p.tiles_state,
+                             p.padded_per_slab, p.slabs, h->desc.H, apply_scales(h->desc))
+            : launch_chained(padded_fused_kernel<D, KIND, 0>, dim3(p.G_state), dim3(C::THREADS), C::SMEM_BYTES, s, mk, mv, mq,
+                             my, h->partials, h->state, h->operand, counters, ctrl, h->status, h->desc.N, p.tiles_state,
+                             p.padded_per_slab, p.slabs, h->desc.H, apply_scales(h->desc));
     if (e != cudaSuccess) return e;
     mark(h, 1, s);
     return cudaGetLastError();
@@ -828,7 +847,12 @@ cudaError_t set_attrs_d(int kind)
     if constexpr (DK == DV && (DV == 40 || DV == 80 || DV == 160)) {
         if (e != cudaSuccess) return e;
 #define LF_K(KV) \
-    e = cudaFuncSetAttribute(padded_fused_kernel<DV, KV>, cudaFuncAttributeMaxDynamicSharedMemorySize, PaddedCfg<DV>::SMEM_BYTES)
+    e = cudaFuncSetAttribute(padded_fused_kernel<DV, KV, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, PaddedCfg<DV>::SMEM_BYTES)
+        LF_DISPATCH_KIND(kind, LF_K)
+#undef LF_K
+        if (e != cudaSuccess) return e;
+#define LF_K(KV) \
+    e = cudaFuncSetAttribute(padded_fused_kernel<DV, KV, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, PaddedCfg<DV>::SMEM_BYTES)
         LF_DISPATCH_KIND(kind, LF_K)
 #undef LF_K
     }

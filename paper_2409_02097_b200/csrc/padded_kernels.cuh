@@ -29,7 +29,9 @@
 //      shared memory), each thread divides its row by the z column (Eq. 5), writes the 16-bit row
 //      over the Q row, and a TMA store (clipped at D channels and N tokens) sends the tile to Y.
 // Every CTA of a slab reads all of its partials, so the host keeps per_slab small enough for that
-// to stay a few hundred KB.  A CTA that has its slab to itself (per_slab = 1) skips 2-3: it builds
+// to stay a few hundred KB — or, where that would leave long runs (large partials: d = 160), asks for the
+// shared form of step 3 (`scatter`): CTA r sums only its share of the rows c, publishes that share of the
+// operand and of the fp32 state, and after a second counter round every CTA copies the whole operand.  A CTA that has its slab to itself (per_slab = 1) skips 2-3: it builds
 // the operand and the fp32 state straight from the accumulator; with more slabs than SMs such a CTA
 // takes several whole slabs one after the other (the K/V tiles of the next slab are fetched while the
 // current one is applied).  The counters are zeroed again by the CTA that finishes last, so every
@@ -118,15 +120,19 @@ __device__ __forceinline__ void phi_row_in_place(uint32_t row_addr, uint32_t sw)
 
 // grid = slabs * per_slab CTAs; CTA g works on slab g / per_slab, run g % per_slab of its tiles (per_slab = 1:
 // grid <= slabs, CTA g on slabs g, g + grid, ...).
-// partials: [slab][run][DKN][DVN] fp32; state: [slab][D*D + D] fp32 (S [c][e], then z [c]); counters: one
-// word per slab, zero between forwards; ctrl: kPaddedCtrlWords words, zero between forwards.
-template <int D, int KIND>
+// partials: [slab][run][DKN][DVN] fp32; state: [slab][D*D + D] fp32 (S [c][e], then z [c]); images (scatter
+// only): [slab][B_BYTES], zero wherever nothing is ever written; counters: two words per slab, zero between
+// forwards; ctrl: kPaddedCtrlWords words, zero between forwards.  SCATTER != 0: instead of every CTA of a slab
+// summing all of its partials, CTA r sums its share of the rows c, publishes that share of the 16-bit operand
+// (and of the fp32 state), and every CTA copies the whole operand once all shares are there — two exchange
+// rounds instead of one, but per_slab times less to read: for slabs whose partials are large (d = 160).
+template <int D, int KIND, int SCATTER>
 __global__ void __launch_bounds__(PaddedCfg<D>::THREADS, 1)
 padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_constant__ CUtensorMap tmap_v,
                     const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_y,
-                    float* __restrict__ partials, float* __restrict__ state, uint32_t* __restrict__ counters,
-                    uint32_t* __restrict__ ctrl, uint32_t* __restrict__ status, int N, int tiles_per_slab,
-                    int per_slab, int slabs, int H, ApplyScales sc)
+                    float* __restrict__ partials, float* __restrict__ state, unsigned char* __restrict__ images,
+                    uint32_t* __restrict__ counters, uint32_t* __restrict__ ctrl, uint32_t* __restrict__ status, int N,
+                    int tiles_per_slab, int per_slab, int slabs, int H, ApplyScales sc)
 {
     using C = PaddedCfg<D>;
     extern __shared__ unsigned char smem_raw[];
@@ -427,7 +433,8 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
         if (per_slab > 1) {
             // 3. all partials of the slab, summed in run order -> the apply operand; this CTA's share of the
             //    rows c also goes to the fp32 state
-            uint32_t* cnt = counters + slab;
+            uint32_t* cnt = counters + 2 * slab;
+            unsigned char* image = images + static_cast<size_t>(slab) * C::B_BYTES;
             if (lane == 0) red_release_gpu_add(cnt, 1u);  // also after a failure: the others must not wait for it
             if (ok) {
                 uint32_t arrived = 0u;
@@ -445,7 +452,9 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                 const float* src0 = partials + static_cast<size_t>(slab) * per_slab * C::PARTIAL_FLOATS;
                 const int c_begin = padded_run_begin(run, D, per_slab), c_end = padded_run_begin(run + 1, D, per_slab);
                 const uint32_t b_addr = smem_u32(bsm);
-                constexpr int kItems = D * C::ECHUNKS;  // rows c >= D of the operand stay zero
+                // rows c >= D of the operand stay zero; with scatter only this CTA's rows are summed here
+                const int row0 = SCATTER != 0 ? c_begin : 0;
+                const int kItems = (SCATTER != 0 ? c_end - c_begin : D) * C::ECHUNKS;  // a constant without SCATTER
                 int item = ctid, p = 0;
                 float acc[8];
                 while (item < kItems) {
@@ -454,7 +463,7 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         if (it2 < kItems) {
-                            const int c2 = it2 / C::ECHUNKS, j2 = it2 - c2 * C::ECHUNKS;
+                            const int r2 = it2 / C::ECHUNKS, j2 = it2 - r2 * C::ECHUNKS, c2 = row0 + r2;
                             const float4* sp = reinterpret_cast<const float4*>(src0 + static_cast<size_t>(p2) * C::PARTIAL_FLOATS +
                                                                               c2 * C::DVN + j2 * 8);
                             a[u] = __ldcg(sp);
@@ -476,15 +485,18 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                                 acc[4] += b[u].x; acc[5] += b[u].y; acc[6] += b[u].z; acc[7] += b[u].w;
                             }
                             if (++p == per_slab) {
-                                const int c = item / C::ECHUNKS, j = item - c * C::ECHUNKS;
+                                const int r = item / C::ECHUNKS, j = item - r * C::ECHUNKS, c = row0 + r;
                                 const uint32_t v0 = to_storage16(acc[0] * sc.operand, dtype) | (static_cast<uint32_t>(to_storage16(acc[1] * sc.operand, dtype)) << 16);
                                 const uint32_t v1 = to_storage16(acc[2] * sc.operand, dtype) | (static_cast<uint32_t>(to_storage16(acc[3] * sc.operand, dtype)) << 16);
                                 const uint32_t v2 = to_storage16(acc[4] * sc.operand, dtype) | (static_cast<uint32_t>(to_storage16(acc[5] * sc.operand, dtype)) << 16);
                                 const uint32_t v3 = to_storage16(acc[6] * sc.operand, dtype) | (static_cast<uint32_t>(to_storage16(acc[7] * sc.operand, dtype)) << 16);
                                 // operand row c, channels 8 j .. 8 j + 7: atom j / 8, chunk position (j % 8) ^ (c % 8)
-                                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(b_addr + (j >> 3) * C::B_ATOM_BYTES + c * 128 + (((j & 7) ^ (c & 7)) << 4)),
-                                             "r"(v0), "r"(v1), "r"(v2), "r"(v3)
-                                             : "memory");
+                                const uint32_t b_off = (j >> 3) * C::B_ATOM_BYTES + c * 128 + (((j & 7) ^ (c & 7)) << 4);
+                                if (SCATTER != 0)
+                                    __stcg(reinterpret_cast<uint4*>(image + b_off), make_uint4(v0, v1, v2, v3));
+                                else
+                                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(b_addr + b_off), "r"(v0), "r"(v1), "r"(v2), "r"(v3)
+                                                 : "memory");
                                 if (c >= c_begin && c < c_end) {
                                     if (j < D / 8) {
                                         float4* sp = reinterpret_cast<float4*>(st + c * D + j * 8);
@@ -498,6 +510,34 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
                                 item += C::CONSUMER_THREADS;
                             }
                         }
+                    }
+                }
+            }
+            if (SCATTER != 0) {
+                // second round: every share of the operand image is there -> copy it (eight loads in flight)
+                __syncwarp();
+                if (lane == 0) red_release_gpu_add(&cnt[1], 1u);
+                if (ok) {
+                    uint32_t arrived = 0u;
+                    if (lane == 0) arrived = counter_wait(&cnt[1], 0u, static_cast<uint32_t>(C::ARRIVALS * per_slab)) ? 1u : 0u;
+                    arrived = __shfl_sync(0xffffffffu, arrived, 0);
+                    if (arrived == 0u) {
+                        ok = false;
+                        if (lane == 0) report_wait_expired(status);
+                    }
+                }
+                if (ok) {
+                    const uint4* src = reinterpret_cast<const uint4*>(image);
+                    uint4* dst = reinterpret_cast<uint4*>(bsm);
+                    constexpr int kVec = C::B_BYTES / 16;
+                    for (int i0 = ctid; i0 < kVec; i0 += 8 * C::CONSUMER_THREADS) {
+                        uint4 v[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if (i0 + u * C::CONSUMER_THREADS < kVec) v[u] = __ldcg(src + i0 + u * C::CONSUMER_THREADS);
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if (i0 + u * C::CONSUMER_THREADS < kVec) dst[i0 + u * C::CONSUMER_THREADS] = v[u];
                     }
                 }
             }
@@ -571,7 +611,7 @@ padded_fused_kernel(const __grid_constant__ CUtensorMap tmap_k, const __grid_con
     if (tid == 0) {
         __threadfence();
         if (atomicAdd(&ctrl[0], 1u) == gridDim.x - 1) {
-            for (int s = 0; s < slabs; ++s) counters[s] = 0u;
+            for (int s = 0; s < 2 * slabs; ++s) counters[s] = 0u;
             ctrl[0] = 0u;
             __threadfence();
         }

@@ -66,6 +66,11 @@ def test_workspace_bytes_is_pure_host_and_monotone():
     # one CTA per slab (d = 160: a partial is 110 KB, so slabs are not shared): no partials at all
     assert _ws(attn.make_desc(2, 8, 256, 160, variant="fused")) == \
         (16 * 160 * 161 * 4 + 255) // 256 * 256 + 256 + 256 + 256
+    # long runs with large partials: 8 CTAs per slab share the summing; partials, state, the 16-bit operand per
+    # slab (3 atoms x 160 rows x 128 bytes), counters + control, status
+    assert _ws(attn.make_desc(2, 8, 1024, 160, variant="fused")) == \
+        (16 * 8 * 160 * 176 * 4 + 255) // 256 * 256 + (16 * 160 * 161 * 4 + 255) // 256 * 256 + \
+        (16 * 3 * 160 * 128 + 255) // 256 * 256 + 256 + 256 + 256
     # more slabs than SMs: whole slabs per CTA, no partials either
     assert _ws(attn.make_desc(2, 100, 256, 40, variant="fused")) == \
         (200 * 40 * 41 * 4 + 255) // 256 * 256 + (200 * 8 + 255) // 256 * 256 + 256 + 256
@@ -216,7 +221,7 @@ AUTO_POLICY = [
     ((2, 20, 576, 64), "fused", 1), ((2, 2, 144, 64), "cluster", 1),
     ((2, 8, 4096, 40), "fused", 1), ((2, 8, 1024, 80), "fused", 1), ((2, 8, 256, 160), "fused", 1),
     ((2, 8, 64, 160), "fused", 1), ((2, 100, 256, 160), "fused", 1), ((2, 100, 8192, 160), "fused", 1),
-    ((2, 100, 131072, 160), "split", 3), ((2, 8, 1000, 160), "split", 3), ((1, 1, 100000, 160), "split", 3),
+    ((2, 100, 131072, 160), "split", 3), ((2, 8, 1000, 160), "fused", 1), ((1, 1, 100000, 160), "fused", 1),
     ((2, 8, 16384, 160), "fused", 1), ((32, 8, 4096, 40), "fused", 1), ((2, 8, 4096, 128), "split", 3),
     ((2, 8, 64, 128), "cluster", 1), ((300, 1, 4096, 64), "stream", 3),
 ]
@@ -235,6 +240,8 @@ def test_auto_policy_without_a_device():
     assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 1024, 80), 148)[2] == 64         # 4 per slab
     assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 256, 160), 148)[2] == 16         # one per slab
     assert attn.linfusion_attn_plan(attn.make_desc(32, 8, 4096, 40), 148)[2] == 148       # whole slabs in turn
+    assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 1024, 160), 148)[2] == 128       # 8 per slab, sharing the summing
+    assert attn.linfusion_attn_plan(attn.make_desc(1, 1, 100000, 160), 148)[2] == 131
     # a requested variant is kept; a smaller device changes the split
     assert attn.linfusion_attn_plan(attn.make_desc(2, 8, 4096, 40, variant="split"), 148)[0] == "split"
     assert attn.linfusion_attn_plan(attn.make_desc(2, 20, 4096, 64), 74)[2] == 74         # 40 of 74 SMs would be too few

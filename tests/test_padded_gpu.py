@@ -18,7 +18,8 @@ WIDTHS = [40, 80, 160]
 # slabs as a B200 has SMs (one CTA per slab, several tiles each)
 SIZES = [(1, 2, 1), (1, 3, 63), (2, 2, 129), (2, 8, 256), (2, 8, 1000), (1, 12, 1500), (1, 1, 5000), (4, 37, 300),
          (4, 50, 300), (1, 149, 129), (3, 111, 64),   # more slabs than SMs: a CTA takes two or three whole slabs in turn
-         (1, 150, 8200)]                              # ... of 65 tiles each: one long accumulation chain per slab
+         (1, 150, 8200),                              # ... of 65 tiles each: one long accumulation chain per slab
+         (2, 8, 1500), (1, 1, 30000)]                 # long runs on few slabs: the CTAs of a slab share the summing (two rounds)
 
 
 @pytest.mark.parametrize("d", WIDTHS)

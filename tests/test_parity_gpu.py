@@ -154,7 +154,7 @@ def test_auto_policy_follows_the_measured_crossovers():
                        ((2, 2, 144, 64), "cluster"), ((2, 8, 4096, 40), "fused"), ((2, 8, 1024, 80), "fused"),
                        ((2, 8, 64, 160), "fused"), ((2, 8, 256, 160), "fused"), ((2, 100, 256, 160), "fused"),
                        ((2, 100, 64, 160), "fused"), ((2, 100, 8192, 160), "fused"), ((2, 100, 131072, 160), "split"),
-                       ((2, 8, 1000, 160), "split"), ((1, 1, 100000, 160), "split"), ((2, 8, 16384, 160), "fused"), ((2, 8, 4096, 128), "split")]:
+                       ((2, 8, 1000, 160), "fused"), ((1, 1, 100000, 160), "fused"), ((2, 8, 16384, 160), "fused"), ((2, 8, 4096, 128), "split")]:
         op = attn.LinFusionAttention(*dims)
         assert op.variant == want, (dims, op.variant)
         op.close()
