@@ -195,10 +195,8 @@ linfusion_status_t make_plan(const linfusion_attn_desc_t* d, int sm_count, Plan*
         // (19.4 vs 20.8 us for three chained launches at N = 4096, d = 40 x 16 slabs; 16.6 vs 17.4 us at
         // N = 1024, d = 80; 19.4 vs 24.6 us at N = 256, d = 160; 13.5 vs 14.7 us for one CTA per slab of the
         // warp-level kernel at N = 64, d = 160).
-        // Not where it would leave most of the machine idle on long runs: the CTAs of a slab all read all of its
-        // partial states, which keeps their number small at d = 160 (a partial is 110 KB), e.g. 16 CTAs of
-        // eight tiles at N = 1000, d = 160 x 16 slabs (54 vs 34 us for the three launches) or 14 CTAs on a single
-        // slab of 100 000 tokens (357 vs 115 us).
+        // Not where it would leave most of the machine idle on runs of more than three tiles (few CTAs per slab
+        // because the partial states are large and sharing their summing does not pay: padded_per_slab()).
         const int pk = padded_width(dk, dv) ? padded_per_slab(d->N, slabs, sm_count, dv) : 0;
         const int padded_ctas = slabs > sm_count ? sm_count : slabs * pk;
         const int padded_run = pk > 0 ? (fused_tiles + pk - 1) / pk : 0;
